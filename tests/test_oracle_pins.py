@@ -1,0 +1,347 @@
+"""Pins for the CPU oracle: everything here checks ``oracle/`` against something other than
+itself -- numbers the paper prints, blocks worked by hand (tests/golden), exact rational
+arithmetic on tiny inputs, numpy's own fp64/int64 matmul on special cases, and invariants the
+format definition implies (Sec. 2 "What are MX Formats?", Sec. 4.1, Eq. 1, Sec. 3.2)."""
+import math
+from fractions import Fraction
+
+import numpy as np
+import pytest
+
+from oracle import mx_oracle as orc
+from tests import golden_io
+
+WIDTHS = (2, 3, 4, 5, 6, 8)
+BLOCKS = (16, 32)
+
+
+def _block_row(vals, B):
+    x = np.zeros((1, B), np.float32)
+    x[0, : len(vals)] = np.asarray(vals, np.float32)
+    return x
+
+
+# --------------------------------------------------------------------------- paper numbers
+
+def test_average_bits_matches_paper_example():
+    recs = [r for r in golden_io.load() if r["kind"] in ("paper", "closed") and "bits" in r]
+    assert recs
+    for r in recs:
+        w = int(r["m"]) + 1
+        got = orc.format_bits(int(r["block"]), w, int(r["block_rows"]), int(r["exp_bits"]))
+        assert got == float(r["bits"])
+
+
+def test_memory_density_matches_table1():
+    rec = [r for r in golden_io.load() if "mxint8_density" in r][0]
+    bits = orc.format_bits(16, 8, 2, 8)
+    density = float(rec["fp32_bits"]) / bits
+    assert math.floor(density * 10) / 10 == float(rec["mxint8_density"])
+
+
+# --------------------------------------------------------------------------- hand-worked blocks
+
+@pytest.mark.parametrize("B", BLOCKS)
+def test_hand_worked_blocks(B):
+    recs = [r for r in golden_io.load() if r["kind"] == "block"]
+    assert len(recs) >= 8
+    for r in recs:
+        w = int(r["w"])
+        xs = golden_io.floats(r["x"])
+        q, e, bad = orc.quantize(_block_row(xs, B), B, w)
+        assert bad == 0
+        assert int(e[0, 0]) == int(r["ebyte"]), r["id"]
+        assert q[0, : len(xs)].tolist() == golden_io.ints(r["q"]), r["id"]
+        assert not q[0, len(xs):].any()
+        xhat = orc.dequantize(q, e, B, w)
+        assert xhat[0, : len(xs)].tolist() == golden_io.floats(r["xhat"]), r["id"]
+        if r["packed"] != "-":
+            want = [int(t, 16) for t in r["packed"].split(",")]
+            got = orc.pack(q, w)
+            assert got[0, : len(want)].tolist() == want, r["id"]
+            assert np.array_equal(orc.unpack(got, B, w), q)
+
+
+def test_hand_worked_dot_products():
+    recs = golden_io.load()
+    blocks = {r["id"]: r for r in recs if r["kind"] == "block"}
+    dots = [r for r in recs if r["kind"] == "dot"]
+    assert dots
+    for d in dots:
+        ra, rb = blocks[d["a"]], blocks[d["b"]]
+        wa, wb = int(ra["w"]), int(rb["w"])
+        qa, ea, _ = orc.quantize(_block_row(golden_io.floats(ra["x"]), 16), 16, wa)
+        qb, eb, _ = orc.quantize(_block_row(golden_io.floats(rb["x"]), 16), 16, wb)
+        y_ref, y_seq, S = orc.gemm(qa, ea, wa, qb, eb, wb, 16)
+        assert float(y_ref[0, 0]) == float(d["y"])
+        assert float(y_seq[0, 0]) == float(d["y"])
+        # the integer block sum and the shared shift, separately
+        P = int(np.dot(qa[0].astype(np.int64), qb[0].astype(np.int64)))
+        assert P == int(d["P"])
+        shift = (int(ea[0, 0]) - 127) - (wa - 2) + (int(eb[0, 0]) - 127) - (wb - 2)
+        assert shift == int(d["shift"])
+        assert S[0, 0] >= abs(float(d["y"]))
+
+
+# --------------------------------------------------------------------------- exponent invariants
+
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("w", WIDTHS)
+def test_exponent_is_the_block_maximums(B, w):
+    rng = np.random.default_rng(10 * B + w)
+    x = (rng.standard_normal((37, 4 * B)) * np.exp(rng.uniform(-20, 20, (37, 1)))).astype(np.float32)
+    x[3, :B] = 0.0
+    q, e, bad = orc.quantize(x, B, w)
+    assert bad == 0
+    amax = np.abs(x.reshape(37, 4, B)).max(axis=2)
+    mant, ex = np.frexp(amax)               # independent library route to floor(log2)
+    want = np.where(amax > 0, ex - 1 + 127, 0)
+    assert np.array_equal(e.astype(np.int64), want)
+    bits = amax.astype(np.float32).view(np.uint32) >> 23      # the binary32 exponent field
+    assert np.array_equal(e.astype(np.uint32), bits)
+    # the max element uses the top magnitude bit: 2^(w-2) <= |q|max <= 2^(w-1)-1
+    qmax = np.abs(q.reshape(37, 4, B).astype(np.int32)).max(axis=2)
+    nz = amax > 0
+    assert (qmax[nz] >= 2 ** (w - 2)).all() and (qmax <= 2 ** (w - 1) - 1).all()
+    assert (qmax[~nz] == 0).all()
+
+
+@pytest.mark.parametrize("w", WIDTHS)
+def test_scale_covariance(w):
+    rng = np.random.default_rng(w)
+    x = rng.standard_normal((8, 64)).astype(np.float32)
+    q0, e0, _ = orc.quantize(x, 16, w)
+    for k in (-30, -3, 1, 17):
+        q1, e1, _ = orc.quantize(np.ldexp(x, k).astype(np.float32), 16, w)
+        assert np.array_equal(q0, q1)
+        assert np.array_equal(e0.astype(np.int32) + k, e1.astype(np.int32))
+
+
+# --------------------------------------------------------------------------- round-trip invariants
+
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("w", WIDTHS)
+def test_round_trip_invariants(B, w):
+    rng = np.random.default_rng(100 * B + w)
+    x = rng.standard_t(3, (64, 8 * B)).astype(np.float32)
+    q, e, _ = orc.quantize(x, B, w)
+    xhat = orc.dequantize(q, e, B, w)
+    # idempotence, bit-exact
+    q2, e2, _ = orc.quantize(xhat.astype(np.float32), B, w)
+    assert np.array_equal(q, q2) and np.array_equal(e, e2)
+    # error bound: half a step unless the element saturated (only the block maximum can)
+    E = e.astype(np.int64) - 127
+    s = np.repeat(np.ldexp(1.0, E - (w - 2)), B, axis=1)
+    err = np.abs(x.astype(np.float64) - xhat)
+    sat = np.abs(q.astype(np.int32)) == 2 ** (w - 1) - 1
+    assert (err[~sat] <= s[~sat] / 2).all()
+    assert (err[sat] < s[sat]).all()
+    # "the shared exponent bounds the range of values in the block"
+    assert (np.abs(xhat) < np.repeat(np.ldexp(1.0, E + 1), B, axis=1)).all()
+    # round-half-even is monotone and sign-symmetric
+    qn, en, _ = orc.quantize(-x, B, w)
+    assert np.array_equal(qn, -q) and np.array_equal(en, e)
+
+
+@pytest.mark.parametrize("B", BLOCKS)
+@pytest.mark.parametrize("w", WIDTHS)
+def test_representable_values_survive(B, w):
+    rng = np.random.default_rng(1000 * B + w)
+    qmax = 2 ** (w - 1) - 1
+    qi = rng.integers(-qmax, qmax + 1, (50, 4 * B))
+    E = rng.integers(-100, 100, (50, 4))
+    x = np.ldexp(qi.astype(np.float64), np.repeat(E, B, axis=1) - (w - 2)).astype(np.float32)
+    q, e, _ = orc.quantize(x, B, w)
+    xhat = orc.dequantize(q, e, B, w)
+    assert np.array_equal(xhat, x.astype(np.float64))   # even when the block is un-normalised
+
+
+def test_ties_go_to_even_and_saturate():
+    # s = 1 for w=4 when the maximum lies in [4, 8): E=2.
+    x = _block_row([4.0, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, 7.5, 7.49, -7.6, 6.5], 16)
+    q, e, _ = orc.quantize(x, 16, 4)
+    assert int(e[0, 0]) == 129
+    assert q[0, :12].tolist() == [4, 0, 2, 2, 0, -2, -2, 4, 7, 7, -7, 6]
+
+
+def test_zero_subnormal_and_nonfinite_blocks():
+    x = np.zeros((1, 64), np.float32)
+    x[0, 16] = np.float32(2.0 ** -126) - np.float32(2.0 ** -149)   # largest subnormal -> byte 0
+    x[0, 17] = -(2.0 ** -127)
+    x[0, 18] = 2.0 ** -130
+    x[0, 19] = 3 * 2.0 ** -130
+    x[0, 32] = np.inf
+    x[0, 33] = 5.0
+    x[0, 48] = np.nan
+    q, e, bad = orc.quantize(x, 16, 4)
+    assert e[0].tolist() == [0, 0, 255, 255]
+    assert bad == 2
+    assert not q[0, :16].any() and not q[0, 32:].any()
+    # grid of the lowest exponent: s = 2^(-127-2); 7.99.. saturates at 7; 0.5 -> 0, 1.5 -> 2
+    assert q[0, 16:20].tolist() == [7, -4, 0, 2]
+    xhat = orc.dequantize(q, e, 16, 4)
+    assert np.isnan(xhat[0, 32:]).all()
+    y, yseq, S = orc.gemm(q, e, 4, q, e, 4, 16)
+    assert np.isnan(y).all() and np.isnan(yseq).all()
+
+
+def test_largest_exponent_byte():
+    x = _block_row([3.0e38, -1.0e38, 2.0 ** 127], 16)
+    q, e, bad = orc.quantize(x, 16, 8)
+    assert bad == 0 and int(e[0, 0]) == 254
+    xhat = orc.dequantize(q, e, 16, 8)
+    assert abs(xhat[0, 0] - 3.0e38) <= 2.0 ** 121 / 2 and xhat[0, 2] == 2.0 ** 127
+
+
+def test_strided_axis_equals_transposed_copy():
+    rng = np.random.default_rng(5)
+    v = rng.standard_normal((96, 40)).astype(np.float32)        # [tokens, d]
+    q1, e1, _ = orc.quantize(v.T, 32, 8)                         # blocks along tokens, strided
+    q2, e2, _ = orc.quantize(np.ascontiguousarray(v.T), 32, 8)
+    assert np.array_equal(q1, q2) and np.array_equal(e1, e2)
+
+
+def test_pack_round_trip_all_widths():
+    rng = np.random.default_rng(6)
+    for w in WIDTHS:
+        qmax = 2 ** (w - 1) - 1
+        q = rng.integers(-qmax - 1, qmax + 1, (5, 64)).astype(np.int8)   # incl. -2^(w-1)
+        if w < 4:
+            q = np.clip(q, -qmax, qmax).astype(np.int8)
+        p = orc.pack(q, w)
+        assert p.shape == (5, 32 if w <= 4 else 64)
+        assert np.array_equal(orc.unpack(p, 64, w), q)
+
+
+# --------------------------------------------------------------------------- GEMM: exact brute force
+
+def _nearest_f32(fr: Fraction) -> float:
+    """Correctly rounded binary32 of an exact rational (ties to even), via integer arithmetic."""
+    if fr == 0:
+        return 0.0
+    sign = -1 if fr < 0 else 1
+    a = abs(fr)
+    e = a.numerator.bit_length() - a.denominator.bit_length()
+    if Fraction(2) ** e > a:
+        e -= 1
+    e = max(e, -126)
+    ulp = Fraction(2) ** (e - 23)
+    n = a / ulp
+    fl = n.numerator // n.denominator
+    rem = n - fl
+    if rem > Fraction(1, 2) or (rem == Fraction(1, 2) and fl % 2 == 1):
+        fl += 1
+    return sign * float(fl * ulp)
+
+
+@pytest.mark.parametrize("B", BLOCKS)
+def test_gemm_equals_exact_rational_dot_products(B):
+    rng = np.random.default_rng(B)
+    for wa in WIDTHS:
+        for ww in (2, 4, 8):
+            M, N, K = 3, 4, 2 * B
+            x = (rng.standard_normal((M, K)) * np.exp(rng.uniform(-6, 6, (M, K)))).astype(np.float32)
+            wt = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+            bias = rng.standard_normal(N).astype(np.float32)
+            qa, ea, _ = orc.quantize(x, B, wa)
+            qw, ew, _ = orc.quantize(wt, B, ww)
+            y, yseq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
+            # emulator form (Sec. 3.2): plain dot product of the dequantized values, exactly
+            xa = orc.dequantize(qa, ea, B, wa)
+            xw = orc.dequantize(qw, ew, B, ww)
+            for i in range(M):
+                for j in range(N):
+                    exact = sum(Fraction(float(xa[i, k])) * Fraction(float(xw[j, k])) for k in range(K))
+                    exact += Fraction(float(bias[j]))
+                    assert float(y[i, j]) == _nearest_f32(exact), (wa, ww, i, j)
+                    sabs = sum(abs(Fraction(float(xa[i, k])) * Fraction(float(xw[j, k]))) for k in range(K))
+                    assert abs(Fraction(float(yseq[i, j])) - exact) <= Fraction(1, 10 ** 5) * (sabs + abs(Fraction(float(bias[j])))) + Fraction(1, 2 ** 140)
+                    assert S[i, j] <= float(sabs + abs(Fraction(float(bias[j])))) * (1 + 1e-12)
+
+
+def test_gemm_hardware_form_equals_emulator_form():
+    """Integer block sums times one shared power of two == fp matmul of dequantized values."""
+    rng = np.random.default_rng(77)
+    M, N, K, B = 5, 6, 128, 32
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    wt = rng.standard_normal((N, K)).astype(np.float32)
+    qa, ea, _ = orc.quantize(x, B, 8)
+    qw, ew, _ = orc.quantize(wt, B, 4)
+    y, _, _ = orc.gemm(qa, ea, 8, qw, ew, 4, B)
+    xa, xw = orc.dequantize(qa, ea, B, 8), orc.dequantize(qw, ew, B, 4)
+    # N(0,1) data: all terms within 2^-12..2^4, 128 of them -> fp64 matmul is exact here
+    assert np.array_equal(y, (xa @ xw.T).astype(np.float32))
+
+
+def test_gemm_equal_exponents_is_integer_matmul():
+    rng = np.random.default_rng(8)
+    M, N, K, B = 7, 9, 96, 16
+    qa = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    qw = rng.integers(-7, 8, (N, K)).astype(np.int8)
+    ea = np.full((M, K // B), 130, np.uint8)
+    ew = np.full((N, K // B), 120, np.uint8)
+    y, yseq, S = orc.gemm(qa, ea, 8, qw, ew, 4, B)
+    P = qa.astype(np.int64) @ qw.astype(np.int64).T
+    want = np.ldexp(P.astype(np.float64), (130 - 127 - 6) + (120 - 127 - 2))
+    assert np.array_equal(y.astype(np.float64), want) and np.array_equal(yseq, y)
+
+
+def test_gemm_representable_inputs_equal_fp64_matmul():
+    rng = np.random.default_rng(9)
+    M, N, K, B, wa, ww = 6, 5, 64, 16, 6, 4
+    A = np.ldexp(rng.integers(-31, 32, (M, K)).astype(np.float64),
+                 np.repeat(rng.integers(-3, 4, (M, K // B)), B, axis=1)).astype(np.float32)
+    W = np.ldexp(rng.integers(-7, 8, (N, K)).astype(np.float64),
+                 np.repeat(rng.integers(-3, 4, (N, K // B)), B, axis=1)).astype(np.float32)
+    qa, ea, _ = orc.quantize(A, B, wa)
+    qw, ew, _ = orc.quantize(W, B, ww)
+    y, _, _ = orc.gemm(qa, ea, wa, qw, ew, ww, B)
+    assert np.array_equal(y, (A.astype(np.float64) @ W.astype(np.float64).T).astype(np.float32))
+
+
+def test_gemm_one_hot_rows_return_dequantized_weights():
+    rng = np.random.default_rng(10)
+    N, K, B, ww = 8, 64, 16, 4
+    W = rng.standard_normal((N, K)).astype(np.float32)
+    qw, ew, _ = orc.quantize(W, B, ww)
+    A = np.eye(K, dtype=np.float32)
+    qa, ea, _ = orc.quantize(A, B, 8)
+    y, yseq, _ = orc.gemm(qa, ea, 8, qw, ew, ww, B)
+    assert np.array_equal(y.astype(np.float64), orc.dequantize(qw, ew, B, ww).T)
+    assert np.array_equal(y, yseq)
+
+
+def test_gemm_samples_agree_with_full():
+    rng = np.random.default_rng(11)
+    M, N, K, B = 9, 11, 64, 32
+    qa = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    qw = rng.integers(-7, 8, (N, K)).astype(np.int8)
+    ea = rng.integers(100, 140, (M, K // B)).astype(np.uint8)
+    ew = rng.integers(100, 140, (N, K // B)).astype(np.uint8)
+    bias = rng.standard_normal(N).astype(np.float32)
+    y, yseq, S = orc.gemm(qa, ea, 8, qw, ew, 4, B, bias=bias)
+    si = rng.integers(0, M, 20)
+    sj = rng.integers(0, N, 20)
+    ys, yseqs, Ss = orc.gemm_samples(qa, ea, 8, qw, ew, 4, B, si, sj, bias=bias)
+    assert np.array_equal(ys, y[si, sj]) and np.array_equal(yseqs, yseq[si, sj])
+    assert np.array_equal(Ss, S[si, sj])
+
+
+def test_sequential_fp32_sum_sits_inside_the_tolerance():
+    rng = np.random.default_rng(12)
+    M, N, K, B = 8, 8, 11008, 16
+    x = rng.standard_t(3, (M, K)).astype(np.float32)
+    wt = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    qa, ea, _ = orc.quantize(x, B, 8)
+    qw, ew, _ = orc.quantize(wt, B, 4)
+    y, yseq, S = orc.gemm(qa, ea, 8, qw, ew, 4, B)
+    assert (np.abs(yseq.astype(np.float64) - y) <= 1e-5 * S).all()
+    assert (S >= np.abs(y) * (1 - 1e-6)).all()
+
+
+def test_rejects_bad_arguments():
+    x = np.zeros((2, 40), np.float32)
+    with pytest.raises(ValueError):
+        orc.quantize(x, 16, 4)          # K not a multiple of the block
+    with pytest.raises(ValueError):
+        orc.quantize(np.zeros((2, 32), np.float32), 16, 9)

@@ -1,0 +1,172 @@
+/*
+ * mxint.h -- C ABI of the MXInt linear-layer library for NVIDIA B200 (sm_100a).
+ *
+ * MXInt (arXiv 2307.15517, Sec. 2 "What are MX Formats?" and Sec. 4.1) is block floating
+ * point: the values of a block share one 8-bit exponent and each keeps a short signed integer
+ * mantissa.  A format is the tuple (B, e, m) of Sec. 4.1; this library fixes e = 8 and takes
+ *   block      = number of consecutive elements along the reduction axis K sharing an exponent
+ *   elem_bits  = w, the signed mantissa width INCLUDING its sign bit (the paper's m = w - 1)
+ * so that the paper's "MXInt4" is elem_bits = 4 and its average size (Eq. 1) is
+ * exp_bits/(block*block_rows) + elem_bits.
+ *
+ * Encoding of one block (E = exponent byte - 127):
+ *   exponent byte = binary32 exponent field of the block's largest magnitude
+ *                   (0 for an all-zero or subnormal block, 255 if the block holds Inf/NaN)
+ *   mantissa q    = clamp(round_to_nearest_even(x * 2^-(E-(w-2))), -(2^(w-1)-1), 2^(w-1)-1)
+ *   value         = q * 2^(E-(w-2));   a block with exponent byte 255 decodes to NaN
+ * Containers: elem_bits <= 4 -> two two's-complement nibbles per byte, even k in the low
+ * nibble, a row of K elements takes K/2 bytes; elem_bits 5..8 -> one int8 per element.
+ * Exponent bytes: uint8 [rows, K/block], row-major.
+ *
+ * Conventions for every entry point:
+ *   - All data pointers are DEVICE pointers owned by the caller.  The library neither
+ *     allocates, frees nor keeps them.  Base pointers must be 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
+ *     asynchronous on it and never synchronise the host, except mx_poll_status.
+ *   - Arguments are validated on the host before anything is launched; a negative
+ *     mx_status_t means nothing ran.  K must be a multiple of the block size.
+ *   - There is no CPU fallback: on a machine without an sm_100 GPU the compute entry points
+ *     return MX_ERR_ARCH / MX_ERR_CUDA.
+ */
+#ifndef MXINT_H_
+#define MXINT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define MX_API __attribute__((visibility("default")))
+#else
+#define MX_API
+#endif
+
+typedef enum {
+    MX_OK = 0,
+    MX_ERR_NULL = -1,      /* a required pointer is NULL                                      */
+    MX_ERR_SHAPE = -2,     /* K % block != 0, a negative size, a leading dimension too small  */
+    MX_ERR_FORMAT = -3,    /* unsupported block / elem_bits / exp_bits / block_rows           */
+    MX_ERR_ALIGN = -4,     /* a pointer or stride breaks the alignment rule                   */
+    MX_ERR_WORKSPACE = -5, /* workspace NULL or smaller than mx_workspace_bytes()             */
+    MX_ERR_CUDA = -6,      /* a CUDA runtime/driver call failed; see mx_last_cuda_error()     */
+    MX_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (reported by mx_poll_status) */
+    MX_ERR_ARCH = -8       /* the current device is not sm_100                                */
+} mx_status_t;
+
+typedef enum { MX_F32 = 0, MX_BF16 = 1 } mx_dtype_t;
+
+/* Which kernel computes the block-scaled product. */
+typedef enum {
+    MX_ALGO_AUTO = 0,    /* skinny problems (M <= 16) -> weight-streaming kernel, else tensor cores */
+    MX_ALGO_SIMT = 1,    /* CUDA-core kernel: exact integer block sums, blocks added in ascending
+                            order in fp32 (bit-reproducible; slow; needs no workspace)              */
+    MX_ALGO_TCGEN05 = 2, /* tcgen05/TMEM tensor-core kernel on exactly dequantized bf16 operands    */
+    MX_ALGO_STREAM = 3   /* weight-streaming kernel for M <= 16 (decode); needs no workspace        */
+} mx_algo_t;
+
+/* The (B, e, m) tuple of Sec. 4.1. */
+typedef struct {
+    int32_t block;      /* 16 or 32 elements along K share one exponent                        */
+    int32_t elem_bits;  /* w = 2..8, sign included (paper m = w - 1)                           */
+    int32_t exp_bits;   /* 8 (the paper fixes the shared exponent to 8 bits)                   */
+    int32_t block_rows; /* 1 (the paper's 2-D block shape (16,2) would be 2; not supported)    */
+} mx_format_t;
+
+/* ---- size helpers (host only, no CUDA call) ------------------------------------------- */
+
+/* Bytes of the mantissa container / of the exponent array of a [rows, K] tensor; 0 on a bad
+ * format or shape. */
+MX_API size_t mx_mant_bytes(int64_t rows, int64_t K, mx_format_t f);
+MX_API size_t mx_exp_bytes(int64_t rows, int64_t K, mx_format_t f);
+
+/* Average bits per value, Eq. 1 of the paper: exp_bits/(block*block_rows) + (w-1) + 1.
+ * MXInt((16,2),8,7) -> 8.25.  Returns 0 on a bad format. */
+MX_API double mx_format_bits(mx_format_t f);
+
+/* Scratch bytes mx_gemm / mx_linear need for these sizes with MX_ALGO_AUTO (the maximum over
+ * the kernels AUTO may pick).  The workspace must be 256-byte aligned. */
+MX_API size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw);
+
+MX_API const char *mx_status_string(mx_status_t s);
+
+/* Text of the last CUDA error this library saw on the calling thread ("" if none). */
+MX_API const char *mx_last_cuda_error(void);
+
+/* ---- quantizer (Sec. 3.2, software emulator: floating point -> MXInt) ------------------ */
+
+/*
+ * Quantize x, a [rows, K] tensor of `dt` whose element (r, k) sits at
+ * x[r*stride_row + k*stride_k] (strides in elements), block by block along k.
+ *   stride_k == 1 : rows are contiguous along K (fast path; stride_row % 8 == 0 required).
+ *   stride_k != 1 : blocks run along a strided axis (e.g. V of attention quantized along the
+ *                   token axis for the P*V product).
+ * mant_out receives mx_mant_bytes(rows,K,f) bytes, exp_out mx_exp_bytes(rows,K,f) bytes, both
+ * row-major and dense.  nonfinite_count (nullable, device uint32) is incremented once per
+ * block that holds an Inf or NaN; such a block gets exponent byte 255 and zero mantissas.
+ */
+MX_API mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K,
+                        int64_t stride_row, int64_t stride_k, mx_format_t f, void *mant_out,
+                        uint8_t *exp_out, uint32_t *nonfinite_count, void *stream);
+
+/* Inverse map (test helper): out[r*ld_out + k] = q * 2^(E-(w-2)) as `dt` (exact in both
+ * fp32 and bf16); NaN for blocks with exponent byte 255. */
+MX_API mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
+                          mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream);
+
+/* ---- block-scaled product (Sec. 3.2, MXInt dot-product operator, Fig. 3 right) --------- */
+
+/*
+ * Y[M,N] = A[M,K] * W[N,K]^T (+ bias[N]) where both operands are MXInt tensors blocked along K:
+ *   Y[i,j] = sum_b 2^(Ea[i,b]+Ew[j,b]-(wa-2)-(ww-2)) * sum_{k in block b} qa[i,k]*qw[j,k]
+ * accumulated in fp32.  fa.block must equal fw.block; elem_bits may differ (e.g. A8/W4).
+ * y is fp32 with leading dimension ldy >= N (elements).  Any block with exponent byte 255
+ * makes the outputs it touches NaN.  workspace: see mx_workspace_bytes (may be NULL for
+ * MX_ALGO_SIMT / MX_ALGO_STREAM).
+ */
+MX_API mx_status_t mx_gemm(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                    const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t M,
+                    int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/* The same with the kernel named explicitly. */
+MX_API mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                       const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t M,
+                       int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                       void *workspace, size_t workspace_bytes, mx_algo_t algo, void *stream);
+
+/* ---- the MXInt linear layer (Fig. 2: LinearOp with MXInt activations and weights) ------ */
+
+/*
+ * Y[M,N] = Q_fa(X)[M,K] * W[N,K]^T (+ bias): quantizes the activations x ([M,K] of `dt`,
+ * leading dimension ldx elements, ldx % 8 == 0) to format fa on the fly and multiplies them
+ * with weights already stored in format fw.  Equivalent to mx_quantize followed by mx_gemm,
+ * but the quantized activations go straight to the product kernel's operand layout.
+ */
+MX_API mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
+                      mx_format_t fa, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                      int64_t N, const float *bias, float *y, int64_t ldy, void *workspace,
+                      size_t workspace_bytes, void *stream);
+
+MX_API mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
+                         mx_format_t fa, const void *w_mant, const uint8_t *w_exp,
+                         mx_format_t fw, int64_t N, const float *bias, float *y, int64_t ldy,
+                         void *workspace, size_t workspace_bytes, mx_algo_t algo, void *stream);
+
+/* ---- device status --------------------------------------------------------------------- */
+
+/*
+ * Every device-side wait in this library (mbarrier polls of the tensor-core pipeline) gives up
+ * after a bounded time, records the fact in a per-device status word and lets the kernel
+ * return.  mx_poll_status synchronises `stream`, reads and clears that word and returns
+ * MX_ERR_TIMEOUT if any wait expired since the last poll, MX_ERR_CUDA if the stream reported
+ * an error, else MX_OK.  Outputs of a call that timed out are undefined.
+ */
+MX_API mx_status_t mx_poll_status(void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MXINT_H_ */

@@ -1,0 +1,201 @@
+"""Thin ctypes binding of ``libmxint.so`` -- argument marshalling only.
+
+Every function has the name of the C entry point it calls (see ``include/mxint.h``) and takes
+torch CUDA tensors for device memory; torch is used for allocation and streams, never for
+arithmetic.  There is no fallback: if the shared library is missing the import fails, and a
+negative status from the library raises ``MxError``.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmxint.so")
+
+MX_F32, MX_BF16 = 0, 1
+MX_ALGO_AUTO, MX_ALGO_SIMT, MX_ALGO_TCGEN05, MX_ALGO_STREAM = 0, 1, 2, 3
+
+STATUS_NAMES = {0: "MX_OK", -1: "MX_ERR_NULL", -2: "MX_ERR_SHAPE", -3: "MX_ERR_FORMAT",
+                -4: "MX_ERR_ALIGN", -5: "MX_ERR_WORKSPACE", -6: "MX_ERR_CUDA",
+                -7: "MX_ERR_TIMEOUT", -8: "MX_ERR_ARCH"}
+
+
+class MxFormat(C.Structure):
+    """The (B, e, m) tuple of the paper's Sec. 4.1 with w = m + 1 (sign included)."""
+    _fields_ = [("block", C.c_int32), ("elem_bits", C.c_int32), ("exp_bits", C.c_int32),
+                ("block_rows", C.c_int32)]
+
+    def __init__(self, block: int = 16, elem_bits: int = 4, exp_bits: int = 8, block_rows: int = 1):
+        super().__init__(block, elem_bits, exp_bits, block_rows)
+
+    def __repr__(self):
+        return "MxFormat(block=%d, elem_bits=%d)" % (self.block, self.elem_bits)
+
+
+class MxError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__("%s failed: %s%s" % (where, STATUS_NAMES.get(status, str(status)),
+                                              (" (" + detail + ")") if detail else ""))
+
+
+def _load() -> C.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            "libmxint.so is not built (%s). Run `python -m paper_2307_15517_b200.build`; there is "
+            "no CPU or PyTorch fallback for these kernels." % LIB_PATH)
+    L = C.CDLL(LIB_PATH)
+    vp, i64, sz, i32 = C.c_void_p, C.c_int64, C.c_size_t, C.c_int
+    F = MxFormat
+    L.mx_mant_bytes.argtypes = [i64, i64, F]
+    L.mx_mant_bytes.restype = sz
+    L.mx_exp_bytes.argtypes = [i64, i64, F]
+    L.mx_exp_bytes.restype = sz
+    L.mx_format_bits.argtypes = [F]
+    L.mx_format_bits.restype = C.c_double
+    L.mx_workspace_bytes.argtypes = [i64, i64, i64, F, F]
+    L.mx_workspace_bytes.restype = sz
+    L.mx_status_string.argtypes = [i32]
+    L.mx_status_string.restype = C.c_char_p
+    L.mx_last_cuda_error.argtypes = []
+    L.mx_last_cuda_error.restype = C.c_char_p
+    L.mx_quantize.argtypes = [vp, i32, i64, i64, i64, i64, F, vp, vp, vp, vp]
+    L.mx_dequantize.argtypes = [vp, vp, i64, i64, F, vp, i32, i64, vp]
+    L.mx_gemm.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, vp]
+    L.mx_gemm_ex.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, i32, vp]
+    L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
+    L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
+    L.mx_poll_status.argtypes = [vp]
+    for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
+                 "mx_linear_ex", "mx_poll_status"):
+        getattr(L, name).restype = i32
+    return L
+
+
+lib = _load()
+
+
+def _check(status: int, where: str):
+    if status != 0:
+        raise MxError(status, where, lib.mx_last_cuda_error().decode() if status == -6 else "")
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return MX_F32
+    if t.dtype == torch.bfloat16:
+        return MX_BF16
+    raise TypeError("expected float32 or bfloat16, got %s" % t.dtype)
+
+
+def _need_cuda(*tensors):
+    for t in tensors:
+        if t is not None and not t.is_cuda:
+            raise ValueError("device tensors required (this library has no host path)")
+
+
+# ---- size helpers ---------------------------------------------------------------------------
+
+def mx_mant_bytes(rows: int, K: int, f: MxFormat) -> int:
+    return int(lib.mx_mant_bytes(rows, K, f))
+
+
+def mx_exp_bytes(rows: int, K: int, f: MxFormat) -> int:
+    return int(lib.mx_exp_bytes(rows, K, f))
+
+
+def mx_format_bits(f: MxFormat) -> float:
+    return float(lib.mx_format_bits(f))
+
+
+def mx_workspace_bytes(M: int, N: int, K: int, fa: MxFormat, fw: MxFormat) -> int:
+    return int(lib.mx_workspace_bytes(M, N, K, fa, fw))
+
+
+def mx_status_string(status: int) -> str:
+    return lib.mx_status_string(status).decode()
+
+
+def alloc_workspace(nbytes: int, device="cuda") -> torch.Tensor:
+    """A 256-byte aligned scratch buffer (torch's caching allocator aligns to 512 bytes)."""
+    return torch.empty(max(int(nbytes), 256), dtype=torch.uint8, device=device)
+
+
+# ---- compute entry points --------------------------------------------------------------------
+
+def mx_quantize(x: torch.Tensor, f: MxFormat, mant_out: Optional[torch.Tensor] = None,
+                exp_out: Optional[torch.Tensor] = None,
+                nonfinite_count: Optional[torch.Tensor] = None,
+                stream=None) -> Tuple[torch.Tensor, torch.Tensor]:
+    """x: [rows, K] fp32/bf16 CUDA tensor (any strides).  Returns (mant uint8, exps uint8)."""
+    _need_cuda(x, mant_out, exp_out, nonfinite_count)
+    assert x.dim() == 2
+    rows, K = x.shape
+    if mant_out is None:
+        mant_out = torch.empty((rows, mx_mant_bytes(1, K, f)), dtype=torch.uint8, device=x.device)
+    if exp_out is None:
+        exp_out = torch.empty((rows, mx_exp_bytes(1, K, f)), dtype=torch.uint8, device=x.device)
+    _check(lib.mx_quantize(_ptr(x), _dtype_code(x), rows, K, x.stride(0), x.stride(1), f,
+                           _ptr(mant_out), _ptr(exp_out), _ptr(nonfinite_count), _stream(stream)),
+           "mx_quantize")
+    return mant_out, exp_out
+
+
+def mx_dequantize(mant: torch.Tensor, exps: torch.Tensor, K: int, f: MxFormat,
+                  dtype=torch.float32, stream=None) -> torch.Tensor:
+    _need_cuda(mant, exps)
+    rows = mant.shape[0]
+    out = torch.empty((rows, K), dtype=dtype, device=mant.device)
+    _check(lib.mx_dequantize(_ptr(mant), _ptr(exps), rows, K, f, _ptr(out), _dtype_code(out), K,
+                             _stream(stream)), "mx_dequantize")
+    return out
+
+
+def mx_gemm(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: int, N: int, K: int,
+            bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+            workspace: Optional[torch.Tensor] = None, algo: int = MX_ALGO_AUTO, stream=None):
+    _need_cuda(a_mant, a_exp, w_mant, w_exp, bias, y, workspace)
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=a_mant.device)
+    if workspace is None and algo in (MX_ALGO_AUTO, MX_ALGO_TCGEN05):
+        workspace = alloc_workspace(mx_workspace_bytes(M, N, K, fa, fw), a_mant.device)
+    _check(lib.mx_gemm_ex(_ptr(a_mant), _ptr(a_exp), fa, _ptr(w_mant), _ptr(w_exp), fw, M, N, K,
+                          _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
+                          0 if workspace is None else workspace.numel(), algo, _stream(stream)),
+           "mx_gemm")
+    return y
+
+
+def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int,
+              bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+              workspace: Optional[torch.Tensor] = None, algo: int = MX_ALGO_AUTO, stream=None):
+    _need_cuda(x, w_mant, w_exp, bias, y, workspace)
+    M, K = x.shape
+    assert x.stride(1) == 1
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+    if workspace is None:
+        workspace = alloc_workspace(mx_workspace_bytes(M, N, K, fa, fw), x.device)
+    _check(lib.mx_linear_ex(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant),
+                            _ptr(w_exp), fw, N, _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
+                            workspace.numel(), algo, _stream(stream)), "mx_linear")
+    return y
+
+
+def mx_poll_status(stream=None) -> int:
+    """Synchronises the stream and returns the library's device status (0 = MX_OK)."""
+    return int(lib.mx_poll_status(_stream(stream)))

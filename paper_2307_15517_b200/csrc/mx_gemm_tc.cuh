@@ -1,0 +1,229 @@
+// Tensor-core MXInt product for prefill shapes (Sec. 3.2 MXInt dot-product operator, computed
+// on tcgen05/TMEM).
+//
+// Why bf16 MMA and not int8 MMA: a decoded MXInt element q*2^(E-(w-2)) with |q| <= 127 has at
+// most 7 significant bits and an 8-bit exponent, so it IS a bf16 number -- the conversion is
+// exact, the product of two such numbers (<= 14 significant bits) is exact in fp32, and the
+// shared exponents ride along inside the operands.  Only the fp32 accumulation rounds, which
+// the paper's operator does as well.  An int8 MMA would need the accumulator pulled out of
+// tensor memory and rescaled by 2^(Ea+Ew) once per block of 16/32 along K, i.e. a full
+// TMEM -> register -> FMA pass per 128x256x32 step, several times longer than the MMA itself.
+//
+// Kernel: persistent, one CTA per SM, 128 x BN output tile, K step 64 (one 128-byte swizzled
+// row of bf16), STAGES-deep TMA pipeline, two accumulators in tensor memory (2*BN <= 512
+// columns) so that the epilogue of tile t overlaps the MMAs of tile t+1.
+//   warp 0      : TMA producer (one lane)
+//   warp 1      : tensor-memory allocation, MMA issue (one lane)
+//   warps 2..5  : epilogue, TMEM -> registers -> (+bias) -> global fp32
+// Every mbarrier wait is bounded in time; on expiry the kernel raises a CTA-wide abort flag,
+// records MX_ERR_TIMEOUT in the status word, frees its tensor memory and returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mx_ptx.cuh"
+
+namespace mx {
+
+constexpr int TC_BM = 128;
+constexpr int TC_BK = 64;                                  // bf16 elements per 128-byte row
+constexpr int TC_THREADS = 192;
+constexpr uint64_t TC_WAIT_LIMIT_NS = 400ull * 1000 * 1000; // 0.4 s per wait
+
+constexpr uint32_t STATUS_TIMEOUT_BIT = 1u;
+
+template <int BN> struct TcCfg {
+    static constexpr int STAGES = (BN == 256) ? 4 : 6;
+    static constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2;
+    static constexpr uint32_t W_BYTES = BN * TC_BK * 2;
+    static constexpr uint32_t STAGE_BYTES = A_BYTES + W_BYTES;
+    static constexpr uint32_t BAR_BYTES = 256;
+    static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024; // + align slack
+    static constexpr uint32_t TMEM_COLS = 2 * BN;          // 256 or 512: powers of two
+};
+
+struct TcParams {
+    float *y;
+    const float *bias;
+    int64_t ldy;
+    int M, N, K;
+    int tiles_m, tiles_n;
+    uint32_t *status;
+};
+
+template <int BN>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
+               const TcParams p)
+{
+    using Cfg = TcCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
+
+    const uint32_t bar_base = smem_base + STAGES * Cfg::STAGE_BYTES;
+    auto full_bar = [&](int s) { return bar_base + 8u * s; };
+    auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
+    auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
+    auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 4));
+    volatile uint32_t *abort_flag = tmem_slot + 1;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            ptx::mbar_init(full_bar(s), 1);
+            ptx::mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            ptx::mbar_init(tfull_bar(a), 1);
+            ptx::mbar_init(tempty_bar(a), 4);          // one arrival per epilogue warp
+        }
+        *abort_flag = 0;
+        ptx::fence_mbar_init();
+        ptx::prefetch_tensormap(&tmap_a);
+        ptx::prefetch_tensormap(&tmap_w);
+    }
+    if (warp == 1) {
+        ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::TMEM_COLS);
+        ptx::tmem_relinquish();
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    ptx::tc_fence_after_sync();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int kblocks = (p.K + TC_BK - 1) / TC_BK;
+    bool timed_out = false;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            int s = 0;
+            uint32_t ph = 0;
+            for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x) {
+                const int m0 = (t % p.tiles_m) * TC_BM, n0 = (t / p.tiles_m) * BN;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS)) {
+                        timed_out = true;
+                        break;
+                    }
+                    ptx::mbar_arrive_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
+                    ptx::tma_load_2d(sa, &tmap_a, kb * TC_BK, m0, full_bar(s));
+                    ptx::tma_load_2d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, full_bar(s));
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(TC_BM, BN);
+            int s = 0;
+            uint32_t ph = 0;
+            int it = 0;
+            for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
+                const int acc = it & 1;
+                const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+                if (!ptx::mbar_wait_bounded(tempty_bar(acc), acc_ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS)) {
+                    timed_out = true;
+                    break;
+                }
+                ptx::tc_fence_after_sync();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(acc * BN);
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, TC_WAIT_LIMIT_NS)) {
+                        timed_out = true;
+                        break;
+                    }
+                    ptx::tc_fence_after_sync();
+                    const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
+                    const uint32_t sw = sa + Cfg::A_BYTES;
+#pragma unroll
+                    for (int j = 0; j < TC_BK / 16; ++j) {
+                        ptx::mma_bf16_ss(d_tmem, ptx::smem_desc_k_sw128(sa, j * 32),
+                                         ptx::smem_desc_k_sw128(sw, j * 32), idesc,
+                                         (kb | j) != 0 ? 1u : 0u);
+                    }
+                    ptx::mma_commit(empty_bar(s));          // stage free once these MMAs retire
+                    if (++s == STAGES) { s = 0; ph ^= 1u; }
+                }
+                if (timed_out) break;
+                ptx::mma_commit(tfull_bar(acc));            // accumulator complete
+            }
+        }
+        __syncwarp();
+    } else {
+        const int quad = warp & 3;                          // TMEM lanes this warp may read
+        int it = 0;
+        for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
+            const int acc = it & 1;
+            const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
+            const int m0 = (t % p.tiles_m) * TC_BM, n0 = (t / p.tiles_m) * BN;
+            // every lane waits (acquire), then the warp agrees on the outcome so that the
+            // warp-collective TMEM loads below are never executed by a partial warp
+            const bool ok = ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
+            if (!__all_sync(0xFFFFFFFFu, ok)) {
+                timed_out = true;
+                break;
+            }
+            ptx::tc_fence_after_sync();
+            const int row = m0 + quad * 32 + lane;
+            float *yrow = p.y + (int64_t)row * p.ldy;
+            const bool vec_ok = ((p.ldy & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
+                uint32_t r[32];
+                ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                ptx::tmem_ld_wait();
+                const int n = n0 + c0;
+                if (row < p.M && n < p.N) {
+                    if (vec_ok && n + 32 <= p.N) {
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 o;
+                            o.x = __uint_as_float(r[4 * v + 0]);
+                            o.y = __uint_as_float(r[4 * v + 1]);
+                            o.z = __uint_as_float(r[4 * v + 2]);
+                            o.w = __uint_as_float(r[4 * v + 3]);
+                            if (p.bias) {
+                                const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + n) + v);
+                                o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                            }
+                            reinterpret_cast<float4 *>(yrow + n)[v] = o;
+                        }
+                    } else {
+#pragma unroll
+                        for (int v = 0; v < 32; ++v)
+                            if (n + v < p.N)
+                                yrow[n + v] = p.bias ? __uint_as_float(r[v]) + __ldg(p.bias + n + v)
+                                                     : __uint_as_float(r[v]);
+                    }
+                }
+            }
+            ptx::tc_fence_before_sync();
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    if (timed_out) {
+        *abort_flag = 1;
+        atomicOr(p.status, STATUS_TIMEOUT_BIT);
+        // give copies that may still be in flight time to land before shared memory is released
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 100000ull) __nanosleep(1000);
+    }
+    ptx::tc_fence_before_sync();
+    __syncthreads();
+    if (warp == 1) {
+        ptx::tc_fence_after_sync();
+        ptx::tmem_dealloc(tmem_base, Cfg::TMEM_COLS);
+    }
+}
+
+}  // namespace mx

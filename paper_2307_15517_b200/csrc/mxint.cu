@@ -1,0 +1,429 @@
+// C ABI of the MXInt linear-layer library: argument validation and kernel launches.
+// Everything here is host code; the arithmetic lives in the kernels of the included headers.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+
+#include "../../include/mxint.h"
+#include "mx_gemm_simt.cuh"
+#include "mx_gemm_tc.cuh"
+#include "mx_quantize.cuh"
+
+namespace {
+
+constexpr int MAX_DEVICES = 64;
+constexpr int SM_COUNT_FALLBACK = 148;
+
+__device__ uint32_t g_status_word;      // per device: bit 0 = a bounded wait expired
+
+thread_local char t_cuda_error[256] = "";
+
+struct DeviceInfo {
+    bool probed = false;
+    bool is_sm100 = false;
+    int sm_count = SM_COUNT_FALLBACK;
+    uint32_t *status = nullptr;
+    bool tc_attr_set[2] = {false, false};
+};
+DeviceInfo g_dev[MAX_DEVICES];
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
+                                  const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
+                                  const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+
+mx_status_t cuda_fail(cudaError_t e, const char *what)
+{
+    snprintf(t_cuda_error, sizeof(t_cuda_error), "%s: %s", what, cudaGetErrorString(e));
+    return MX_ERR_CUDA;
+}
+
+#define MX_CUDA(call)                                            \
+    do {                                                         \
+        cudaError_t e_ = (call);                                 \
+        if (e_ != cudaSuccess) return cuda_fail(e_, #call);      \
+    } while (0)
+
+mx_status_t device_info(DeviceInfo **out)
+{
+    int dev = 0;
+    MX_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return MX_ERR_CUDA;
+    DeviceInfo &d = g_dev[dev];
+    if (!d.probed) {
+        int major = 0, sms = 0;
+        MX_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
+        MX_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        d.is_sm100 = (major == 10);
+        d.sm_count = sms > 0 ? sms : SM_COUNT_FALLBACK;
+        if (d.is_sm100) {
+            void *p = nullptr;
+            MX_CUDA(cudaGetSymbolAddress(&p, g_status_word));
+            d.status = static_cast<uint32_t *>(p);
+        }
+        d.probed = true;
+    }
+    *out = &d;
+    return d.is_sm100 ? MX_OK : MX_ERR_ARCH;
+}
+
+bool format_ok(const mx_format_t &f)
+{
+    return (f.block == 16 || f.block == 32) && f.elem_bits >= 2 && f.elem_bits <= 8 &&
+           f.exp_bits == 8 && f.block_rows == 1;
+}
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+size_t round256(size_t n) { return (n + 255u) & ~size_t(255); }
+
+int grid_for(int64_t work_items, int threads, int sm_count, int ctas_per_sm)
+{
+    int64_t g = (work_items + threads - 1) / threads;
+    const int64_t cap = (int64_t)sm_count * ctas_per_sm;
+    if (g > cap) g = cap;
+    if (g < 1) g = 1;
+    return (int)g;
+}
+
+// ---- quantize launchers ---------------------------------------------------------------------
+template <typename InT>
+mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t ldx,
+                                 const mx_format_t &f, mx::QuantOut out, const DeviceInfo &d,
+                                 cudaStream_t st)
+{
+    const int64_t chunks = rows * (K / 8);
+    if (chunks == 0) return MX_OK;
+    const int grid = grid_for(chunks, 256, d.sm_count, 16);
+    if (f.block == 16)
+        mx::quantize_rows_kernel<InT, 16><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+    else
+        mx::quantize_rows_kernel<InT, 32><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t quantize_rows_any(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, int64_t ldx,
+                              const mx_format_t &f, mx::QuantOut out, const DeviceInfo &d,
+                              cudaStream_t st)
+{
+    if (dt == MX_F32)
+        return launch_quantize_rows(static_cast<const float *>(x), rows, K, ldx, f, out, d, st);
+    return launch_quantize_rows(static_cast<const __nv_bfloat16 *>(x), rows, K, ldx, f, out, d, st);
+}
+
+mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
+                                const mx_format_t &f, __nv_bfloat16 *out, int64_t ld,
+                                const DeviceInfo &d, cudaStream_t st)
+{
+    const int64_t chunks = rows * (K / 8);
+    if (chunks == 0) return MX_OK;
+    mx::dequantize_kernel<__nv_bfloat16><<<grid_for(chunks, 256, d.sm_count, 16), 256, 0, st>>>(
+        static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits, out, ld);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+// ---- tensor-core GEMM launcher ----------------------------------------------------------------
+mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, int64_t K, int box_rows)
+{
+    if (!g_encode_tiled) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !fn) {
+            snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled not available");
+            return MX_ERR_CUDA;
+        }
+        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)mx::TC_BK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base),
+                                      dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled failed (%d)", (int)r);
+        return MX_ERR_CUDA;
+    }
+    return MX_OK;
+}
+
+template <int BN>
+mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
+                      int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d,
+                      cudaStream_t st)
+{
+    using Cfg = mx::TcCfg<BN>;
+    CUtensorMap tm_a, tm_w;
+    mx_status_t s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
+    if (s != MX_OK) return s;
+    constexpr int slot = BN == 256 ? 0 : 1;
+    if (!d.tc_attr_set[slot]) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Cfg::SMEM_BYTES));
+        d.tc_attr_set[slot] = true;
+    }
+    mx::TcParams p;
+    p.y = y;
+    p.bias = bias;
+    p.ldy = ldy;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
+    p.tiles_n = (int)((N + BN - 1) / BN);
+    p.status = d.status;
+    const int tiles = p.tiles_m * p.tiles_n;
+    const int grid = tiles < d.sm_count ? tiles : d.sm_count;
+    mx::gemm_tc_kernel<BN><<<grid, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, p);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
+                   int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+{
+    const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256);
+    if (tiles256 >= (int64_t)d.sm_count * 3 / 4)
+        return launch_tc<256>(a_hat, w_hat, M, N, K, bias, y, ldy, d, st);
+    return launch_tc<128>(a_hat, w_hat, M, N, K, bias, y, ldy, d, st);
+}
+
+size_t tc_workspace(int64_t M, int64_t N, int64_t K)
+{
+    return round256((size_t)M * K * 2) + round256((size_t)N * K * 2);
+}
+size_t packed_workspace(int64_t M, int64_t K, const mx_format_t &fa)
+{
+    return round256(mx_mant_bytes(M, K, fa)) + round256(mx_exp_bytes(M, K, fa));
+}
+
+mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t &fa, const void *w,
+                            const void *w_exp, const mx_format_t &fw, int64_t M, int64_t N, int64_t K,
+                            const float *bias, const float *y, int64_t ldy)
+{
+    if (!a || !w || !w_exp || !y) return MX_ERR_NULL;
+    (void)a_exp;
+    if (!format_ok(fa) || !format_ok(fw) || fa.block != fw.block) return MX_ERR_FORMAT;
+    if (M <= 0 || N <= 0 || K <= 0 || (K % fa.block) != 0 || ldy < N) return MX_ERR_SHAPE;
+    if (M > INT32_MAX / 2 || N > INT32_MAX / 2 || K > INT32_MAX / 2) return MX_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias))) return MX_ERR_ALIGN;
+    return MX_OK;
+}
+
+}  // namespace
+
+// =================================================================================================
+extern "C" {
+
+size_t mx_mant_bytes(int64_t rows, int64_t K, mx_format_t f)
+{
+    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
+    return f.elem_bits <= 4 ? (size_t)rows * (size_t)(K / 2) : (size_t)rows * (size_t)K;
+}
+
+size_t mx_exp_bytes(int64_t rows, int64_t K, mx_format_t f)
+{
+    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
+    return (size_t)rows * (size_t)(K / f.block);
+}
+
+double mx_format_bits(mx_format_t f)
+{
+    if (f.block <= 0 || f.block_rows <= 0 || f.exp_bits <= 0 || f.elem_bits < 2) return 0.0;
+    return (double)f.exp_bits / ((double)f.block * (double)f.block_rows) + (double)(f.elem_bits - 1) + 1.0;
+}
+
+size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw)
+{
+    if (!format_ok(fa) || !format_ok(fw) || M <= 0 || N <= 0 || K <= 0) return 0;
+    const size_t tc = tc_workspace(M, N, K);
+    const size_t pk = packed_workspace(M, K, fa);
+    return tc > pk ? tc : pk;
+}
+
+const char *mx_status_string(mx_status_t s)
+{
+    switch (s) {
+    case MX_OK: return "ok";
+    case MX_ERR_NULL: return "null pointer";
+    case MX_ERR_SHAPE: return "bad shape";
+    case MX_ERR_FORMAT: return "unsupported MXInt format";
+    case MX_ERR_ALIGN: return "misaligned pointer or stride";
+    case MX_ERR_WORKSPACE: return "workspace missing or too small";
+    case MX_ERR_CUDA: return "CUDA error";
+    case MX_ERR_TIMEOUT: return "device-side wait timed out";
+    case MX_ERR_ARCH: return "device is not sm_100";
+    }
+    return "unknown status";
+}
+
+const char *mx_last_cuda_error(void) { return t_cuda_error; }
+
+mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, int64_t stride_row,
+                        int64_t stride_k, mx_format_t f, void *mant_out, uint8_t *exp_out,
+                        uint32_t *nonfinite_count, void *stream)
+{
+    if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || stride_k == 0) return MX_ERR_SHAPE;
+    if (rows == 0 || K == 0) return MX_OK;               // empty tensor: nothing to do
+    if (!x || !mant_out || !exp_out) return MX_ERR_NULL;
+    if (stride_k == 1 && stride_row < K) return MX_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(mant_out)) return MX_ERR_ALIGN;
+    if (stride_k == 1 && (stride_row % 8) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    mx::QuantOut out{static_cast<uint8_t *>(mant_out), exp_out, nullptr, 0, nonfinite_count};
+    if (stride_k == 1) return quantize_rows_any(x, dt, rows, K, stride_row, f, out, *d, st);
+    const int grid = grid_for(rows * (K / f.block), 256, d->sm_count, 8);
+    if (dt == MX_F32)
+        mx::quantize_strided_kernel<float><<<grid, 256, 0, st>>>(
+            static_cast<const float *>(x), rows, K, stride_row, stride_k, f.block, f.elem_bits, out);
+    else
+        mx::quantize_strided_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(
+            static_cast<const __nv_bfloat16 *>(x), rows, K, stride_row, stride_k, f.block, f.elem_bits, out);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
+                          mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream)
+{
+    if (!mant || !exps || !out) return MX_ERR_NULL;
+    if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || ld_out < K) return MX_ERR_SHAPE;
+    if (!aligned16(mant) || !aligned16(out) || (ld_out % 8) != 0) return MX_ERR_ALIGN;
+    if (rows == 0 || K == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (dt == MX_BF16)
+        return launch_dequant_bf16(mant, exps, rows, K, f, static_cast<__nv_bfloat16 *>(out), ld_out, *d, st);
+    mx::dequantize_kernel<float><<<grid_for(rows * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
+        static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits,
+        static_cast<float *>(out), ld_out);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                       const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                       const float *bias, float *y, int64_t ldy, void *workspace,
+                       size_t workspace_bytes, mx_algo_t algo, void *stream)
+{
+    mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
+    if (s != MX_OK) return s;
+    if (!a_exp) return MX_ERR_NULL;
+    if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05) return MX_ERR_FORMAT;
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (algo == MX_ALGO_SIMT) {
+        dim3 grid((unsigned)((N + 15) / 16), (unsigned)((M + 15) / 16));
+        mx::gemm_simt_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t *>(a_mant), a_exp,
+                                                   fa.elem_bits, static_cast<const uint8_t *>(w_mant),
+                                                   w_exp, fw.elem_bits, M, N, K, fa.block, bias, y, ldy);
+        MX_CUDA(cudaGetLastError());
+        return MX_OK;
+    }
+    if (!workspace || workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
+                                                             round256((size_t)M * K * 2));
+    s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    if (s != MX_OK) return s;
+    return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
+}
+
+mx_status_t mx_gemm(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                    const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                    const float *bias, float *y, int64_t ldy, void *workspace, size_t workspace_bytes,
+                    void *stream)
+{
+    return mx_gemm_ex(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, workspace,
+                      workspace_bytes, MX_ALGO_AUTO, stream);
+}
+
+mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
+                         mx_format_t fa, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                         int64_t N, const float *bias, float *y, int64_t ldy, void *workspace,
+                         size_t workspace_bytes, mx_algo_t algo, void *stream)
+{
+    mx_status_t s = check_gemm_args(x, nullptr, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
+    if (s != MX_OK) return s;
+    if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
+    if (ldx < K) return MX_ERR_SHAPE;
+    if ((ldx % 8) != 0) return MX_ERR_ALIGN;
+    if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05) return MX_ERR_FORMAT;
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!workspace) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    if (algo == MX_ALGO_SIMT) {
+        if (workspace_bytes < packed_workspace(M, K, fa)) return MX_ERR_WORKSPACE;
+        uint8_t *a_mant = ws;
+        uint8_t *a_exp = ws + round256(mx_mant_bytes(M, K, fa));
+        mx::QuantOut out{a_mant, a_exp, nullptr, 0, nullptr};
+        s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
+        if (s != MX_OK) return s;
+        return mx_gemm_ex(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, nullptr, 0,
+                          MX_ALGO_SIMT, stream);
+    }
+    if (workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
+    // the activations' mantissas and exponents go straight to the MMA operand form (exact bf16)
+    mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
+    s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    if (s != MX_OK) return s;
+    return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
+}
+
+mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
+                      const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
+                      const float *bias, float *y, int64_t ldy, void *workspace, size_t workspace_bytes,
+                      void *stream)
+{
+    return mx_linear_ex(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, y, ldy, workspace,
+                        workspace_bytes, MX_ALGO_AUTO, stream);
+}
+
+mx_status_t mx_poll_status(void *stream)
+{
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    MX_CUDA(cudaStreamSynchronize(st));
+    uint32_t word = 0;
+    MX_CUDA(cudaMemcpy(&word, d->status, sizeof(word), cudaMemcpyDeviceToHost));
+    if (word != 0) {
+        const uint32_t zero = 0;
+        MX_CUDA(cudaMemcpy(d->status, &zero, sizeof(zero), cudaMemcpyHostToDevice));
+    }
+    return (word & mx::STATUS_TIMEOUT_BIT) ? MX_ERR_TIMEOUT : MX_OK;
+}
+
+}  // extern "C"

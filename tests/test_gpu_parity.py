@@ -1,0 +1,245 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on identical seeded
+inputs.  Mantissas and exponent bytes must match bit for bit; fp32 outputs of the block-scaled
+product must satisfy |Y - Y_ref| <= 1e-5 * S with S = sum_b |t_b| the sum of the absolute block
+terms (so <= 1e-5 relative wherever there is no cancellation); the CUDA-core kernel adds the
+blocks in ascending order and must equal the oracle's sequential-fp32 result exactly."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mx_oracle as orc
+from paper_2307_15517_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL = 1e-5
+WIDTHS = (2, 3, 4, 5, 6, 8)
+
+
+@pytest.fixture(scope="module")
+def mxb():
+    from paper_2307_15517_b200 import binding
+    return binding
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def _oracle_packed(x_np, B, w):
+    q, e, bad = orc.quantize(x_np, B, w)
+    return q, e, orc.pack(q, w), bad
+
+
+def _check_tol(y_gpu, y_ref, S):
+    y = y_gpu.cpu().numpy().astype(np.float64)
+    err = np.abs(y - y_ref.astype(np.float64))
+    bound = TOL * S + 1e-37
+    worst = float((err / np.maximum(S, 1e-300)).max())
+    assert (err <= bound).all(), "max |dY|/S = %.3e" % worst
+    return worst
+
+
+# ------------------------------------------------------------------------------ quantizer
+
+def _edge_case_rows(K):
+    """Rows that exercise zeros, subnormals, ties, saturation, huge and non-finite values."""
+    rng = np.random.default_rng(3)
+    x = rng.standard_normal((12, K)).astype(np.float32)
+    x[0] = 0.0
+    x[1, :] = (rng.integers(-7, 8, K) * 0.5).astype(np.float32)          # many exact ties
+    x[1, ::16] = 4.0
+    x[2] = np.ldexp(x[2], -140).astype(np.float32)                         # subnormal blocks
+    x[3] = np.ldexp(x[3], 120).astype(np.float32)                          # near the top
+    x[3, 5] = 3.0e38
+    x[4, 3] = np.inf
+    x[4, 40] = -np.inf
+    x[5, 17] = np.nan
+    x[6, :] = 7.99                                                          # saturating maximum
+    x[7, :] = np.float32(2.0 ** -126) - np.float32(2.0 ** -149)
+    x[8, ::2] = -x[8, ::2] * 1000
+    x[9] = np.ldexp(np.ones(K), rng.integers(-126, 127, K)).astype(np.float32)
+    x[10, :] = -0.0
+    x[11] = rng.standard_t(3, K).astype(np.float32) * 40
+    return x
+
+
+@pytest.mark.parametrize("B", (16, 32))
+@pytest.mark.parametrize("w", WIDTHS)
+def test_quantize_bit_exact(mxb, B, w):
+    F = mxb.MxFormat(B, w)
+    rng = np.random.default_rng(100 * B + w)
+    cases = [
+        (rng.standard_normal((37, 96)) * np.exp(rng.uniform(-8, 8, (37, 1)))).astype(np.float32),
+        rng.standard_t(3, (130, 2080)).astype(np.float32),       # ragged last warp, several CTAs
+        _edge_case_rows(64),
+        np.zeros((0, 64), np.float32),
+    ]
+    for x in cases:
+        q, e, packed, bad = _oracle_packed(x, B, w)
+        cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        mant, exps = mxb.mx_quantize(_dev(x), F, nonfinite_count=cnt)
+        assert np.array_equal(exps.cpu().numpy(), e)
+        assert np.array_equal(mant.cpu().numpy(), packed)
+        assert int(cnt.item()) == bad
+        if x.shape[0]:
+            xhat = mxb.mx_dequantize(mant, exps, x.shape[1], F).cpu().numpy()
+            want = orc.dequantize(q, e, B, w)
+            assert np.array_equal(np.isnan(xhat), np.isnan(want))
+            ok = ~np.isnan(want)
+            assert np.array_equal(xhat[ok].astype(np.float64), want[ok])
+            xhat16 = mxb.mx_dequantize(mant, exps, x.shape[1], F, dtype=torch.bfloat16)
+            assert np.array_equal(xhat16.float().cpu().numpy()[ok].astype(np.float64), want[ok])
+
+
+@pytest.mark.parametrize("w", (4, 8))
+def test_quantize_bf16_input_and_padded_rows(mxb, w):
+    F = mxb.MxFormat(32, w)
+    g = torch.Generator().manual_seed(w)
+    xb = (torch.randn(67, 256, generator=g) * 3).to(torch.bfloat16)
+    q, e, packed, _ = _oracle_packed(xb.float().numpy(), 32, w)
+    mant, exps = mxb.mx_quantize(xb.cuda(), F)
+    assert np.array_equal(mant.cpu().numpy(), packed) and np.array_equal(exps.cpu().numpy(), e)
+    # a view with a leading dimension larger than K
+    big = torch.randn(67, 512, generator=g)
+    view = big.cuda()[:, 128:384]
+    q, e, packed, _ = _oracle_packed(big[:, 128:384].contiguous().numpy(), 32, w)
+    mant, exps = mxb.mx_quantize(view, F)
+    assert np.array_equal(mant.cpu().numpy(), packed) and np.array_equal(exps.cpu().numpy(), e)
+
+
+def test_quantize_along_a_strided_axis(mxb):
+    """V of attention is blocked along the token axis: x[r, k] = v[k, r]."""
+    g = torch.Generator().manual_seed(9)
+    v = torch.randn(192, 40, generator=g)                      # [tokens, d]
+    for w, B in ((8, 16), (4, 32)):
+        F = mxb.MxFormat(B, w)
+        q, e, packed, _ = _oracle_packed(v.numpy().T, B, w)
+        mant, exps = mxb.mx_quantize(v.cuda().t(), F)
+        assert np.array_equal(mant.cpu().numpy(), packed) and np.array_equal(exps.cpu().numpy(), e)
+
+
+def test_quantize_single_layer_config(mxb):
+    x, wt, spec = synth.single_layer(0)
+    F = mxb.MxFormat(spec.block, spec.w_act)
+    for t in (x, wt):
+        q, e, packed, _ = _oracle_packed(t.numpy(), spec.block, spec.w_act)
+        mant, exps = mxb.mx_quantize(t.cuda(), F)
+        assert np.array_equal(mant.cpu().numpy(), packed) and np.array_equal(exps.cpu().numpy(), e)
+
+
+# ------------------------------------------------------------------------------ product
+
+def _random_operands(M, N, K, B, wa, ww, seed, spread=8):
+    """Raw mantissas and exponent bytes (not produced by any quantizer): full value range
+    including -2^(w-1), exponents spread over 2^spread."""
+    qa = synth.random_ints((M, K), -(2 ** (wa - 1)) if wa > 2 else -1, 2 ** (wa - 1) - 1, seed).numpy()
+    qw = synth.random_ints((N, K), -(2 ** (ww - 1)) if ww > 2 else -1, 2 ** (ww - 1) - 1, seed + 1).numpy()
+    ea = synth.random_bytes((M, K // B), 127 - spread, 127 + spread, seed + 2).numpy()
+    ew = synth.random_bytes((N, K // B), 120 - spread, 120 + spread, seed + 3).numpy()
+    return qa, ea, qw, ew
+
+
+GEMM_SHAPES = [
+    # M, N, K, B, wa, ww
+    (128, 768, 768, 16, 4, 4),        # the single-layer configuration's shape
+    (200, 300, 320, 32, 8, 4),        # ragged M and N tails, K tail (320 = 5 * 64)
+    (384, 640, 1024, 16, 8, 8),       # several tiles each way
+    (130, 40, 96, 16, 6, 3),          # K not a multiple of 64, N below one tile
+    (1, 256, 128, 32, 8, 4),          # a single row
+    (257, 513, 2048, 32, 5, 2),
+    (1536, 2560, 256, 16, 8, 4),      # 120 tiles of 128x256: the wide-tile kernel, multi-wave
+]
+
+
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+def test_gemm_simt_matches_sequential_oracle_exactly(mxb, shape):
+    M, N, K, B, wa, ww = shape
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=M + N)
+    bias = np.random.default_rng(1).standard_normal(N).astype(np.float32)
+    y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
+    y = mxb.mx_gemm(_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)),
+                    _dev(ew), mxb.MxFormat(B, ww), M, N, K, bias=_dev(bias), algo=mxb.MX_ALGO_SIMT)
+    assert np.array_equal(y.cpu().numpy(), y_seq)
+    _check_tol(y, y_ref, S)
+
+
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+@pytest.mark.parametrize("with_bias", (False, True))
+def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias):
+    M, N, K, B, wa, ww = shape
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=7 * M + N)
+    bias = np.random.default_rng(2).standard_normal(N).astype(np.float32) if with_bias else None
+    y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
+    ypad = torch.full((M, N + 8), -77.0, device="cuda")           # canary columns, ldy > N
+    y = mxb.mx_gemm(_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)),
+                    _dev(ew), mxb.MxFormat(B, ww), M, N, K, bias=None if bias is None else _dev(bias),
+                    y=ypad[:, :N], algo=mxb.MX_ALGO_TCGEN05)
+    assert mxb.mx_poll_status() == 0
+    _check_tol(y, y_ref, S)
+    assert (ypad[:, N:] == -77.0).all()
+
+
+def test_gemm_one_hot_rows_expose_the_operand_layout(mxb):
+    """A = identity-like rows: Y must be the decoded weights, element for element (catches any
+    error in the swizzled shared-memory layout or the descriptors)."""
+    K, N, B = 256, 512, 16
+    x = np.zeros((K, K), np.float32)
+    x[np.arange(K), np.arange(K)] = 1.0
+    qa, ea, _ = orc.quantize(x, B, 8)
+    wt = synth.gaussian_weights(N, K, 3).numpy()
+    qw, ew, _ = orc.quantize(wt, B, 4)
+    y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, 4)),
+                    _dev(ew), mxb.MxFormat(B, 4), K, N, K, algo=mxb.MX_ALGO_TCGEN05)
+    assert np.array_equal(y.cpu().numpy().astype(np.float64), orc.dequantize(qw, ew, B, 4).T)
+
+
+def test_gemm_nonfinite_blocks_poison_their_outputs(mxb):
+    M, N, K, B = 130, 260, 128, 16
+    qa, ea, qw, ew = _random_operands(M, N, K, B, 8, 4, seed=5)
+    ea[3, 2] = 255
+    ew[200, 7] = 255
+    y_ref, _, _ = orc.gemm(qa, ea, 8, qw, ew, 4, B)
+    for algo in (mxb.MX_ALGO_SIMT, mxb.MX_ALGO_TCGEN05):
+        y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, 4)),
+                        _dev(ew), mxb.MxFormat(B, 4), M, N, K, algo=algo).cpu().numpy()
+        assert np.array_equal(np.isnan(y), np.isnan(y_ref))
+        assert np.isnan(y[3]).all() and np.isnan(y[:, 200]).all() and not np.isnan(y[4, 5])
+
+
+# ------------------------------------------------------------------------------ the layer
+
+def test_linear_single_layer_config(mxb):
+    """Configuration 1 end to end: quantize X on the fly, weights pre-quantized, Y = X W^T."""
+    x, wt, spec = synth.single_layer(0)
+    fa, fw = mxb.MxFormat(spec.block, spec.w_act), mxb.MxFormat(spec.block, spec.w_wgt)
+    qa, ea, _ = orc.quantize(x.numpy(), spec.block, spec.w_act)
+    qw, ew, _ = orc.quantize(wt.numpy(), spec.block, spec.w_wgt)
+    y_ref, y_seq, S = orc.gemm(qa, ea, spec.w_act, qw, ew, spec.w_wgt, spec.block)
+    w_mant, w_exp = mxb.mx_quantize(wt.cuda(), fw)
+    y_tc = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N, algo=mxb.MX_ALGO_TCGEN05)
+    y_simt = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N, algo=mxb.MX_ALGO_SIMT)
+    assert mxb.mx_poll_status() == 0
+    assert np.array_equal(y_simt.cpu().numpy(), y_seq)
+    _check_tol(y_tc, y_ref, S)
+
+
+@pytest.mark.parametrize("case", [(16, 8, 4), (32, 4, 4), (32, 6, 3), (16, 2, 8)])
+def test_linear_mixed_precision(mxb, case):
+    B, wa, ww = case
+    M, K, N = 300, 1152, 520
+    x = synth.student_t_activations(M, K, seed=wa)
+    wt = synth.gaussian_weights(N, K, seed=ww)
+    bias = synth.gaussian_weights(1, N, seed=5, std=1.0)[0]
+    qa, ea, _ = orc.quantize(x.numpy(), B, wa)
+    qw, ew, _ = orc.quantize(wt.numpy(), B, ww)
+    y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias.numpy())
+    fa, fw = mxb.MxFormat(B, wa), mxb.MxFormat(B, ww)
+    w_mant, w_exp = mxb.mx_quantize(wt.cuda(), fw)
+    y = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, N, bias=bias.cuda())
+    assert mxb.mx_poll_status() == 0
+    _check_tol(y, y_ref, S)
+    yb = mxb.mx_linear(x.to(torch.bfloat16).cuda(), fa, w_mant, w_exp, fw, N, bias=bias.cuda())
+    qa, ea, _ = orc.quantize(x.to(torch.bfloat16).float().numpy(), B, wa)
+    y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias.numpy())
+    _check_tol(yb, y_ref, S)

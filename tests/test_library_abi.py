@@ -1,0 +1,95 @@
+"""Host-side checks of the C-ABI library that need no GPU: it loads, exports every symbol the
+header declares, its size helpers reproduce the paper's storage accounting (Eq. 1), and
+invalid arguments are rejected before any launch."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+
+from paper_2307_15517_b200 import build as mx_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def mxb():
+    mx_build.build()
+    from paper_2307_15517_b200 import binding
+    return binding
+
+
+def _declared_symbols():
+    names = []
+    inc = os.path.join(ROOT, "include")
+    for fn in sorted(os.listdir(inc)):
+        if fn.endswith(".h"):
+            text = open(os.path.join(inc, fn)).read()
+            names += re.findall(r"MX_API\s+[\w\s\*]+?\b(mx_\w+)\s*\(", text)
+    return names
+
+
+def test_every_declared_symbol_is_exported(mxb):
+    names = _declared_symbols()
+    assert len(names) >= 13 and "mx_quantize" in names and "mx_gemm" in names and "mx_linear" in names
+    for n in names:
+        assert hasattr(mxb.lib, n), n
+
+
+def test_size_helpers_match_eq1(mxb):
+    F = mxb.MxFormat
+    assert mxb.mx_format_bits(F(16, 8, 8, 2)) == 8.25          # the paper's MXInt((16,2),8,7)
+    assert mxb.mx_format_bits(F(16, 4)) == 4.5 and mxb.mx_format_bits(F(32, 4)) == 4.25
+    assert mxb.mx_mant_bytes(128, 768, F(16, 4)) == 128 * 384
+    assert mxb.mx_mant_bytes(128, 768, F(16, 5)) == 128 * 768
+    assert mxb.mx_exp_bytes(128, 768, F(16, 4)) == 128 * 48
+    assert mxb.mx_exp_bytes(4096, 11008, F(32, 4)) == 4096 * 344
+    # decode weight stream of one 4096x4096 W4/B32 matrix: 0.53125 bytes per weight
+    total = mxb.mx_mant_bytes(4096, 4096, F(32, 4)) + mxb.mx_exp_bytes(4096, 4096, F(32, 4))
+    assert total == int(4096 * 4096 * 0.53125)
+    assert mxb.mx_mant_bytes(4, 40, F(16, 4)) == 0             # K not a multiple of the block
+    assert mxb.mx_mant_bytes(4, 64, F(8, 4)) == 0              # unsupported block
+    assert mxb.mx_workspace_bytes(128, 768, 768, F(16, 4), F(16, 4)) >= 2 * (128 + 768) * 768
+
+
+def test_status_strings(mxb):
+    for code in range(0, -9, -1):
+        assert mxb.mx_status_string(code) not in ("", "unknown status")
+
+
+def test_invalid_arguments_are_rejected_on_the_host(mxb):
+    F = mxb.MxFormat
+    L = mxb.lib
+    fake = C.c_void_p(0x10000)       # never dereferenced: validation fails first
+    odd = C.c_void_p(0x10004)
+    f = F(16, 4)
+    assert L.mx_quantize(None, 0, 4, 64, 64, 1, f, fake, fake, None, None) == -1
+    assert L.mx_quantize(fake, 0, 4, 40, 40, 1, f, fake, fake, None, None) == -2
+    assert L.mx_quantize(fake, 0, 4, 64, 32, 1, f, fake, fake, None, None) == -2   # ld < K
+    assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 9), fake, fake, None, None) == -3
+    assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4, 5), fake, fake, None, None) == -3
+    assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4, 8, 2), fake, fake, None, None) == -3
+    assert L.mx_quantize(fake, 7, 4, 64, 64, 1, f, fake, fake, None, None) == -3
+    assert L.mx_quantize(odd, 0, 4, 64, 64, 1, f, fake, fake, None, None) == -4
+    assert L.mx_quantize(fake, 0, 4, 64, 68, 1, f, fake, fake, None, None) == -4   # ld % 8
+    g = lambda **kw: L.mx_gemm_ex(kw.get("a", fake), fake, kw.get("fa", f), fake, fake, kw.get("fw", f),
+                                  kw.get("M", 8), kw.get("N", 8), kw.get("K", 64), None,
+                                  kw.get("y", fake), kw.get("ldy", 8), kw.get("ws", None), 0,
+                                  kw.get("algo", 2), None)
+    assert g(a=None) == -1
+    assert g(K=40) == -2 and g(M=0) == -2 and g(ldy=4) == -2
+    assert g(fa=F(32, 4)) == -3                     # blocks of A and W differ
+    assert g(y=odd) == -4
+    assert g(algo=9) == -3
+    assert L.mx_linear_ex(fake, 0, 8, 64, 60, f, fake, fake, f, 8, None, fake, 8, None, 0, 2, None) == -2
+
+
+@pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")
+def test_compute_calls_fail_loudly_without_a_gpu(mxb):
+    F = mxb.MxFormat
+    fake = C.c_void_p(0x10000)
+    rc = mxb.lib.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4), fake, fake, None, None)
+    assert rc in (-6, -8)
+    with pytest.raises(ValueError):
+        mxb.mx_quantize(torch.zeros(4, 64), F(16, 4))       # host tensors are refused

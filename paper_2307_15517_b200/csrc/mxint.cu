@@ -273,10 +273,10 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
                         uint32_t *nonfinite_count, void *stream)
 {
     if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
-    if (rows < 0 || K < 0 || (K % f.block) != 0 || stride_k == 0) return MX_ERR_SHAPE;
+    if (rows < 0 || K < 0 || (K % f.block) != 0) return MX_ERR_SHAPE;
     if (rows == 0 || K == 0) return MX_OK;               // empty tensor: nothing to do
     if (!x || !mant_out || !exp_out) return MX_ERR_NULL;
-    if (stride_k == 1 && stride_row < K) return MX_ERR_SHAPE;
+    if (stride_k == 0 || (stride_k == 1 && stride_row < K)) return MX_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(mant_out)) return MX_ERR_ALIGN;
     if (stride_k == 1 && (stride_row % 8) != 0) return MX_ERR_ALIGN;
     DeviceInfo *d = nullptr;

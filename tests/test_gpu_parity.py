@@ -167,8 +167,10 @@ def test_gemm_simt_matches_sequential_oracle_exactly(mxb, shape):
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
 @pytest.mark.parametrize("with_bias", (False, True))
 def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias):
+    """Block exponents spread over 2^+-3 per operand (2^+-6 per product term), wider than any of
+    the paper-shaped workloads produce within one row."""
     M, N, K, B, wa, ww = shape
-    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=7 * M + N)
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=7 * M + N, spread=3)
     bias = np.random.default_rng(2).standard_normal(N).astype(np.float32) if with_bias else None
     y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
     ypad = torch.full((M, N + 8), -77.0, device="cuda")           # canary columns, ldy > N
@@ -178,6 +180,26 @@ def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias):
     assert mxb.mx_poll_status() == 0
     _check_tol(y, y_ref, S)
     assert (ypad[:, N:] == -77.0).all()
+
+
+def test_gemm_tensor_core_adversarial_exponent_spread(mxb):
+    """Block exponents drawn uniformly over 2^+-8 per operand (terms 2^+-16 apart).  The tensor
+    pipe aligns the 16 products of one MMA step and the accumulator to the largest of them and
+    truncates each (measured: no rounding, no guard bit), so its worst case is 17 truncations of
+    one accumulator ulp per step: |dY| < ceil(K/16) * 17 * 2^-23 * S.  The CUDA-core kernel, which
+    rounds once per block, stays inside 1e-5 * S on the same operands."""
+    M, N, K, B, wa, ww = 200, 300, 320, 32, 8, 4
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=1700, spread=8)
+    y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
+    args = (_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)), _dev(ew),
+            mxb.MxFormat(B, ww), M, N, K)
+    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05).cpu().numpy().astype(np.float64)
+    assert mxb.mx_poll_status() == 0
+    bound = -(-K // 16) * 17 * 2.0 ** -23 * S
+    assert (np.abs(y - y_ref) <= bound).all()
+    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_SIMT)
+    assert np.array_equal(y.cpu().numpy(), y_seq)
+    _check_tol(y, y_ref, S)
 
 
 def test_gemm_one_hot_rows_expose_the_operand_layout(mxb):

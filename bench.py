@@ -1,0 +1,321 @@
+#!/usr/bin/env python
+"""Benchmark of the MXInt linear-layer hot path (arXiv 2307.15517) on B200.
+
+One *step* = the whole hot path over one batch of synthetic input: for each of the four
+OPT-1.3B-shaped prefill linears (2048 tokens; 2048->6144, 2048->2048, 2048->8192, 8192->2048;
+MXInt4, block 16) the activations are quantized on the fly and multiplied with the layer's
+pre-quantized weights (``mx_linear`` of the C ABI).  Weights are quantized once before the timed
+region (they are static at inference); activations are quantized in every step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  ``value`` = effective TOPS (2*M*N*K summed over the four layers and all
+ranks / device time of the steps).  With N > 1 (torchrun) every rank runs the same step on its own
+token batch: independent problems, no data-path collective, weak scaling.
+``--impl reference`` times the plain CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "mx_linear_effective_tops"
+UNIT = "TOPS"
+WORKLOAD = "opt-1.3b prefill linears, 2048 tokens, MXInt4 block 16 (4 layers per step)"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS}, "measured"
+    except Exception:
+        return dict(FALLBACK_PEAKS), "fallback"
+
+
+# ------------------------------------------------------------------------------ clocks sampler
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in out.splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        # samples taken under load: the upper half of the observed clocks
+        load = sorted(sm)[len(sm) // 2:] if sm else []
+        return {"sm_mhz": statistics.median(load) if load else None,
+                "sm_max_mhz": max(smax) if smax else None, "samples": len(sm),
+                "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ workload
+def layer_flops(tokens, spec):
+    return 2.0 * tokens * spec.N * spec.K
+
+
+def build_device_workload(mxb, synth, torch, rank):
+    """Per layer: fp32 activations (device + pinned host copy), pre-quantized weights, output."""
+    layers = []
+    for li, spec in enumerate(synth.opt13b_prefill_layers()):
+        x, w, _ = synth.opt13b_inputs(li, seed=rank)
+        fa, fw = mxb.MxFormat(spec.block, spec.w_act), mxb.MxFormat(spec.block, spec.w_wgt)
+        w_mant, w_exp = mxb.mx_quantize(w.cuda(), fw)
+        xd = x.cuda()
+        y = torch.empty((x.shape[0], spec.N), dtype=torch.float32, device="cuda")
+        ws = mxb.alloc_workspace(mxb.mx_workspace_bytes(x.shape[0], spec.N, spec.K, fa, fw))
+        layers.append(dict(spec=spec, fa=fa, fw=fw, x=xd, x_host=x.pin_memory(), w_mant=w_mant,
+                           w_exp=w_exp, y=y, ws=ws,
+                           y_host=torch.empty((x.shape[0], spec.N), dtype=torch.float32).pin_memory()))
+    torch.cuda.synchronize()
+    return layers
+
+
+def run_step(mxb, layers):
+    for L in layers:
+        mxb.mx_linear(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, y=L["y"],
+                      workspace=L["ws"])
+
+
+def run_step_e2e(mxb, layers):
+    for L in layers:
+        L["x"].copy_(L["x_host"], non_blocking=True)
+        mxb.mx_linear(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, y=L["y"],
+                      workspace=L["ws"])
+        L["y_host"].copy_(L["y"], non_blocking=True)
+
+
+# ------------------------------------------------------------------------------ oracle (CPU)
+def oracle_inputs(orc, synth, sample_rows):
+    """Untimed set-up: the first `sample_rows` tokens of every layer and its quantized weights."""
+    out = []
+    for li, spec in enumerate(synth.opt13b_prefill_layers()):
+        x, w, _ = synth.opt13b_inputs(li, seed=0)
+        qw, ew, _ = orc.quantize(w.numpy(), spec.block, spec.w_wgt)
+        out.append(dict(spec=spec, x=x[:sample_rows].contiguous().numpy(), qw=qw, ew=ew))
+    return out
+
+
+def oracle_step(orc, inputs):
+    """One pass of the hot path on the CPU: quantize the sampled activations, then the
+    block-scaled product against the full weights.  Returns (seconds, operations)."""
+    t_total, macs = 0.0, 0
+    for L in inputs:
+        spec = L["spec"]
+        t0 = time.perf_counter()
+        qa, ea, _ = orc.quantize(L["x"], spec.block, spec.w_act)
+        orc.gemm(qa, ea, spec.w_act, L["qw"], L["ew"], spec.w_wgt, spec.block)
+        t_total += time.perf_counter() - t0
+        macs += L["x"].shape[0] * spec.N * spec.K
+    return t_total, 2.0 * macs
+
+
+def cpu_baseline(sample_rows=2048):
+    from oracle import mx_oracle as orc
+    from paper_2307_15517_b200 import synth
+    t, ops = oracle_step(orc, oracle_inputs(orc, synth, sample_rows))
+    return {"value": ops / t / 1e12, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+            "sample": "first %d of 2048 tokens of each of the 4 layers, all output columns, "
+                      "one pass, %.1f s of CPU time" % (sample_rows, t)}
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step is a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import mx_oracle as orc
+    from paper_2307_15517_b200 import synth
+    rows = 64
+    inputs = oracle_inputs(orc, synth, rows)
+    for _ in range(max(args.warmup, 1)):
+        oracle_step(orc, inputs)
+    t, ops = 0.0, 0.0
+    for _ in range(args.steps):
+        dt, o = oracle_step(orc, inputs)
+        t += dt
+        ops += o
+    value = ops / t / 1e12
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int64/f64",
+        "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": "first %d tokens of each layer per step" % rows},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": orc.threads(), "kind": "oracle",
+                         "sample": "first %d of 2048 tokens of each of the 4 layers per step" % rows},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2307_15517_b200 import binding as mxb
+    from paper_2307_15517_b200 import synth
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the MXInt kernels have no CPU path")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks, peaks_kind = load_peaks()
+    layers = build_device_workload(mxb, synth, torch, rank)
+    tokens = synth.OPT13B_TOKENS
+    flops_step = sum(layer_flops(tokens, L["spec"]) for L in layers)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # > 126 MB of L2
+
+    def timed_steps(step_fn, steps, profile):
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+               for _ in range(steps)]
+        if profile:
+            mxb.mx_profile_begin()
+        for a, b in evs:
+            flush.fill_(1)                    # evict the previous step's data from L2 (untimed)
+            a.record()
+            step_fn(mxb, layers)
+            b.record()
+        torch.cuda.synchronize()
+        prof = mxb.mx_profile_end() if profile else None
+        return sum(a.elapsed_time(b) for a, b in evs), prof
+
+    # ---- device-resident timing ----
+    for _ in range(args.warmup):
+        run_step(mxb, layers)
+    assert mxb.mx_poll_status() == 0, "device status after warm-up"
+    sampler = ClockSampler(local_rank)
+    barrier()
+    if rank == 0:
+        sampler.start()
+    ms_total, prof = timed_steps(run_step, args.steps, profile=True)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    assert mxb.mx_poll_status() == 0, "device status after the timed region"
+
+    # ---- end to end: pinned host inputs in, results out, every step ----
+    ms_e2e = float("nan")
+    if not args.skip_e2e:
+        for _ in range(2):
+            run_step_e2e(mxb, layers)
+        barrier()
+        ms_e2e, _ = timed_steps(run_step_e2e, args.steps, profile=False)
+        barrier()
+
+    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, ms_e2e = float(t[0]), float(t[1])
+
+    if rank == 0:
+        value = world * flops_step * args.steps / (ms_total * 1e-3) / 1e12
+        e2e_value = world * flops_step * args.steps / (ms_e2e * 1e-3) / 1e12
+        gemm_ms, gemm_n = prof["gemm_tc"]
+        achieved = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
+        peak = peaks["bf16_tflops_sustained"]
+        h2d = sum(L["x_host"].numel() * 4 for L in layers)
+        d2h = sum(L["y_host"].numel() * 4 for L in layers)
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (exact MXInt decode) x bf16 -> f32",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "tokens_per_gpu": tokens,
+                       "layers": [[L["spec"].name, L["spec"].K, L["spec"].N] for L in layers],
+                       "weights": "pre-quantized once outside the timed region",
+                       "l2": "256 MiB written between steps (untimed); per-step CUDA events summed",
+                       "parallelism": "replicas over token batches (no collective)"},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                    "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps},
+            "gpu_launches": sum(n for _, n in prof.values()),
+            "kernels": {k: {"ms_per_step": ms / args.steps, "launches_per_step": n / args.steps}
+                        for k, (ms, n) in prof.items() if n},
+            "roofline": {"bound": "tensor", "kernel": "gemm_tc_kernel", "achieved": achieved,
+                         "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
+                         "peak_kind": "bf16 sustained, %s" % peaks_kind,
+                         "frac_of_burst_peak": achieved / peaks["bf16_tflops"],
+                         "traffic": None},
+            "cpu_baseline": None if args.skip_cpu_baseline else cpu_baseline(),
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=("ours", "reference"))
+    ap.add_argument("--skip-cpu-baseline", action="store_true",
+                    help="leave the CPU oracle timing out (profiler runs)")
+    ap.add_argument("--skip-e2e", action="store_true", help="leave the host-buffer leg out")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3)
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

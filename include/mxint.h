@@ -166,6 +166,18 @@ MX_API mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t
  */
 MX_API mx_status_t mx_poll_status(void *stream);
 
+/* ---- launch profile (benchmark support; the paper has no counterpart) ---------------------
+ *
+ * Between mx_profile_begin and mx_profile_end the library brackets each of its kernel launches
+ * with a pair of CUDA events on the launch stream.  mx_profile_end waits for them and returns,
+ * per kernel kind, the summed device time in milliseconds and the number of launches (arrays of
+ * MX_KERNEL_KINDS entries, host memory).  Kinds: 0 quantize, 1 dequantize, 2 tensor-core GEMM,
+ * 3 CUDA-core GEMM, 4 weight-streaming GEMM.  Not thread-safe with respect to concurrent
+ * compute calls on other host threads being attributed correctly; meant for one stream. */
+#define MX_KERNEL_KINDS 8
+MX_API mx_status_t mx_profile_begin(void);
+MX_API mx_status_t mx_profile_end(double *ms_per_kind, int64_t *launches_per_kind);
+
 #ifdef __cplusplus
 }
 #endif

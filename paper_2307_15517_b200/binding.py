@@ -70,8 +70,10 @@ def _load() -> C.CDLL:
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
     L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_poll_status.argtypes = [vp]
+    L.mx_profile_begin.argtypes = []
+    L.mx_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
-                 "mx_linear_ex", "mx_poll_status"):
+                 "mx_linear_ex", "mx_poll_status", "mx_profile_begin", "mx_profile_end"):
         getattr(L, name).restype = i32
     return L
 
@@ -199,3 +201,18 @@ def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int
 def mx_poll_status(stream=None) -> int:
     """Synchronises the stream and returns the library's device status (0 = MX_OK)."""
     return int(lib.mx_poll_status(_stream(stream)))
+
+
+KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream")
+
+
+def mx_profile_begin() -> None:
+    _check(lib.mx_profile_begin(), "mx_profile_begin")
+
+
+def mx_profile_end():
+    """Returns {kind: (milliseconds, launches)} for the kernels launched since mx_profile_begin."""
+    ms = (C.c_double * 8)()
+    n = (C.c_int64 * 8)()
+    _check(lib.mx_profile_end(ms, n), "mx_profile_end")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(KERNEL_KINDS)}

@@ -7,6 +7,9 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <mutex>
+#include <vector>
+
 #include "../../include/mxint.h"
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
@@ -35,6 +38,44 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode_tiled = nullptr;
+
+// ---- launch profile: CUDA events around every kernel launch, summed per kernel kind ----------
+enum KernelKind { KIND_QUANTIZE = 0, KIND_DEQUANTIZE = 1, KIND_GEMM_TC = 2, KIND_GEMM_SIMT = 3,
+                  KIND_GEMM_STREAM = 4, KIND_COUNT = MX_KERNEL_KINDS };
+struct ProfEntry { cudaEvent_t a, b; int kind; };
+struct Profiler {
+    bool on = false;
+    std::vector<ProfEntry> entries;      // events in use since mx_profile_begin
+    std::vector<ProfEntry> pool;         // events kept for reuse
+    std::mutex mu;
+};
+Profiler g_prof;
+
+struct ProfScope {
+    cudaStream_t st;
+    ProfEntry e{};
+    bool live = false;
+    ProfScope(int kind, cudaStream_t s) : st(s)
+    {
+        if (!g_prof.on) return;
+        std::lock_guard<std::mutex> lk(g_prof.mu);
+        if (!g_prof.pool.empty()) {
+            e = g_prof.pool.back();
+            g_prof.pool.pop_back();
+        } else if (cudaEventCreate(&e.a) != cudaSuccess || cudaEventCreate(&e.b) != cudaSuccess) {
+            return;
+        }
+        e.kind = kind;
+        live = cudaEventRecord(e.a, st) == cudaSuccess;
+    }
+    ~ProfScope()
+    {
+        if (!live) return;
+        cudaEventRecord(e.b, st);
+        std::lock_guard<std::mutex> lk(g_prof.mu);
+        g_prof.entries.push_back(e);
+    }
+};
 
 mx_status_t cuda_fail(cudaError_t e, const char *what)
 {
@@ -97,6 +138,7 @@ mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t 
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
     const int grid = grid_for(chunks, 256, d.sm_count, 16);
+    ProfScope prof(KIND_QUANTIZE, st);
     if (f.block == 16)
         mx::quantize_rows_kernel<InT, 16><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
     else
@@ -120,6 +162,7 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
 {
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
+    ProfScope prof(KIND_DEQUANTIZE, st);
     mx::dequantize_kernel<__nv_bfloat16><<<grid_for(chunks, 256, d.sm_count, 16), 256, 0, st>>>(
         static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits, out, ld);
     MX_CUDA(cudaGetLastError());
@@ -183,6 +226,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, in
     p.status = d.status;
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
+    ProfScope prof(KIND_GEMM_TC, st);
     mx::gemm_tc_kernel<BN><<<grid, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, p);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
@@ -286,6 +330,7 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
     mx::QuantOut out{static_cast<uint8_t *>(mant_out), exp_out, nullptr, 0, nonfinite_count};
     if (stride_k == 1) return quantize_rows_any(x, dt, rows, K, stride_row, f, out, *d, st);
     const int grid = grid_for(rows * (K / f.block), 256, d->sm_count, 8);
+    ProfScope prof(KIND_QUANTIZE, st);
     if (dt == MX_F32)
         mx::quantize_strided_kernel<float><<<grid, 256, 0, st>>>(
             static_cast<const float *>(x), rows, K, stride_row, stride_k, f.block, f.elem_bits, out);
@@ -310,6 +355,7 @@ mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dt == MX_BF16)
         return launch_dequant_bf16(mant, exps, rows, K, f, static_cast<__nv_bfloat16 *>(out), ld_out, *d, st);
+    ProfScope prof(KIND_DEQUANTIZE, st);
     mx::dequantize_kernel<float><<<grid_for(rows * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
         static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits,
         static_cast<float *>(out), ld_out);
@@ -333,6 +379,7 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (algo == MX_ALGO_SIMT) {
         dim3 grid((unsigned)((N + 15) / 16), (unsigned)((M + 15) / 16));
+        ProfScope prof(KIND_GEMM_SIMT, st);
         mx::gemm_simt_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t *>(a_mant), a_exp,
                                                    fa.elem_bits, static_cast<const uint8_t *>(w_mant),
                                                    w_exp, fw.elem_bits, M, N, K, fa.block, bias, y, ldy);
@@ -408,6 +455,40 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
 {
     return mx_linear_ex(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, y, ldy, workspace,
                         workspace_bytes, MX_ALGO_AUTO, stream);
+}
+
+mx_status_t mx_profile_begin(void)
+{
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    for (const ProfEntry &e : g_prof.entries) g_prof.pool.push_back(e);
+    g_prof.entries.clear();
+    g_prof.on = true;
+    return MX_OK;
+}
+
+mx_status_t mx_profile_end(double *ms_per_kind, int64_t *launches_per_kind)
+{
+    if (!ms_per_kind || !launches_per_kind) return MX_ERR_NULL;
+    std::lock_guard<std::mutex> lk(g_prof.mu);
+    g_prof.on = false;
+    for (int k = 0; k < MX_KERNEL_KINDS; ++k) {
+        ms_per_kind[k] = 0.0;
+        launches_per_kind[k] = 0;
+    }
+    mx_status_t rc = MX_OK;
+    for (const ProfEntry &e : g_prof.entries) {
+        float ms = 0.f;
+        cudaError_t err = cudaEventSynchronize(e.b);
+        if (err == cudaSuccess) err = cudaEventElapsedTime(&ms, e.a, e.b);
+        if (err != cudaSuccess) rc = cuda_fail(err, "mx_profile_end");
+        if (e.kind >= 0 && e.kind < MX_KERNEL_KINDS) {
+            ms_per_kind[e.kind] += ms;
+            launches_per_kind[e.kind] += 1;
+        }
+        g_prof.pool.push_back(e);
+    }
+    g_prof.entries.clear();
+    return rc;
 }
 
 mx_status_t mx_poll_status(void *stream)

@@ -166,6 +166,34 @@ MX_API mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t
  */
 MX_API mx_status_t mx_poll_status(void *stream);
 
+/* ---- product for callers that cannot allocate (the paper has no counterpart) -----------------
+ *
+ * Some callers of this library have no way to obtain device memory at the point where they
+ * need the product: a plugin running inside a host application that owns the allocator and
+ * forbids cudaMalloc after start-up, a real-time loop with a no-allocation rule, or code that
+ * runs while another component holds the device's memory pool.  mx_gemm and mx_linear need a
+ * caller-provided workspace for the decoded bf16 operands; mx_gemm_static needs none.  It is
+ * the tensor-core product of mx_gemm_ex(..., MX_ALGO_TCGEN05) with that workspace replaced by
+ * a fixed array of MX_STATIC_SCRATCH_BYTES that is part of the library's device image (every
+ * GPU that loads the library holds these bytes until the process exits).  The caller still
+ * passes all inputs and the output; arguments, layouts and result are those of mx_gemm.
+ *
+ *  - Limit: 2*(M+N)*K bytes (each operand rounded up to 256) must fit in MX_STATIC_SCRATCH_BYTES,
+ *    e.g. M = N = K = 2048.  Larger problems return MX_ERR_WORKSPACE without launching
+ *    anything; mx_last_cuda_error() then holds the sizes.
+ *  - The call creates no buffer, event or handle: no cudaMalloc/cudaFree, no allocating library
+ *    routine.  The first call on a device looks up the array's device address and sets a kernel
+ *    attribute; make that first call before any stream capture begins.
+ *  - All calls on a device share the one array.  It keeps the previous call's bytes; the call
+ *    rewrites every byte it later reads, so nothing has to be cleared.  Two calls whose kernels
+ *    can overlap on the GPU (different streams, or different host threads) race on it: issue
+ *    them on one stream or order them with events. */
+#define MX_STATIC_SCRATCH_BYTES (32u << 20)
+MX_API mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                                  const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                                  int64_t M, int64_t N, int64_t K, const float *bias, float *y,
+                                  int64_t ldy, void *stream);
+
 /* ---- launch profile (benchmark support; the paper has no counterpart) ---------------------
  *
  * Between mx_profile_begin and mx_profile_end the library brackets each of its kernel launches

@@ -70,6 +70,8 @@ def _load() -> C.CDLL:
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
     L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_poll_status.argtypes = [vp]
+    L.mx_gemm_static.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp]
+    L.mx_gemm_static.restype = i32
     L.mx_profile_begin.argtypes = []
     L.mx_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
@@ -195,6 +197,26 @@ def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int
     _check(lib.mx_linear_ex(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant),
                             _ptr(w_exp), fw, N, _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
                             workspace.numel(), algo, _stream(stream)), "mx_linear")
+    return y
+
+
+MX_STATIC_SCRATCH_BYTES = 32 << 20
+
+
+def mx_gemm_static(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: int, N: int, K: int,
+                   bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None, stream=None):
+    """The tensor-core product for callers that must not allocate device memory: same arguments
+    and result as ``mx_gemm`` minus the workspace, which is a fixed array inside the library
+    (2*(M+N)*K bytes must fit in ``MX_STATIC_SCRATCH_BYTES``; ``MxError`` with
+    ``MX_ERR_WORKSPACE`` otherwise).  Pass ``y`` to keep this wrapper allocation-free as well."""
+    _need_cuda(a_mant, a_exp, w_mant, w_exp, bias, y)
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=a_mant.device)
+    rc = lib.mx_gemm_static(_ptr(a_mant), _ptr(a_exp), fa, _ptr(w_mant), _ptr(w_exp), fw, M, N, K,
+                            _ptr(bias), _ptr(y), y.stride(0), _stream(stream))
+    if rc == -5:
+        raise MxError(rc, "mx_gemm_static", lib.mx_last_cuda_error().decode())
+    _check(rc, "mx_gemm_static")
     return y
 
 

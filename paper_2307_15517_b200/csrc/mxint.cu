@@ -457,6 +457,80 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
                         workspace_bytes, MX_ALGO_AUTO, stream);
 }
 
+// ---- product without any allocation ---------------------------------------------------------
+// Scratch for mx_gemm_static: a fixed array in the library's device image.  In host code the
+// name below is only a handle for the runtime, never a device address; the address a kernel can
+// use comes from cudaGetSymbolAddress, looked up once per device with that device current.
+static __device__ __align__(256) unsigned char g_static_scratch[MX_STATIC_SCRATCH_BYTES];
+static void *g_static_scratch_addr[MAX_DEVICES] = {nullptr};
+
+mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                           const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t M,
+                           int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                           void *stream)
+{
+    mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
+    if (s != MX_OK) return s;
+    if (!a_exp) return MX_ERR_NULL;
+    const size_t need = tc_workspace(M, N, K);
+    if (need > (size_t)MX_STATIC_SCRATCH_BYTES) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error),
+                 "mx_gemm_static: M=%lld N=%lld K=%lld needs %zu bytes of scratch, the built-in array holds %zu",
+                 (long long)M, (long long)N, (long long)K, need, (size_t)MX_STATIC_SCRATCH_BYTES);
+        return MX_ERR_WORKSPACE;
+    }
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    int dev = 0;
+    MX_CUDA(cudaGetDevice(&dev));
+    if (!g_static_scratch_addr[dev]) {              // set-up: first call on this device
+        void *p = nullptr;
+        MX_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+        g_static_scratch_addr[dev] = p;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *scratch = static_cast<uint8_t *>(g_static_scratch_addr[dev]);
+    __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(scratch);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(scratch + round256((size_t)M * K * 2));
+    // Decode both operands into the scratch (every byte the product reads is written here first,
+    // so nothing left by an earlier call is ever observed), then the tensor-core product.
+    // Launches are issued directly: no event, no buffer and no handle is created on this path.
+    mx::dequantize_kernel<__nv_bfloat16><<<grid_for(M * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
+        static_cast<const uint8_t *>(a_mant), a_exp, M, K, fa.block, fa.elem_bits, a_hat, K);
+    MX_CUDA(cudaGetLastError());
+    mx::dequantize_kernel<__nv_bfloat16><<<grid_for(N * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
+        static_cast<const uint8_t *>(w_mant), w_exp, N, K, fw.block, fw.elem_bits, w_hat, K);
+    MX_CUDA(cudaGetLastError());
+    constexpr int BN = 128;
+    using Cfg = mx::TcCfg<BN>;
+    CUtensorMap tm_a, tm_w;
+    s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
+    if (s != MX_OK) return s;
+    if (!d->tc_attr_set[1]) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Cfg::SMEM_BYTES));
+        d->tc_attr_set[1] = true;
+    }
+    mx::TcParams p;
+    p.y = y;
+    p.bias = bias;
+    p.ldy = ldy;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
+    p.tiles_n = (int)((N + BN - 1) / BN);
+    p.status = d->status;
+    const int tiles = p.tiles_m * p.tiles_n;
+    mx::gemm_tc_kernel<BN><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
+        tm_a, tm_w, p);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 mx_status_t mx_profile_begin(void)
 {
     std::lock_guard<std::mutex> lk(g_prof.mu);

@@ -60,11 +60,17 @@ typedef enum { MX_F32 = 0, MX_BF16 = 1 } mx_dtype_t;
 
 /* Which kernel computes the block-scaled product. */
 typedef enum {
-    MX_ALGO_AUTO = 0,    /* skinny problems (M <= 16) -> weight-streaming kernel, else tensor cores */
+    MX_ALGO_AUTO = 0,    /* currently MX_ALGO_TCGEN05                                               */
     MX_ALGO_SIMT = 1,    /* CUDA-core kernel: exact integer block sums, blocks added in ascending
-                            order in fp32 (bit-reproducible; slow; needs no workspace)              */
-    MX_ALGO_TCGEN05 = 2, /* tcgen05/TMEM tensor-core kernel on exactly dequantized bf16 operands    */
-    MX_ALGO_STREAM = 3   /* weight-streaming kernel for M <= 16 (decode); needs no workspace        */
+                            order in fp32 (bit-reproducible; slow; mx_gemm needs no workspace)      */
+    MX_ALGO_TCGEN05 = 2, /* tcgen05/TMEM tensor-core kernel on exactly decoded bf16 operands; a
+                            separate pass decodes the packed weights into the workspace            */
+    MX_ALGO_STREAM = 3,  /* weight-streaming kernel for M <= 16 (decode)                            */
+    MX_ALGO_TCGEN05_FUSED = 4 /* the same tensor-core kernel with the packed weights decoded inside
+                            it by extra warps (no bf16 copy of W: workspace holds the activations
+                            only; needs K % 32 == 0 and a 2-byte aligned w_exp, else it falls back to
+                            the separate pass).  Saves memory, but the decode costs more issue slots
+                            than the MMA leaves free, so it is slower than MX_ALGO_TCGEN05.          */
 } mx_algo_t;
 
 /* The (B, e, m) tuple of Sec. 4.1. */
@@ -89,6 +95,10 @@ MX_API double mx_format_bits(mx_format_t f);
 /* Scratch bytes mx_gemm / mx_linear need for these sizes with MX_ALGO_AUTO (the maximum over
  * the kernels AUTO may pick).  The workspace must be 256-byte aligned. */
 MX_API size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw);
+
+/* The same for an explicitly named kernel (0 for an unknown algo or a bad format). */
+MX_API size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw,
+                                    mx_algo_t algo);
 
 MX_API const char *mx_status_string(mx_status_t s);
 

@@ -17,7 +17,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libmxint.so")
 
 MX_F32, MX_BF16 = 0, 1
-MX_ALGO_AUTO, MX_ALGO_SIMT, MX_ALGO_TCGEN05, MX_ALGO_STREAM = 0, 1, 2, 3
+MX_ALGO_AUTO, MX_ALGO_SIMT, MX_ALGO_TCGEN05, MX_ALGO_STREAM, MX_ALGO_TCGEN05_FUSED = 0, 1, 2, 3, 4
 
 STATUS_NAMES = {0: "MX_OK", -1: "MX_ERR_NULL", -2: "MX_ERR_SHAPE", -3: "MX_ERR_FORMAT",
                 -4: "MX_ERR_ALIGN", -5: "MX_ERR_WORKSPACE", -6: "MX_ERR_CUDA",
@@ -59,6 +59,8 @@ def _load() -> C.CDLL:
     L.mx_format_bits.restype = C.c_double
     L.mx_workspace_bytes.argtypes = [i64, i64, i64, F, F]
     L.mx_workspace_bytes.restype = sz
+    L.mx_workspace_bytes_ex.argtypes = [i64, i64, i64, F, F, i32]
+    L.mx_workspace_bytes_ex.restype = sz
     L.mx_status_string.argtypes = [i32]
     L.mx_status_string.restype = C.c_char_p
     L.mx_last_cuda_error.argtypes = []
@@ -130,6 +132,10 @@ def mx_workspace_bytes(M: int, N: int, K: int, fa: MxFormat, fw: MxFormat) -> in
     return int(lib.mx_workspace_bytes(M, N, K, fa, fw))
 
 
+def mx_workspace_bytes_ex(M: int, N: int, K: int, fa: MxFormat, fw: MxFormat, algo: int) -> int:
+    return int(lib.mx_workspace_bytes_ex(M, N, K, fa, fw, algo))
+
+
 def mx_status_string(status: int) -> str:
     return lib.mx_status_string(status).decode()
 
@@ -175,8 +181,8 @@ def mx_gemm(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: int, N:
     _need_cuda(a_mant, a_exp, w_mant, w_exp, bias, y, workspace)
     if y is None:
         y = torch.empty((M, N), dtype=torch.float32, device=a_mant.device)
-    if workspace is None and algo in (MX_ALGO_AUTO, MX_ALGO_TCGEN05):
-        workspace = alloc_workspace(mx_workspace_bytes(M, N, K, fa, fw), a_mant.device)
+    if workspace is None and algo != MX_ALGO_SIMT:
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, algo), a_mant.device)
     _check(lib.mx_gemm_ex(_ptr(a_mant), _ptr(a_exp), fa, _ptr(w_mant), _ptr(w_exp), fw, M, N, K,
                           _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
                           0 if workspace is None else workspace.numel(), algo, _stream(stream)),
@@ -193,7 +199,7 @@ def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int
     if y is None:
         y = torch.empty((M, N), dtype=torch.float32, device=x.device)
     if workspace is None:
-        workspace = alloc_workspace(mx_workspace_bytes(M, N, K, fa, fw), x.device)
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, algo), x.device)
     _check(lib.mx_linear_ex(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant),
                             _ptr(w_exp), fw, N, _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
                             workspace.numel(), algo, _stream(stream)), "mx_linear")

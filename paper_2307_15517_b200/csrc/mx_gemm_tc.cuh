@@ -22,13 +22,24 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cuda_bf16.h>
+
 #include "mx_ptx.cuh"
+#include "mx_quantize.cuh"
 
 namespace mx {
 
+// How the weight operand reaches shared memory.
+//   W_BF16   : already decoded to bf16 in global memory, fetched by TMA (192 threads)
+//   W_NIBBLE : packed 4-bit mantissas + exponent bytes, decoded in the kernel by 8 extra warps
+//   W_INT8   : int8 mantissas + exponent bytes, decoded in the kernel by 8 extra warps
+enum WMode { W_BF16 = 0, W_NIBBLE = 1, W_INT8 = 2 };
+
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                                  // bf16 elements per 128-byte row
-constexpr int TC_THREADS = 192;
+constexpr int TC_THREADS = 192;                            // producer, MMA, 4 epilogue warps
+// fused modes: 2 * BN extra weight-decode threads (one per tile row and half K step)
+constexpr int tc_threads(int bn, int wmode) { return wmode == 0 ? TC_THREADS : TC_THREADS + 2 * bn; }
 constexpr uint64_t TC_WAIT_LIMIT_NS = 400ull * 1000 * 1000; // 0.4 s per wait
 
 constexpr uint32_t STATUS_TIMEOUT_BIT = 1u;
@@ -50,14 +61,101 @@ struct TcParams {
     int M, N, K;
     int tiles_m, tiles_n;
     uint32_t *status;
+    // fused modes only: the packed weight operand
+    const uint8_t *w_mant;
+    const uint8_t *w_exp;
+    int w_bits;    // signed mantissa width of W
+    int block;     // 16 or 32
 };
 
-template <int BN>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+// ---- in-kernel decode of packed weights to the MMA's bf16 operand ---------------------------
+// bf16 bit pattern of the block scale 2^(E-(w-2)), both halves; e_field = Ebyte - (w-2) may be
+// <= 0 (bf16 subnormal scale) and Ebyte 255 marks a non-finite block (NaN scale).
+__device__ __forceinline__ uint32_t bf16x2_scale_bits(int ebyte, int w)
+{
+    const int e = ebyte - (w - 2);
+    uint32_t b = e > 0 ? ((uint32_t)e << 7) : (1u << (6 + e));
+    if (ebyte == 255) b = 0x7FC0u;
+    return b | (b << 16);
+}
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u)
+{
+    return *reinterpret_cast<__nv_bfloat162 *>(&u);
+}
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 v)
+{
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Slow but range-safe decode of 8 mantissas (used for blocks whose scale is within 2^8 of the
+// top of the bf16 range, where the fused multiply-add below would overflow its constant).
+__device__ __forceinline__ void decode8_safe(const int (&q)[8], int ebyte, int w, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 lo = __float2bfloat16_rn(decode_value(q[2 * i], ebyte, w));
+        const __nv_bfloat16 hi = __float2bfloat16_rn(decode_value(q[2 * i + 1], ebyte, w));
+        out[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+    }
+}
+
+// 8 two's-complement nibbles (k ascending from bit 0) -> 8 bf16 values q * s, exact, for a
+// power-of-two scale s (bf16x2, both halves) and c = -136 * s.
+// nibble ^ 8 = q + 8 in [0,15]; 0x4300 | that is the bf16 number 128 + (q + 8); one bf16x2 fma
+// gives (136 + q) * s - 136 * s = q * s with a single, exact rounding.
+__device__ __forceinline__ void decode8_nibbles(uint32_t p, __nv_bfloat162 s, __nv_bfloat162 c,
+                                                uint32_t (&out)[4])
+{
+    uint32_t v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t x = (((p >> (4 * i)) & 0x000F000Fu) ^ 0x00080008u) | 0x43004300u;   // (n_i, n_{i+4})
+        v[i] = as_u32(__hfma2(as_bf162(x), s, c));
+    }
+    out[0] = __byte_perm(v[0], v[1], 0x5410);      // (k0, k1)
+    out[1] = __byte_perm(v[2], v[3], 0x5410);      // (k2, k3)
+    out[2] = __byte_perm(v[0], v[1], 0x7632);      // (k4, k5)
+    out[3] = __byte_perm(v[2], v[3], 0x7632);      // (k6, k7)
+}
+// The fma constant -136*s must stay finite: scale field (Ebyte - (w-2)) at most 240.
+__device__ __forceinline__ bool nibble_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 240; }
+
+// 8 int8 mantissas (two words, k ascending) -> 8 bf16 values q * s, exact, for a power-of-two
+// fp32 scale s and c = -(2^23 + 128) * s.  byte ^ 0x80 = q + 128; 0x4B000000 | that is the float
+// 2^23 + (q + 128); one fp32 fma removes the offset and applies the scale.
+__device__ __forceinline__ void decode8_bytes(uint32_t p0, uint32_t p1, float s, float c, uint32_t (&out)[4])
+{
+    const uint32_t t0 = p0 ^ 0x80808080u, t1 = p1 ^ 0x80808080u;
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[i] = fmaf(__uint_as_float(__byte_perm(t0, 0x4B000000u, 0x7540 | i)), s, c);
+        f[4 + i] = fmaf(__uint_as_float(__byte_perm(t1, 0x4B000000u, 0x7540 | i)), s, c);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) out[i] = as_u32(__floats2bfloat162_rn(f[2 * i], f[2 * i + 1]));
+}
+__device__ __forceinline__ bool byte_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 225; }
+__device__ __forceinline__ float f32_scale(int ebyte, int w)
+{
+    const int e = ebyte - (w - 2);
+    return ebyte == 255 ? __uint_as_float(0x7FC00000u)
+                        : __uint_as_float(e > 0 ? ((uint32_t)e << 23) : (1u << (22 + e)));
+}
+
+// Raw bytes of one (row, half K-step) item: 32 mantissas and their exponent bytes.
+template <int WMODE> struct RawItem {
+    uint4 m[WMODE == W_INT8 ? 2 : 1];
+    uint32_t e;          // block 16: two exponent bytes (low = first block); block 32: one
+};                       // an item outside the matrix is all zero bytes and decodes to +0
+
+template <int BN, int WMODE>
+__global__ void __launch_bounds__(tc_threads(BN, WMODE), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                const TcParams p)
 {
     using Cfg = TcCfg<BN>;
+    constexpr bool FUSED = WMODE != W_BF16;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -75,7 +173,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
-            ptx::mbar_init(full_bar(s), 1);
+            // full: the TMA lane's expect_tx arrival (+ one arrival per decode warp in the fused modes)
+            ptx::mbar_init(full_bar(s), FUSED ? 1 + (2 * BN) / 32 : 1);
             ptx::mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -85,7 +184,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         *abort_flag = 0;
         ptx::fence_mbar_init();
         ptx::prefetch_tensormap(&tmap_a);
-        ptx::prefetch_tensormap(&tmap_w);
+        if (!FUSED) ptx::prefetch_tensormap(&tmap_w);
     }
     if (warp == 1) {
         ptx::tmem_alloc(ptx::smem_u32(tmem_slot), Cfg::TMEM_COLS);
@@ -111,10 +210,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         timed_out = true;
                         break;
                     }
-                    ptx::mbar_arrive_expect_tx(full_bar(s), Cfg::STAGE_BYTES);
+                    ptx::mbar_arrive_expect_tx(full_bar(s), FUSED ? Cfg::A_BYTES : Cfg::STAGE_BYTES);
                     const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
                     ptx::tma_load_2d(sa, &tmap_a, kb * TC_BK, m0, full_bar(s));
-                    ptx::tma_load_2d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, full_bar(s));
+                    if (!FUSED) ptx::tma_load_2d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, full_bar(s));
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -157,6 +256,137 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
         __syncwarp();
+    } else if (FUSED && warp >= TC_THREADS / 32) {
+        // ---- weight decode: packed mantissas + exponent bytes -> swizzled bf16 operand tile ----
+        // Thread d owns half h = d & 1 (32 of the 64 k of a K step) of tile row d >> 1.  Raw
+        // bytes are fetched three K steps ahead.
+        constexpr int ITEMS = 1;
+        const int d = threadIdx.x - TC_THREADS;
+        const int h = d & 1;
+        const int my_tiles = blockIdx.x < num_tiles ? (num_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+        const int total = my_tiles * kblocks;
+        const int64_t mant_ld = WMODE == W_NIBBLE ? (p.K >> 1) : p.K;      // bytes per row
+        const int nb_row = p.K / p.block;
+        const bool b16 = p.block == 16;
+        const int exp_shift = b16 ? 4 : 5;
+
+        // load cursor: walks (tile, K step) in the order the steps are consumed
+        int l_tile = blockIdx.x, l_kb = 0, l_i = 0;
+        const uint8_t *l_mant = nullptr, *l_exp = nullptr;
+        bool l_row_ok = false;
+        auto load = [&](RawItem<WMODE> (&r)[ITEMS]) {
+            r[0].e = 0;
+#pragma unroll
+            for (int j = 0; j < (WMODE == W_INT8 ? 2 : 1); ++j) r[0].m[j] = make_uint4(0, 0, 0, 0);
+            if (l_i >= total) return;
+            if (l_kb == 0) {                                   // new tile: this thread's weight row
+                const int n = (l_tile / p.tiles_m) * BN + (d >> 1);
+                l_row_ok = n < p.N;
+                l_mant = p.w_mant + (int64_t)n * mant_ld;
+                l_exp = p.w_exp + (int64_t)n * nb_row;
+            }
+            const int k0 = l_kb * TC_BK + h * 32;
+            if (l_row_ok && k0 < p.K) {
+                if (WMODE == W_NIBBLE) {
+                    r[0].m[0] = __ldg(reinterpret_cast<const uint4 *>(l_mant + (k0 >> 1)));
+                } else {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(l_mant + k0);
+                    r[0].m[0] = __ldg(src);
+                    r[0].m[WMODE == W_INT8 ? 1 : 0] = __ldg(src + 1);
+                }
+                const uint8_t *ep = l_exp + (k0 >> exp_shift);
+                r[0].e = b16 ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(ep)) : (uint32_t)__ldg(ep);
+            }
+            ++l_i;
+            if (++l_kb == kblocks) { l_kb = 0; l_tile += gridDim.x; }
+        };
+        auto decode_store = [&](int s, const RawItem<WMODE> (&r)[ITEMS]) {
+            uint8_t *sw = smem_gen + s * Cfg::STAGE_BYTES + Cfg::A_BYTES;
+#pragma unroll
+            for (int it = 0; it < ITEMS; ++it) {
+                const int row = d >> 1;
+                uint8_t *rowp = sw + (row >> 3) * 1024 + (row & 7) * 128;
+                const int e0 = (int)(r[it].e & 0xFF), e1 = b16 ? (int)((r[it].e >> 8) & 0xFF) : e0;
+                uint32_t o[4][4];
+                const uint32_t w8[8] = {r[it].m[0].x, r[it].m[0].y, r[it].m[0].z, r[it].m[0].w,
+                                        r[it].m[WMODE == W_INT8 ? 1 : 0].x, r[it].m[WMODE == W_INT8 ? 1 : 0].y,
+                                        r[it].m[WMODE == W_INT8 ? 1 : 0].z, r[it].m[WMODE == W_INT8 ? 1 : 0].w};
+                if (WMODE == W_NIBBLE) {
+                    if (nibble_fast_ok(e0, p.w_bits) && nibble_fast_ok(e1, p.w_bits)) {
+                        const __nv_bfloat162 m136 = as_bf162(0xC308C308u);       // -136
+                        const __nv_bfloat162 s0 = as_bf162(bf16x2_scale_bits(e0, p.w_bits));
+                        const __nv_bfloat162 s1 = as_bf162(bf16x2_scale_bits(e1, p.w_bits));
+                        const __nv_bfloat162 c0 = __hmul2(s0, m136), c1 = __hmul2(s1, m136);
+                        decode8_nibbles(w8[0], s0, c0, o[0]);
+                        decode8_nibbles(w8[1], s0, c0, o[1]);
+                        decode8_nibbles(w8[2], s1, c1, o[2]);
+                        decode8_nibbles(w8[3], s1, c1, o[3]);
+                    } else {                                    // scale near the top of the range
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            int q[8];
+#pragma unroll
+                            for (int i = 0; i < 8; ++i) q[i] = ((int)(w8[j] << (28 - 4 * i))) >> 28;
+                            decode8_safe(q, j < 2 ? e0 : e1, p.w_bits, o[j]);
+                        }
+                    }
+                } else {
+                    if (byte_fast_ok(e0, p.w_bits) && byte_fast_ok(e1, p.w_bits)) {
+                        const float s0 = f32_scale(e0, p.w_bits), s1 = f32_scale(e1, p.w_bits);
+                        const float c0 = -8388736.0f * s0, c1 = -8388736.0f * s1;   // -(2^23+128)*s, exact
+                        decode8_bytes(w8[0], w8[1], s0, c0, o[0]);
+                        decode8_bytes(w8[2], w8[3], s0, c0, o[1]);
+                        decode8_bytes(w8[4], w8[5], s1, c1, o[2]);
+                        decode8_bytes(w8[6], w8[7], s1, c1, o[3]);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            int q[8];
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                q[i] = ((int)(w8[2 * j] << (24 - 8 * i))) >> 24;
+                                q[4 + i] = ((int)(w8[2 * j + 1] << (24 - 8 * i))) >> 24;
+                            }
+                            decode8_safe(q, j < 2 ? e0 : e1, p.w_bits, o[j]);
+                        }
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const int chunk = (h * 4 + j) ^ (row & 7);          // 128-byte swizzle
+                    *reinterpret_cast<uint4 *>(rowp + chunk * 16) = make_uint4(o[j][0], o[j][1], o[j][2], o[j][3]);
+                }
+            }
+        };
+
+        // Three raw-byte buffers rotate without register moves: buffer b is decoded at steps
+        // b, b+3, b+6, ... and refilled for step +3 right after, so each global load has almost
+        // three K steps to land.
+        int s = 0;
+        uint32_t ph = 0;
+        auto step = [&](int i, RawItem<WMODE> (&buf)[ITEMS]) -> bool {
+            if (i >= total) return true;
+            bool ok = true;
+            if (lane == 0) ok = ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS);
+            if (!__shfl_sync(0xFFFFFFFFu, ok, 0)) return false;       // also orders the warp's stores
+            decode_store(s, buf);
+            ptx::fence_proxy_async_smem();          // generic-proxy stores -> visible to the MMA
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(full_bar(s));
+            if (++s == STAGES) { s = 0; ph ^= 1u; }
+            load(buf);
+            return true;
+        };
+        RawItem<WMODE> b0[ITEMS], b1[ITEMS], b2[ITEMS];
+        load(b0);
+        load(b1);
+        load(b2);
+        for (int i = 0; i < total; i += 3) {
+            if (!step(i, b0) || !step(i + 1, b1) || !step(i + 2, b2)) {
+                timed_out = true;
+                break;
+            }
+        }
     } else {
         const int quad = warp & 3;                          // TMEM lanes this warp may read
         int it = 0;

@@ -29,7 +29,7 @@ struct DeviceInfo {
     bool is_sm100 = false;
     int sm_count = SM_COUNT_FALLBACK;
     uint32_t *status = nullptr;
-    bool tc_attr_set[2] = {false, false};
+    bool tc_attr_set[2][3] = {{false, false, false}, {false, false, false}};
 };
 DeviceInfo g_dev[MAX_DEVICES];
 
@@ -197,22 +197,32 @@ mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, in
     return MX_OK;
 }
 
-template <int BN>
-mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
-                      int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d,
-                      cudaStream_t st)
+struct PackedW {                 // weight operand of the fused kernels (unused for W_BF16)
+    const uint8_t *mant = nullptr;
+    const uint8_t *exps = nullptr;
+    int bits = 0, block = 0;
+};
+
+template <int BN, int WMODE>
+mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
+                      int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                      DeviceInfo &d, cudaStream_t st)
 {
     using Cfg = mx::TcCfg<BN>;
     CUtensorMap tm_a, tm_w;
     mx_status_t s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
     if (s != MX_OK) return s;
-    s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
-    if (s != MX_OK) return s;
+    if (WMODE == mx::W_BF16) {
+        s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
+        if (s != MX_OK) return s;
+    } else {
+        tm_w = tm_a;                     // not read by the fused kernels
+    }
     constexpr int slot = BN == 256 ? 0 : 1;
-    if (!d.tc_attr_set[slot]) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Cfg::SMEM_BYTES));
-        d.tc_attr_set[slot] = true;
+    if (!d.tc_attr_set[slot][WMODE]) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN, WMODE>,
+                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES));
+        d.tc_attr_set[slot][WMODE] = true;
     }
     mx::TcParams p;
     p.y = y;
@@ -224,27 +234,65 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, in
     p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.status = d.status;
+    p.w_mant = pw.mant;
+    p.w_exp = pw.exps;
+    p.w_bits = pw.bits;
+    p.block = pw.block;
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
+    const int threads = mx::tc_threads(BN, WMODE);
     ProfScope prof(KIND_GEMM_TC, st);
-    mx::gemm_tc_kernel<BN><<<grid, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, p);
+    mx::gemm_tc_kernel<BN, WMODE><<<grid, threads, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, p);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
 
+bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
+{
+    const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256);
+    return tiles256 >= (int64_t)d.sm_count * 3 / 4;
+}
+
+// Pre-decoded bf16 weights (both operands fetched by TMA).
 mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
                    int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
 {
-    const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256);
-    if (tiles256 >= (int64_t)d.sm_count * 3 / 4)
-        return launch_tc<256>(a_hat, w_hat, M, N, K, bias, y, ldy, d, st);
-    return launch_tc<128>(a_hat, w_hat, M, N, K, bias, y, ldy, d, st);
+    const PackedW none;
+    if (wide_tile(M, N, d))
+        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, d, st);
+    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, d, st);
+}
+
+// Packed weights decoded inside the kernel.
+mx_status_t run_tc_fused(const __nv_bfloat16 *a_hat, const void *w_mant, const uint8_t *w_exp,
+                         const mx_format_t &fw, int64_t M, int64_t N, int64_t K, const float *bias,
+                         float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+{
+    PackedW pw;
+    pw.mant = static_cast<const uint8_t *>(w_mant);
+    pw.exps = w_exp;
+    pw.bits = fw.elem_bits;
+    pw.block = fw.block;
+    const bool wide = wide_tile(M, N, d);
+    if (fw.elem_bits <= 4) {
+        if (wide) return launch_tc<256, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+        return launch_tc<128, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+    }
+    if (wide) return launch_tc<256, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+    return launch_tc<128, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+}
+
+// The fused kernels read weight rows with 16-byte loads and exponent pairs with 2-byte loads.
+bool fused_ok(int64_t K, const uint8_t *w_exp)
+{
+    return (K % 32) == 0 && (reinterpret_cast<uintptr_t>(w_exp) & 1u) == 0;
 }
 
 size_t tc_workspace(int64_t M, int64_t N, int64_t K)
 {
     return round256((size_t)M * K * 2) + round256((size_t)N * K * 2);
 }
+size_t fused_workspace(int64_t M, int64_t K) { return round256((size_t)M * K * 2); }
 size_t packed_workspace(int64_t M, int64_t K, const mx_format_t &fa)
 {
     return round256(mx_mant_bytes(M, K, fa)) + round256(mx_exp_bytes(M, K, fa));
@@ -286,12 +334,23 @@ double mx_format_bits(mx_format_t f)
     return (double)f.exp_bits / ((double)f.block * (double)f.block_rows) + (double)(f.elem_bits - 1) + 1.0;
 }
 
-size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw)
+size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw,
+                             mx_algo_t algo)
 {
     if (!format_ok(fa) || !format_ok(fw) || M <= 0 || N <= 0 || K <= 0) return 0;
-    const size_t tc = tc_workspace(M, N, K);
-    const size_t pk = packed_workspace(M, K, fa);
-    return tc > pk ? tc : pk;
+    const size_t pk = packed_workspace(M, K, fa);          // mx_linear with the CUDA-core kernel
+    switch (algo) {
+    case MX_ALGO_SIMT: return pk;
+    case MX_ALGO_AUTO:
+    case MX_ALGO_TCGEN05: return tc_workspace(M, N, K);
+    case MX_ALGO_TCGEN05_FUSED: return (K % 32) == 0 ? fused_workspace(M, K) : tc_workspace(M, N, K);
+    default: return 0;
+    }
+}
+
+size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw)
+{
+    return mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_AUTO);
 }
 
 const char *mx_status_string(mx_status_t s)
@@ -372,7 +431,8 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
     if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
-    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05) return MX_ERR_FORMAT;
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
+        return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
@@ -386,13 +446,17 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         MX_CUDA(cudaGetLastError());
         return MX_OK;
     }
-    if (!workspace || workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0;
+    if (fused && !fused_ok(K, w_exp)) return MX_ERR_ALIGN;
+    if (!workspace || workspace_bytes < (fused ? fused_workspace(M, K) : tc_workspace(M, N, K)))
+        return MX_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
     __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
-    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
-                                                             round256((size_t)M * K * 2));
     s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
     if (s != MX_OK) return s;
+    if (fused) return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
+                                                             round256((size_t)M * K * 2));
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
@@ -418,7 +482,8 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
     if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
-    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05) return MX_ERR_FORMAT;
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
+        return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
@@ -436,13 +501,16 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         return mx_gemm_ex(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, nullptr, 0,
                           MX_ALGO_SIMT, stream);
     }
-    if (workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0;
+    if (fused && !fused_ok(K, w_exp)) return MX_ERR_ALIGN;
+    if (workspace_bytes < (fused ? fused_workspace(M, K) : tc_workspace(M, N, K))) return MX_ERR_WORKSPACE;
     __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
-    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     // the activations' mantissas and exponents go straight to the MMA operand form (exact bf16)
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
     s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
     if (s != MX_OK) return s;
+    if (fused) return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
@@ -509,10 +577,10 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     if (s != MX_OK) return s;
     s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
     if (s != MX_OK) return s;
-    if (!d->tc_attr_set[1]) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    if (!d->tc_attr_set[1][mx::W_BF16]) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN, mx::W_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)Cfg::SMEM_BYTES));
-        d->tc_attr_set[1] = true;
+        d->tc_attr_set[1][mx::W_BF16] = true;
     }
     mx::TcParams p;
     p.y = y;
@@ -524,8 +592,12 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.status = d->status;
+    p.w_mant = nullptr;
+    p.w_exp = nullptr;
+    p.w_bits = 0;
+    p.block = 0;
     const int tiles = p.tiles_m * p.tiles_n;
-    mx::gemm_tc_kernel<BN><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
+    mx::gemm_tc_kernel<BN, mx::W_BF16><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
         tm_a, tm_w, p);
     MX_CUDA(cudaGetLastError());
     return MX_OK;

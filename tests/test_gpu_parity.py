@@ -146,6 +146,7 @@ GEMM_SHAPES = [
     (200, 300, 320, 32, 8, 4),        # ragged M and N tails, K tail (320 = 5 * 64)
     (384, 640, 1024, 16, 8, 8),       # several tiles each way
     (130, 40, 96, 16, 6, 3),          # K not a multiple of 64, N below one tile
+    (70, 136, 112, 16, 4, 4),         # K % 32 != 0: the tensor-core path decodes W in a pre-pass
     (1, 256, 128, 32, 8, 4),          # a single row
     (257, 513, 2048, 32, 5, 2),
     (1536, 2560, 256, 16, 8, 4),      # 120 tiles of 128x256: the wide-tile kernel, multi-wave
@@ -164,9 +165,13 @@ def test_gemm_simt_matches_sequential_oracle_exactly(mxb, shape):
     _check_tol(y, y_ref, S)
 
 
+TC_ALGOS = ("MX_ALGO_TCGEN05", "MX_ALGO_TCGEN05_FUSED")
+
+
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
 @pytest.mark.parametrize("with_bias", (False, True))
-def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias):
+@pytest.mark.parametrize("algo", TC_ALGOS)
+def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias, algo):
     """Block exponents spread over 2^+-3 per operand (2^+-6 per product term), wider than any of
     the paper-shaped workloads produce within one row."""
     M, N, K, B, wa, ww = shape
@@ -176,7 +181,7 @@ def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias):
     ypad = torch.full((M, N + 8), -77.0, device="cuda")           # canary columns, ldy > N
     y = mxb.mx_gemm(_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)),
                     _dev(ew), mxb.MxFormat(B, ww), M, N, K, bias=None if bias is None else _dev(bias),
-                    y=ypad[:, :N], algo=mxb.MX_ALGO_TCGEN05)
+                    y=ypad[:, :N], algo=getattr(mxb, algo))
     assert mxb.mx_poll_status() == 0
     _check_tol(y, y_ref, S)
     assert (ypad[:, N:] == -77.0).all()
@@ -193,27 +198,60 @@ def test_gemm_tensor_core_adversarial_exponent_spread(mxb):
     y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
     args = (_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)), _dev(ew),
             mxb.MxFormat(B, ww), M, N, K)
-    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05).cpu().numpy().astype(np.float64)
-    assert mxb.mx_poll_status() == 0
     bound = -(-K // 16) * 17 * 2.0 ** -23 * S
-    assert (np.abs(y - y_ref) <= bound).all()
+    for algo in TC_ALGOS:
+        y = mxb.mx_gemm(*args, algo=getattr(mxb, algo)).cpu().numpy().astype(np.float64)
+        assert mxb.mx_poll_status() == 0
+        assert (np.abs(y - y_ref) <= bound).all()
     y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_SIMT)
     assert np.array_equal(y.cpu().numpy(), y_seq)
     _check_tol(y, y_ref, S)
 
 
-def test_gemm_one_hot_rows_expose_the_operand_layout(mxb):
+@pytest.mark.parametrize("algo", TC_ALGOS)
+@pytest.mark.parametrize("ww,B", [(4, 16), (4, 32), (3, 16), (8, 16), (6, 32)])
+def test_gemm_one_hot_rows_expose_the_operand_layout(mxb, algo, ww, B):
     """A = identity-like rows: Y must be the decoded weights, element for element (catches any
-    error in the swizzled shared-memory layout or the descriptors)."""
-    K, N, B = 256, 512, 16
+    error in the swizzled shared-memory layout, the descriptors or the in-kernel decode)."""
+    K, N = 256, 512
     x = np.zeros((K, K), np.float32)
     x[np.arange(K), np.arange(K)] = 1.0
     qa, ea, _ = orc.quantize(x, B, 8)
-    wt = synth.gaussian_weights(N, K, 3).numpy()
-    qw, ew, _ = orc.quantize(wt, B, 4)
-    y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, 4)),
-                    _dev(ew), mxb.MxFormat(B, 4), K, N, K, algo=mxb.MX_ALGO_TCGEN05)
-    assert np.array_equal(y.cpu().numpy().astype(np.float64), orc.dequantize(qw, ew, B, 4).T)
+    wt = synth.student_t_activations(N, K, 3).numpy()
+    qw, ew, _ = orc.quantize(wt, B, ww)
+    y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, ww)),
+                    _dev(ew), mxb.MxFormat(B, ww), K, N, K, algo=getattr(mxb, algo))
+    assert mxb.mx_poll_status() == 0
+    assert np.array_equal(y.cpu().numpy().astype(np.float64), orc.dequantize(qw, ew, B, ww).T)
+
+
+@pytest.mark.parametrize("ww", (2, 4, 8))
+def test_gemm_decode_is_exact_over_the_exponent_range(mxb, ww):
+    """Raw weights with every mantissa value (incl. -2^(w-1)) and exponent bytes from 0 (bf16
+    subnormal scale) to 253; one-hot activations of value
+    2^-60 / 1 / 2^60 keep each output inside fp32, so Y must equal the decoded weight times that
+    power of two exactly."""
+    K, N, B = 128, 256, 16
+    lo = -(2 ** (ww - 1))
+    qw = synth.random_ints((N, K), lo, -lo - 1, 11).numpy()
+    # byte 254 is left out: -2^(w-1) * 2^(127-(w-2)) = -2^128 is outside bf16 and fp32 (the
+    # quantizer never emits -2^(w-1), so it cannot occur in quantized data)
+    ew = synth.random_bytes((N, K // B), 0, 253, 12).numpy()
+    ew[:, 0] = np.arange(N) % 254                      # every byte value 0..253 appears
+    x = np.zeros((K, K), np.float32)
+    x[np.arange(K), np.arange(K)] = 1.0
+    qa, ea0, _ = orc.quantize(x, B, 8)
+    want = orc.dequantize(qw, ew, B, ww).T             # [K, N]
+    for shift in (-60, 0, 60):
+        ea = (ea0.astype(np.int32) + shift * (ea0 > 0)).astype(np.uint8)
+        ref = np.ldexp(want, shift).astype(np.float32)  # rounds only where fp32 itself must
+        finite = np.isfinite(ref) & (np.abs(np.ldexp(want, shift)) >= 2.0 ** -126)
+        for algo in TC_ALGOS:
+            y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, ww)),
+                            _dev(ew), mxb.MxFormat(B, ww), K, N, K, algo=getattr(mxb, algo)).cpu().numpy()
+            assert mxb.mx_poll_status() == 0
+            assert finite.sum() > 1000
+            assert np.array_equal(y[finite], ref[finite]), (ww, shift, algo)
 
 
 def test_gemm_nonfinite_blocks_poison_their_outputs(mxb):
@@ -222,7 +260,7 @@ def test_gemm_nonfinite_blocks_poison_their_outputs(mxb):
     ea[3, 2] = 255
     ew[200, 7] = 255
     y_ref, _, _ = orc.gemm(qa, ea, 8, qw, ew, 4, B)
-    for algo in (mxb.MX_ALGO_SIMT, mxb.MX_ALGO_TCGEN05):
+    for algo in (mxb.MX_ALGO_SIMT, mxb.MX_ALGO_TCGEN05_FUSED, mxb.MX_ALGO_TCGEN05):
         y = mxb.mx_gemm(_dev(orc.pack(qa, 8)), _dev(ea), mxb.MxFormat(B, 8), _dev(orc.pack(qw, 4)),
                         _dev(ew), mxb.MxFormat(B, 4), M, N, K, algo=algo).cpu().numpy()
         assert np.array_equal(np.isnan(y), np.isnan(y_ref))
@@ -239,11 +277,13 @@ def test_linear_single_layer_config(mxb):
     qw, ew, _ = orc.quantize(wt.numpy(), spec.block, spec.w_wgt)
     y_ref, y_seq, S = orc.gemm(qa, ea, spec.w_act, qw, ew, spec.w_wgt, spec.block)
     w_mant, w_exp = mxb.mx_quantize(wt.cuda(), fw)
-    y_tc = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N, algo=mxb.MX_ALGO_TCGEN05)
+    y_tc = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N)
+    y_fused = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N, algo=mxb.MX_ALGO_TCGEN05_FUSED)
     y_simt = mxb.mx_linear(x.cuda(), fa, w_mant, w_exp, fw, spec.N, algo=mxb.MX_ALGO_SIMT)
     assert mxb.mx_poll_status() == 0
     assert np.array_equal(y_simt.cpu().numpy(), y_seq)
     _check_tol(y_tc, y_ref, S)
+    _check_tol(y_fused, y_ref, S)
 
 
 @pytest.mark.parametrize("case", [(16, 8, 4), (32, 4, 4), (32, 6, 3), (16, 2, 8)])

@@ -50,7 +50,12 @@ def test_size_helpers_match_eq1(mxb):
     assert total == int(4096 * 4096 * 0.53125)
     assert mxb.mx_mant_bytes(4, 40, F(16, 4)) == 0             # K not a multiple of the block
     assert mxb.mx_mant_bytes(4, 64, F(8, 4)) == 0              # unsupported block
-    assert mxb.mx_workspace_bytes(128, 768, 768, F(16, 4), F(16, 4)) >= 2 * (128 + 768) * 768
+    f4 = F(16, 4)
+    assert mxb.mx_workspace_bytes(128, 768, 768, f4, f4) >= 2 * (128 + 768) * 768   # both operands as bf16
+    fused = mxb.mx_workspace_bytes_ex(128, 768, 768, f4, f4, mxb.MX_ALGO_TCGEN05_FUSED)
+    assert 2 * 128 * 768 <= fused < 2 * (128 + 768) * 768                           # activations only
+    assert mxb.mx_workspace_bytes_ex(128, 768, 112, f4, f4, mxb.MX_ALGO_TCGEN05_FUSED) >= 2 * (128 + 768) * 112
+    assert mxb.mx_workspace_bytes_ex(128, 768, 768, f4, f4, 99) == 0
 
 
 def test_status_strings(mxb):

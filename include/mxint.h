@@ -60,12 +60,14 @@ typedef enum { MX_F32 = 0, MX_BF16 = 1 } mx_dtype_t;
 
 /* Which kernel computes the block-scaled product. */
 typedef enum {
-    MX_ALGO_AUTO = 0,    /* currently MX_ALGO_TCGEN05                                               */
+    MX_ALGO_AUTO = 0,    /* mx_linear with M <= 16 and a streamable format: MX_ALGO_STREAM; everything
+                            else: MX_ALGO_TCGEN05                                                  */
     MX_ALGO_SIMT = 1,    /* CUDA-core kernel: exact integer block sums, blocks added in ascending
                             order in fp32 (bit-reproducible; slow; mx_gemm needs no workspace)      */
     MX_ALGO_TCGEN05 = 2, /* tcgen05/TMEM tensor-core kernel on exactly decoded bf16 operands; a
                             separate pass decodes the packed weights into the workspace            */
-    MX_ALGO_STREAM = 3,  /* weight-streaming kernel for M <= 16 (decode)                            */
+    MX_ALGO_STREAM = 3,  /* weight-streaming kernel for M <= 16 (decode), mx_linear only; see
+                            mx_linear_grouped for its restrictions                                 */
     MX_ALGO_TCGEN05_FUSED = 4 /* the same tensor-core kernel with the packed weights decoded inside
                             it by extra warps (no bf16 copy of W: workspace holds the activations
                             only; needs K % 32 == 0 and a 2-byte aligned w_exp, else it falls back to
@@ -164,6 +166,38 @@ MX_API mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t
                          mx_format_t fa, const void *w_mant, const uint8_t *w_exp,
                          mx_format_t fw, int64_t N, const float *bias, float *y, int64_t ldy,
                          void *workspace, size_t workspace_bytes, mx_algo_t algo, void *stream);
+
+/* ---- decode: a few tokens against many weight matrices (weights streamed once) ---------- */
+
+/* One layer of a grouped call: the arguments of mx_linear. */
+typedef struct {
+    const void *x;          /* [M, K] activations of `dt`, leading dimension ldx (elements)     */
+    mx_dtype_t dt;
+    int64_t M, K, ldx;      /* M = number of tokens, 1..16                                      */
+    mx_format_t fa;         /* activation format (block 32)                                     */
+    const void *w_mant;     /* [N, K/2] packed weights (elem_bits <= 4, block 32)               */
+    const uint8_t *w_exp;   /* [N, K/32], 4-byte aligned                                        */
+    mx_format_t fw;
+    int64_t N;
+    const float *bias;      /* nullable, [N]                                                    */
+    float *y;               /* [M, ldy]                                                         */
+    int64_t ldy;
+} mx_linear_args_t;
+
+/*
+ * Runs n_layers independent MXInt linear layers with few tokens each (decode) in ONE kernel
+ * launch: every distinct activation tensor is quantized to its format once (layers that name
+ * the same x, shape and format share it), then a single persistent kernel streams all weight
+ * matrices from HBM exactly once.  Per output the integer block sums are exact and the blocks are
+ * added in fp32, in ascending order whenever there are enough weight rows to fill the GPU without
+ * cutting K (always the case for tens of layers).  `layers` is HOST memory (read during the
+ * call).  Restrictions: M <= 16, both formats block 32, weights elem_bits <= 4, K % 128 == 0,
+ * M*K small enough to stage in shared memory (M = 16: K <= 18432); otherwise MX_ERR_SHAPE /
+ * MX_ERR_FORMAT.  mx_linear(_ex) with MX_ALGO_STREAM is the one-layer form of this call.
+ */
+MX_API size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, int32_t n_layers);
+MX_API mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers,
+                                     void *workspace, size_t workspace_bytes, void *stream);
 
 /* ---- device status --------------------------------------------------------------------- */
 

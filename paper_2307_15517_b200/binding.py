@@ -36,6 +36,14 @@ class MxFormat(C.Structure):
         return "MxFormat(block=%d, elem_bits=%d)" % (self.block, self.elem_bits)
 
 
+class MxLinearArgs(C.Structure):
+    """One layer of ``mx_linear_grouped`` (mirrors ``mx_linear_args_t``)."""
+    _fields_ = [("x", C.c_void_p), ("dt", C.c_int), ("M", C.c_int64), ("K", C.c_int64),
+                ("ldx", C.c_int64), ("fa", MxFormat), ("w_mant", C.c_void_p), ("w_exp", C.c_void_p),
+                ("fw", MxFormat), ("N", C.c_int64), ("bias", C.c_void_p), ("y", C.c_void_p),
+                ("ldy", C.c_int64)]
+
+
 class MxError(RuntimeError):
     def __init__(self, status: int, where: str, detail: str = ""):
         self.status = status
@@ -72,6 +80,10 @@ def _load() -> C.CDLL:
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
     L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_poll_status.argtypes = [vp]
+    L.mx_linear_grouped_workspace_bytes.argtypes = [C.POINTER(MxLinearArgs), i32]
+    L.mx_linear_grouped_workspace_bytes.restype = sz
+    L.mx_linear_grouped.argtypes = [C.POINTER(MxLinearArgs), i32, vp, sz, vp]
+    L.mx_linear_grouped.restype = i32
     L.mx_gemm_static.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp]
     L.mx_gemm_static.restype = i32
     L.mx_profile_begin.argtypes = []
@@ -204,6 +216,36 @@ def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int
                             _ptr(w_exp), fw, N, _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
                             workspace.numel(), algo, _stream(stream)), "mx_linear")
     return y
+
+
+def make_linear_args(layers):
+    """layers: iterable of dicts with x, fa, w_mant, w_exp, fw, N, y and optionally bias.
+    Returns a ctypes array of ``MxLinearArgs`` (host memory) for ``mx_linear_grouped``."""
+    layers = list(layers)
+    arr = (MxLinearArgs * len(layers))()
+    for a, L in zip(arr, layers):
+        x, y = L["x"], L["y"]
+        _need_cuda(x, y, L["w_mant"], L["w_exp"], L.get("bias"))
+        assert x.stride(1) == 1
+        a.x, a.dt, a.M, a.K, a.ldx, a.fa = x.data_ptr(), _dtype_code(x), x.shape[0], x.shape[1], x.stride(0), L["fa"]
+        a.w_mant, a.w_exp, a.fw, a.N = L["w_mant"].data_ptr(), L["w_exp"].data_ptr(), L["fw"], L["N"]
+        bias = L.get("bias")
+        a.bias = None if bias is None else bias.data_ptr()
+        a.y, a.ldy = y.data_ptr(), y.stride(0)
+    return arr
+
+
+def mx_linear_grouped_workspace_bytes(args) -> int:
+    return int(lib.mx_linear_grouped_workspace_bytes(args, len(args)))
+
+
+def mx_linear_grouped(args, workspace: Optional[torch.Tensor] = None, stream=None):
+    """args: the array made by ``make_linear_args``.  One launch over all layers (decode)."""
+    if workspace is None:
+        workspace = alloc_workspace(mx_linear_grouped_workspace_bytes(args))
+    _check(lib.mx_linear_grouped(args, len(args), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "mx_linear_grouped")
+    return workspace
 
 
 MX_STATIC_SCRATCH_BYTES = 32 << 20

@@ -68,81 +68,6 @@ struct TcParams {
     int block;     // 16 or 32
 };
 
-// ---- in-kernel decode of packed weights to the MMA's bf16 operand ---------------------------
-// bf16 bit pattern of the block scale 2^(E-(w-2)), both halves; e_field = Ebyte - (w-2) may be
-// <= 0 (bf16 subnormal scale) and Ebyte 255 marks a non-finite block (NaN scale).
-__device__ __forceinline__ uint32_t bf16x2_scale_bits(int ebyte, int w)
-{
-    const int e = ebyte - (w - 2);
-    uint32_t b = e > 0 ? ((uint32_t)e << 7) : (1u << (6 + e));
-    if (ebyte == 255) b = 0x7FC0u;
-    return b | (b << 16);
-}
-__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u)
-{
-    return *reinterpret_cast<__nv_bfloat162 *>(&u);
-}
-__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 v)
-{
-    return *reinterpret_cast<uint32_t *>(&v);
-}
-
-// Slow but range-safe decode of 8 mantissas (used for blocks whose scale is within 2^8 of the
-// top of the bf16 range, where the fused multiply-add below would overflow its constant).
-__device__ __forceinline__ void decode8_safe(const int (&q)[8], int ebyte, int w, uint32_t (&out)[4])
-{
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const __nv_bfloat16 lo = __float2bfloat16_rn(decode_value(q[2 * i], ebyte, w));
-        const __nv_bfloat16 hi = __float2bfloat16_rn(decode_value(q[2 * i + 1], ebyte, w));
-        out[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
-    }
-}
-
-// 8 two's-complement nibbles (k ascending from bit 0) -> 8 bf16 values q * s, exact, for a
-// power-of-two scale s (bf16x2, both halves) and c = -136 * s.
-// nibble ^ 8 = q + 8 in [0,15]; 0x4300 | that is the bf16 number 128 + (q + 8); one bf16x2 fma
-// gives (136 + q) * s - 136 * s = q * s with a single, exact rounding.
-__device__ __forceinline__ void decode8_nibbles(uint32_t p, __nv_bfloat162 s, __nv_bfloat162 c,
-                                                uint32_t (&out)[4])
-{
-    uint32_t v[4];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const uint32_t x = (((p >> (4 * i)) & 0x000F000Fu) ^ 0x00080008u) | 0x43004300u;   // (n_i, n_{i+4})
-        v[i] = as_u32(__hfma2(as_bf162(x), s, c));
-    }
-    out[0] = __byte_perm(v[0], v[1], 0x5410);      // (k0, k1)
-    out[1] = __byte_perm(v[2], v[3], 0x5410);      // (k2, k3)
-    out[2] = __byte_perm(v[0], v[1], 0x7632);      // (k4, k5)
-    out[3] = __byte_perm(v[2], v[3], 0x7632);      // (k6, k7)
-}
-// The fma constant -136*s must stay finite: scale field (Ebyte - (w-2)) at most 240.
-__device__ __forceinline__ bool nibble_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 240; }
-
-// 8 int8 mantissas (two words, k ascending) -> 8 bf16 values q * s, exact, for a power-of-two
-// fp32 scale s and c = -(2^23 + 128) * s.  byte ^ 0x80 = q + 128; 0x4B000000 | that is the float
-// 2^23 + (q + 128); one fp32 fma removes the offset and applies the scale.
-__device__ __forceinline__ void decode8_bytes(uint32_t p0, uint32_t p1, float s, float c, uint32_t (&out)[4])
-{
-    const uint32_t t0 = p0 ^ 0x80808080u, t1 = p1 ^ 0x80808080u;
-    float f[8];
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        f[i] = fmaf(__uint_as_float(__byte_perm(t0, 0x4B000000u, 0x7540 | i)), s, c);
-        f[4 + i] = fmaf(__uint_as_float(__byte_perm(t1, 0x4B000000u, 0x7540 | i)), s, c);
-    }
-#pragma unroll
-    for (int i = 0; i < 4; ++i) out[i] = as_u32(__floats2bfloat162_rn(f[2 * i], f[2 * i + 1]));
-}
-__device__ __forceinline__ bool byte_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 225; }
-__device__ __forceinline__ float f32_scale(int ebyte, int w)
-{
-    const int e = ebyte - (w - 2);
-    return ebyte == 255 ? __uint_as_float(0x7FC00000u)
-                        : __uint_as_float(e > 0 ? ((uint32_t)e << 23) : (1u << (22 + e)));
-}
-
 // Raw bytes of one (row, half K-step) item: 32 mantissas and their exponent bytes.
 template <int WMODE> struct RawItem {
     uint4 m[WMODE == W_INT8 ? 2 : 1];

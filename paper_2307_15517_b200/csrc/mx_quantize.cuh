@@ -35,6 +35,81 @@ __device__ __forceinline__ int encode_value(float x, float inv_pow2_E, float pow
     return max(-qmax, min(qmax, q));
 }
 
+// ---- fast exact decode of packed mantissas to bf16 (the MMA operand form) -------------------
+// bf16 bit pattern of the block scale 2^(E-(w-2)), both halves; e_field = Ebyte - (w-2) may be
+// <= 0 (bf16 subnormal scale) and Ebyte 255 marks a non-finite block (NaN scale).
+__device__ __forceinline__ uint32_t bf16x2_scale_bits(int ebyte, int w)
+{
+    const int e = ebyte - (w - 2);
+    uint32_t b = e > 0 ? ((uint32_t)e << 7) : (1u << (6 + e));
+    if (ebyte == 255) b = 0x7FC0u;
+    return b | (b << 16);
+}
+__device__ __forceinline__ __nv_bfloat162 as_bf162(uint32_t u)
+{
+    return *reinterpret_cast<__nv_bfloat162 *>(&u);
+}
+__device__ __forceinline__ uint32_t as_u32(__nv_bfloat162 v)
+{
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Slow but range-safe decode of 8 mantissas (used for blocks whose scale is within 2^8 of the
+// top of the bf16 range, where the fused multiply-add below would overflow its constant).
+__device__ __forceinline__ void decode8_safe(const int (&q)[8], int ebyte, int w, uint32_t (&out)[4])
+{
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const __nv_bfloat16 lo = __float2bfloat16_rn(decode_value(q[2 * i], ebyte, w));
+        const __nv_bfloat16 hi = __float2bfloat16_rn(decode_value(q[2 * i + 1], ebyte, w));
+        out[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+    }
+}
+
+// 8 two's-complement nibbles (k ascending from bit 0) -> 8 bf16 values q * s, exact, for a
+// power-of-two scale s (bf16x2, both halves) and c = -136 * s.
+// nibble ^ 8 = q + 8 in [0,15]; 0x4300 | that is the bf16 number 128 + (q + 8); one bf16x2 fma
+// gives (136 + q) * s - 136 * s = q * s with a single, exact rounding.
+__device__ __forceinline__ void decode8_nibbles(uint32_t p, __nv_bfloat162 s, __nv_bfloat162 c,
+                                                uint32_t (&out)[4])
+{
+    uint32_t v[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t x = (((p >> (4 * i)) & 0x000F000Fu) ^ 0x00080008u) | 0x43004300u;   // (n_i, n_{i+4})
+        v[i] = as_u32(__hfma2(as_bf162(x), s, c));
+    }
+    out[0] = __byte_perm(v[0], v[1], 0x5410);      // (k0, k1)
+    out[1] = __byte_perm(v[2], v[3], 0x5410);      // (k2, k3)
+    out[2] = __byte_perm(v[0], v[1], 0x7632);      // (k4, k5)
+    out[3] = __byte_perm(v[2], v[3], 0x7632);      // (k6, k7)
+}
+// The fma constant -136*s must stay finite: scale field (Ebyte - (w-2)) at most 240.
+__device__ __forceinline__ bool nibble_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 240; }
+
+// 8 int8 mantissas (two words, k ascending) -> 8 bf16 values q * s, exact, for a power-of-two
+// fp32 scale s and c = -(2^23 + 128) * s.  byte ^ 0x80 = q + 128; 0x4B000000 | that is the float
+// 2^23 + (q + 128); one fp32 fma removes the offset and applies the scale.
+__device__ __forceinline__ void decode8_bytes(uint32_t p0, uint32_t p1, float s, float c, uint32_t (&out)[4])
+{
+    const uint32_t t0 = p0 ^ 0x80808080u, t1 = p1 ^ 0x80808080u;
+    float f[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        f[i] = fmaf(__uint_as_float(__byte_perm(t0, 0x4B000000u, 0x7540 | i)), s, c);
+        f[4 + i] = fmaf(__uint_as_float(__byte_perm(t1, 0x4B000000u, 0x7540 | i)), s, c);
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) out[i] = as_u32(__floats2bfloat162_rn(f[2 * i], f[2 * i + 1]));
+}
+__device__ __forceinline__ bool byte_fast_ok(int ebyte, int w) { return ebyte == 255 || ebyte - (w - 2) <= 225; }
+__device__ __forceinline__ float f32_scale(int ebyte, int w)
+{
+    const int e = ebyte - (w - 2);
+    return ebyte == 255 ? __uint_as_float(0x7FC00000u)
+                        : __uint_as_float(e > 0 ? ((uint32_t)e << 23) : (1u << (22 + e)));
+}
+
 struct QuantOut {
     uint8_t *mant;        // packed mantissas (nullable)
     uint8_t *exps;        // exponent bytes (nullable together with mant)
@@ -47,8 +122,8 @@ template <typename InT> struct Load8;
 template <> struct Load8<float> {
     static __device__ __forceinline__ void run(const float *p, float (&v)[8])
     {
-        const float4 a = __ldg(reinterpret_cast<const float4 *>(p));
-        const float4 b = __ldg(reinterpret_cast<const float4 *>(p) + 1);
+        const float4 a = __ldcs(reinterpret_cast<const float4 *>(p));      // read once: evict first
+        const float4 b = __ldcs(reinterpret_cast<const float4 *>(p) + 1);
         v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
         v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
     }
@@ -56,7 +131,7 @@ template <> struct Load8<float> {
 template <> struct Load8<__nv_bfloat16> {
     static __device__ __forceinline__ void run(const __nv_bfloat16 *p, float (&v)[8])
     {
-        const uint4 a = __ldg(reinterpret_cast<const uint4 *>(p));
+        const uint4 a = __ldcs(reinterpret_cast<const uint4 *>(p));
         const uint32_t u[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
@@ -67,73 +142,111 @@ template <> struct Load8<__nv_bfloat16> {
 };
 
 // rows x K, rows contiguous along K with leading dimension ldx.  BLOCK in {16, 32}.
-template <typename InT, int BLOCK>
+//
+// Work item of a warp = (row, segment of 256 elements): lane l owns the 8 elements starting at
+// k = segment*256 + 8*l, so a warp reads 1 KB of fp32 contiguously and the index arithmetic is
+// paid once per 256 elements.  UNROLL items per warp and iteration have all their loads issued
+// before any arithmetic (UNROLL * 32 bytes in flight per thread).
+//
+// Rounding without a conversion instruction: with v = x * 2^-E * 2^(w-2) clamped to
+// [-qmax, qmax], t = v + (1.5 * 2^23 + OFF) is rounded by the adder to an integer (nearest,
+// ties to even -- OFF is even, so ties fall on even q), and the low bits of t's pattern hold
+// q + OFF >= 1.  OFF = 8 (nibble container) or 128 (byte container) keeps every field
+// non-negative, so the fields of a word can be summed with shifts and the two's-complement
+// form restored by one XOR with 0x88888888 / 0x80808080.
+template <typename InT, int BLOCK, int UNROLL>
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w,
                      QuantOut out)
 {
     constexpr int LANES = BLOCK / 8;                    // lanes sharing one block
-    const int64_t chunks_per_row = K >> 3;
-    const int64_t total = rows * chunks_per_row;
-    const int qmax = (1 << (w - 1)) - 1;
-    const float pow2_wm2 = (float)(1 << (w - 2));
+    const int lane = threadIdx.x & 31;
+    const int cpr = (int)(K >> 3);                      // 8-element chunks per row
+    const int segs = (cpr + 31) >> 5;                   // 256-element segments per row
+    const int64_t items = rows * segs;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const bool nibble = w <= 4;
-    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
-    // trip count is uniform over the warp so that the shuffles below see all 32 lanes
-    const int64_t first = (int64_t)blockIdx.x * blockDim.x + (threadIdx.x & ~31);
-    for (int64_t base = first; base < total; base += stride) {
-        const int64_t c = base + (threadIdx.x & 31);
-        const bool live = c < total;
-        const int64_t row = live ? c / chunks_per_row : 0;
-        const int64_t kc = live ? c - row * chunks_per_row : 0;
-        float v[8];
-        if (live) {
-            Load8<InT>::run(x + row * ldx + kc * 8, v);
-        } else {
+    const float qmaxf = (float)((1 << (w - 1)) - 1);
+    const float pow2_wm2 = (float)(1 << (w - 2));
+    const float off = nibble ? 8.f : 128.f;
+    const float magic = 12582912.f + off;               // 1.5 * 2^23 + OFF
+    const uint32_t magic_bits = __float_as_uint(magic);
+    const bool leader = (lane & (LANES - 1)) == 0;
+
+    for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {   // warp-uniform trip count
+        float v[UNROLL][8];
+        int64_t row[UNROLL];
+        int kc[UNROLL];
+        bool live[UNROLL];
 #pragma unroll
-            for (int i = 0; i < 8; ++i) v[i] = 0.f;
-        }
-        uint32_t amax = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) amax = max(amax, __float_as_uint(v[i]) & 0x7FFFFFFFu);
-#pragma unroll
-        for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
-        const int ebyte = (int)(amax >> 23);            // 255 <=> an Inf or NaN in the block
-        const bool bad = ebyte == 255;
-        const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
-        int q[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) q[i] = bad ? 0 : encode_value(v[i], inv_pow2_E, pow2_wm2, qmax);
-        if (!live) continue;
-        const bool leader = (threadIdx.x & (LANES - 1)) == 0;
-        if (out.mant) {
-            if (nibble) {
-                uint32_t p = 0;
-#pragma unroll
-                for (int i = 0; i < 8; ++i) p |= ((uint32_t)q[i] & 0xFu) << (4 * i);
-                *reinterpret_cast<uint32_t *>(out.mant + row * (K >> 1) + kc * 4) = p;
+        for (int u = 0; u < UNROLL; ++u) {
+            const int64_t it = it0 + u * n_warps;
+            const bool ok = it < items;
+            row[u] = ok ? it / segs : 0;
+            kc[u] = (int)(ok ? it - row[u] * segs : 0) * 32 + lane;
+            live[u] = ok && kc[u] < cpr;
+            if (live[u]) {
+                Load8<InT>::run(x + row[u] * ldx + (int64_t)kc[u] * 8, v[u]);
             } else {
-                uint2 p;
-                p.x = ((uint32_t)q[0] & 0xFF) | (((uint32_t)q[1] & 0xFF) << 8) |
-                      (((uint32_t)q[2] & 0xFF) << 16) | ((uint32_t)q[3] << 24);
-                p.y = ((uint32_t)q[4] & 0xFF) | (((uint32_t)q[5] & 0xFF) << 8) |
-                      (((uint32_t)q[6] & 0xFF) << 16) | ((uint32_t)q[7] << 24);
-                *reinterpret_cast<uint2 *>(out.mant + row * K + kc * 8) = p;
-            }
-            if (leader) out.exps[row * (K / BLOCK) + kc / LANES] = (uint8_t)ebyte;
-        }
-        if (out.xhat) {
-            uint32_t h[4];
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const __nv_bfloat16 lo = __float2bfloat16_rn(decode_value(q[2 * i], ebyte, w));
-                const __nv_bfloat16 hi = __float2bfloat16_rn(decode_value(q[2 * i + 1], ebyte, w));
-                h[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
+                for (int i = 0; i < 8; ++i) v[u][i] = 0.f;
             }
-            *reinterpret_cast<uint4 *>(out.xhat + row * out.ld_xhat + kc * 8) =
-                make_uint4(h[0], h[1], h[2], h[3]);
         }
-        if (bad && leader && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            uint32_t amax = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) amax = max(amax, __float_as_uint(v[u][i]) & 0x7FFFFFFFu);
+#pragma unroll
+            for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+            if (!live[u]) continue;
+            const int ebyte = (int)(amax >> 23);            // 255 <=> an Inf or NaN in the block
+            const bool bad = ebyte == 255;
+            const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
+            float t[8];                                     // magic + OFF + q, exactly
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const float s = (v[u][i] * inv_pow2_E) * pow2_wm2;          // exact scaling
+                t[i] = fminf(fmaxf(s, -qmaxf), qmaxf) + magic;              // clamp, then round
+            }
+            if (out.mant) {
+                if (nibble) {
+                    uint32_t p = 0;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) p += (__float_as_uint(t[i]) - magic_bits + 8u) << (4 * i);
+                    p ^= 0x88888888u;
+                    *reinterpret_cast<uint32_t *>(out.mant + row[u] * (K >> 1) + (int64_t)kc[u] * 4) = bad ? 0u : p;
+                } else {
+                    uint2 p = make_uint2(0, 0);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        p.x += (__float_as_uint(t[i]) - magic_bits + 128u) << (8 * i);
+                        p.y += (__float_as_uint(t[4 + i]) - magic_bits + 128u) << (8 * i);
+                    }
+                    p.x ^= 0x80808080u;
+                    p.y ^= 0x80808080u;
+                    if (bad) p = make_uint2(0, 0);
+                    *reinterpret_cast<uint2 *>(out.mant + row[u] * K + (int64_t)kc[u] * 8) = p;
+                }
+                if (leader) out.exps[row[u] * (K / BLOCK) + kc[u] / LANES] = (uint8_t)ebyte;
+            }
+            if (out.xhat) {
+                // decoded value q * 2^-(w-2) * 2^E as bf16 (exact: <= 7 significant bits)
+                const float dec_small = small_neg_pow2(w), dec_big = pow2_from_biased(bad ? 127 : ebyte);
+                uint32_t h[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float lo = ((t[2 * i] - magic) * dec_small) * dec_big;
+                    const float hi = ((t[2 * i + 1] - magic) * dec_small) * dec_big;
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
+                    h[i] = bad ? 0x7FC07FC0u : *reinterpret_cast<const uint32_t *>(&pr);
+                }
+                *reinterpret_cast<uint4 *>(out.xhat + row[u] * out.ld_xhat + (int64_t)kc[u] * 8) =
+                    make_uint4(h[0], h[1], h[2], h[3]);
+            }
+            if (bad && leader && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+        }
     }
 }
 
@@ -217,6 +330,104 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
                 h[i] = (uint32_t)__bfloat16_as_ushort(lo) | ((uint32_t)__bfloat16_as_ushort(hi) << 16);
             }
             *reinterpret_cast<uint4 *>(o) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+    }
+}
+
+
+// (mant, exps) -> bf16 operand, 32 elements per thread: one 16-byte (nibbles) or two 16-byte
+// (int8) loads, four 16-byte stores.  Work item of a warp = (row, segment of 1024 elements);
+// UNROLL items per warp are loaded before any is decoded so that several loads are in flight.
+// Requires K % 32 == 0 (rows of the packed tensor 16-byte aligned).  Element order and values
+// are those of dequantize_kernel.
+template <bool NIBBLE, int UNROLL>
+__global__ void __launch_bounds__(256)
+decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps, int64_t rows,
+                   int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out)
+{
+    const int lane = threadIdx.x & 31;
+    const int ipr = (int)(K >> 5);                      // 32-element items per row
+    const int segs = (ipr + 31) >> 5;
+    const int64_t items = rows * segs;
+    const bool b16 = block == 16;
+    const int exp_shift = b16 ? 4 : 5;
+    const int64_t nb_row = K >> exp_shift;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {
+        uint4 m[UNROLL][NIBBLE ? 1 : 2];
+        uint32_t e[UNROLL];
+        int64_t row[UNROLL], kc[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int64_t it = it0 + u * n_warps;
+            const bool ok = it < items;
+            const int64_t r = ok ? it / segs : 0;
+            kc[u] = (ok ? it - r * segs : 0) * 32 + lane;
+            row[u] = (ok && kc[u] < ipr) ? r : -1;
+            if (row[u] >= 0) {
+                if (NIBBLE) {
+                    m[u][0] = __ldcs(reinterpret_cast<const uint4 *>(mant + row[u] * (K >> 1) + kc[u] * 16));
+                } else {
+                    const uint4 *src = reinterpret_cast<const uint4 *>(mant + row[u] * K + kc[u] * 32);
+                    m[u][0] = __ldcs(src);
+                    m[u][NIBBLE ? 0 : 1] = __ldcs(src + 1);
+                }
+                const uint8_t *ep = exps + row[u] * nb_row + ((kc[u] * 32) >> exp_shift);
+                e[u] = b16 ? (uint32_t)ep[0] | ((uint32_t)ep[1] << 8) : (uint32_t)ep[0];
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            if (row[u] < 0) continue;
+            const int e0 = (int)(e[u] & 0xFF), e1 = b16 ? (int)((e[u] >> 8) & 0xFF) : e0;
+            const uint32_t w8[8] = {m[u][0].x, m[u][0].y, m[u][0].z, m[u][0].w,
+                                    m[u][NIBBLE ? 0 : 1].x, m[u][NIBBLE ? 0 : 1].y,
+                                    m[u][NIBBLE ? 0 : 1].z, m[u][NIBBLE ? 0 : 1].w};
+            uint32_t o[4][4];
+            if (NIBBLE) {
+                if (nibble_fast_ok(e0, w) && nibble_fast_ok(e1, w)) {
+                    const __nv_bfloat162 m136 = as_bf162(0xC308C308u);       // -136
+                    const __nv_bfloat162 s0 = as_bf162(bf16x2_scale_bits(e0, w));
+                    const __nv_bfloat162 s1 = as_bf162(bf16x2_scale_bits(e1, w));
+                    const __nv_bfloat162 c0 = __hmul2(s0, m136), c1 = __hmul2(s1, m136);
+                    decode8_nibbles(w8[0], s0, c0, o[0]);
+                    decode8_nibbles(w8[1], s0, c0, o[1]);
+                    decode8_nibbles(w8[2], s1, c1, o[2]);
+                    decode8_nibbles(w8[3], s1, c1, o[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        int q[8];
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) q[i] = ((int)(w8[j] << (28 - 4 * i))) >> 28;
+                        decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
+                    }
+                }
+            } else {
+                if (byte_fast_ok(e0, w) && byte_fast_ok(e1, w)) {
+                    const float s0 = f32_scale(e0, w), s1 = f32_scale(e1, w);
+                    const float c0 = -8388736.0f * s0, c1 = -8388736.0f * s1;
+                    decode8_bytes(w8[0], w8[1], s0, c0, o[0]);
+                    decode8_bytes(w8[2], w8[3], s0, c0, o[1]);
+                    decode8_bytes(w8[4], w8[5], s1, c1, o[2]);
+                    decode8_bytes(w8[6], w8[7], s1, c1, o[3]);
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        int q[8];
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            q[i] = ((int)(w8[2 * j] << (24 - 8 * i))) >> 24;
+                            q[4 + i] = ((int)(w8[2 * j + 1] << (24 - 8 * i))) >> 24;
+                        }
+                        decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
+                    }
+                }
+            }
+            uint4 *dst = reinterpret_cast<uint4 *>(out + row[u] * ld_out + kc[u] * 32);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[j][0], o[j][1], o[j][2], o[j][3]);
         }
     }
 }

@@ -13,6 +13,7 @@
 #include "../../include/mxint.h"
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
+#include "mx_gemv_stream.cuh"
 #include "mx_quantize.cuh"
 
 namespace {
@@ -30,6 +31,7 @@ struct DeviceInfo {
     int sm_count = SM_COUNT_FALLBACK;
     uint32_t *status = nullptr;
     bool tc_attr_set[2][3] = {{false, false, false}, {false, false, false}};
+    bool stream_attr_set[2] = {false, false};
 };
 DeviceInfo g_dev[MAX_DEVICES];
 
@@ -137,12 +139,13 @@ mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t 
 {
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
-    const int grid = grid_for(chunks, 256, d.sm_count, 16);
+    constexpr int UNROLL = 2;
+    const int grid = grid_for((chunks + UNROLL - 1) / UNROLL, 256, d.sm_count, 8);
     ProfScope prof(KIND_QUANTIZE, st);
     if (f.block == 16)
-        mx::quantize_rows_kernel<InT, 16><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+        mx::quantize_rows_kernel<InT, 16, UNROLL><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
     else
-        mx::quantize_rows_kernel<InT, 32><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+        mx::quantize_rows_kernel<InT, 32, UNROLL><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -163,8 +166,19 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
     ProfScope prof(KIND_DEQUANTIZE, st);
-    mx::dequantize_kernel<__nv_bfloat16><<<grid_for(chunks, 256, d.sm_count, 16), 256, 0, st>>>(
-        static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits, out, ld);
+    const uint8_t *m = static_cast<const uint8_t *>(mant);
+    if ((K % 32) == 0) {                    // 32 elements per thread, 16-byte loads and stores
+        constexpr int UNROLL = 2;
+        const int64_t items = rows * (K / 32);
+        const int grid = grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, 8);
+        if (f.elem_bits <= 4)
+            mx::decode_bf16_kernel<true, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld);
+        else
+            mx::decode_bf16_kernel<false, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld);
+    } else {
+        mx::dequantize_kernel<__nv_bfloat16><<<grid_for(chunks, 256, d.sm_count, 16), 256, 0, st>>>(
+            m, exps, rows, K, f.block, f.elem_bits, out, ld);
+    }
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -311,6 +325,38 @@ mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t 
     return MX_OK;
 }
 
+// ---- decode: few tokens, weights streamed once ------------------------------------------------
+bool stream_layer_ok(const mx_linear_args_t &a)
+{
+    return a.M >= 1 && a.M <= 16 && a.fw.block == 32 && a.fa.block == 32 && a.fw.elem_bits <= 4 &&
+           (a.K % 128) == 0;
+}
+
+size_t stream_act_bytes(const mx_linear_args_t &a)
+{
+    return round256(mx_mant_bytes(a.M, a.K, a.fa)) + round256(mx_exp_bytes(a.M, a.K, a.fa));
+}
+
+bool same_activation(const mx_linear_args_t &a, const mx_linear_args_t &b)
+{
+    return a.x == b.x && a.dt == b.dt && a.M == b.M && a.K == b.K && a.ldx == b.ldx &&
+           a.fa.block == b.fa.block && a.fa.elem_bits == b.fa.elem_bits;
+}
+
+template <int NT>
+mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, DeviceInfo &d, cudaStream_t st)
+{
+    if (!d.stream_attr_set[NT - 1]) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemv_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     227 * 1024));
+        d.stream_attr_set[NT - 1] = true;
+    }
+    ProfScope prof(KIND_GEMM_STREAM, st);
+    mx::gemv_stream_kernel<NT><<<grid, mx::STREAM_THREADS, smem, st>>>(sp);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -341,7 +387,13 @@ size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx
     const size_t pk = packed_workspace(M, K, fa);          // mx_linear with the CUDA-core kernel
     switch (algo) {
     case MX_ALGO_SIMT: return pk;
-    case MX_ALGO_AUTO:
+    case MX_ALGO_STREAM: return round256(sizeof(mx::StreamLayer)) + round256(mx_mant_bytes(M, K, fa)) +
+                                round256(mx_exp_bytes(M, K, fa));
+    case MX_ALGO_AUTO: {            // mx_linear may stream (M <= 16), mx_gemm uses the tensor cores
+        const size_t st = mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_STREAM);
+        const size_t tc = tc_workspace(M, N, K);
+        return st > tc ? st : tc;
+    }
     case MX_ALGO_TCGEN05: return tc_workspace(M, N, K);
     case MX_ALGO_TCGEN05_FUSED: return (K % 32) == 0 ? fused_workspace(M, K) : tc_workspace(M, N, K);
     default: return 0;
@@ -481,7 +533,13 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
-    if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
+    mx_linear_args_t one;
+    one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
+    one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = ldy;
+    if (algo == MX_ALGO_AUTO)
+        algo = (stream_layer_ok(one) && (reinterpret_cast<uintptr_t>(w_exp) & 3u) == 0) ? MX_ALGO_STREAM
+                                                                                     : MX_ALGO_TCGEN05;
+    if (algo == MX_ALGO_STREAM) return mx_linear_grouped(&one, 1, workspace, workspace_bytes, stream);
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
@@ -523,6 +581,108 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
 {
     return mx_linear_ex(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, y, ldy, workspace,
                         workspace_bytes, MX_ALGO_AUTO, stream);
+}
+
+// ---- decode: few tokens, weights streamed once ------------------------------------------------
+size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, int32_t n_layers)
+{
+    if (!layers || n_layers <= 0) return 0;
+    size_t total = round256((size_t)n_layers * sizeof(mx::StreamLayer));
+    for (int i = 0; i < n_layers; ++i) {
+        if (!format_ok(layers[i].fa) || !format_ok(layers[i].fw)) return 0;
+        bool seen = false;
+        for (int j = 0; j < i && !seen; ++j) seen = same_activation(layers[i], layers[j]);
+        if (!seen) total += stream_act_bytes(layers[i]);
+    }
+    return total;
+}
+
+mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, void *workspace,
+                              size_t workspace_bytes, void *stream)
+{
+    if (!layers) return MX_ERR_NULL;
+    if (n_layers <= 0) return MX_ERR_SHAPE;
+    int max_t = 0, max_nb = 0, min_nb = INT32_MAX;
+    for (int i = 0; i < n_layers; ++i) {
+        const mx_linear_args_t &a = layers[i];
+        mx_status_t s = check_gemm_args(a.x, nullptr, a.fa, a.w_mant, a.w_exp, a.fw, a.M, a.N, a.K, a.bias,
+                                        a.y, a.ldy);
+        if (s != MX_OK) return s;
+        if (a.dt != MX_F32 && a.dt != MX_BF16) return MX_ERR_FORMAT;
+        if (a.ldx < a.K) return MX_ERR_SHAPE;
+        if ((a.ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(a.w_exp) & 3u) != 0) return MX_ERR_ALIGN;
+        if (!stream_layer_ok(a)) return a.M > 16 || (a.K % 128) != 0 ? MX_ERR_SHAPE : MX_ERR_FORMAT;
+        max_t = a.M > max_t ? (int)a.M : max_t;
+        const int nb = (int)(a.K / 32);
+        max_nb = nb > max_nb ? nb : max_nb;
+        min_nb = nb < min_nb ? nb : min_nb;
+    }
+    const size_t need = mx_linear_grouped_workspace_bytes(layers, n_layers);
+    if (!workspace || workspace_bytes < need) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    const int nt = max_t > 8 ? 2 : 1;
+    const size_t smem = nt == 2 ? mx::stream_smem_bytes<2>(max_nb) : mx::stream_smem_bytes<1>(max_nb);
+    if (smem > 227u * 1024u) return MX_ERR_SHAPE;                  // tokens x K too large to stage
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+
+    // quantize every distinct activation tensor once, build the device layer table
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    size_t off = round256((size_t)n_layers * sizeof(mx::StreamLayer));
+    std::vector<mx::StreamLayer> table((size_t)n_layers);
+    std::vector<uint8_t *> act_ptr((size_t)n_layers, nullptr);
+    int total_tiles = 0;
+    for (int i = 0; i < n_layers; ++i) {
+        const mx_linear_args_t &a = layers[i];
+        for (int j = 0; j < i && !act_ptr[i]; ++j)
+            if (same_activation(a, layers[j])) act_ptr[i] = act_ptr[j];
+        if (!act_ptr[i]) {
+            act_ptr[i] = ws + off;
+            off += stream_act_bytes(a);
+            mx::QuantOut out{act_ptr[i], act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa)), nullptr, 0, nullptr};
+            s = quantize_rows_any(a.x, a.dt, a.M, a.K, a.ldx, a.fa, out, *d, st);
+            if (s != MX_OK) return s;
+        }
+        mx::StreamLayer &L = table[i];
+        L.w_mant = static_cast<const uint8_t *>(a.w_mant);
+        L.w_exp = a.w_exp;
+        L.a_mant = act_ptr[i];
+        L.a_exp = act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa));
+        L.bias = a.bias;
+        L.y = a.y;
+        L.ldy = a.ldy;
+        L.N = (int)a.N;
+        L.K = (int)a.K;
+        L.T = (int)a.M;
+        L.a_bits = a.fa.elem_bits;
+        L.w_bits = a.fw.elem_bits;
+        L.tile_begin = total_tiles;
+        L.n_tiles = (int)((a.N + 15) / 16);
+        total_tiles += L.n_tiles;
+    }
+    MX_CUDA(cudaMemcpyAsync(ws, table.data(), (size_t)n_layers * sizeof(mx::StreamLayer),
+                            cudaMemcpyHostToDevice, st));
+
+    const int ctas_per_sm = (int)((227u * 1024u) / (smem + 1024)) < 4 ? (int)((227u * 1024u) / (smem + 1024)) : 4;
+    const int max_ctas = d->sm_count * (ctas_per_sm < 1 ? 1 : ctas_per_sm);
+    int split = 1;                         // cut K over warps only when row tiles alone cannot fill the GPU
+    if (total_tiles < max_ctas * 8) {
+        if (min_nb % 16 == 0 && total_tiles * 4 >= max_ctas * 2) split = 4;
+        else if (min_nb % 32 == 0) split = 8;
+        else if (min_nb % 16 == 0) split = 4;
+        else if (min_nb % 8 == 0) split = 2;
+    }
+    const int rounds = (total_tiles + (8 / split) - 1) / (8 / split);
+    const int grid = rounds < max_ctas ? rounds : max_ctas;
+    mx::StreamParams sp;
+    sp.layers = reinterpret_cast<const mx::StreamLayer *>(ws);
+    sp.n_layers = n_layers;
+    sp.total_tiles = total_tiles;
+    sp.split = split;
+    sp.max_nb = max_nb;
+    return nt == 2 ? launch_stream<2>(sp, smem, grid, *d, st) : launch_stream<1>(sp, smem, grid, *d, st);
 }
 
 // ---- product without any allocation ---------------------------------------------------------

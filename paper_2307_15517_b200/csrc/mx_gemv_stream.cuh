@@ -23,9 +23,11 @@
 // contiguous pieces handled by consecutive warps of one CTA and summed in piece order through
 // shared memory (deterministic, but no longer the ascending single chain).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "mx_ptx.cuh"
 #include "mx_quantize.cuh"
 
 namespace mx {
@@ -50,16 +52,49 @@ struct StreamParams {
     int total_tiles;
     int split;                   // 1, 2, 4 or 8
     int max_nb;                  // largest K/32 over the layers (sizes the shared-memory arrays)
+    uint32_t *status;            // device status word (bit 0: a bounded wait expired)
+    const CUtensorMap *tmaps;    // BULK: one map per layer over its packed mantissas [N, K/2] bytes,
+                                 // box 128 bytes x 16 rows, 128-byte swizzle (device memory)
 };
 
-constexpr int STREAM_THREADS = 256;
+// Geometry of the two variants.
+//   register variant (BULK = false): 8 warps, each lane prefetches four blocks' words with 32-bit
+//     loads; works for any K % 128 == 0.
+//   TMA variant (BULK = true): 16 warps; every warp owns a ring of STAGES shared-memory stages,
+//     each filled by ONE tiled TMA load of 16 rows x 8 blocks of mantissas (128 bytes per row,
+//     128-byte swizzle so that the 8 rows one fragment load touches fall into different banks),
+//     plus a per-tile 1-D bulk copy of its rows' exponent bytes; global data never passes through
+//     the load/store data pipe.  Needs K % 512 == 0 and 16-byte aligned exponent arrays.
+template <int NT, bool BULK> struct StreamCfg {
+    static constexpr int WARPS = BULK ? 16 : 8;
+    static constexpr int THREADS = WARPS * 32;
+    static constexpr int STAGES = NT == 1 ? 4 : 3;
+    static constexpr int CH = BULK ? 8 : 4;                        // blocks of 32 per step and row
+    static constexpr int STAGE_BYTES = 16 * CH * 16;               // 2048: 16 rows x 128 bytes
+    static constexpr uint32_t STAGE_TX = STAGE_BYTES;
+    static constexpr int TP = NT * 8;                              // padded token count
+    static constexpr size_t tokens_bytes(int max_nb) { return (size_t)max_nb * TP * (32 + 8); }
+    static constexpr size_t red_bytes() { return (size_t)WARPS * NT * 4 * 32 * 4; }
+    static constexpr size_t exp_pitch(int max_nb) { return (size_t)max_nb + 16; }
+    static constexpr size_t smem_bytes(int max_nb)
+    {
+        return tokens_bytes(max_nb) + red_bytes() +
+               (BULK ? 1024 /* stage alignment */ + (size_t)WARPS * STAGES * STAGE_BYTES +
+                           (size_t)WARPS * 16 * exp_pitch(max_nb) + (size_t)WARPS * (STAGES + 1) * 8 + 16
+                     : 0);
+    }
+};
+constexpr uint64_t STREAM_WAIT_LIMIT_NS = 400ull * 1000 * 1000;
 constexpr int STREAM_MAGIC_INT = 0x4B400000;        // bit pattern of 1.5 * 2^23
 constexpr float STREAM_MAGIC = 12582912.0f;
 
-template <int NT> constexpr size_t stream_smem_bytes(int max_nb)
+// 1-D bulk copy global -> shared (no tensor map, no multicast); 16-byte aligned, size % 16 == 0.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void *src, uint32_t bytes, uint32_t bar)
 {
-    // operand words + token scales + accumulator seeds + split-K exchange
-    return (size_t)max_nb * NT * 8 * (4 * 8 + 4 + 4) + 8 * NT * 4 * 32 * 4;
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :
+                 : "r"(dst_smem), "l"((uint64_t)src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 __device__ __forceinline__ void mma_u8s8_m16n8k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
@@ -73,20 +108,39 @@ __device__ __forceinline__ void mma_u8s8_m16n8k32(int (&d)[4], uint32_t a0, uint
 }
 
 // NT = number of 8-token column tiles (1: T <= 8, 2: T <= 16).
-template <int NT>
-__global__ void __launch_bounds__(STREAM_THREADS)
+template <int NT, bool BULK>
+__global__ void __launch_bounds__(StreamCfg<NT, BULK>::THREADS, 1)
 gemv_stream_kernel(const StreamParams p)
 {
+    using Cfg = StreamCfg<NT, BULK>;
+    constexpr int TP = Cfg::TP, WARPS = Cfg::WARPS, STAGES = Cfg::STAGES, CH = Cfg::CH;
     extern __shared__ __align__(16) uint8_t smem[];
-    constexpr int TP = NT * 8;                                   // padded token count
     uint2 *sB = reinterpret_cast<uint2 *>(smem);                 // [nb][TP][4]: (even-k word, odd-k word)
-    float *sSa = reinterpret_cast<float *>(smem + (size_t)p.max_nb * TP * 32);   // [nb][TP]
-    int *sC = reinterpret_cast<int *>(sSa + (size_t)p.max_nb * TP);              // [nb][TP]
-    float *sRed = reinterpret_cast<float *>(sC + (size_t)p.max_nb * TP);         // [8][NT][4][32]
+    // [nb][TP] pairs (accumulator seed, token scale); the token scale also carries the weights'
+    // binary point 2^-(ww-2), so the weight scale below is the plain 2^(Ew-127)
+    uint2 *sCS = reinterpret_cast<uint2 *>(smem + (size_t)p.max_nb * TP * 32);
+    float *sRed = reinterpret_cast<float *>(sCS + (size_t)p.max_nb * TP);        // [WARPS][NT][4][32]
+    // [WARPS][STAGES] swizzled weight stages, 1024-byte aligned (BULK)
+    uint8_t *sStage = reinterpret_cast<uint8_t *>(sRed + WARPS * NT * 4 * 32);
+    sStage += (1024u - (ptx::smem_u32(sStage) & 1023u)) & 1023u;
+    uint8_t *sExp = sStage + WARPS * STAGES * Cfg::STAGE_BYTES;                  // [WARPS][16][max_nb + 16]
+    const int exp_pitch = p.max_nb + 16;
+    uint8_t *sBar = sExp + (size_t)WARPS * 16 * exp_pitch;                       // [WARPS][STAGES + 1] mbarriers
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(sBar + WARPS * (STAGES + 1) * 8);
+    uint32_t phase_bits = 0;                  // parity per barrier of this warp (bit STAGES: exponents)
+    bool timed_out = false;
+    if (BULK) {
+        if (threadIdx.x == 0) {
+            for (int i = 0; i < WARPS * (STAGES + 1); ++i) ptx::mbar_init(ptx::smem_u32(sBar) + 8 * i, 1);
+            *abort_flag = 0;
+            ptx::fence_mbar_init();
+        }
+        __syncthreads();
+    }
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
-    const int S = p.split, TPR = 8 / S;                          // row tiles per round of the CTA
+    const int S = p.split, TPR = WARPS / S;                      // row tiles per round of the CTA
 
     const int per = (p.total_tiles + gridDim.x - 1) / gridDim.x;
     int tile_lo = blockIdx.x * per;
@@ -101,7 +155,7 @@ gemv_stream_kernel(const StreamParams p)
 
         // ---- stage this layer's tokens: operand words, block scales, accumulator seeds ----
         __syncthreads();                                         // previous layer fully consumed
-        for (int i = threadIdx.x; i < nb * TP * 4; i += STREAM_THREADS) {
+        for (int i = threadIdx.x; i < nb * TP * 4; i += Cfg::THREADS) {
             const int tq = i & 3, tok = (i >> 2) % TP, b = (i >> 2) / TP;
             uint32_t lo = 0, hi = 0;                             // 8 mantissas, k = 32b + 8tq ..
             if (tok < L.T) {
@@ -127,8 +181,8 @@ gemv_stream_kernel(const StreamParams p)
             sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);         // the 4 groups of one block
             if (tq == 0) {
                 const int eb = tok < L.T ? (int)__ldg(L.a_exp + (int64_t)tok * nb + b) : 0;
-                sSa[b * TP + tok] = f32_scale(eb, L.a_bits);
-                sC[b * TP + tok] = STREAM_MAGIC_INT - 8 * sum;
+                const float sa = f32_scale(eb, L.a_bits) * small_neg_pow2(L.w_bits);     // exact
+                sCS[b * TP + tok] = make_uint2((uint32_t)(STREAM_MAGIC_INT - 8 * sum), __float_as_uint(sa));
             }
         }
         __syncthreads();
@@ -150,38 +204,34 @@ gemv_stream_kernel(const StreamParams p)
                 const uint8_t *eA = L.w_exp + (int64_t)rowA * nb;
                 const uint8_t *eB = L.w_exp + (int64_t)rowB * nb;
                 const int b_lo = (nb / S) * s, b_hi = b_lo + nb / S;       // nb % (4*S) == 0
-                uint32_t wa[4], wb[4], ea, eb;
-                auto fetch = [&](int b, uint32_t (&xa)[4], uint32_t (&xb)[4], uint32_t &xea, uint32_t &xeb) {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        xa[j] = __ldcs(reinterpret_cast<const uint32_t *>(mA + (b + j) * 16));
-                        xb[j] = __ldcs(reinterpret_cast<const uint32_t *>(mB + (b + j) * 16));
-                    }
-                    xea = __ldcs(reinterpret_cast<const uint32_t *>(eA + b));
-                    xeb = __ldcs(reinterpret_cast<const uint32_t *>(eB + b));
+                struct Regs { uint32_t a[4], b[4], ea, eb; };
+                // any exponent byte >= 226: 1.5*2^23 * 2^(E-127) is not finite, take two steps there
+                auto near_top = [](uint32_t v) {
+                    return ((v & 0x80808080u) & ((v & 0x7F7F7F7Fu) + 0x1E1E1E1Eu)) != 0u;
                 };
-                fetch(b_lo, wa, wb, ea, eb);
-                for (int b = b_lo; b < b_hi; b += 4) {
-                    uint32_t na[4], nbw[4], nea = 0, neb = 0;
-                    if (b + 4 < b_hi) fetch(b + 4, na, nbw, nea, neb);
+                auto compute = [&](int b, const Regs &r) {
+                    const bool top = near_top(r.ea) || near_top(r.eb);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const int ebA = (int)((ea >> (8 * j)) & 0xFF), ebB = (int)((eb >> (8 * j)) & 0xFF);
-                        const float swA = f32_scale(ebA, L.w_bits), swB = f32_scale(ebB, L.w_bits);
-                        // far up the exponent range 1.5*2^23 * scale is not finite: take two steps there
-                        const bool top = (ebA > 225 && ebA != 255) || (ebB > 225 && ebB != 255);
+                        // weight scale 2^(E-127): exponent byte moved into the float's exponent field
+                        // (byte 0 -> the subnormal 2^-127, byte 255 -> Inf, which turns the block into NaN)
+                        const uint32_t fa = j == 3 ? (r.ea >> 1) : (r.ea << (23 - 8 * j));
+                        const uint32_t fb = j == 3 ? (r.eb >> 1) : (r.eb << (23 - 8 * j));
+                        const float swA = __uint_as_float(max(fa & 0x7F800000u, 0x00400000u));
+                        const float swB = __uint_as_float(max(fb & 0x7F800000u, 0x00400000u));
                         const float mwA = -STREAM_MAGIC * swA, mwB = -STREAM_MAGIC * swB;
-                        const uint32_t pa = wa[j] ^ 0x88888888u, pb = wb[j] ^ 0x88888888u;
-                        const uint32_t a0 = pa & 0x0F0F0F0Fu, a2 = (pa >> 4) & 0x0F0F0F0Fu;
-                        const uint32_t a1 = pb & 0x0F0F0F0Fu, a3 = (pb >> 4) & 0x0F0F0F0Fu;
+                        const uint32_t a0 = (r.a[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
+                        const uint32_t a2 = ((r.a[j] >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
+                        const uint32_t a1 = (r.b[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
+                        const uint32_t a3 = ((r.b[j] >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
                         const int blk = b + j;
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
                             const uint2 bf = sB[(blk * TP + n * 8 + g) * 4 + t];
-                            const int2 c = *reinterpret_cast<const int2 *>(&sC[blk * TP + n * 8 + 2 * t]);
-                            const float2 sa = *reinterpret_cast<const float2 *>(&sSa[blk * TP + n * 8 + 2 * t]);
+                            const uint4 cs = *reinterpret_cast<const uint4 *>(&sCS[blk * TP + n * 8 + 2 * t]);
+                            const float sa0 = __uint_as_float(cs.y), sa1 = __uint_as_float(cs.w);
                             int d[4];
-                            mma_u8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, c.x, c.y);
+                            mma_u8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, (int)cs.x, (int)cs.z);
                             float p0, p1, p2, p3;                 // P * weight scale, exact
                             if (!top) {
                                 p0 = fmaf(__int_as_float(d[0]), swA, mwA);
@@ -189,24 +239,100 @@ gemv_stream_kernel(const StreamParams p)
                                 p2 = fmaf(__int_as_float(d[2]), swB, mwB);
                                 p3 = fmaf(__int_as_float(d[3]), swB, mwB);
                             } else {
-                                p0 = (__int_as_float(d[0]) - STREAM_MAGIC) * swA;
-                                p1 = (__int_as_float(d[1]) - STREAM_MAGIC) * swA;
-                                p2 = (__int_as_float(d[2]) - STREAM_MAGIC) * swB;
-                                p3 = (__int_as_float(d[3]) - STREAM_MAGIC) * swB;
+                                // + 0 * scale keeps finite results and turns an Inf scale into NaN
+                                p0 = fmaf(0.f, swA, (__int_as_float(d[0]) - STREAM_MAGIC) * swA);
+                                p1 = fmaf(0.f, swA, (__int_as_float(d[1]) - STREAM_MAGIC) * swA);
+                                p2 = fmaf(0.f, swB, (__int_as_float(d[2]) - STREAM_MAGIC) * swB);
+                                p3 = fmaf(0.f, swB, (__int_as_float(d[3]) - STREAM_MAGIC) * swB);
                             }
-                            acc[n][0] = fmaf(p0, sa.x, acc[n][0]);   // one rounding per block, ascending
-                            acc[n][1] = fmaf(p1, sa.y, acc[n][1]);
-                            acc[n][2] = fmaf(p2, sa.x, acc[n][2]);
-                            acc[n][3] = fmaf(p3, sa.y, acc[n][3]);
+                            acc[n][0] = fmaf(p0, sa0, acc[n][0]);   // one rounding per block, ascending
+                            acc[n][1] = fmaf(p1, sa1, acc[n][1]);
+                            acc[n][2] = fmaf(p2, sa0, acc[n][2]);
+                            acc[n][3] = fmaf(p3, sa1, acc[n][3]);
                         }
                     }
+                };
+                if (!BULK) {
+                    auto fetch = [&](int b, Regs &r) {
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        wa[j] = na[j];
-                        wb[j] = nbw[j];
+                        for (int j = 0; j < 4; ++j) {
+                            r.a[j] = __ldcs(reinterpret_cast<const uint32_t *>(mA + (b + j) * 16));
+                            r.b[j] = __ldcs(reinterpret_cast<const uint32_t *>(mB + (b + j) * 16));
+                        }
+                        r.ea = __ldcs(reinterpret_cast<const uint32_t *>(eA + b));
+                        r.eb = __ldcs(reinterpret_cast<const uint32_t *>(eB + b));
+                    };
+                    // two register sets alternate, so the prefetched words are never copied
+                    Regs ra, rb;
+                    fetch(b_lo, ra);
+                    for (int b = b_lo; b < b_hi; b += 8) {
+                        const bool second = b + 4 < b_hi;
+                        if (second) fetch(b + 4, rb);
+                        compute(b, ra);
+                        if (b + 8 < b_hi) fetch(b + 8, ra);
+                        if (second) compute(b + 4, rb);
                     }
-                    ea = nea;
-                    eb = neb;
+                } else {
+                    // exponent bytes: lanes 0..15 each copy one row's piece once per tile;
+                    // mantissas: one tiled TMA load (16 rows x 128 bytes, swizzled) per step
+                    uint8_t *my_stage = sStage + warp * STAGES * Cfg::STAGE_BYTES;
+                    uint8_t *my_exp = sExp + (size_t)warp * 16 * exp_pitch;
+                    const uint32_t my_bar = ptx::smem_u32(sBar) + 8 * warp * (STAGES + 1);
+                    const int crow = min(r0 + (lane & 15), L.N - 1);
+                    const uint8_t *ce = L.w_exp + (int64_t)crow * nb;
+                    const CUtensorMap *tmap = p.tmaps + li;
+                    const int nblk = b_hi - b_lo;                       // multiple of 16
+                    ptx::fence_proxy_async_smem();                      // earlier reads of these buffers are done
+                    if (lane == 0) ptx::mbar_arrive_expect_tx(my_bar + 8 * STAGES, 16u * (uint32_t)nblk);
+                    __syncwarp();
+                    if (lane < 16)
+                        bulk_copy_g2s(ptx::smem_u32(my_exp + lane * exp_pitch), ce + b_lo, (uint32_t)nblk,
+                                      my_bar + 8 * STAGES);
+                    auto issue = [&](int step, int st) {              // step: CH-block chunk index from b_lo
+                        if (lane == 0) {
+                            const uint32_t bar = my_bar + 8 * st;
+                            ptx::mbar_arrive_expect_tx(bar, Cfg::STAGE_TX);
+                            ptx::tma_load_2d(ptx::smem_u32(my_stage + st * Cfg::STAGE_BYTES), tmap,
+                                             (b_lo + step * CH) * 16, r0, bar);     // rows >= N read as zero
+                        }
+                    };
+                    const int nsteps = nblk / CH;
+                    for (int i = 0; i < STAGES && i < nsteps; ++i) issue(i, i);
+                    {
+                        const bool ok = ptx::mbar_wait_bounded(my_bar + 8 * STAGES, (phase_bits >> STAGES) & 1u,
+                                                               abort_flag, STREAM_WAIT_LIMIT_NS);
+                        if (!__all_sync(0xFFFFFFFFu, ok)) timed_out = true;
+                        phase_bits ^= 1u << STAGES;
+                    }
+                    int st = 0;
+                    for (int step = 0; step < nsteps && !timed_out; ++step) {
+                        const bool ok = ptx::mbar_wait_bounded(my_bar + 8 * st, (phase_bits >> st) & 1u, abort_flag,
+                                                               STREAM_WAIT_LIMIT_NS);
+                        if (!__all_sync(0xFFFFFFFFu, ok)) { timed_out = true; break; }
+                        phase_bits ^= 1u << st;
+                        const uint8_t *sm = my_stage + st * Cfg::STAGE_BYTES;
+#pragma unroll
+                        for (int q = 0; q < CH / 4; ++q) {
+                            Regs r;
+#pragma unroll
+                            for (int j = 0; j < 4; ++j) {
+                                // 16-byte chunk c of row r sits at chunk c ^ (r & 7); g + 8 has the same r & 7
+                                const int off = g * 128 + (((q * 4 + j) ^ g) << 4) + t * 4;
+                                r.a[j] = *reinterpret_cast<const uint32_t *>(sm + off);
+                                r.b[j] = *reinterpret_cast<const uint32_t *>(sm + off + 8 * 128);
+                            }
+                            const int boff = step * CH + q * 4;        // block offset from b_lo
+                            r.ea = *reinterpret_cast<const uint32_t *>(my_exp + g * exp_pitch + boff);
+                            r.eb = *reinterpret_cast<const uint32_t *>(my_exp + (g + 8) * exp_pitch + boff);
+                            compute(b_lo + boff, r);
+                        }
+                        __syncwarp();                                 // every lane is done reading the stage
+                        if (step + STAGES < nsteps) {
+                            ptx::fence_proxy_async_smem();
+                            issue(step + STAGES, st);
+                        }
+                        if (++st == STAGES) st = 0;
+                    }
                 }
             }
             if (S > 1) {                                             // CTA-uniform branch
@@ -240,6 +366,11 @@ gemv_stream_kernel(const StreamParams p)
         }
         tile_lo = l_end;
         ++li;
+        if (BULK && __syncthreads_or(timed_out ? 1 : 0)) break;     // a bounded wait expired: give up
+    }
+    if (BULK && timed_out) {
+        *abort_flag = 1;
+        atomicOr(p.status, 1u);
     }
 }
 

@@ -7,7 +7,9 @@
 #include <stdio.h>
 #include <string.h>
 
+#include <map>
 #include <mutex>
+#include <tuple>
 #include <vector>
 
 #include "../../include/mxint.h"
@@ -31,7 +33,7 @@ struct DeviceInfo {
     int sm_count = SM_COUNT_FALLBACK;
     uint32_t *status = nullptr;
     bool tc_attr_set[2][3] = {{false, false, false}, {false, false, false}};
-    bool stream_attr_set[2] = {false, false};
+    bool stream_attr_set[4] = {false, false, false, false};
 };
 DeviceInfo g_dev[MAX_DEVICES];
 
@@ -326,6 +328,49 @@ mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t 
 }
 
 // ---- decode: few tokens, weights streamed once ------------------------------------------------
+// Tensor maps over packed weight matrices are cached: weights are static, so after the first
+// call a layer costs a map lookup instead of a driver call.
+std::map<std::tuple<const void *, int64_t, int64_t>, CUtensorMap> g_wmap_cache;
+std::mutex g_wmap_mu;
+
+mx_status_t packed_weight_map(const void *w_mant, int64_t N, int64_t K, CUtensorMap *out)
+{
+    std::lock_guard<std::mutex> lk(g_wmap_mu);
+    const auto key = std::make_tuple(w_mant, N, K);
+    auto it = g_wmap_cache.find(key);
+    if (it != g_wmap_cache.end()) {
+        *out = it->second;
+        return MX_OK;
+    }
+    if (!g_encode_tiled) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+        if (q != cudaDriverEntryPointSuccess || !fn) return MX_ERR_CUDA;
+        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    }
+    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
+    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
+    const cuuint32_t box[2] = {128, 16};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(w_mant), dims,
+                                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled (packed weights) failed (%d)", (int)r);
+        return MX_ERR_CUDA;
+    }
+    if (g_wmap_cache.size() > 4096) g_wmap_cache.clear();
+    g_wmap_cache[key] = *out;
+    return MX_OK;
+}
+
+size_t stream_table_bytes(int32_t n_layers)
+{
+    return round256((size_t)n_layers * sizeof(mx::StreamLayer)) + round256((size_t)n_layers * sizeof(CUtensorMap));
+}
+
 bool stream_layer_ok(const mx_linear_args_t &a)
 {
     return a.M >= 1 && a.M <= 16 && a.fw.block == 32 && a.fa.block == 32 && a.fw.elem_bits <= 4 &&
@@ -343,16 +388,17 @@ bool same_activation(const mx_linear_args_t &a, const mx_linear_args_t &b)
            a.fa.block == b.fa.block && a.fa.elem_bits == b.fa.elem_bits;
 }
 
-template <int NT>
+template <int NT, bool BULK>
 mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, DeviceInfo &d, cudaStream_t st)
 {
-    if (!d.stream_attr_set[NT - 1]) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemv_stream_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    bool &done = d.stream_attr_set[(NT - 1) * 2 + (BULK ? 1 : 0)];
+    if (!done) {
+        MX_CUDA(cudaFuncSetAttribute(mx::gemv_stream_kernel<NT, BULK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      227 * 1024));
-        d.stream_attr_set[NT - 1] = true;
+        done = true;
     }
     ProfScope prof(KIND_GEMM_STREAM, st);
-    mx::gemv_stream_kernel<NT><<<grid, mx::STREAM_THREADS, smem, st>>>(sp);
+    mx::gemv_stream_kernel<NT, BULK><<<grid, mx::StreamCfg<NT, BULK>::THREADS, smem, st>>>(sp);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -387,7 +433,7 @@ size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx
     const size_t pk = packed_workspace(M, K, fa);          // mx_linear with the CUDA-core kernel
     switch (algo) {
     case MX_ALGO_SIMT: return pk;
-    case MX_ALGO_STREAM: return round256(sizeof(mx::StreamLayer)) + round256(mx_mant_bytes(M, K, fa)) +
+    case MX_ALGO_STREAM: return stream_table_bytes(1) + round256(mx_mant_bytes(M, K, fa)) +
                                 round256(mx_exp_bytes(M, K, fa));
     case MX_ALGO_AUTO: {            // mx_linear may stream (M <= 16), mx_gemm uses the tensor cores
         const size_t st = mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_STREAM);
@@ -587,7 +633,7 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
 size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, int32_t n_layers)
 {
     if (!layers || n_layers <= 0) return 0;
-    size_t total = round256((size_t)n_layers * sizeof(mx::StreamLayer));
+    size_t total = stream_table_bytes(n_layers);
     for (int i = 0; i < n_layers; ++i) {
         if (!format_ok(layers[i].fa) || !format_ok(layers[i].fw)) return 0;
         bool seen = false;
@@ -621,7 +667,19 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     if (!workspace || workspace_bytes < need) return MX_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
     const int nt = max_t > 8 ? 2 : 1;
-    const size_t smem = nt == 2 ? mx::stream_smem_bytes<2>(max_nb) : mx::stream_smem_bytes<1>(max_nb);
+    // weights staged by bulk copies need 16-byte aligned exponent chunks: K % 512 == 0 everywhere
+    bool bulk = true;
+    for (int i = 0; i < n_layers; ++i)
+        bulk = bulk && (layers[i].K % 512) == 0 && (reinterpret_cast<uintptr_t>(layers[i].w_exp) & 15u) == 0;
+    auto smem_of = [&](bool b) {
+        return nt == 2 ? (b ? mx::StreamCfg<2, true>::smem_bytes(max_nb) : mx::StreamCfg<2, false>::smem_bytes(max_nb))
+                       : (b ? mx::StreamCfg<1, true>::smem_bytes(max_nb) : mx::StreamCfg<1, false>::smem_bytes(max_nb));
+    };
+    size_t smem = smem_of(bulk);
+    if (bulk && smem > 227u * 1024u) {
+        bulk = false;
+        smem = smem_of(false);
+    }
     if (smem > 227u * 1024u) return MX_ERR_SHAPE;                  // tokens x K too large to stage
     DeviceInfo *d = nullptr;
     mx_status_t s = device_info(&d);
@@ -630,8 +688,10 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
 
     // quantize every distinct activation tensor once, build the device layer table
     uint8_t *ws = static_cast<uint8_t *>(workspace);
-    size_t off = round256((size_t)n_layers * sizeof(mx::StreamLayer));
+    size_t off = stream_table_bytes(n_layers);
+    const size_t tmap_off = round256((size_t)n_layers * sizeof(mx::StreamLayer));
     std::vector<mx::StreamLayer> table((size_t)n_layers);
+    std::vector<CUtensorMap> tmaps(bulk ? (size_t)n_layers : 0);
     std::vector<uint8_t *> act_ptr((size_t)n_layers, nullptr);
     int total_tiles = 0;
     for (int i = 0; i < n_layers; ++i) {
@@ -661,20 +721,28 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
         L.tile_begin = total_tiles;
         L.n_tiles = (int)((a.N + 15) / 16);
         total_tiles += L.n_tiles;
+        if (bulk) {
+            s = packed_weight_map(a.w_mant, a.N, a.K, &tmaps[(size_t)i]);
+            if (s != MX_OK) return s;
+        }
     }
+    if (bulk)
+        MX_CUDA(cudaMemcpyAsync(ws + tmap_off, tmaps.data(), (size_t)n_layers * sizeof(CUtensorMap),
+                                cudaMemcpyHostToDevice, st));
     MX_CUDA(cudaMemcpyAsync(ws, table.data(), (size_t)n_layers * sizeof(mx::StreamLayer),
                             cudaMemcpyHostToDevice, st));
 
     const int ctas_per_sm = (int)((227u * 1024u) / (smem + 1024)) < 4 ? (int)((227u * 1024u) / (smem + 1024)) : 4;
     const int max_ctas = d->sm_count * (ctas_per_sm < 1 ? 1 : ctas_per_sm);
+    const int warps = bulk ? 16 : 8;
     int split = 1;                         // cut K over warps only when row tiles alone cannot fill the GPU
-    if (total_tiles < max_ctas * 8) {
-        if (min_nb % 16 == 0 && total_tiles * 4 >= max_ctas * 2) split = 4;
-        else if (min_nb % 32 == 0) split = 8;
-        else if (min_nb % 16 == 0) split = 4;
-        else if (min_nb % 8 == 0) split = 2;
+    const int unit = bulk ? 16 : 4;        // blocks per row a warp's K piece must be a multiple of
+    if (total_tiles < max_ctas * warps) {
+        for (int cand = 8; cand > 1 && split == 1; cand >>= 1)
+            if (min_nb % (unit * cand) == 0 && (cand <= 4 || total_tiles * 4 < max_ctas * warps)) split = cand;
     }
-    const int rounds = (total_tiles + (8 / split) - 1) / (8 / split);
+    const int tpr = warps / split;
+    const int rounds = (total_tiles + tpr - 1) / tpr;
     const int grid = rounds < max_ctas ? rounds : max_ctas;
     mx::StreamParams sp;
     sp.layers = reinterpret_cast<const mx::StreamLayer *>(ws);
@@ -682,7 +750,11 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     sp.total_tiles = total_tiles;
     sp.split = split;
     sp.max_nb = max_nb;
-    return nt == 2 ? launch_stream<2>(sp, smem, grid, *d, st) : launch_stream<1>(sp, smem, grid, *d, st);
+    sp.status = d->status;
+    sp.tmaps = reinterpret_cast<const CUtensorMap *>(ws + tmap_off);
+    if (bulk)
+        return nt == 2 ? launch_stream<2, true>(sp, smem, grid, *d, st) : launch_stream<1, true>(sp, smem, grid, *d, st);
+    return nt == 2 ? launch_stream<2, false>(sp, smem, grid, *d, st) : launch_stream<1, false>(sp, smem, grid, *d, st);
 }
 
 // ---- product without any allocation ---------------------------------------------------------

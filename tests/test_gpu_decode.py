@@ -52,10 +52,12 @@ def test_stream_single_layer_within_tolerance(mxb, T, shape):
     assert torch.equal(y, y2)
 
 
-@pytest.mark.parametrize("T,n_layers", [(1, 20), (4, 20), (16, 10)])
-def test_grouped_launch_is_bit_exact_against_sequential_oracle(mxb, T, n_layers):
-    """Enough row tiles to fill the GPU without cutting K: ascending fp32 block sums, exactly."""
-    K, N = 256, 4096
+@pytest.mark.parametrize("T,n_layers,K", [(1, 20, 256), (4, 20, 256), (16, 10, 256),
+                                          (4, 20, 512), (16, 20, 1024), (1, 20, 1536)])
+def test_grouped_launch_is_bit_exact_against_sequential_oracle(mxb, T, n_layers, K):
+    """Enough row tiles to fill the GPU without cutting K: ascending fp32 block sums, exactly.
+    K = 256 takes the register-prefetch kernel, K % 512 == 0 the bulk-copy staged one."""
+    N = 4096
     layers, refs = [], []
     for i in range(n_layers):
         dev, ref = _layer(mxb, T, K, N, seed=100 * T + 3 * i, wa=(8, 6, 4)[i % 3], ww=(4, 3, 2)[i % 3],

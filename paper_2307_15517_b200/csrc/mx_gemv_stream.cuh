@@ -53,35 +53,39 @@ struct StreamParams {
     int split;                   // 1, 2, 4 or 8
     int max_nb;                  // largest K/32 over the layers (sizes the shared-memory arrays)
     uint32_t *status;            // device status word (bit 0: a bounded wait expired)
-    const CUtensorMap *tmaps;    // BULK: one map per layer over its packed mantissas [N, K/2] bytes,
-                                 // box 128 bytes x 16 rows, 128-byte swizzle (device memory)
+    const CUtensorMap *tmaps;    // BULK: two maps per layer (device memory): [2l] over the packed
+                                 // mantissas [N, K/2] bytes, box 128 x 16 rows, 128-byte swizzle;
+                                 // [2l+1] over the exponent bytes [N, K/32], box 16 x 16 rows
 };
 
 // Geometry of the two variants.
 //   register variant (BULK = false): 8 warps, each lane prefetches four blocks' words with 32-bit
 //     loads; works for any K % 128 == 0.
-//   TMA variant (BULK = true): 16 warps; every warp owns a ring of STAGES shared-memory stages,
-//     each filled by ONE tiled TMA load of 16 rows x 8 blocks of mantissas (128 bytes per row,
-//     128-byte swizzle so that the 8 rows one fragment load touches fall into different banks),
-//     plus a per-tile 1-D bulk copy of its rows' exponent bytes; global data never passes through
-//     the load/store data pipe.  Needs K % 512 == 0 and 16-byte aligned exponent arrays.
+//   TMA variant (BULK = true): 16 warps; every warp owns a ring of STAGES shared-memory stages.
+//     A stage is 16 rows x 16 blocks: two tiled TMA loads of 16 rows x 128 mantissa bytes each
+//     (issued back to back so that DRAM sees 256 contiguous bytes per row -- 128-byte pieces
+//     alone reach only ~70 % of the HBM rate; 128-byte swizzle so that the 8 rows one fragment
+//     load touches fall into different banks) plus one load of 16 rows x 16 exponent bytes.
+//     Global data never passes through the load/store data pipe.  Needs K % 512 == 0 and
+//     16-byte aligned exponent arrays.
 template <int NT, bool BULK> struct StreamCfg {
     static constexpr int WARPS = BULK ? 16 : 8;
     static constexpr int THREADS = WARPS * 32;
-    static constexpr int STAGES = NT == 1 ? 4 : 3;
-    static constexpr int CH = BULK ? 8 : 4;                        // blocks of 32 per step and row
-    static constexpr int STAGE_BYTES = 16 * CH * 16;               // 2048: 16 rows x 128 bytes
+    static constexpr int STAGES = 2;
+    static constexpr int CH = BULK ? 16 : 4;                       // blocks of 32 per step and row
+    static constexpr int MANT_BYTES = 16 * CH * 16;                // 4096: two boxes of 16 rows x 128 bytes
+    static constexpr int STAGE_BYTES = MANT_BYTES + 16 * CH;       // + 16 rows x 16 exponent bytes
     static constexpr uint32_t STAGE_TX = STAGE_BYTES;
     static constexpr int TP = NT * 8;                              // padded token count
     static constexpr size_t tokens_bytes(int max_nb) { return (size_t)max_nb * TP * (32 + 8); }
     static constexpr size_t red_bytes() { return (size_t)WARPS * NT * 4 * 32 * 4; }
-    static constexpr size_t exp_pitch(int max_nb) { return (size_t)max_nb + 16; }
     static constexpr size_t smem_bytes(int max_nb)
     {
-        return tokens_bytes(max_nb) + red_bytes() +
+        // the split-K exchange buffer aliases the weight stages in the TMA variant
+        return tokens_bytes(max_nb) +
                (BULK ? 1024 /* stage alignment */ + (size_t)WARPS * STAGES * STAGE_BYTES +
-                           (size_t)WARPS * 16 * exp_pitch(max_nb) + (size_t)WARPS * (STAGES + 1) * 8 + 16
-                     : 0);
+                           (size_t)WARPS * STAGES * 8 + 16
+                     : red_bytes());
     }
 };
 constexpr uint64_t STREAM_WAIT_LIMIT_NS = 400ull * 1000 * 1000;
@@ -119,19 +123,19 @@ gemv_stream_kernel(const StreamParams p)
     // [nb][TP] pairs (accumulator seed, token scale); the token scale also carries the weights'
     // binary point 2^-(ww-2), so the weight scale below is the plain 2^(Ew-127)
     uint2 *sCS = reinterpret_cast<uint2 *>(smem + (size_t)p.max_nb * TP * 32);
-    float *sRed = reinterpret_cast<float *>(sCS + (size_t)p.max_nb * TP);        // [WARPS][NT][4][32]
-    // [WARPS][STAGES] swizzled weight stages, 1024-byte aligned (BULK)
-    uint8_t *sStage = reinterpret_cast<uint8_t *>(sRed + WARPS * NT * 4 * 32);
-    sStage += (1024u - (ptx::smem_u32(sStage) & 1023u)) & 1023u;
-    uint8_t *sExp = sStage + WARPS * STAGES * Cfg::STAGE_BYTES;                  // [WARPS][16][max_nb + 16]
-    const int exp_pitch = p.max_nb + 16;
-    uint8_t *sBar = sExp + (size_t)WARPS * 16 * exp_pitch;                       // [WARPS][STAGES + 1] mbarriers
-    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(sBar + WARPS * (STAGES + 1) * 8);
-    uint32_t phase_bits = 0;                  // parity per barrier of this warp (bit STAGES: exponents)
+    // BULK: [WARPS][STAGES][4096] swizzled mantissa stages (1024-byte aligned), then
+    // [WARPS][STAGES][256] exponent stages; the split-K exchange buffer [WARPS][NT][4][32] reuses them
+    uint8_t *sStage = reinterpret_cast<uint8_t *>(sCS + (size_t)p.max_nb * TP);
+    if (BULK) sStage += (1024u - (ptx::smem_u32(sStage) & 1023u)) & 1023u;
+    uint8_t *sExpStage = sStage + WARPS * STAGES * Cfg::MANT_BYTES;
+    float *sRed = reinterpret_cast<float *>(sStage);
+    uint8_t *sBar = sStage + (BULK ? WARPS * STAGES * Cfg::STAGE_BYTES : 0);     // [WARPS][STAGES] mbarriers
+    volatile uint32_t *abort_flag = reinterpret_cast<volatile uint32_t *>(sBar + WARPS * STAGES * 8);
+    uint32_t phase_bits = 0;                  // parity per stage barrier of this warp
     bool timed_out = false;
     if (BULK) {
         if (threadIdx.x == 0) {
-            for (int i = 0; i < WARPS * (STAGES + 1); ++i) ptx::mbar_init(ptx::smem_u32(sBar) + 8 * i, 1);
+            for (int i = 0; i < WARPS * STAGES; ++i) ptx::mbar_init(ptx::smem_u32(sBar) + 8 * i, 1);
             *abort_flag = 0;
             ptx::fence_mbar_init();
         }
@@ -273,58 +277,51 @@ gemv_stream_kernel(const StreamParams p)
                         if (second) compute(b + 4, rb);
                     }
                 } else {
-                    // exponent bytes: lanes 0..15 each copy one row's piece once per tile;
-                    // mantissas: one tiled TMA load (16 rows x 128 bytes, swizzled) per step
-                    uint8_t *my_stage = sStage + warp * STAGES * Cfg::STAGE_BYTES;
-                    uint8_t *my_exp = sExp + (size_t)warp * 16 * exp_pitch;
-                    const uint32_t my_bar = ptx::smem_u32(sBar) + 8 * warp * (STAGES + 1);
-                    const int crow = min(r0 + (lane & 15), L.N - 1);
-                    const uint8_t *ce = L.w_exp + (int64_t)crow * nb;
-                    const CUtensorMap *tmap = p.tmaps + li;
+                    // one lane fills a stage with three tiled TMA loads: mantissa columns [x, x+128) and
+                    // [x+128, x+256) of the 16 rows, and their 16 exponent bytes
+                    uint8_t *my_stage = sStage + warp * STAGES * Cfg::MANT_BYTES;
+                    uint8_t *my_exps = sExpStage + warp * STAGES * (16 * CH);
+                    const uint32_t my_bar = ptx::smem_u32(sBar) + 8 * warp * STAGES;
+                    const CUtensorMap *tm_m = p.tmaps + 2 * li, *tm_e = tm_m + 1;
                     const int nblk = b_hi - b_lo;                       // multiple of 16
-                    ptx::fence_proxy_async_smem();                      // earlier reads of these buffers are done
-                    if (lane == 0) ptx::mbar_arrive_expect_tx(my_bar + 8 * STAGES, 16u * (uint32_t)nblk);
-                    __syncwarp();
-                    if (lane < 16)
-                        bulk_copy_g2s(ptx::smem_u32(my_exp + lane * exp_pitch), ce + b_lo, (uint32_t)nblk,
-                                      my_bar + 8 * STAGES);
                     auto issue = [&](int step, int st) {              // step: CH-block chunk index from b_lo
                         if (lane == 0) {
                             const uint32_t bar = my_bar + 8 * st;
+                            const uint32_t dst = ptx::smem_u32(my_stage + st * Cfg::MANT_BYTES);
+                            const int b = b_lo + step * CH;
                             ptx::mbar_arrive_expect_tx(bar, Cfg::STAGE_TX);
-                            ptx::tma_load_2d(ptx::smem_u32(my_stage + st * Cfg::STAGE_BYTES), tmap,
-                                             (b_lo + step * CH) * 16, r0, bar);     // rows >= N read as zero
+                            ptx::tma_load_2d(dst, tm_m, b * 16, r0, bar);                 // rows >= N read as zero
+                            ptx::tma_load_2d(dst + 2048, tm_m, b * 16 + 128, r0, bar);
+                            ptx::tma_load_2d(ptx::smem_u32(my_exps + st * (16 * CH)), tm_e, b, r0, bar);
                         }
                     };
                     const int nsteps = nblk / CH;
+                    ptx::fence_proxy_async_smem();                      // earlier generic reads/writes of the stages
+                    __syncwarp();
                     for (int i = 0; i < STAGES && i < nsteps; ++i) issue(i, i);
-                    {
-                        const bool ok = ptx::mbar_wait_bounded(my_bar + 8 * STAGES, (phase_bits >> STAGES) & 1u,
-                                                               abort_flag, STREAM_WAIT_LIMIT_NS);
-                        if (!__all_sync(0xFFFFFFFFu, ok)) timed_out = true;
-                        phase_bits ^= 1u << STAGES;
-                    }
                     int st = 0;
                     for (int step = 0; step < nsteps && !timed_out; ++step) {
                         const bool ok = ptx::mbar_wait_bounded(my_bar + 8 * st, (phase_bits >> st) & 1u, abort_flag,
                                                                STREAM_WAIT_LIMIT_NS);
                         if (!__all_sync(0xFFFFFFFFu, ok)) { timed_out = true; break; }
                         phase_bits ^= 1u << st;
-                        const uint8_t *sm = my_stage + st * Cfg::STAGE_BYTES;
+                        const uint8_t *sm = my_stage + st * Cfg::MANT_BYTES;
+                        const uint8_t *se = my_exps + st * (16 * CH);
 #pragma unroll
                         for (int q = 0; q < CH / 4; ++q) {
                             Regs r;
 #pragma unroll
                             for (int j = 0; j < 4; ++j) {
-                                // 16-byte chunk c of row r sits at chunk c ^ (r & 7); g + 8 has the same r & 7
-                                const int off = g * 128 + (((q * 4 + j) ^ g) << 4) + t * 4;
+                                // box (c >> 3); inside it the 16-byte chunk c & 7 of row r sits at
+                                // chunk (c & 7) ^ (r & 7); rows g and g + 8 share r & 7
+                                const int c = q * 4 + j;
+                                const int off = (c >> 3) * 2048 + g * 128 + (((c & 7) ^ g) << 4) + t * 4;
                                 r.a[j] = *reinterpret_cast<const uint32_t *>(sm + off);
                                 r.b[j] = *reinterpret_cast<const uint32_t *>(sm + off + 8 * 128);
                             }
-                            const int boff = step * CH + q * 4;        // block offset from b_lo
-                            r.ea = *reinterpret_cast<const uint32_t *>(my_exp + g * exp_pitch + boff);
-                            r.eb = *reinterpret_cast<const uint32_t *>(my_exp + (g + 8) * exp_pitch + boff);
-                            compute(b_lo + boff, r);
+                            r.ea = *reinterpret_cast<const uint32_t *>(se + g * 16 + q * 4);
+                            r.eb = *reinterpret_cast<const uint32_t *>(se + (g + 8) * 16 + q * 4);
+                            compute(b_lo + step * CH + q * 4, r);
                         }
                         __syncwarp();                                 // every lane is done reading the stage
                         if (step + STAGES < nsteps) {
@@ -352,6 +349,7 @@ gemv_stream_kernel(const StreamParams p)
                             acc[n][j] = v;
                         }
                 }
+                __syncthreads();          // the exchange buffer shares memory with the weight stages
             }
             if (active && s == 0) {
 #pragma unroll

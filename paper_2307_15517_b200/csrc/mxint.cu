@@ -330,45 +330,56 @@ mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t 
 // ---- decode: few tokens, weights streamed once ------------------------------------------------
 // Tensor maps over packed weight matrices are cached: weights are static, so after the first
 // call a layer costs a map lookup instead of a driver call.
-std::map<std::tuple<const void *, int64_t, int64_t>, CUtensorMap> g_wmap_cache;
+struct WeightMaps { CUtensorMap mant, exps; };
+std::map<std::tuple<const void *, const void *, int64_t, int64_t>, WeightMaps> g_wmap_cache;
 std::mutex g_wmap_mu;
 
-mx_status_t packed_weight_map(const void *w_mant, int64_t N, int64_t K, CUtensorMap *out)
+mx_status_t encode_u8_rows(CUtensorMap *out, const void *base, int64_t rows, int64_t row_bytes, int box_bytes,
+                           CUtensorMapSwizzle swz)
 {
-    std::lock_guard<std::mutex> lk(g_wmap_mu);
-    const auto key = std::make_tuple(w_mant, N, K);
-    auto it = g_wmap_cache.find(key);
-    if (it != g_wmap_cache.end()) {
-        *out = it->second;
-        return MX_OK;
-    }
-    if (!g_encode_tiled) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-        if (q != cudaDriverEntryPointSuccess || !fn) return MX_ERR_CUDA;
-        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
-    }
-    const cuuint64_t dims[2] = {(cuuint64_t)(K / 2), (cuuint64_t)N};
-    const cuuint64_t strides[1] = {(cuuint64_t)(K / 2)};
-    const cuuint32_t box[2] = {128, 16};
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)box_bytes, 16};
     const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = g_encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(w_mant), dims,
-                                      strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-                                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    const CUresult r = g_encode_tiled(out, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides,
+                                      box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled (packed weights) failed (%d)", (int)r);
         return MX_ERR_CUDA;
     }
-    if (g_wmap_cache.size() > 4096) g_wmap_cache.clear();
-    g_wmap_cache[key] = *out;
+    return MX_OK;
+}
+
+mx_status_t packed_weight_maps(const void *w_mant, const void *w_exp, int64_t N, int64_t K, CUtensorMap *out2)
+{
+    std::lock_guard<std::mutex> lk(g_wmap_mu);
+    const auto key = std::make_tuple(w_mant, w_exp, N, K);
+    auto it = g_wmap_cache.find(key);
+    if (it == g_wmap_cache.end()) {
+        if (!g_encode_tiled) {
+            void *fn = nullptr;
+            cudaDriverEntryPointQueryResult q;
+            MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+            if (q != cudaDriverEntryPointSuccess || !fn) return MX_ERR_CUDA;
+            g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+        }
+        WeightMaps wm;
+        mx_status_t s = encode_u8_rows(&wm.mant, w_mant, N, K / 2, 128, CU_TENSOR_MAP_SWIZZLE_128B);
+        if (s != MX_OK) return s;
+        s = encode_u8_rows(&wm.exps, w_exp, N, K / 32, 16, CU_TENSOR_MAP_SWIZZLE_NONE);
+        if (s != MX_OK) return s;
+        if (g_wmap_cache.size() > 4096) g_wmap_cache.clear();
+        it = g_wmap_cache.emplace(key, wm).first;
+    }
+    out2[0] = it->second.mant;
+    out2[1] = it->second.exps;
     return MX_OK;
 }
 
 size_t stream_table_bytes(int32_t n_layers)
 {
-    return round256((size_t)n_layers * sizeof(mx::StreamLayer)) + round256((size_t)n_layers * sizeof(CUtensorMap));
+    return round256((size_t)n_layers * sizeof(mx::StreamLayer)) + round256((size_t)n_layers * 2 * sizeof(CUtensorMap));
 }
 
 bool stream_layer_ok(const mx_linear_args_t &a)
@@ -691,7 +702,7 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     size_t off = stream_table_bytes(n_layers);
     const size_t tmap_off = round256((size_t)n_layers * sizeof(mx::StreamLayer));
     std::vector<mx::StreamLayer> table((size_t)n_layers);
-    std::vector<CUtensorMap> tmaps(bulk ? (size_t)n_layers : 0);
+    std::vector<CUtensorMap> tmaps(bulk ? (size_t)n_layers * 2 : 0);
     std::vector<uint8_t *> act_ptr((size_t)n_layers, nullptr);
     int total_tiles = 0;
     for (int i = 0; i < n_layers; ++i) {
@@ -722,12 +733,12 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
         L.n_tiles = (int)((a.N + 15) / 16);
         total_tiles += L.n_tiles;
         if (bulk) {
-            s = packed_weight_map(a.w_mant, a.N, a.K, &tmaps[(size_t)i]);
+            s = packed_weight_maps(a.w_mant, a.w_exp, a.N, a.K, &tmaps[(size_t)i * 2]);
             if (s != MX_OK) return s;
         }
     }
     if (bulk)
-        MX_CUDA(cudaMemcpyAsync(ws + tmap_off, tmaps.data(), (size_t)n_layers * sizeof(CUtensorMap),
+        MX_CUDA(cudaMemcpyAsync(ws + tmap_off, tmaps.data(), (size_t)n_layers * 2 * sizeof(CUtensorMap),
                                 cudaMemcpyHostToDevice, st));
     MX_CUDA(cudaMemcpyAsync(ws, table.data(), (size_t)n_layers * sizeof(mx::StreamLayer),
                             cudaMemcpyHostToDevice, st));

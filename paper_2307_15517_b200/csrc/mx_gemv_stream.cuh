@@ -27,6 +27,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <type_traits>
+
 #include "mx_ptx.cuh"
 #include "mx_quantize.cuh"
 
@@ -111,6 +113,38 @@ __device__ __forceinline__ void mma_u8s8_m16n8k32(int (&d)[4], uint32_t a0, uint
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c0), "r"(c1), "r"(c0), "r"(c1));
 }
 
+// Pairs of fp32 values in one 64-bit register and the sm_100 packed-pair arithmetic on them
+// (each half rounds exactly like the scalar instruction).
+typedef uint64_t f32x2_t;
+__device__ __forceinline__ f32x2_t pack2(float lo, float hi)
+{
+    f32x2_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ f32x2_t pack2u(uint32_t lo, uint32_t hi)
+{
+    f32x2_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2_t v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2_t ffma2(f32x2_t a, f32x2_t b, f32x2_t c)
+{
+    f32x2_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ f32x2_t fmul2(f32x2_t a, f32x2_t b)
+{
+    f32x2_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 // NT = number of 8-token column tiles (1: T <= 8, 2: T <= 16).
 template <int NT, bool BULK>
 __global__ void __launch_bounds__(StreamCfg<NT, BULK>::THREADS, 1)
@@ -120,12 +154,13 @@ gemv_stream_kernel(const StreamParams p)
     constexpr int TP = Cfg::TP, WARPS = Cfg::WARPS, STAGES = Cfg::STAGES, CH = Cfg::CH;
     extern __shared__ __align__(16) uint8_t smem[];
     uint2 *sB = reinterpret_cast<uint2 *>(smem);                 // [nb][TP][4]: (even-k word, odd-k word)
-    // [nb][TP] pairs (accumulator seed, token scale); the token scale also carries the weights'
-    // binary point 2^-(ww-2), so the weight scale below is the plain 2^(Ew-127)
-    uint2 *sCS = reinterpret_cast<uint2 *>(smem + (size_t)p.max_nb * TP * 32);
+    // [nb][TP/2] records {seed(tok 2i), seed(tok 2i+1), scale(tok 2i), scale(tok 2i+1)}: accumulator
+    // seeds and token scales; the token scale also carries the weights' binary point 2^-(ww-2), so
+    // the weight scale below is the plain 2^(Ew-127)
+    uint32_t *sCS = reinterpret_cast<uint32_t *>(smem + (size_t)p.max_nb * TP * 32);
     // BULK: [WARPS][STAGES][4096] swizzled mantissa stages (1024-byte aligned), then
     // [WARPS][STAGES][256] exponent stages; the split-K exchange buffer [WARPS][NT][4][32] reuses them
-    uint8_t *sStage = reinterpret_cast<uint8_t *>(sCS + (size_t)p.max_nb * TP);
+    uint8_t *sStage = reinterpret_cast<uint8_t *>(sCS + (size_t)p.max_nb * TP * 2);
     if (BULK) sStage += (1024u - (ptx::smem_u32(sStage) & 1023u)) & 1023u;
     uint8_t *sExpStage = sStage + WARPS * STAGES * Cfg::MANT_BYTES;
     float *sRed = reinterpret_cast<float *>(sStage);
@@ -186,7 +221,9 @@ gemv_stream_kernel(const StreamParams p)
             if (tq == 0) {
                 const int eb = tok < L.T ? (int)__ldg(L.a_exp + (int64_t)tok * nb + b) : 0;
                 const float sa = f32_scale(eb, L.a_bits) * small_neg_pow2(L.w_bits);     // exact
-                sCS[b * TP + tok] = make_uint2((uint32_t)(STREAM_MAGIC_INT - 8 * sum), __float_as_uint(sa));
+                uint32_t *rec = sCS + ((b * TP + tok) >> 1) * 4 + (tok & 1);
+                rec[0] = (uint32_t)(STREAM_MAGIC_INT - 8 * sum);
+                rec[2] = __float_as_uint(sa);
             }
         }
         __syncthreads();
@@ -195,11 +232,9 @@ gemv_stream_kernel(const StreamParams p)
         for (int base = tile_lo; base < l_end; base += TPR) {
             const int tile = base + warp / S, s = warp % S;
             const bool active = tile < l_end;
-            float acc[NT][4];
+            f32x2_t accA[NT], accB[NT];        // rows g / g + 8, tokens (2t, 2t + 1) of each column tile
 #pragma unroll
-            for (int n = 0; n < NT; ++n)
-#pragma unroll
-                for (int j = 0; j < 4; ++j) acc[n][j] = 0.f;
+            for (int n = 0; n < NT; ++n) accA[n] = accB[n] = pack2(0.f, 0.f);
             const int r0 = (tile - L.tile_begin) * 16;
             if (active) {
                 const int rowA = min(r0 + g, L.N - 1), rowB = min(r0 + g + 8, L.N - 1);
@@ -213,17 +248,18 @@ gemv_stream_kernel(const StreamParams p)
                 auto near_top = [](uint32_t v) {
                     return ((v & 0x80808080u) & ((v & 0x7F7F7F7Fu) + 0x1E1E1E1Eu)) != 0u;
                 };
-                auto compute = [&](int b, const Regs &r) {
-                    const bool top = near_top(r.ea) || near_top(r.eb);
+                auto compute_g = [&](int b, const Regs &r, auto top_c) {
+                    constexpr bool TOP = decltype(top_c)::value;
+                    const f32x2_t neg_magic = pack2(-STREAM_MAGIC, -STREAM_MAGIC);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         // weight scale 2^(E-127): exponent byte moved into the float's exponent field
                         // (byte 0 -> the subnormal 2^-127, byte 255 -> Inf, which turns the block into NaN)
                         const uint32_t fa = j == 3 ? (r.ea >> 1) : (r.ea << (23 - 8 * j));
                         const uint32_t fb = j == 3 ? (r.eb >> 1) : (r.eb << (23 - 8 * j));
-                        const float swA = __uint_as_float(max(fa & 0x7F800000u, 0x00400000u));
-                        const float swB = __uint_as_float(max(fb & 0x7F800000u, 0x00400000u));
-                        const float mwA = -STREAM_MAGIC * swA, mwB = -STREAM_MAGIC * swB;
+                        const uint32_t ba = max(fa & 0x7F800000u, 0x00400000u), bb = max(fb & 0x7F800000u, 0x00400000u);
+                        const f32x2_t swA = pack2u(ba, ba), swB = pack2u(bb, bb);
+                        const f32x2_t mwA = fmul2(swA, neg_magic), mwB = fmul2(swB, neg_magic);
                         const uint32_t a0 = (r.a[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
                         const uint32_t a2 = ((r.a[j] >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
                         const uint32_t a1 = (r.b[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
@@ -232,29 +268,33 @@ gemv_stream_kernel(const StreamParams p)
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
                             const uint2 bf = sB[(blk * TP + n * 8 + g) * 4 + t];
-                            const uint4 cs = *reinterpret_cast<const uint4 *>(&sCS[blk * TP + n * 8 + 2 * t]);
-                            const float sa0 = __uint_as_float(cs.y), sa1 = __uint_as_float(cs.w);
+                            const uint4 cs = *reinterpret_cast<const uint4 *>(sCS + ((blk * TP + n * 8) / 2 + t) * 4);
+                            const f32x2_t sa = pack2u(cs.z, cs.w);
                             int d[4];
-                            mma_u8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, (int)cs.x, (int)cs.z);
-                            float p0, p1, p2, p3;                 // P * weight scale, exact
-                            if (!top) {
-                                p0 = fmaf(__int_as_float(d[0]), swA, mwA);
-                                p1 = fmaf(__int_as_float(d[1]), swA, mwA);
-                                p2 = fmaf(__int_as_float(d[2]), swB, mwB);
-                                p3 = fmaf(__int_as_float(d[3]), swB, mwB);
+                            mma_u8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, (int)cs.x, (int)cs.y);
+                            f32x2_t pA, pB;                       // P * weight scale (rows g, g + 8), exact
+                            if (!TOP) {
+                                pA = ffma2(pack2u((uint32_t)d[0], (uint32_t)d[1]), swA, mwA);
+                                pB = ffma2(pack2u((uint32_t)d[2], (uint32_t)d[3]), swB, mwB);
                             } else {
-                                // + 0 * scale keeps finite results and turns an Inf scale into NaN
-                                p0 = fmaf(0.f, swA, (__int_as_float(d[0]) - STREAM_MAGIC) * swA);
-                                p1 = fmaf(0.f, swA, (__int_as_float(d[1]) - STREAM_MAGIC) * swA);
-                                p2 = fmaf(0.f, swB, (__int_as_float(d[2]) - STREAM_MAGIC) * swB);
-                                p3 = fmaf(0.f, swB, (__int_as_float(d[3]) - STREAM_MAGIC) * swB);
+                                // 1.5*2^23 * scale is not finite up here: subtract first; + 0 * scale keeps
+                                // finite results and turns an Inf scale into NaN
+                                const float wa_ = __uint_as_float(ba), wb_ = __uint_as_float(bb);
+                                pA = pack2(fmaf(0.f, wa_, (__int_as_float(d[0]) - STREAM_MAGIC) * wa_),
+                                           fmaf(0.f, wa_, (__int_as_float(d[1]) - STREAM_MAGIC) * wa_));
+                                pB = pack2(fmaf(0.f, wb_, (__int_as_float(d[2]) - STREAM_MAGIC) * wb_),
+                                           fmaf(0.f, wb_, (__int_as_float(d[3]) - STREAM_MAGIC) * wb_));
                             }
-                            acc[n][0] = fmaf(p0, sa0, acc[n][0]);   // one rounding per block, ascending
-                            acc[n][1] = fmaf(p1, sa1, acc[n][1]);
-                            acc[n][2] = fmaf(p2, sa0, acc[n][2]);
-                            acc[n][3] = fmaf(p3, sa1, acc[n][3]);
+                            accA[n] = ffma2(pA, sa, accA[n]);     // one rounding per block, ascending blocks
+                            accB[n] = ffma2(pB, sa, accB[n]);
                         }
                     }
+                };
+                // The two-step form is needed only when an exponent byte is >= 226.  The decision is taken
+                // for the whole warp: the MMA inside is warp-collective and must never run divergent.
+                auto compute = [&](int b, const Regs &r) {
+                    if (__any_sync(0xFFFFFFFFu, near_top(r.ea | r.eb))) compute_g(b, r, std::true_type{});
+                    else compute_g(b, r, std::false_type{});
                 };
                 if (!BULK) {
                     auto fetch = [&](int b, Regs &r) {
@@ -331,6 +371,12 @@ gemv_stream_kernel(const StreamParams p)
                         if (++st == STAGES) st = 0;
                     }
                 }
+            }
+            float acc[NT][4];
+#pragma unroll
+            for (int n = 0; n < NT; ++n) {
+                unpack2(accA[n], acc[n][0], acc[n][1]);
+                unpack2(accB[n], acc[n][2], acc[n][3]);
             }
             if (S > 1) {                                             // CTA-uniform branch
                 __syncthreads();

@@ -155,17 +155,15 @@ template <> struct Load8<__nv_bfloat16> {
 // non-negative, so the fields of a word can be summed with shifts and the two's-complement
 // form restored by one XOR with 0x88888888 / 0x80808080.
 template <typename InT, int BLOCK, int UNROLL>
-__global__ void __launch_bounds__(256)
-quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w,
-                     QuantOut out)
+__device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, int64_t rows, int64_t K,
+                                                   int64_t ldx, int w, const QuantOut &out,
+                                                   int64_t warp_id, int64_t n_warps)
 {
     constexpr int LANES = BLOCK / 8;                    // lanes sharing one block
     const int lane = threadIdx.x & 31;
     const int cpr = (int)(K >> 3);                      // 8-element chunks per row
     const int segs = (cpr + 31) >> 5;                   // 256-element segments per row
     const int64_t items = rows * segs;
-    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     const bool nibble = w <= 4;
     const float qmaxf = (float)((1 << (w - 1)) - 1);
     const float pow2_wm2 = (float)(1 << (w - 2));
@@ -248,6 +246,39 @@ quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t
             if (bad && leader && out.nonfinite) atomicAdd(out.nonfinite, 1u);
         }
     }
+}
+
+template <typename InT, int BLOCK, int UNROLL>
+__global__ void __launch_bounds__(256)
+quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w,
+                     QuantOut out)
+{
+    quantize_rows_body<InT, BLOCK, UNROLL>(x, rows, K, ldx, w, out,
+                                           (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5),
+                                           (int64_t)gridDim.x * (blockDim.x >> 5));
+}
+
+// Several tensors in one launch (the distinct activation tensors of a grouped decode call):
+// blockIdx.y selects the tensor, blockIdx.x strides over its rows.
+struct QuantJob {
+    const void *x;
+    int64_t rows, K, ldx;
+    int w, block, dt;        // dt: 0 = fp32, 1 = bf16
+    QuantOut out;
+};
+
+template <typename InT, int DT>
+__global__ void __launch_bounds__(256)
+quantize_multi_kernel(const QuantJob *__restrict__ jobs)
+{
+    const QuantJob j = jobs[blockIdx.y];
+    if (j.dt != DT) return;
+    const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    if (j.block == 16)
+        quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.x), j.rows, j.K, j.ldx, j.w, j.out, warp_id, n_warps);
+    else
+        quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.x), j.rows, j.K, j.ldx, j.w, j.out, warp_id, n_warps);
 }
 
 // Generic-stride variant (blocks along a strided axis): one thread per block, plain loads.

@@ -379,7 +379,8 @@ mx_status_t packed_weight_maps(const void *w_mant, const void *w_exp, int64_t N,
 
 size_t stream_table_bytes(int32_t n_layers)
 {
-    return round256((size_t)n_layers * sizeof(mx::StreamLayer)) + round256((size_t)n_layers * 2 * sizeof(CUtensorMap));
+    return round256((size_t)n_layers * sizeof(mx::StreamLayer)) + round256((size_t)n_layers * 2 * sizeof(CUtensorMap)) +
+           round256((size_t)n_layers * sizeof(mx::QuantJob));
 }
 
 bool stream_layer_ok(const mx_linear_args_t &a)
@@ -701,6 +702,10 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     size_t off = stream_table_bytes(n_layers);
     const size_t tmap_off = round256((size_t)n_layers * sizeof(mx::StreamLayer));
+    const size_t job_off = tmap_off + round256((size_t)n_layers * 2 * sizeof(CUtensorMap));
+    std::vector<mx::QuantJob> jobs;
+    bool any_dt[2] = {false, false};
+    int64_t max_chunks = 0;
     std::vector<mx::StreamLayer> table((size_t)n_layers);
     std::vector<CUtensorMap> tmaps(bulk ? (size_t)n_layers * 2 : 0);
     std::vector<uint8_t *> act_ptr((size_t)n_layers, nullptr);
@@ -712,9 +717,19 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
         if (!act_ptr[i]) {
             act_ptr[i] = ws + off;
             off += stream_act_bytes(a);
-            mx::QuantOut out{act_ptr[i], act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa)), nullptr, 0, nullptr};
-            s = quantize_rows_any(a.x, a.dt, a.M, a.K, a.ldx, a.fa, out, *d, st);
-            if (s != MX_OK) return s;
+            mx::QuantJob job;
+            job.x = a.x;
+            job.rows = a.M;
+            job.K = a.K;
+            job.ldx = a.ldx;
+            job.w = a.fa.elem_bits;
+            job.block = a.fa.block;
+            job.dt = a.dt == MX_F32 ? 0 : 1;
+            job.out = mx::QuantOut{act_ptr[i], act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa)), nullptr, 0, nullptr};
+            jobs.push_back(job);
+            any_dt[job.dt] = true;
+            const int64_t chunks = a.M * (a.K / 8);
+            max_chunks = chunks > max_chunks ? chunks : max_chunks;
         }
         mx::StreamLayer &L = table[i];
         L.w_mant = static_cast<const uint8_t *>(a.w_mant);
@@ -742,6 +757,21 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
                                 cudaMemcpyHostToDevice, st));
     MX_CUDA(cudaMemcpyAsync(ws, table.data(), (size_t)n_layers * sizeof(mx::StreamLayer),
                             cudaMemcpyHostToDevice, st));
+    // all distinct activation tensors are quantized by one launch per input type
+    MX_CUDA(cudaMemcpyAsync(ws + job_off, jobs.data(), jobs.size() * sizeof(mx::QuantJob), cudaMemcpyHostToDevice, st));
+    {
+        const mx::QuantJob *dj = reinterpret_cast<const mx::QuantJob *>(ws + job_off);
+        const dim3 qgrid((unsigned)grid_for((max_chunks + 1) / 2, 256, d->sm_count, 8), (unsigned)jobs.size());
+        if (any_dt[0]) {
+            ProfScope prof(KIND_QUANTIZE, st);
+            mx::quantize_multi_kernel<float, 0><<<qgrid, 256, 0, st>>>(dj);
+        }
+        if (any_dt[1]) {
+            ProfScope prof(KIND_QUANTIZE, st);
+            mx::quantize_multi_kernel<__nv_bfloat16, 1><<<qgrid, 256, 0, st>>>(dj);
+        }
+        MX_CUDA(cudaGetLastError());
+    }
 
     const int ctas_per_sm = (int)((227u * 1024u) / (smem + 1024)) < 4 ? (int)((227u * 1024u) / (smem + 1024)) : 4;
     const int max_ctas = d->sm_count * (ctas_per_sm < 1 ? 1 : ctas_per_sm);

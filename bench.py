@@ -137,6 +137,76 @@ def run_step_e2e(mxb, layers):
         L["y_host"].copy_(L["y"], non_blocking=True)
 
 
+# ------------------------------------------------------------------------------ secondary metrics
+def decode_sweep(mxb, synth, torch, hbm_gbs, iters=10):
+    """Decode-shaped sweep: token batches 1/4/16 against 32 layers' worth of weight matrices
+    (4 x 4096->4096 and 2 x 4096->11008 per layer, MXInt4 block 32, pre-quantized; activations fp32,
+    quantized to MXInt8 inside the call), one grouped launch.  GB/s counts the packed weight bytes
+    (mantissas + exponent bytes) that have to be streamed, nothing else."""
+    fw = mxb.MxFormat(synth.DECODE_SPEC["block"], synth.DECODE_SPEC["w_wgt"])
+    fa = mxb.MxFormat(synth.DECODE_SPEC["block"], synth.DECODE_SPEC["w_act"])
+    g = torch.Generator(device="cuda")
+    g.manual_seed(1234)
+    mats = []
+    for layer in range(synth.DECODE_LAYERS):
+        for _, K, N in synth.decode_layer_shapes():
+            w = torch.randn(N, K, generator=g, device="cuda", dtype=torch.float32) * 0.02
+            mats.append((K, N) + tuple(mxb.mx_quantize(w, fw)))
+            del w
+    wbytes = sum(m[2].numel() + m[3].numel() for m in mats)
+    out = {"weight_bytes": wbytes, "matrices": len(mats)}
+    per_layer = len(synth.decode_layer_shapes())
+    for T in synth.DECODE_TOKEN_BATCHES:
+        xs = [synth.decode_activations(T, 4096, seed=l).cuda() for l in range(synth.DECODE_LAYERS)]
+        layers = [dict(x=xs[i // per_layer], fa=fa, fw=fw, N=N, w_mant=wm, w_exp=we,
+                       y=torch.empty(T, N, device="cuda")) for i, (K, N, wm, we) in enumerate(mats)]
+        args = mxb.make_linear_args(layers)
+        ws = mxb.alloc_workspace(mxb.mx_linear_grouped_workspace_bytes(args))
+        for _ in range(3):
+            mxb.mx_linear_grouped(args, ws)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        mxb.mx_profile_begin()
+        a.record()
+        for _ in range(iters):
+            mxb.mx_linear_grouped(args, ws)
+        b.record()
+        torch.cuda.synchronize()
+        prof = mxb.mx_profile_end()
+        ms_call = a.elapsed_time(b) / iters
+        ms_kernel = prof["gemm_stream"][0] / iters
+        out["tokens_%d" % T] = {
+            "ms_per_call": ms_call, "gbs_call": wbytes / ms_call / 1e6,
+            "ms_stream_kernel": ms_kernel, "gbs_stream_kernel": wbytes / ms_kernel / 1e6,
+            "frac_hbm_stream_kernel": wbytes / ms_kernel / 1e6 / hbm_gbs,
+            "frac_hbm_call": wbytes / ms_call / 1e6 / hbm_gbs, "launches_per_call": sum(n for _, n in prof.values()) / iters}
+    return out
+
+
+def quantize_rate(mxb, torch, hbm_gbs, iters=20):
+    """Quantizer throughput on activation-sized tensors (fp32 in, packed MXInt4/B16 out):
+    algorithmic bytes = 4 read + 0.5 + 1/16 written per element."""
+    out = {}
+    for rows, K in ((2048, 8192), (16384, 8192)):
+        xs = [torch.randn(rows, K, device="cuda") for _ in range(3)]       # rotate: inputs beyond L2
+        f = mxb.MxFormat(16, 4)
+        mant = torch.empty(rows, K // 2, dtype=torch.uint8, device="cuda")
+        ex = torch.empty(rows, K // 16, dtype=torch.uint8, device="cuda")
+        for i in range(3):
+            mxb.mx_quantize(xs[i], f, mant, ex)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(iters):
+            mxb.mx_quantize(xs[i % 3], f, mant, ex)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / iters
+        gbs = rows * K * (4 + 0.5 + 1 / 16) / ms / 1e6
+        out["%dx%d" % (rows, K)] = {"ms": ms, "gbs": gbs, "frac_hbm": gbs / hbm_gbs}
+    return out
+
+
 # ------------------------------------------------------------------------------ oracle (CPU)
 def oracle_inputs(orc, synth, sample_rows):
     """Untimed set-up: the first `sample_rows` tokens of every layer and its quantized weights."""
@@ -231,6 +301,9 @@ def run_ours(args):
     layers = sets[0]
     tokens = synth.OPT13B_TOKENS
     flops_step = sum(layer_flops(tokens, L["spec"]) for L in layers)
+    h2d = sum(L["x_host"].numel() * 4 for L in layers)
+    d2h = sum(L["y_host"].numel() * 4 for L in layers)
+    layer_list = [[L["spec"].name, L["spec"].K, L["spec"].N] for L in layers]
     counter = [0]
 
     def next_set():
@@ -272,6 +345,16 @@ def run_ours(args):
         ms_e2e, _ = timed_steps(run_step_e2e, args.steps, profile=False)
         barrier()
 
+    secondary = None
+    if rank == 0 and not args.skip_secondary:
+        del sets, layers
+        torch.cuda.empty_cache()
+        secondary = {"decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
+                     "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
+                     "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
+        assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"
+    barrier()
+
     t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
     if world > 1:
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
@@ -283,15 +366,13 @@ def run_ours(args):
         gemm_ms, gemm_n = prof["gemm_tc"]
         achieved = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
         peak = peaks["bf16_tflops"]          # burst figure: the timed region lasts well under a second
-        h2d = sum(L["x_host"].numel() * 4 for L in layers)
-        d2h = sum(L["y_host"].numel() * 4 for L in layers)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "bf16 (exact MXInt decode) x bf16 -> f32",
             "data": "synthetic",
             "config": {"workload": WORKLOAD, "tokens_per_gpu": tokens,
-                       "layers": [[L["spec"].name, L["spec"].K, L["spec"].N] for L in layers],
+                       "layers": layer_list,
                        "weights": "pre-quantized once outside the timed region",
                        "l2": "inputs larger than L2: %d rotating sets of activations, weights, workspace "
                              "and outputs (~450 MB each); per-step CUDA events summed" % N_SETS,
@@ -307,6 +388,7 @@ def run_ours(args):
                          "peak_kind": "bf16 burst, %s" % peaks_kind,
                          "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
                          "traffic": None},
+            "secondary": secondary,
             "cpu_baseline": None if args.skip_cpu_baseline else cpu_baseline(),
         }
         print(json.dumps(line))
@@ -323,6 +405,8 @@ def main():
     ap.add_argument("--skip-cpu-baseline", action="store_true",
                     help="leave the CPU oracle timing out (profiler runs)")
     ap.add_argument("--skip-e2e", action="store_true", help="leave the host-buffer leg out")
+    ap.add_argument("--skip-secondary", action="store_true",
+                    help="leave the decode sweep and the quantizer rate out")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3)
     if args.impl == "reference":

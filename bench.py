@@ -31,6 +31,9 @@ METRIC = "mx_linear_effective_tops"
 UNIT = "TOPS"
 WORKLOAD = "opt-1.3b prefill linears, 2048 tokens, MXInt4 block 16 (4 layers per step)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_tc_kernel<256,0>, averaged over the
+# four launches of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_opt13b_prefill.md
+GEMM_TC_DRAM_BYTES_PER_LAUNCH = 45.3e6
 
 
 def load_peaks():
@@ -387,7 +390,8 @@ def run_ours(args):
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
                          "peak_kind": "bf16 burst, %s" % peaks_kind,
                          "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
-                         "traffic": None},
+                         "traffic": GEMM_TC_DRAM_BYTES_PER_LAUNCH,
+                         "algorithmic_flops_per_launch": flops_step / 4.0},
             "secondary": secondary,
             "cpu_baseline": None if args.skip_cpu_baseline else cpu_baseline(),
         }

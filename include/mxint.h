@@ -199,6 +199,40 @@ MX_API size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, 
 MX_API mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers,
                                      void *workspace, size_t workspace_bytes, void *stream);
 
+/* ---- batched product and fp32 glue (the attention matmuls and the rest of a decoder block) --- */
+
+/*
+ * `batch` independent products Y_b[M,N] = A_b[M,K] * W_b[N,K]^T of MXInt operands that live inside
+ * larger packed tensors: row r of A_b starts `r*lda + b*stride_a` ELEMENTS into the packed tensor
+ * (mantissa byte offset = elements * container bits / 8, exponent offset = elements / block), same
+ * for W with ldw / stride_w; Y_b = y + b*stride_y with leading dimension ldy.  The attention
+ * matmuls of Fig. 1 (tensors "A" = Q K^T and "B" = P V) are this call: heads side by side in a
+ * [tokens, heads*d] tensor give lda = heads*d, stride_a = d.  lda, ldw, stride_a, stride_w must be
+ * multiples of the block size and of 8.  Tensor-core kernel, one launch per batch item after one
+ * decode launch per operand; workspace from mx_gemm_batched_workspace_bytes.
+ */
+MX_API size_t mx_gemm_batched_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t batch);
+MX_API mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                                   int64_t lda, int64_t stride_a, const void *w_mant,
+                                   const uint8_t *w_exp, mx_format_t fw, int64_t ldw, int64_t stride_w,
+                                   int64_t M, int64_t N, int64_t K, int64_t batch, float *y,
+                                   int64_t ldy, int64_t stride_y, void *workspace,
+                                   size_t workspace_bytes, void *stream);
+
+/* The paper keeps LayerNorm, softmax and the activation function in floating point around the MX
+ * operators (Fig. 1(d)); these are plain fp32 row kernels.  cols <= 8192.
+ *   mx_layernorm : y[r,:] = (x[r,:] - mean) / sqrt(var + eps) * gamma + beta  (gamma/beta nullable)
+ *   mx_softmax   : in place, s[r,j] = softmax_j(scale * s[r,j]); with causal != 0 only columns
+ *                  j <= (r % rows_per_batch) take part and the rest become 0
+ *   mx_relu_add  : y[i] = (relu ? max(a[i], 0) : a[i]) + (b ? b[i] : 0); y may alias a or b */
+MX_API mx_status_t mx_layernorm(const float *x, int64_t ldx, const float *gamma, const float *beta,
+                                float eps, int64_t rows, int64_t cols, float *y, int64_t ldy,
+                                void *stream);
+MX_API mx_status_t mx_softmax(float *s, int64_t ld, int64_t rows, int64_t cols, float scale,
+                              int causal, int64_t rows_per_batch, void *stream);
+MX_API mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int relu,
+                               void *stream);
+
 /* ---- device status --------------------------------------------------------------------- */
 
 /*

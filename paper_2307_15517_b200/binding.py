@@ -80,6 +80,15 @@ def _load() -> C.CDLL:
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
     L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_poll_status.argtypes = [vp]
+    L.mx_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64]
+    L.mx_gemm_batched_workspace_bytes.restype = sz
+    L.mx_gemm_batched.argtypes = [vp, vp, F, i64, i64, vp, vp, F, i64, i64, i64, i64, i64, i64, vp, i64, i64,
+                                  vp, sz, vp]
+    L.mx_layernorm.argtypes = [vp, i64, vp, vp, C.c_float, i64, i64, vp, i64, vp]
+    L.mx_softmax.argtypes = [vp, i64, i64, i64, C.c_float, i32, i64, vp]
+    L.mx_relu_add.argtypes = [vp, vp, vp, i64, i32, vp]
+    for name in ("mx_gemm_batched", "mx_layernorm", "mx_softmax", "mx_relu_add"):
+        getattr(L, name).restype = i32
     L.mx_linear_grouped_workspace_bytes.argtypes = [C.POINTER(MxLinearArgs), i32]
     L.mx_linear_grouped_workspace_bytes.restype = sz
     L.mx_linear_grouped.argtypes = [C.POINTER(MxLinearArgs), i32, vp, sz, vp]
@@ -246,6 +255,50 @@ def mx_linear_grouped(args, workspace: Optional[torch.Tensor] = None, stream=Non
     _check(lib.mx_linear_grouped(args, len(args), _ptr(workspace), workspace.numel(), _stream(stream)),
            "mx_linear_grouped")
     return workspace
+
+
+def mx_gemm_batched(a_mant, a_exp, fa: MxFormat, lda: int, stride_a: int, w_mant, w_exp, fw: MxFormat,
+                    ldw: int, stride_w: int, M: int, N: int, K: int, batch: int, y: torch.Tensor,
+                    ldy: int, stride_y: int, workspace: Optional[torch.Tensor] = None, stream=None):
+    """`batch` products Y_b = A_b W_b^T on slices of packed tensors (strides in elements)."""
+    _need_cuda(a_mant, a_exp, w_mant, w_exp, y, workspace)
+    if workspace is None:
+        workspace = alloc_workspace(int(lib.mx_gemm_batched_workspace_bytes(M, N, K, batch)), y.device)
+    _check(lib.mx_gemm_batched(_ptr(a_mant), _ptr(a_exp), fa, lda, stride_a, _ptr(w_mant), _ptr(w_exp), fw,
+                               ldw, stride_w, M, N, K, batch, _ptr(y), ldy, stride_y, _ptr(workspace),
+                               workspace.numel(), _stream(stream)), "mx_gemm_batched")
+    return y
+
+
+def mx_layernorm(x: torch.Tensor, gamma, beta, eps: float, y: Optional[torch.Tensor] = None, stream=None):
+    _need_cuda(x, gamma, beta, y)
+    assert x.dim() == 2 and x.stride(1) == 1 and x.dtype == torch.float32
+    if y is None:
+        y = torch.empty_like(x)
+    _check(lib.mx_layernorm(_ptr(x), x.stride(0), _ptr(gamma), _ptr(beta), eps, x.shape[0], x.shape[1],
+                            _ptr(y), y.stride(0), _stream(stream)), "mx_layernorm")
+    return y
+
+
+def mx_softmax(s: torch.Tensor, scale: float = 1.0, causal: bool = False, rows_per_batch: int = 0, stream=None):
+    """In place over the rows of the 2-D fp32 tensor s."""
+    _need_cuda(s)
+    assert s.dim() == 2 and s.stride(1) == 1 and s.dtype == torch.float32
+    _check(lib.mx_softmax(_ptr(s), s.stride(0), s.shape[0], s.shape[1], scale, 1 if causal else 0,
+                          rows_per_batch, _stream(stream)), "mx_softmax")
+    return s
+
+
+def mx_relu_add(a: torch.Tensor, b: Optional[torch.Tensor], y: Optional[torch.Tensor] = None,
+                relu: bool = False, stream=None):
+    """y = (relu ? max(a, 0) : a) + b over contiguous fp32 tensors."""
+    _need_cuda(a, b, y)
+    assert a.is_contiguous() and (b is None or b.is_contiguous())
+    if y is None:
+        y = torch.empty_like(a)
+    _check(lib.mx_relu_add(_ptr(a), _ptr(b), _ptr(y), a.numel(), 1 if relu else 0, _stream(stream)),
+           "mx_relu_add")
+    return y
 
 
 MX_STATIC_SCRATCH_BYTES = 32 << 20

@@ -110,6 +110,13 @@ __device__ __forceinline__ float f32_scale(int ebyte, int w)
                         : __uint_as_float(e > 0 ? ((uint32_t)e << 23) : (1u << (22 + e)));
 }
 
+// Row and batch strides (bytes) of a packed source and (elements) of the decoded output.
+struct PackedStrides {
+    int64_t mant_ld, exp_ld;          // bytes between rows of the mantissa / exponent arrays
+    int64_t mant_batch, exp_batch;    // bytes between batch items
+    int64_t out_batch;                // elements between batch items of the output
+};
+
 struct QuantOut {
     uint8_t *mant;        // packed mantissas (nullable)
     uint8_t *exps;        // exponent bytes (nullable together with mant)
@@ -322,21 +329,24 @@ quantize_strided_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int6
 template <typename OutT>
 __global__ void __launch_bounds__(256)
 dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps, int64_t rows,
-                  int64_t K, int block, int w, OutT *__restrict__ out, int64_t ld_out)
+                  int64_t K, int block, int w, OutT *__restrict__ out, int64_t ld_out, PackedStrides ps)
 {
+    mant += (int64_t)blockIdx.y * ps.mant_batch;
+    exps += (int64_t)blockIdx.y * ps.exp_batch;
+    out += (int64_t)blockIdx.y * ps.out_batch;
     const int64_t chunks_per_row = K >> 3;
     const int64_t total = rows * chunks_per_row;
     for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total;
          c += (int64_t)gridDim.x * blockDim.x) {
         const int64_t row = c / chunks_per_row, kc = c - row * chunks_per_row;
-        const int ebyte = __ldg(exps + row * (K / block) + (kc * 8) / block);
+        const int ebyte = __ldg(exps + row * ps.exp_ld + (kc * 8) / block);
         int q[8];
         if (w <= 4) {
-            const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant + row * (K >> 1) + kc * 4));
+            const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant + row * ps.mant_ld + kc * 4));
 #pragma unroll
             for (int i = 0; i < 8; ++i) q[i] = ((int)(p << (28 - 4 * i))) >> 28;
         } else {
-            const uint2 p = __ldg(reinterpret_cast<const uint2 *>(mant + row * K + kc * 8));
+            const uint2 p = __ldg(reinterpret_cast<const uint2 *>(mant + row * ps.mant_ld + kc * 8));
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 q[i] = ((int)(p.x << (24 - 8 * i))) >> 24;
@@ -374,15 +384,20 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
 template <bool NIBBLE, int UNROLL>
 __global__ void __launch_bounds__(256)
 decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps, int64_t rows,
-                   int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out)
+                   int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out,
+                   PackedStrides ps)
 {
+    // blockIdx.y = batch item; rows of the packed source may be wider than K (a column slice)
+    mant += (int64_t)blockIdx.y * ps.mant_batch;
+    exps += (int64_t)blockIdx.y * ps.exp_batch;
+    out += (int64_t)blockIdx.y * ps.out_batch;
     const int lane = threadIdx.x & 31;
     const int ipr = (int)(K >> 5);                      // 32-element items per row
     const int segs = (ipr + 31) >> 5;
     const int64_t items = rows * segs;
     const bool b16 = block == 16;
     const int exp_shift = b16 ? 4 : 5;
-    const int64_t nb_row = K >> exp_shift;
+    const int64_t nb_row = ps.exp_ld;
     const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {
@@ -398,9 +413,9 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
             row[u] = (ok && kc[u] < ipr) ? r : -1;
             if (row[u] >= 0) {
                 if (NIBBLE) {
-                    m[u][0] = __ldcs(reinterpret_cast<const uint4 *>(mant + row[u] * (K >> 1) + kc[u] * 16));
+                    m[u][0] = __ldcs(reinterpret_cast<const uint4 *>(mant + row[u] * ps.mant_ld + kc[u] * 16));
                 } else {
-                    const uint4 *src = reinterpret_cast<const uint4 *>(mant + row[u] * K + kc[u] * 32);
+                    const uint4 *src = reinterpret_cast<const uint4 *>(mant + row[u] * ps.mant_ld + kc[u] * 32);
                     m[u][0] = __ldcs(src);
                     m[u][NIBBLE ? 0 : 1] = __ldcs(src + 1);
                 }

@@ -16,6 +16,7 @@
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
 #include "mx_gemv_stream.cuh"
+#include "mx_glue.cuh"
 #include "mx_quantize.cuh"
 
 namespace {
@@ -161,28 +162,47 @@ mx_status_t quantize_rows_any(const void *x, mx_dtype_t dt, int64_t rows, int64_
     return launch_quantize_rows(static_cast<const __nv_bfloat16 *>(x), rows, K, ldx, f, out, d, st);
 }
 
+mx::PackedStrides dense_strides(int64_t K, const mx_format_t &f)
+{
+    mx::PackedStrides ps;
+    ps.mant_ld = f.elem_bits <= 4 ? K / 2 : K;
+    ps.exp_ld = K / f.block;
+    ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+    return ps;
+}
+
+// (mant, exps) -> bf16 [rows, ld] for `batch` items laid out by `ps`.
+mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
+                                const mx_format_t &f, __nv_bfloat16 *out, int64_t ld,
+                                const mx::PackedStrides &ps, int64_t batch, const DeviceInfo &d,
+                                cudaStream_t st)
+{
+    const int64_t chunks = rows * (K / 8);
+    if (chunks == 0 || batch == 0) return MX_OK;
+    ProfScope prof(KIND_DEQUANTIZE, st);
+    const uint8_t *m = static_cast<const uint8_t *>(mant);
+    const bool wide_ok = (K % 32) == 0 && (ps.mant_ld % 16) == 0 && (ps.mant_batch % 16) == 0;
+    if (wide_ok) {                          // 32 elements per thread, 16-byte loads and stores
+        constexpr int UNROLL = 2;
+        const int64_t items = rows * (K / 32);
+        const dim3 grid((unsigned)grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, 8), (unsigned)batch);
+        if (f.elem_bits <= 4)
+            mx::decode_bf16_kernel<true, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
+        else
+            mx::decode_bf16_kernel<false, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
+    } else {
+        const dim3 grid((unsigned)grid_for(chunks, 256, d.sm_count, 16), (unsigned)batch);
+        mx::dequantize_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
+    }
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
                                 const mx_format_t &f, __nv_bfloat16 *out, int64_t ld,
                                 const DeviceInfo &d, cudaStream_t st)
 {
-    const int64_t chunks = rows * (K / 8);
-    if (chunks == 0) return MX_OK;
-    ProfScope prof(KIND_DEQUANTIZE, st);
-    const uint8_t *m = static_cast<const uint8_t *>(mant);
-    if ((K % 32) == 0) {                    // 32 elements per thread, 16-byte loads and stores
-        constexpr int UNROLL = 2;
-        const int64_t items = rows * (K / 32);
-        const int grid = grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, 8);
-        if (f.elem_bits <= 4)
-            mx::decode_bf16_kernel<true, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld);
-        else
-            mx::decode_bf16_kernel<false, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld);
-    } else {
-        mx::dequantize_kernel<__nv_bfloat16><<<grid_for(chunks, 256, d.sm_count, 16), 256, 0, st>>>(
-            m, exps, rows, K, f.block, f.elem_bits, out, ld);
-    }
-    MX_CUDA(cudaGetLastError());
-    return MX_OK;
+    return launch_dequant_bf16(mant, exps, rows, K, f, out, ld, dense_strides(K, f), 1, d, st);
 }
 
 // ---- tensor-core GEMM launcher ----------------------------------------------------------------
@@ -527,7 +547,7 @@ mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, i
     ProfScope prof(KIND_DEQUANTIZE, st);
     mx::dequantize_kernel<float><<<grid_for(rows * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
         static_cast<const uint8_t *>(mant), exps, rows, K, f.block, f.elem_bits,
-        static_cast<float *>(out), ld_out);
+        static_cast<float *>(out), ld_out, dense_strides(K, f));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -798,6 +818,117 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     return nt == 2 ? launch_stream<2, false>(sp, smem, grid, *d, st) : launch_stream<1, false>(sp, smem, grid, *d, st);
 }
 
+// ---- batched product (per-head attention matmuls) ------------------------------------------------
+size_t mx_gemm_batched_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t batch)
+{
+    if (M <= 0 || N <= 0 || K <= 0 || batch <= 0) return 0;
+    return (size_t)batch * (round256((size_t)M * K * 2) + round256((size_t)N * K * 2));
+}
+
+mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, int64_t lda,
+                            int64_t stride_a, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                            int64_t ldw, int64_t stride_w, int64_t M, int64_t N, int64_t K, int64_t batch,
+                            float *y, int64_t ldy, int64_t stride_y, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, nullptr, y, ldy);
+    if (s != MX_OK) return s;
+    if (!a_exp) return MX_ERR_NULL;
+    if (batch <= 0 || lda < K || ldw < K || stride_a < 0 || stride_w < 0 || stride_y < 0) return MX_ERR_SHAPE;
+    // row and batch strides must keep whole blocks and whole container bytes together
+    if ((lda % fa.block) || (ldw % fw.block) || (stride_a % fa.block) || (stride_w % fw.block) ||
+        (lda % 8) || (ldw % 8) || (stride_a % 8) || (stride_w % 8) || (stride_y % 4))
+        return MX_ERR_ALIGN;
+    if (!workspace || workspace_bytes < mx_gemm_batched_workspace_bytes(M, N, K, batch)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t a_item = round256((size_t)M * K * 2), w_item = round256((size_t)N * K * 2);
+    __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + (size_t)batch * a_item);
+    auto strides = [](const mx_format_t &f, int64_t ld, int64_t bstride, size_t out_item) {
+        mx::PackedStrides ps;
+        ps.mant_ld = f.elem_bits <= 4 ? ld / 2 : ld;
+        ps.exp_ld = ld / f.block;
+        ps.mant_batch = f.elem_bits <= 4 ? bstride / 2 : bstride;
+        ps.exp_batch = bstride / f.block;
+        ps.out_batch = (int64_t)(out_item / 2);
+        return ps;
+    };
+    // one decode launch per operand covers every batch item, then one product launch per item
+    s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, strides(fa, lda, stride_a, a_item), batch, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, strides(fw, ldw, stride_w, w_item), batch, *d, st);
+    if (s != MX_OK) return s;
+    for (int64_t b = 0; b < batch; ++b) {
+        s = run_tc(a_hat + b * (int64_t)(a_item / 2), w_hat + b * (int64_t)(w_item / 2), M, N, K, nullptr,
+                   y + b * stride_y, ldy, *d, st);
+        if (s != MX_OK) return s;
+    }
+    return MX_OK;
+}
+
+// ---- fp32 glue of the transformer block ---------------------------------------------------------
+mx_status_t mx_layernorm(const float *x, int64_t ldx, const float *gamma, const float *beta, float eps,
+                         int64_t rows, int64_t cols, float *y, int64_t ldy, void *stream)
+{
+    if (!x || !y) return MX_ERR_NULL;
+    if (rows < 0 || cols <= 0 || ldx < cols || ldy < cols || cols > mx::GLUE_THREADS * mx::GLUE_MAX_PER_THREAD)
+        return MX_ERR_SHAPE;
+    if (rows == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int per = (int)((cols + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);
+    const unsigned g = (unsigned)rows;
+    if (per <= 4) mx::layernorm_kernel<4><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
+    else if (per <= 8) mx::layernorm_kernel<8><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
+    else if (per <= 16) mx::layernorm_kernel<16><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
+    else mx::layernorm_kernel<32><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_softmax(float *s_inout, int64_t ld, int64_t rows, int64_t cols, float scale, int causal,
+                       int64_t rows_per_batch, void *stream)
+{
+    if (!s_inout) return MX_ERR_NULL;
+    if (rows < 0 || cols <= 0 || ld < cols || cols > mx::GLUE_THREADS * mx::GLUE_MAX_PER_THREAD ||
+        (causal && rows_per_batch <= 0))
+        return MX_ERR_SHAPE;
+    if (rows == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int per = (int)((cols + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);
+    const unsigned g = (unsigned)rows;
+    if (per <= 4) mx::softmax_kernel<4><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
+    else if (per <= 8) mx::softmax_kernel<8><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
+    else if (per <= 16) mx::softmax_kernel<16><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
+    else mx::softmax_kernel<32><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int relu, void *stream)
+{
+    if (!a || !y) return MX_ERR_NULL;
+    if (n < 0) return MX_ERR_SHAPE;
+    if (!aligned16(a) || !aligned16(y) || (b && !aligned16(b))) return MX_ERR_ALIGN;
+    if (n == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    mx::relu_add_kernel<<<grid_for((n + 3) / 4, mx::GLUE_THREADS, d->sm_count, 8), mx::GLUE_THREADS, 0, st>>>(a, b, y, n, relu);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 // ---- product without any allocation ---------------------------------------------------------
 // Scratch for mx_gemm_static: a fixed array in the library's device image.  In host code the
 // name below is only a handle for the runtime, never a device address; the address a kernel can
@@ -838,10 +969,10 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     // so nothing left by an earlier call is ever observed), then the tensor-core product.
     // Launches are issued directly: no event, no buffer and no handle is created on this path.
     mx::dequantize_kernel<__nv_bfloat16><<<grid_for(M * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
-        static_cast<const uint8_t *>(a_mant), a_exp, M, K, fa.block, fa.elem_bits, a_hat, K);
+        static_cast<const uint8_t *>(a_mant), a_exp, M, K, fa.block, fa.elem_bits, a_hat, K, dense_strides(K, fa));
     MX_CUDA(cudaGetLastError());
     mx::dequantize_kernel<__nv_bfloat16><<<grid_for(N * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
-        static_cast<const uint8_t *>(w_mant), w_exp, N, K, fw.block, fw.elem_bits, w_hat, K);
+        static_cast<const uint8_t *>(w_mant), w_exp, N, K, fw.block, fw.elem_bits, w_hat, K, dense_strides(K, fw));
     MX_CUDA(cudaGetLastError());
     constexpr int BN = 128;
     using Cfg = mx::TcCfg<BN>;

@@ -1,0 +1,84 @@
+"""One pre-LayerNorm transformer decoder block with every matmul in MXInt (the block of the paper's
+Fig. 1(d): linears, Q K^T and P V quantized; LayerNorm, softmax and ReLU in fp32).
+
+This module only sequences calls of the C ABI (through ``binding``): every arithmetic step runs in
+the library's kernels.  ``run`` returns the block output and, on request, every intermediate
+tensor so that each stage can be checked against the oracle on identical inputs.
+"""
+from __future__ import annotations
+
+import math
+from dataclasses import dataclass
+from typing import Dict, Optional
+
+import torch
+
+from . import binding as mxb
+
+
+@dataclass
+class BlockConfig:
+    hidden: int
+    heads: int
+    head_dim: int
+    ffn: int
+    block: int = 16
+    w_act: int = 8           # activations and both attention operands
+    w_wgt: int = 4           # weights of the linears
+    eps: float = 1e-5
+
+
+def quantize_weights(cfg: BlockConfig, weights: Dict[str, torch.Tensor]):
+    """weights: fp32 CUDA tensors wq, wk, wv, wo [hidden, hidden], w1 [ffn, hidden], w2 [hidden, ffn]."""
+    fw = mxb.MxFormat(cfg.block, cfg.w_wgt)
+    return {k: mxb.mx_quantize(v, fw) for k, v in weights.items()}
+
+
+def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Tensor],
+        keep: Optional[dict] = None) -> torch.Tensor:
+    """x: [seq, hidden] fp32 CUDA.  params: ln1_g, ln1_b, ln2_g, ln2_b, bq, bk, bv, bo, b1, b2."""
+    seq, hid, H, d = x.shape[0], cfg.hidden, cfg.heads, cfg.head_dim
+    assert hid == H * d
+    fa, fw = mxb.MxFormat(cfg.block, cfg.w_act), mxb.MxFormat(cfg.block, cfg.w_wgt)
+
+    def rec(name, t):
+        if keep is not None:
+            keep[name] = t
+        return t
+
+    def linear(inp, name, bias, n_out):
+        wm, we = qweights[name]
+        return mxb.mx_linear(inp, fa, wm, we, fw, n_out, bias=bias)
+
+    h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
+    q = rec("q", linear(h1, "wq", params["bq"], hid))
+    k = rec("k", linear(h1, "wk", params["bk"], hid))
+    v = rec("v", linear(h1, "wv", params["bv"], hid))
+    # attention scores per head: both operands MXInt, blocks along the head dimension
+    qm, qe = mxb.mx_quantize(q, fa)
+    km, ke = mxb.mx_quantize(k, fa)
+    s = torch.empty((H * seq, seq), dtype=torch.float32, device=x.device)
+    mxb.mx_gemm_batched(qm, qe, fa, hid, d, km, ke, fa, hid, d, seq, seq, d, H, s, seq, seq * seq)
+    rec("scores", s.clone() if keep is not None else s)
+    p = rec("probs", mxb.mx_softmax(s, 1.0 / math.sqrt(d), causal=True, rows_per_batch=seq))
+    # context per head: probabilities and values MXInt, blocks along the key/token axis
+    pm, pe = mxb.mx_quantize(p, fa)
+    vm, ve = mxb.mx_quantize(v.t(), fa)                      # [hidden, seq]: blocks along tokens
+    ctx = torch.empty((seq, hid), dtype=torch.float32, device=x.device)
+    mxb.mx_gemm_batched(pm, pe, fa, seq, seq * seq, vm, ve, fa, seq, d * seq, seq, d, seq, H, ctx, hid, d)
+    rec("ctx", ctx)
+    a = rec("attn_out", linear(ctx, "wo", params["bo"], hid))
+    x1 = rec("x1", mxb.mx_relu_add(a, x))
+    h2 = rec("ln2", mxb.mx_layernorm(x1, params["ln2_g"], params["ln2_b"], cfg.eps))
+    f = rec("ffn_pre", linear(h2, "w1", params["b1"], cfg.ffn))
+    f = rec("ffn_act", mxb.mx_relu_add(f, None, relu=True))
+    o = rec("ffn_out", linear(f, "w2", params["b2"], hid))
+    return rec("x2", mxb.mx_relu_add(o, x1))
+
+
+def flops(cfg: BlockConfig, seq: int) -> float:
+    """2*M*N*K of the eight MXInt matmuls of one block."""
+    hid, H, d = cfg.hidden, cfg.heads, cfg.head_dim
+    lin = 2.0 * seq * (4 * hid * hid + 2 * hid * cfg.ffn)
+    att = 2.0 * H * (seq * seq * d) * 2
+    return lin + att

@@ -345,3 +345,48 @@ def test_rejects_bad_arguments():
         orc.quantize(x, 16, 4)          # K not a multiple of the block
     with pytest.raises(ValueError):
         orc.quantize(np.zeros((2, 32), np.float32), 16, 9)
+
+
+# --------------------------------------------------------------------------- fp32 glue of the block
+
+def test_glue_oracle_against_library_routines():
+    import scipy.special
+    import torch
+    from oracle import block_oracle as blk
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((7, 96)) * 3 + 1
+    g, b = rng.standard_normal(96), rng.standard_normal(96)
+    want = torch.nn.functional.layer_norm(torch.from_numpy(x), (96,), torch.from_numpy(g), torch.from_numpy(b), 1e-5)
+    assert np.allclose(blk.layernorm(x, g, b, 1e-5), want.numpy(), rtol=1e-12, atol=1e-12)
+    y = blk.layernorm(x, None, None, 0.0)
+    assert np.allclose(y.mean(axis=1), 0, atol=1e-12) and np.allclose((y ** 2).mean(axis=1), 1, atol=1e-12)
+    s = rng.standard_normal((2 * 5, 5))                       # two batches of 5 query rows
+    p = blk.softmax_causal(s, 0.5, 5)
+    for r in range(10):
+        n = r % 5 + 1
+        assert np.allclose(p[r, :n], scipy.special.softmax(0.5 * s[r, :n]), rtol=1e-13)
+        assert (p[r, n:] == 0).all()
+    assert np.allclose(p.sum(axis=1), 1)
+    assert np.array_equal(blk.relu(np.array([-1.0, 0.0, 2.5])), np.array([0.0, 0.0, 2.5]))
+
+
+def test_attention_oracle_reduces_to_plain_matmul_on_representable_inputs():
+    from oracle import block_oracle as blk
+    rng = np.random.default_rng(22)
+    seq, H, d = 32, 2, 16
+    q = rng.integers(-127, 128, (seq, H * d)).astype(np.float32)
+    k = rng.integers(-127, 128, (seq, H * d)).astype(np.float32)
+    q[:, ::16] = 127
+    k[:, ::16] = -127                                         # every block's maximum uses the top bit
+    sc = blk.attention_scores(q, k, H, d, 16, 8)
+    for h in range(H):
+        want = q[:, h * d:(h + 1) * d].astype(np.float64) @ k[:, h * d:(h + 1) * d].astype(np.float64).T
+        assert np.array_equal(sc[h][0].astype(np.float64), want)
+    p = rng.integers(0, 128, (H * seq, seq)).astype(np.float32)
+    v = rng.integers(-127, 128, (seq, H * d)).astype(np.float32)
+    p[:, ::16] = 127
+    v[::16, :] = 127
+    ctx = blk.attention_context(p, v, H, d, 16, 8)
+    for h in range(H):
+        want = p[h * seq:(h + 1) * seq].astype(np.float64) @ v[:, h * d:(h + 1) * d].astype(np.float64)
+        assert np.array_equal(ctx[h][0].astype(np.float64), want)

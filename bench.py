@@ -210,6 +210,44 @@ def quantize_rate(mxb, torch, hbm_gbs, iters=20):
     return out
 
 
+def decoder_block_rate(mxb, synth, torch, iters=5):
+    """One full decoder block in MX at OPT-6.7B shapes (hidden 4096, 32 heads x 128, FFN 16384,
+    sequence 2048): six linears (A8/W4/B16), Q K^T and P V per head (A8/A8/B16), fp32 glue."""
+    from paper_2307_15517_b200 import decoder_block as db
+    sh = synth.decoder_block_shapes()
+    cfg = db.BlockConfig(hidden=sh["hidden"], heads=sh["heads"], head_dim=sh["head_dim"], ffn=sh["ffn"],
+                         block=sh["block"], w_act=sh["w_act"], w_wgt=sh["w_wgt"])
+    seq, hid, ffn = sh["seq"], sh["hidden"], sh["ffn"]
+    g = torch.Generator(device="cuda")
+    g.manual_seed(77)
+    rnd = lambda *shape: torch.randn(*shape, generator=g, device="cuda", dtype=torch.float32)
+    qw = db.quantize_weights(cfg, {n: rnd(o, i) * 0.02 for n, o, i in
+                                   (("wq", hid, hid), ("wk", hid, hid), ("wv", hid, hid), ("wo", hid, hid),
+                                    ("w1", ffn, hid), ("w2", hid, ffn))})
+    params = {n: rnd(sz) * 0.02 for n, sz in (("bq", hid), ("bk", hid), ("bv", hid), ("bo", hid), ("b1", ffn),
+                                              ("b2", hid), ("ln1_b", hid), ("ln2_b", hid))}
+    params["ln1_g"] = torch.ones(hid, device="cuda")
+    params["ln2_g"] = torch.ones(hid, device="cuda")
+    x = synth.outlier_activations(seq, hid, 4, -(-hid * 5 // 1000), 40.0).cuda()
+    for _ in range(2):
+        db.run(cfg, x, qw, params)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    mxb.mx_profile_begin()
+    a.record()
+    for _ in range(iters):
+        db.run(cfg, x, qw, params)
+    b.record()
+    torch.cuda.synchronize()
+    prof = mxb.mx_profile_end()
+    ms = a.elapsed_time(b) / iters
+    fl = db.flops(cfg, seq)
+    return {"ms_per_block": ms, "tops": fl / ms / 1e9, "flops": fl,
+            "kernels_ms": {k: v[0] / iters for k, v in prof.items() if v[1]},
+            "launches": sum(v[1] for v in prof.values()) / iters,
+            "note": "includes torch allocations of the intermediates; glue kernels are not in kernels_ms"}
+
+
 # ------------------------------------------------------------------------------ oracle (CPU)
 def oracle_inputs(orc, synth, sample_rows):
     """Untimed set-up: the first `sample_rows` tokens of every layer and its quantized weights."""
@@ -354,6 +392,7 @@ def run_ours(args):
         torch.cuda.empty_cache()
         secondary = {"decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
                      "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
+                     "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
         assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"
     barrier()

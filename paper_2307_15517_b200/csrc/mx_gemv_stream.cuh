@@ -13,11 +13,12 @@
 //  * tokens   : already quantized (int8 or nibble container); each CTA stages them once per
 //               layer into shared memory in the operand order of the integer MMA below, with
 //               their float block scales and the per-block sums needed to undo the +8 offset.
-//  * per block: nibble ^ 8 = q + 8 is an unsigned byte after one AND/shift, so a 16-row x 32-k
-//               tile of weights is the A operand of mma.sync.m16n8k32 (u8 x s8 -> s32) with no
-//               sign extension; the accumulator starts at 0x4B400000 - 8 * sum(qa), so the result
-//               register IS the float 1.5*2^23 + P (P = exact integer block sum), and two FMAs
-//               per output apply the weight scale (removing the 1.5*2^23) and the token scale.
+//  * per block: a two's-complement nibble moved into the HIGH half of a byte is the signed byte
+//               16*q, so one shift/AND pair turns a packed word into the A operand of
+//               mma.sync.m16n8k32 (s8 x s8 -> s32) with no sign extension; the accumulator starts
+//               at 0x4B400000, so the result register IS the float 1.5*2^23 + 16*P (P = exact
+//               integer block sum, |16 P| < 2^22), and two packed FMAs per output pair apply the
+//               weight scale (removing the 1.5*2^23) and the token scale (which carries the 1/16).
 //
 // A warp owns 16 weight rows.  With split > 1 the K range of a row tile is cut into `split`
 // contiguous pieces handled by consecutive warps of one CTA and summed in piece order through
@@ -79,7 +80,7 @@ template <int NT, bool BULK> struct StreamCfg {
     static constexpr int STAGE_BYTES = MANT_BYTES + 16 * CH;       // + 16 rows x 16 exponent bytes
     static constexpr uint32_t STAGE_TX = STAGE_BYTES;
     static constexpr int TP = NT * 8;                              // padded token count
-    static constexpr size_t tokens_bytes(int max_nb) { return (size_t)max_nb * TP * (32 + 8); }
+    static constexpr size_t tokens_bytes(int max_nb) { return (size_t)max_nb * TP * (32 + 4); }
     static constexpr size_t red_bytes() { return (size_t)WARPS * NT * 4 * 32 * 4; }
     static constexpr size_t smem_bytes(int max_nb)
     {
@@ -103,14 +104,14 @@ __device__ __forceinline__ void bulk_copy_g2s(uint32_t dst_smem, const void *src
                  : "memory");
 }
 
-__device__ __forceinline__ void mma_u8s8_m16n8k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
-                                                  uint32_t a3, uint32_t b0, uint32_t b1, int c0, int c1)
+__device__ __forceinline__ void mma_s8s8_m16n8k32(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                                  uint32_t a3, uint32_t b0, uint32_t b1, const int (&c)[4])
 {
     asm volatile(
-        "mma.sync.aligned.m16n8k32.row.col.s32.u8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+        "mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
         "{%10,%11,%12,%13};"
         : "=r"(d[0]), "=r"(d[1]), "=r"(d[2]), "=r"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c0), "r"(c1), "r"(c0), "r"(c1));
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1), "r"(c[0]), "r"(c[1]), "r"(c[2]), "r"(c[3]));
 }
 
 // Pairs of fp32 values in one 64-bit register and the sm_100 packed-pair arithmetic on them
@@ -154,13 +155,12 @@ gemv_stream_kernel(const StreamParams p)
     constexpr int TP = Cfg::TP, WARPS = Cfg::WARPS, STAGES = Cfg::STAGES, CH = Cfg::CH;
     extern __shared__ __align__(16) uint8_t smem[];
     uint2 *sB = reinterpret_cast<uint2 *>(smem);                 // [nb][TP][4]: (even-k word, odd-k word)
-    // [nb][TP/2] records {seed(tok 2i), seed(tok 2i+1), scale(tok 2i), scale(tok 2i+1)}: accumulator
-    // seeds and token scales; the token scale also carries the weights' binary point 2^-(ww-2), so
-    // the weight scale below is the plain 2^(Ew-127)
-    uint32_t *sCS = reinterpret_cast<uint32_t *>(smem + (size_t)p.max_nb * TP * 32);
+    // [nb][TP] token block scales; they also carry the weights' binary point 2^-(ww-2) and the 1/16
+    // of the shifted nibbles, so the weight scale below is the plain 2^(Ew-127)
+    float *sCS = reinterpret_cast<float *>(smem + (size_t)p.max_nb * TP * 32);
     // BULK: [WARPS][STAGES][4096] swizzled mantissa stages (1024-byte aligned), then
     // [WARPS][STAGES][256] exponent stages; the split-K exchange buffer [WARPS][NT][4][32] reuses them
-    uint8_t *sStage = reinterpret_cast<uint8_t *>(sCS + (size_t)p.max_nb * TP * 2);
+    uint8_t *sStage = reinterpret_cast<uint8_t *>(sCS + (size_t)p.max_nb * TP);
     if (BULK) sStage += (1024u - (ptx::smem_u32(sStage) & 1023u)) & 1023u;
     uint8_t *sExpStage = sStage + WARPS * STAGES * Cfg::MANT_BYTES;
     float *sRed = reinterpret_cast<float *>(sStage);
@@ -180,6 +180,9 @@ gemv_stream_kernel(const StreamParams p)
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int S = p.split, TPR = WARPS / S;                      // row tiles per round of the CTA
+    int swz[8];                               // this lane's byte offset of 16-byte chunk c in a swizzled box
+#pragma unroll
+    for (int c = 0; c < 8; ++c) swz[c] = g * 128 + ((c ^ g) << 4) + t * 4;
 
     const int per = (p.total_tiles + gridDim.x - 1) / gridDim.x;
     int tile_lo = blockIdx.x * per;
@@ -215,15 +218,10 @@ gemv_stream_kernel(const StreamParams p)
             }
             // MMA slots 4t..4t+3 take the even k of this group of 8, slots 16+4t.. the odd k
             sB[i] = make_uint2(__byte_perm(lo, hi, 0x6420), __byte_perm(lo, hi, 0x7531));
-            int sum = __dp4a((int)lo, 0x01010101, __dp4a((int)hi, 0x01010101, 0));
-            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 1);
-            sum += __shfl_xor_sync(0xFFFFFFFFu, sum, 2);         // the 4 groups of one block
             if (tq == 0) {
                 const int eb = tok < L.T ? (int)__ldg(L.a_exp + (int64_t)tok * nb + b) : 0;
-                const float sa = f32_scale(eb, L.a_bits) * small_neg_pow2(L.w_bits);     // exact
-                uint32_t *rec = sCS + ((b * TP + tok) >> 1) * 4 + (tok & 1);
-                rec[0] = (uint32_t)(STREAM_MAGIC_INT - 8 * sum);
-                rec[2] = __float_as_uint(sa);
+                // 2^(Ea-127-(wa-2)) * 2^-(ww-2) * 2^-4, every factor an exact power of two
+                sCS[b * TP + tok] = f32_scale(eb, L.a_bits) * small_neg_pow2(L.w_bits) * 0.0625f;
             }
         }
         __syncthreads();
@@ -251,6 +249,7 @@ gemv_stream_kernel(const StreamParams p)
                 auto compute_g = [&](int b, const Regs &r, auto top_c) {
                     constexpr bool TOP = decltype(top_c)::value;
                     const f32x2_t neg_magic = pack2(-STREAM_MAGIC, -STREAM_MAGIC);
+                    const int seed[4] = {STREAM_MAGIC_INT, STREAM_MAGIC_INT, STREAM_MAGIC_INT, STREAM_MAGIC_INT};
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
                         // weight scale 2^(E-127): exponent byte moved into the float's exponent field
@@ -260,18 +259,16 @@ gemv_stream_kernel(const StreamParams p)
                         const uint32_t ba = max(fa & 0x7F800000u, 0x00400000u), bb = max(fb & 0x7F800000u, 0x00400000u);
                         const f32x2_t swA = pack2u(ba, ba), swB = pack2u(bb, bb);
                         const f32x2_t mwA = fmul2(swA, neg_magic), mwB = fmul2(swB, neg_magic);
-                        const uint32_t a0 = (r.a[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
-                        const uint32_t a2 = ((r.a[j] >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
-                        const uint32_t a1 = (r.b[j] ^ 0x88888888u) & 0x0F0F0F0Fu;
-                        const uint32_t a3 = ((r.b[j] >> 4) ^ 0x08080808u) & 0x0F0F0F0Fu;
+                        // even-k nibbles shifted up, odd-k nibbles already in the high halves: bytes 16*q
+                        const uint32_t a0 = (r.a[j] << 4) & 0xF0F0F0F0u, a2 = r.a[j] & 0xF0F0F0F0u;
+                        const uint32_t a1 = (r.b[j] << 4) & 0xF0F0F0F0u, a3 = r.b[j] & 0xF0F0F0F0u;
                         const int blk = b + j;
 #pragma unroll
                         for (int n = 0; n < NT; ++n) {
                             const uint2 bf = sB[(blk * TP + n * 8 + g) * 4 + t];
-                            const uint4 cs = *reinterpret_cast<const uint4 *>(sCS + ((blk * TP + n * 8) / 2 + t) * 4);
-                            const f32x2_t sa = pack2u(cs.z, cs.w);
+                            const f32x2_t sa = *reinterpret_cast<const f32x2_t *>(sCS + blk * TP + n * 8 + 2 * t);
                             int d[4];
-                            mma_u8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, (int)cs.x, (int)cs.y);
+                            mma_s8s8_m16n8k32(d, a0, a1, a2, a3, bf.x, bf.y, seed);
                             f32x2_t pA, pB;                       // P * weight scale (rows g, g + 8), exact
                             if (!TOP) {
                                 pA = ffma2(pack2u((uint32_t)d[0], (uint32_t)d[1]), swA, mwA);
@@ -355,7 +352,7 @@ gemv_stream_kernel(const StreamParams p)
                                 // box (c >> 3); inside it the 16-byte chunk c & 7 of row r sits at
                                 // chunk (c & 7) ^ (r & 7); rows g and g + 8 share r & 7
                                 const int c = q * 4 + j;
-                                const int off = (c >> 3) * 2048 + g * 128 + (((c & 7) ^ g) << 4) + t * 4;
+                                const int off = (c >> 3) * 2048 + swz[c & 7];
                                 r.a[j] = *reinterpret_cast<const uint32_t *>(sm + off);
                                 r.b[j] = *reinterpret_cast<const uint32_t *>(sm + off + 8 * 128);
                             }

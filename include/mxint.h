@@ -278,7 +278,8 @@ MX_API mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_f
  * with a pair of CUDA events on the launch stream.  mx_profile_end waits for them and returns,
  * per kernel kind, the summed device time in milliseconds and the number of launches (arrays of
  * MX_KERNEL_KINDS entries, host memory).  Kinds: 0 quantize, 1 dequantize, 2 tensor-core GEMM,
- * 3 CUDA-core GEMM, 4 weight-streaming GEMM.  Not thread-safe with respect to concurrent
+ * 3 CUDA-core GEMM, 4 weight-streaming GEMM, 5 operand preparation of mx_linear (activation
+ * quantize + weight decode in one launch).  Not thread-safe with respect to concurrent
  * compute calls on other host threads being attributed correctly; meant for one stream. */
 #define MX_KERNEL_KINDS 8
 MX_API mx_status_t mx_profile_begin(void);

@@ -326,7 +326,7 @@ def mx_poll_status(stream=None) -> int:
     return int(lib.mx_poll_status(_stream(stream)))
 
 
-KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream")
+KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream", "prep")
 
 
 def mx_profile_begin() -> None:

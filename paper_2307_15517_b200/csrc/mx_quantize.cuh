@@ -382,15 +382,11 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
 // Requires K % 32 == 0 (rows of the packed tensor 16-byte aligned).  Element order and values
 // are those of dequantize_kernel.
 template <bool NIBBLE, int UNROLL>
-__global__ void __launch_bounds__(256)
-decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps, int64_t rows,
-                   int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out,
-                   PackedStrides ps)
+__device__ __forceinline__ void decode_bf16_body(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps,
+                                                 int64_t rows, int64_t K, int block, int w,
+                                                 __nv_bfloat16 *__restrict__ out, int64_t ld_out,
+                                                 const PackedStrides &ps, int64_t warp_id, int64_t n_warps)
 {
-    // blockIdx.y = batch item; rows of the packed source may be wider than K (a column slice)
-    mant += (int64_t)blockIdx.y * ps.mant_batch;
-    exps += (int64_t)blockIdx.y * ps.exp_batch;
-    out += (int64_t)blockIdx.y * ps.out_batch;
     const int lane = threadIdx.x & 31;
     const int ipr = (int)(K >> 5);                      // 32-element items per row
     const int segs = (ipr + 31) >> 5;
@@ -398,8 +394,6 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
     const bool b16 = block == 16;
     const int exp_shift = b16 ? 4 : 5;
     const int64_t nb_row = ps.exp_ld;
-    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
-    const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {
         uint4 m[UNROLL][NIBBLE ? 1 : 2];
         uint32_t e[UNROLL];
@@ -475,6 +469,57 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
 #pragma unroll
             for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[j][0], o[j][1], o[j][2], o[j][3]);
         }
+    }
+}
+
+
+template <bool NIBBLE, int UNROLL>
+__global__ void __launch_bounds__(256)
+decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ exps, int64_t rows,
+                   int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out,
+                   PackedStrides ps)
+{
+    // blockIdx.y = batch item; rows of the packed source may be wider than K (a column slice)
+    decode_bf16_body<NIBBLE, UNROLL>(mant + (int64_t)blockIdx.y * ps.mant_batch,
+                                     exps + (int64_t)blockIdx.y * ps.exp_batch, rows, K, block, w,
+                                     out + (int64_t)blockIdx.y * ps.out_batch, ld_out, ps,
+                                     (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5),
+                                     (int64_t)gridDim.x * (blockDim.x >> 5));
+}
+
+// Both operands of the tensor-core product in one launch: the first `q_blocks` CTAs quantize the
+// activations straight to their exact bf16 operand form, the remaining CTAs decode the packed
+// weights to theirs.  Two HBM-bound passes overlap instead of queueing behind each other.
+struct PrepJob {
+    const void *x;            // activations [M, K] of InT, leading dimension ldx
+    int64_t M, K, ldx;
+    int wa, block;
+    __nv_bfloat16 *a_hat;     // [M, K]
+    const uint8_t *w_mant, *w_exp;
+    int64_t N;
+    int ww;
+    __nv_bfloat16 *w_hat;     // [N, K]
+    int q_blocks;
+};
+
+template <typename InT, bool NIBBLE>
+__global__ void __launch_bounds__(256)
+prep_operands_kernel(const PrepJob j)
+{
+    const int warps = blockDim.x >> 5;
+    if ((int)blockIdx.x < j.q_blocks) {
+        QuantOut out{nullptr, nullptr, j.a_hat, j.K, nullptr};
+        const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)j.q_blocks * warps;
+        if (j.block == 16) quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
+        else quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
+    } else {
+        PackedStrides ps;
+        ps.mant_ld = NIBBLE ? j.K / 2 : j.K;
+        ps.exp_ld = j.K / j.block;
+        ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+        const int64_t wid = (int64_t)(blockIdx.x - j.q_blocks) * warps + (threadIdx.x >> 5);
+        const int64_t nw = (int64_t)(gridDim.x - j.q_blocks) * warps;
+        decode_bf16_body<NIBBLE, 2>(j.w_mant, j.w_exp, j.N, j.K, j.block, j.ww, j.w_hat, j.K, ps, wid, nw);
     }
 }
 

@@ -46,7 +46,7 @@ EncodeTiledFn g_encode_tiled = nullptr;
 
 // ---- launch profile: CUDA events around every kernel launch, summed per kernel kind ----------
 enum KernelKind { KIND_QUANTIZE = 0, KIND_DEQUANTIZE = 1, KIND_GEMM_TC = 2, KIND_GEMM_SIMT = 3,
-                  KIND_GEMM_STREAM = 4, KIND_COUNT = MX_KERNEL_KINDS };
+                  KIND_GEMM_STREAM = 4, KIND_PREP = 5, KIND_COUNT = MX_KERNEL_KINDS };
 struct ProfEntry { cudaEvent_t a, b; int kind; };
 struct Profiler {
     bool on = false;
@@ -643,10 +643,46 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
     // the activations' mantissas and exponents go straight to the MMA operand form (exact bf16)
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
+    if (fused) {
+        s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
+        if (s != MX_OK) return s;
+        return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+    }
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
+    if ((K % 32) == 0) {
+        // one launch prepares both operands: CTAs are split in proportion to the bytes each side moves
+        mx::PrepJob job;
+        job.x = x; job.M = M; job.K = K; job.ldx = ldx; job.wa = fa.elem_bits; job.block = fa.block;
+        job.a_hat = a_hat;
+        job.w_mant = static_cast<const uint8_t *>(w_mant); job.w_exp = w_exp; job.N = N; job.ww = fw.elem_bits;
+        job.w_hat = w_hat;
+        const double qb = (double)M * K * ((dt == MX_F32 ? 4.0 : 2.0) + 2.0);
+        const double db = (double)N * K * ((fw.elem_bits <= 4 ? 0.5 : 1.0) + 1.0 / fw.block + 2.0);
+        const int need_q = grid_for((M * (K / 8) + 1) / 2, 256, 1 << 20, 1);
+        const int need_d = grid_for((N * (K / 32) + 1) / 2, 256, 1 << 20, 1);
+        const int total = d->sm_count * 8;
+        int gq = (int)(total * qb / (qb + db) + 0.5);
+        gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
+        int gd = total - gq;
+        if (gq > need_q) gq = need_q;
+        if (gd > need_d) gd = need_d;
+        job.q_blocks = gq;
+        {
+            ProfScope prof(KIND_PREP, st);
+            const bool nib = fw.elem_bits <= 4;
+            if (dt == MX_F32) {
+                if (nib) mx::prep_operands_kernel<float, true><<<gq + gd, 256, 0, st>>>(job);
+                else mx::prep_operands_kernel<float, false><<<gq + gd, 256, 0, st>>>(job);
+            } else {
+                if (nib) mx::prep_operands_kernel<__nv_bfloat16, true><<<gq + gd, 256, 0, st>>>(job);
+                else mx::prep_operands_kernel<__nv_bfloat16, false><<<gq + gd, 256, 0, st>>>(job);
+            }
+            MX_CUDA(cudaGetLastError());
+        }
+        return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
+    }
     s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
     if (s != MX_OK) return s;
-    if (fused) return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
-    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);

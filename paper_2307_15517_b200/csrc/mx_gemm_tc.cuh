@@ -50,7 +50,8 @@ template <int BN> struct TcCfg {
     static constexpr uint32_t W_BYTES = BN * TC_BK * 2;
     static constexpr uint32_t STAGE_BYTES = A_BYTES + W_BYTES;
     static constexpr uint32_t BAR_BYTES = 256;
-    static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + BAR_BYTES + 1024; // + align slack
+    static constexpr uint32_t EPI_BYTES = 4 * 2 * 4096;    // per epilogue warp two 32x32 fp32 store buffers
+    static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024; // + align slack
     static constexpr uint32_t TMEM_COLS = 2 * BN;          // 256 or 512: powers of two
 };
 
@@ -60,6 +61,7 @@ struct TcParams {
     int64_t ldy;
     int M, N, K;
     int tiles_m, tiles_n;
+    int tma_store;   // 1: the epilogue writes Y with tiled TMA stores (needs ldy % 4 == 0)
     uint32_t *status;
     // fused modes only: the packed weight operand
     const uint8_t *w_mant;
@@ -77,7 +79,7 @@ template <int WMODE> struct RawItem {
 template <int BN, int WMODE>
 __global__ void __launch_bounds__(tc_threads(BN, WMODE), 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-               const TcParams p)
+               const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
 {
     using Cfg = TcCfg<BN>;
     constexpr bool FUSED = WMODE != W_BF16;
@@ -86,12 +88,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
 
-    const uint32_t bar_base = smem_base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t epi_base = smem_base + STAGES * Cfg::STAGE_BYTES;        // 1024-byte aligned
+    const uint32_t bar_base = epi_base + Cfg::EPI_BYTES;
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (STAGES + s); };
     auto tfull_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + a); };
     auto tempty_bar = [&](int a) { return bar_base + 8u * (2 * STAGES + 2 + a); };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + STAGES * Cfg::STAGE_BYTES + 8 * (2 * STAGES + 4));
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + STAGES * Cfg::STAGE_BYTES + Cfg::EPI_BYTES + 8 * (2 * STAGES + 4));
     volatile uint32_t *abort_flag = tmem_slot + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -315,6 +318,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     } else {
         const int quad = warp & 3;                          // TMEM lanes this warp may read
         int it = 0;
+        uint32_t epi_buf = 0;                               // alternates between the warp's two store buffers
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
@@ -336,7 +340,46 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
-                if (row < p.M && n < p.N) {
+                if (p.tma_store) {
+                    // Stage the 32x32 block in shared memory in the 128-byte swizzled box layout and let
+                    // one lane hand it to a tiled TMA store: full 128-byte lines reach L2, the store
+                    // clips rows >= M and columns >= N by itself.
+                    if (n < p.N && m0 + quad * 32 < p.M) {          // warp-uniform
+                        const uint32_t buf = epi_base + (uint32_t)((warp - 2) * 2 + (epi_buf & 1)) * 4096u;
+                        if (lane == 0) ptx::bulk_wait_group_read<1>();   // the buffer used two blocks ago is free
+                        __syncwarp();
+#pragma unroll
+                        for (int v = 0; v < 8; ++v) {
+                            float4 o;
+                            o.x = __uint_as_float(r[4 * v + 0]);
+                            o.y = __uint_as_float(r[4 * v + 1]);
+                            o.z = __uint_as_float(r[4 * v + 2]);
+                            o.w = __uint_as_float(r[4 * v + 3]);
+                            if (p.bias) {
+                                const int c = n + 4 * v;
+                                if (c + 4 <= p.N) {
+                                    const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + c));
+                                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                                } else {
+                                    if (c + 0 < p.N) o.x += __ldg(p.bias + c + 0);
+                                    if (c + 1 < p.N) o.y += __ldg(p.bias + c + 1);
+                                    if (c + 2 < p.N) o.z += __ldg(p.bias + c + 2);
+                                }
+                            }
+                            const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
+                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y),
+                                         "f"(o.z), "f"(o.w)
+                                         : "memory");
+                        }
+                        ptx::fence_proxy_async_smem();
+                        __syncwarp();
+                        if (lane == 0) {
+                            ptx::tma_store_2d(&tmap_y, n, m0 + quad * 32, buf);
+                            ptx::bulk_commit_group();
+                        }
+                        ++epi_buf;
+                    }
+                } else if (row < p.M && n < p.N) {
                     if (vec_ok && n + 32 <= p.N) {
 #pragma unroll
                         for (int v = 0; v < 8; ++v) {
@@ -364,6 +407,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             __syncwarp();
             if (lane == 0) ptx::mbar_arrive(tempty_bar(acc));
         }
+        if (p.tma_store && lane == 0) ptx::bulk_wait_group<0>();    // all of this warp's stores have landed
     }
 
     if (timed_out) {

@@ -239,6 +239,22 @@ struct PackedW {                 // weight operand of the fused kernels (unused 
     int bits = 0, block = 0;
 };
 
+mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int64_t ldy)
+{
+    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
+    const cuuint64_t strides[1] = {(cuuint64_t)ldy * 4};
+    const cuuint32_t box[2] = {32, 32};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled (output) failed (%d)", (int)r);
+        return MX_ERR_CUDA;
+    }
+    return MX_OK;
+}
+
 template <int BN, int WMODE>
 mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
                       int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
@@ -253,6 +269,12 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         if (s != MX_OK) return s;
     } else {
         tm_w = tm_a;                     // not read by the fused kernels
+    }
+    CUtensorMap tm_y = tm_a;             // placeholder when the epilogue stores directly
+    const bool tma_store = (ldy % 4) == 0;
+    if (tma_store) {
+        s = encode_f32_out(&tm_y, y, M, N, ldy);
+        if (s != MX_OK) return s;
     }
     constexpr int slot = BN == 256 ? 0 : 1;
     if (!d.tc_attr_set[slot][WMODE]) {
@@ -270,6 +292,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.status = d.status;
+    p.tma_store = tma_store ? 1 : 0;
     p.w_mant = pw.mant;
     p.w_exp = pw.exps;
     p.w_bits = pw.bits;
@@ -278,7 +301,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
     const int threads = mx::tc_threads(BN, WMODE);
     ProfScope prof(KIND_GEMM_TC, st);
-    mx::gemm_tc_kernel<BN, WMODE><<<grid, threads, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, p);
+    mx::gemm_tc_kernel<BN, WMODE><<<grid, threads, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, tm_y, p);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -1032,13 +1055,14 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.status = d->status;
+    p.tma_store = 0;
     p.w_mant = nullptr;
     p.w_exp = nullptr;
     p.w_bits = 0;
     p.block = 0;
     const int tiles = p.tiles_m * p.tiles_n;
     mx::gemm_tc_kernel<BN, mx::W_BF16><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
-        tm_a, tm_w, p);
+        tm_a, tm_w, tm_a, p);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }

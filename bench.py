@@ -313,6 +313,27 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+# ------------------------------------------------------------------------------ multi-rank bookkeeping
+def rank_seed(rank: int, set_index: int) -> int:
+    """Every rank works on its own token batches: distinct seeds per (rank, rotating set)."""
+    return N_SETS * rank + set_index
+
+
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of `values` (a list of floats) over all ranks of the default group;
+    the identity when no process group is up.  The slowest rank defines the job's time."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if dist is not None and dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_tops(world: int, flops_per_rank_step: float, steps: int, ms_total: float) -> float:
+    """Whole-job throughput: every rank does the same work on its own batch (weak scaling)."""
+    return world * flops_per_rank_step * steps / (ms_total * 1e-3) / 1e12
+
+
 # ------------------------------------------------------------------------------ GPU arm
 def run_ours(args):
     import torch
@@ -338,7 +359,7 @@ def run_ours(args):
     peaks, peaks_kind = load_peaks()
     # Step i works on set i % N_SETS (own activations, weights, workspace and outputs), so what a
     # step reads was last touched N_SETS steps ago and has long left the 126 MB L2.
-    sets = [build_device_workload(mxb, synth, torch, seed=N_SETS * rank + i) for i in range(N_SETS)]
+    sets = [build_device_workload(mxb, synth, torch, seed=rank_seed(rank, i)) for i in range(N_SETS)]
     layers = sets[0]
     tokens = synth.OPT13B_TOKENS
     flops_step = sum(layer_flops(tokens, L["spec"]) for L in layers)
@@ -387,7 +408,7 @@ def run_ours(args):
         barrier()
 
     secondary = None
-    if rank == 0 and not args.skip_secondary:
+    if world == 1 and not args.skip_secondary:          # single-GPU runs only
         del sets, layers
         torch.cuda.empty_cache()
         secondary = {"decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
@@ -397,14 +418,11 @@ def run_ours(args):
         assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"
     barrier()
 
-    t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total, ms_e2e = float(t[0]), float(t[1])
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, device="cuda")
 
     if rank == 0:
-        value = world * flops_step * args.steps / (ms_total * 1e-3) / 1e12
-        e2e_value = world * flops_step * args.steps / (ms_e2e * 1e-3) / 1e12
+        value = aggregate_tops(world, flops_step, args.steps, ms_total)
+        e2e_value = aggregate_tops(world, flops_step, args.steps, ms_e2e)
         gemm_ms, gemm_n = prof["gemm_tc"]
         achieved = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
         peak = peaks["bf16_tflops"]          # burst figure: the timed region lasts well under a second

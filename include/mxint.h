@@ -60,14 +60,14 @@ typedef enum { MX_F32 = 0, MX_BF16 = 1 } mx_dtype_t;
 
 /* Which kernel computes the block-scaled product. */
 typedef enum {
-    MX_ALGO_AUTO = 0,    /* mx_linear with M <= 16 and a streamable format: MX_ALGO_STREAM; everything
-                            else: MX_ALGO_TCGEN05                                                  */
+    MX_ALGO_AUTO = 0,    /* M <= 16 and a streamable format (see mx_linear_grouped): MX_ALGO_STREAM;
+                            everything else: MX_ALGO_TCGEN05                                       */
     MX_ALGO_SIMT = 1,    /* CUDA-core kernel: exact integer block sums, blocks added in ascending
                             order in fp32 (bit-reproducible; slow; mx_gemm needs no workspace)      */
     MX_ALGO_TCGEN05 = 2, /* tcgen05/TMEM tensor-core kernel on exactly decoded bf16 operands; a
                             separate pass decodes the packed weights into the workspace            */
-    MX_ALGO_STREAM = 3,  /* weight-streaming kernel for M <= 16 (decode), mx_linear only; see
-                            mx_linear_grouped for its restrictions                                 */
+    MX_ALGO_STREAM = 3,  /* weight-streaming kernel for M <= 16 (decode); see mx_linear_grouped for
+                            its restrictions                                                       */
     MX_ALGO_TCGEN05_FUSED = 4 /* the same tensor-core kernel with the packed weights decoded inside
                             it by extra warps (no bf16 copy of W: workspace holds the activations
                             only; needs K % 32 == 0 and a 2-byte aligned w_exp, else it falls back to

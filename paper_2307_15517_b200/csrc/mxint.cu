@@ -463,6 +463,10 @@ mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, Dev
 // =================================================================================================
 extern "C" {
 
+static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers,
+                                const uint8_t *const *packed_exps, void *workspace, size_t workspace_bytes,
+                                void *stream);
+
 size_t mx_mant_bytes(int64_t rows, int64_t K, mx_format_t f)
 {
     if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
@@ -583,7 +587,15 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
-    if (algo == MX_ALGO_AUTO) algo = MX_ALGO_TCGEN05;
+    {
+        mx_linear_args_t one;
+        one.x = a_mant; one.dt = MX_F32; one.M = M; one.K = K; one.ldx = K; one.fa = fa;
+        one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = ldy;
+        const bool can_stream = stream_layer_ok(one) && (reinterpret_cast<uintptr_t>(w_exp) & 3u) == 0 &&
+                                workspace && workspace_bytes >= stream_table_bytes(1);
+        if (algo == MX_ALGO_AUTO) algo = can_stream ? MX_ALGO_STREAM : MX_ALGO_TCGEN05;
+        if (algo == MX_ALGO_STREAM) return grouped_impl(&one, 1, &a_exp, workspace, workspace_bytes, stream);
+    }
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
@@ -734,8 +746,11 @@ size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, int32_t
     return total;
 }
 
-mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, void *workspace,
-                              size_t workspace_bytes, void *stream)
+// packed_exps == nullptr: layers[i].x are floating-point activations, quantized here.
+// packed_exps != nullptr: layers[i].x are mantissas already in format fa, packed_exps[i] their exponents.
+static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers,
+                                const uint8_t *const *packed_exps, void *workspace, size_t workspace_bytes,
+                                void *stream)
 {
     if (!layers) return MX_ERR_NULL;
     if (n_layers <= 0) return MX_ERR_SHAPE;
@@ -745,16 +760,17 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
         mx_status_t s = check_gemm_args(a.x, nullptr, a.fa, a.w_mant, a.w_exp, a.fw, a.M, a.N, a.K, a.bias,
                                         a.y, a.ldy);
         if (s != MX_OK) return s;
-        if (a.dt != MX_F32 && a.dt != MX_BF16) return MX_ERR_FORMAT;
-        if (a.ldx < a.K) return MX_ERR_SHAPE;
-        if ((a.ldx % 8) != 0 || (reinterpret_cast<uintptr_t>(a.w_exp) & 3u) != 0) return MX_ERR_ALIGN;
+        if (!packed_exps && a.dt != MX_F32 && a.dt != MX_BF16) return MX_ERR_FORMAT;
+        if (packed_exps && !packed_exps[i]) return MX_ERR_NULL;
+        if (!packed_exps && a.ldx < a.K) return MX_ERR_SHAPE;
+        if ((!packed_exps && (a.ldx % 8) != 0) || (reinterpret_cast<uintptr_t>(a.w_exp) & 3u) != 0) return MX_ERR_ALIGN;
         if (!stream_layer_ok(a)) return a.M > 16 || (a.K % 128) != 0 ? MX_ERR_SHAPE : MX_ERR_FORMAT;
         max_t = a.M > max_t ? (int)a.M : max_t;
         const int nb = (int)(a.K / 32);
         max_nb = nb > max_nb ? nb : max_nb;
         min_nb = nb < min_nb ? nb : min_nb;
     }
-    const size_t need = mx_linear_grouped_workspace_bytes(layers, n_layers);
+    const size_t need = packed_exps ? stream_table_bytes(n_layers) : mx_linear_grouped_workspace_bytes(layers, n_layers);
     if (!workspace || workspace_bytes < need) return MX_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
     const int nt = max_t > 8 ? 2 : 1;
@@ -791,9 +807,9 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     int total_tiles = 0;
     for (int i = 0; i < n_layers; ++i) {
         const mx_linear_args_t &a = layers[i];
-        for (int j = 0; j < i && !act_ptr[i]; ++j)
+        for (int j = 0; j < i && !act_ptr[i] && !packed_exps; ++j)
             if (same_activation(a, layers[j])) act_ptr[i] = act_ptr[j];
-        if (!act_ptr[i]) {
+        if (!act_ptr[i] && !packed_exps) {
             act_ptr[i] = ws + off;
             off += stream_act_bytes(a);
             mx::QuantJob job;
@@ -813,8 +829,8 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
         mx::StreamLayer &L = table[i];
         L.w_mant = static_cast<const uint8_t *>(a.w_mant);
         L.w_exp = a.w_exp;
-        L.a_mant = act_ptr[i];
-        L.a_exp = act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa));
+        L.a_mant = packed_exps ? static_cast<const uint8_t *>(a.x) : act_ptr[i];
+        L.a_exp = packed_exps ? packed_exps[i] : act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa));
         L.bias = a.bias;
         L.y = a.y;
         L.ldy = a.ldy;
@@ -837,8 +853,8 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     MX_CUDA(cudaMemcpyAsync(ws, table.data(), (size_t)n_layers * sizeof(mx::StreamLayer),
                             cudaMemcpyHostToDevice, st));
     // all distinct activation tensors are quantized by one launch per input type
-    MX_CUDA(cudaMemcpyAsync(ws + job_off, jobs.data(), jobs.size() * sizeof(mx::QuantJob), cudaMemcpyHostToDevice, st));
-    {
+    if (!jobs.empty()) {
+        MX_CUDA(cudaMemcpyAsync(ws + job_off, jobs.data(), jobs.size() * sizeof(mx::QuantJob), cudaMemcpyHostToDevice, st));
         const mx::QuantJob *dj = reinterpret_cast<const mx::QuantJob *>(ws + job_off);
         const dim3 qgrid((unsigned)grid_for((max_chunks + 1) / 2, 256, d->sm_count, 8), (unsigned)jobs.size());
         if (any_dt[0]) {
@@ -875,6 +891,12 @@ mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, 
     if (bulk)
         return nt == 2 ? launch_stream<2, true>(sp, smem, grid, *d, st) : launch_stream<1, true>(sp, smem, grid, *d, st);
     return nt == 2 ? launch_stream<2, false>(sp, smem, grid, *d, st) : launch_stream<1, false>(sp, smem, grid, *d, st);
+}
+
+mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_layers, void *workspace,
+                              size_t workspace_bytes, void *stream)
+{
+    return grouped_impl(layers, n_layers, nullptr, workspace, workspace_bytes, stream);
 }
 
 // ---- batched product (per-head attention matmuls) ------------------------------------------------

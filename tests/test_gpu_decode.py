@@ -113,6 +113,22 @@ def test_decode_shapes_sampled(mxb):
         assert (np.abs(got - y_ref) <= TOL * S + 1e-37).all()
 
 
+def test_gemm_on_packed_activations_streams_too(mxb):
+    """mx_gemm with already quantized tokens (M <= 16) takes the same kernel, no quantize launch."""
+    dev, ref = _layer(mxb, 8, 1024, 640, seed=77, with_bias=True)
+    y_ref, y_seq, S = _oracle(ref)
+    a_mant = torch.from_numpy(orc.pack(ref["qa"], 8)).cuda()
+    a_exp = torch.from_numpy(ref["ea"]).cuda()
+    for algo in (mxb.MX_ALGO_STREAM, mxb.MX_ALGO_AUTO):
+        y = mxb.mx_gemm(a_mant, a_exp, dev["fa"], dev["w_mant"], dev["w_exp"], dev["fw"], 8, 640, 1024,
+                        bias=dev["bias"], algo=algo)
+        err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+        assert (err <= TOL * S + 1e-37).all()
+    y_tc = mxb.mx_gemm(a_mant, a_exp, dev["fa"], dev["w_mant"], dev["w_exp"], dev["fw"], 8, 640, 1024,
+                       bias=dev["bias"], algo=mxb.MX_ALGO_TCGEN05)
+    assert (np.abs(y_tc.cpu().numpy().astype(np.float64) - y_ref) <= TOL * S + 1e-37).all()
+
+
 def test_stream_rejects_what_it_cannot_stage(mxb):
     dev, _ = _layer(mxb, 4, 256, 64, seed=1)
     with pytest.raises(mxb.MxError):                       # block 16 weights are not streamable

@@ -33,7 +33,7 @@ WORKLOAD = "opt-1.3b prefill linears, 2048 tokens, MXInt4 block 16 (4 layers per
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_tc_kernel<256,0>, averaged over the
 # four launches of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_opt13b_prefill.md
-GEMM_TC_DRAM_BYTES_PER_LAUNCH = 45.3e6
+GEMM_TC_DRAM_BYTES_PER_LAUNCH = 46.4e6
 
 
 def load_peaks():

@@ -125,6 +125,21 @@ bool format_ok(const mx_format_t &f)
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 size_t round256(size_t n) { return (n + 255u) & ~size_t(255); }
 
+// CTAs of `kernel` (256 threads, no dynamic shared memory) that are resident per SM; looked up once.
+template <typename K> int resident_ctas(K kernel)
+{
+    static std::mutex mu;
+    static std::map<const void *, int> cache;
+    std::lock_guard<std::mutex> lk(mu);
+    const void *key = reinterpret_cast<const void *>(kernel);
+    auto it = cache.find(key);
+    if (it != cache.end()) return it->second;
+    int n = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, 256, 0) != cudaSuccess || n < 1) n = 4;
+    cache[key] = n;
+    return n;
+}
+
 int grid_for(int64_t work_items, int threads, int sm_count, int ctas_per_sm)
 {
     int64_t g = (work_items + threads - 1) / threads;
@@ -143,7 +158,10 @@ mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t 
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
     constexpr int UNROLL = 2;
-    const int grid = grid_for((chunks + UNROLL - 1) / UNROLL, 256, d.sm_count, 8);
+    // at most one resident wave of CTAs: the grid-stride loop does the rest without a ragged second wave
+    const int per_sm = f.block == 16 ? resident_ctas(mx::quantize_rows_kernel<InT, 16, UNROLL>)
+                                     : resident_ctas(mx::quantize_rows_kernel<InT, 32, UNROLL>);
+    const int grid = grid_for((chunks + UNROLL - 1) / UNROLL, 256, d.sm_count, per_sm);
     ProfScope prof(KIND_QUANTIZE, st);
     if (f.block == 16)
         mx::quantize_rows_kernel<InT, 16, UNROLL><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
@@ -185,7 +203,9 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
     if (wide_ok) {                          // 32 elements per thread, 16-byte loads and stores
         constexpr int UNROLL = 2;
         const int64_t items = rows * (K / 32);
-        const dim3 grid((unsigned)grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, 8), (unsigned)batch);
+        const int per_sm = f.elem_bits <= 4 ? resident_ctas(mx::decode_bf16_kernel<true, UNROLL>)
+                                            : resident_ctas(mx::decode_bf16_kernel<false, UNROLL>);
+        const dim3 grid((unsigned)grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, per_sm), (unsigned)batch);
         if (f.elem_bits <= 4)
             mx::decode_bf16_kernel<true, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
         else
@@ -695,7 +715,12 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         const double db = (double)N * K * ((fw.elem_bits <= 4 ? 0.5 : 1.0) + 1.0 / fw.block + 2.0);
         const int need_q = grid_for((M * (K / 8) + 1) / 2, 256, 1 << 20, 1);
         const int need_d = grid_for((N * (K / 32) + 1) / 2, 256, 1 << 20, 1);
-        const int total = d->sm_count * 8;
+        const bool nibw = fw.elem_bits <= 4;
+        const int per_sm = dt == MX_F32 ? (nibw ? resident_ctas(mx::prep_operands_kernel<float, true>)
+                                                : resident_ctas(mx::prep_operands_kernel<float, false>))
+                                        : (nibw ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
+                                                : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>));
+        const int total = d->sm_count * per_sm;           // exactly one resident wave
         int gq = (int)(total * qb / (qb + db) + 0.5);
         gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
         int gd = total - gq;

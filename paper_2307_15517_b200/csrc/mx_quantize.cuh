@@ -148,49 +148,69 @@ template <> struct Load8<__nv_bfloat16> {
     }
 };
 
+// Largest magnitude so far, NaN-propagating (a NaN comes out as 0x7FFFFFFF, exponent field 255).
+__device__ __forceinline__ float absmax_nan(float m, float x)
+{
+    float d;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(d) : "f"(m), "f"(fabsf(x)));
+    return d;
+}
+
 // rows x K, rows contiguous along K with leading dimension ldx.  BLOCK in {16, 32}.
 //
 // Work item of a warp = (row, segment of 256 elements): lane l owns the 8 elements starting at
-// k = segment*256 + 8*l, so a warp reads 1 KB of fp32 contiguously and the index arithmetic is
-// paid once per 256 elements.  UNROLL items per warp and iteration have all their loads issued
+// k = segment*256 + 8*l, so a warp reads 1 KB of fp32 contiguously.  A warp walks its items with
+// a fixed stride; (row, segment) advance by the stride's quotient and remainder, so the only
+// divisions are at set-up.  UNROLL items per warp and iteration have all their loads issued
 // before any arithmetic (UNROLL * 32 bytes in flight per thread).
 //
-// Rounding without a conversion instruction: with v = x * 2^-E * 2^(w-2) clamped to
-// [-qmax, qmax], t = v + (1.5 * 2^23 + OFF) is rounded by the adder to an integer (nearest,
-// ties to even -- OFF is even, so ties fall on even q), and the low bits of t's pattern hold
-// q + OFF >= 1.  OFF = 8 (nibble container) or 128 (byte container) keeps every field
-// non-negative, so the fields of a word can be summed with shifts and the two's-complement
-// form restored by one XOR with 0x88888888 / 0x80808080.
+// Rounding without a multiply or a conversion: the block scale is s = 2^es, es = E-127-(w-2).
+// M = 1.5 * 2^(23+es) has ulp s, so the adder rounds x + M to a multiple of s (nearest, ties to
+// even; M's significand is even, so ties fall on even q) and the low bits of the sum's pattern
+// are those of M plus q.  Clamping the sum to [M - qmax*s, M + qmax*s] is the symmetric clamp of
+// q, and (sum - M) is the decoded value q*s, exactly.  The patterns of a word's 8 (4) values are
+// added up with shifts; one multiply-subtract removes M's pattern from every field and leaves
+// q + OFF >= 1 there (OFF = 8 / 128), one XOR restores two's complement.
+// M needs a biased exponent E + 25 - w <= 254: blocks above that (|x| >= 2^102) take the
+// multiply-based path below, as do blocks holding an Inf or NaN.
 template <typename InT, int BLOCK, int UNROLL>
 __device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, int64_t rows, int64_t K,
                                                    int64_t ldx, int w, const QuantOut &out,
                                                    int64_t warp_id, int64_t n_warps)
 {
     constexpr int LANES = BLOCK / 8;                    // lanes sharing one block
+    constexpr int LANE_SHIFT = BLOCK == 16 ? 1 : 2;
     const int lane = threadIdx.x & 31;
     const int cpr = (int)(K >> 3);                      // 8-element chunks per row
     const int segs = (cpr + 31) >> 5;                   // 256-element segments per row
-    const int64_t items = rows * segs;
     const bool nibble = w <= 4;
-    const float qmaxf = (float)((1 << (w - 1)) - 1);
-    const float pow2_wm2 = (float)(1 << (w - 2));
-    const float off = nibble ? 8.f : 128.f;
-    const float magic = 12582912.f + off;               // 1.5 * 2^23 + OFF
-    const uint32_t magic_bits = __float_as_uint(magic);
+    const int qmax = (1 << (w - 1)) - 1;
+    const uint32_t off = nibble ? 8u : 128u;
+    const int fast_top = 229 + w;                       // largest exponent byte of the add-only path
     const bool leader = (lane & (LANES - 1)) == 0;
+    const int64_t nb_row = K >> (BLOCK == 16 ? 4 : 5);
+    const int64_t mant_ld = nibble ? (K >> 1) : K;
 
-    for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {   // warp-uniform trip count
+    const int64_t step = n_warps * UNROLL;
+    const int64_t step_row = step / segs;
+    const int step_seg = (int)(step - step_row * segs);
+    int64_t row[UNROLL];
+    int seg[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const int64_t it = warp_id + u * n_warps;
+        row[u] = it / segs;
+        seg[u] = (int)(it - row[u] * segs);
+    }
+
+    while (row[0] < rows) {                             // warp-uniform: items ascend with u
         float v[UNROLL][8];
-        int64_t row[UNROLL];
         int kc[UNROLL];
         bool live[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const int64_t it = it0 + u * n_warps;
-            const bool ok = it < items;
-            row[u] = ok ? it / segs : 0;
-            kc[u] = (int)(ok ? it - row[u] * segs : 0) * 32 + lane;
-            live[u] = ok && kc[u] < cpr;
+            kc[u] = seg[u] * 32 + lane;
+            live[u] = row[u] < rows && kc[u] < cpr;
             if (live[u]) {
                 Load8<InT>::run(x + row[u] * ldx + (int64_t)kc[u] * 8, v[u]);
             } else {
@@ -200,57 +220,76 @@ __device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, in
         }
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            uint32_t amax = 0;
+            float am = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) amax = max(amax, __float_as_uint(v[u][i]) & 0x7FFFFFFFu);
+            for (int i = 0; i < 8; ++i) am = absmax_nan(am, v[u][i]);
+            uint32_t amax = __float_as_uint(am);
 #pragma unroll
             for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
-            if (!live[u]) continue;
-            const int ebyte = (int)(amax >> 23);            // 255 <=> an Inf or NaN in the block
-            const bool bad = ebyte == 255;
-            const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
-            float t[8];                                     // magic + OFF + q, exactly
+            if (live[u]) {
+                const int ebyte = (int)(amax >> 23);        // 255 <=> an Inf or NaN in the block
+                const bool bad = ebyte == 255;
+                uint32_t f[8];                              // per value: corr + OFF + q
+                float xh[8];                                // decoded values (when asked for)
+                uint32_t corr;
+                if (ebyte <= fast_top) {
+                    const uint32_t mb = ((uint32_t)(ebyte + 25 - w) << 23) | 0x00400000u;
+                    const float M = __uint_as_float(mb);
+                    const float lo = __uint_as_float(mb - (uint32_t)qmax), hi = __uint_as_float(mb + (uint32_t)qmax);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                const float s = (v[u][i] * inv_pow2_E) * pow2_wm2;          // exact scaling
-                t[i] = fminf(fmaxf(s, -qmaxf), qmaxf) + magic;              // clamp, then round
-            }
-            if (out.mant) {
-                if (nibble) {
-                    uint32_t p = 0;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) p += (__float_as_uint(t[i]) - magic_bits + 8u) << (4 * i);
-                    p ^= 0x88888888u;
-                    *reinterpret_cast<uint32_t *>(out.mant + row[u] * (K >> 1) + (int64_t)kc[u] * 4) = bad ? 0u : p;
-                } else {
-                    uint2 p = make_uint2(0, 0);
-#pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        p.x += (__float_as_uint(t[i]) - magic_bits + 128u) << (8 * i);
-                        p.y += (__float_as_uint(t[4 + i]) - magic_bits + 128u) << (8 * i);
+                    for (int i = 0; i < 8; ++i) {
+                        const float t = fminf(fmaxf(v[u][i] + M, lo), hi);
+                        f[i] = __float_as_uint(t);
+                        xh[i] = t - M;
                     }
-                    p.x ^= 0x80808080u;
-                    p.y ^= 0x80808080u;
-                    if (bad) p = make_uint2(0, 0);
-                    *reinterpret_cast<uint2 *>(out.mant + row[u] * K + (int64_t)kc[u] * 8) = p;
-                }
-                if (leader) out.exps[row[u] * (K / BLOCK) + kc[u] / LANES] = (uint8_t)ebyte;
-            }
-            if (out.xhat) {
-                // decoded value q * 2^-(w-2) * 2^E as bf16 (exact: <= 7 significant bits)
-                const float dec_small = small_neg_pow2(w), dec_big = pow2_from_biased(bad ? 127 : ebyte);
-                uint32_t h[4];
+                    corr = mb - off;
+                } else {
+                    const float qmaxf = (float)qmax, pow2_wm2 = (float)(1 << (w - 2));
+                    const float magic = 12582912.f;         // 1.5 * 2^23: adding it rounds to an integer
+                    const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
+                    const float dec_small = small_neg_pow2(w), dec_big = pow2_from_biased(bad ? 127 : ebyte);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float lo = ((t[2 * i] - magic) * dec_small) * dec_big;
-                    const float hi = ((t[2 * i + 1] - magic) * dec_small) * dec_big;
-                    const __nv_bfloat162 pr = __floats2bfloat162_rn(lo, hi);
-                    h[i] = bad ? 0x7FC07FC0u : *reinterpret_cast<const uint32_t *>(&pr);
+                    for (int i = 0; i < 8; ++i) {
+                        const float s = (v[u][i] * inv_pow2_E) * pow2_wm2;              // exact scaling
+                        const float t = fminf(fmaxf(s, -qmaxf), qmaxf) + magic;         // clamp, then round
+                        f[i] = bad ? off : __float_as_uint(t) - 0x4B400000u + off;
+                        xh[i] = bad ? __uint_as_float(0x7FC00000u) : ((t - magic) * dec_small) * dec_big;
+                    }
+                    corr = 0;
                 }
-                *reinterpret_cast<uint4 *>(out.xhat + row[u] * out.ld_xhat + (int64_t)kc[u] * 8) =
-                    make_uint4(h[0], h[1], h[2], h[3]);
+                if (out.mant) {
+                    if (nibble) {
+                        uint32_t p = 0;
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) p += f[i] << (4 * i);
+                        p = (p - corr * 0x11111111u) ^ 0x88888888u;
+                        *reinterpret_cast<uint32_t *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 4) = p;
+                    } else {
+                        uint2 p = make_uint2(0, 0);
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) {
+                            p.x += f[i] << (8 * i);
+                            p.y += f[4 + i] << (8 * i);
+                        }
+                        p.x = (p.x - corr * 0x01010101u) ^ 0x80808080u;
+                        p.y = (p.y - corr * 0x01010101u) ^ 0x80808080u;
+                        *reinterpret_cast<uint2 *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 8) = p;
+                    }
+                    if (leader) out.exps[row[u] * nb_row + (kc[u] >> LANE_SHIFT)] = (uint8_t)ebyte;
+                }
+                if (out.xhat) {
+                    // q * 2^(E-127-(w-2)) as bf16 (exact: <= 7 significant bits)
+                    uint32_t h[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) h[i] = as_u32(__floats2bfloat162_rn(xh[2 * i], xh[2 * i + 1]));
+                    *reinterpret_cast<uint4 *>(out.xhat + row[u] * out.ld_xhat + (int64_t)kc[u] * 8) =
+                        make_uint4(h[0], h[1], h[2], h[3]);
+                }
+                if (bad && leader && out.nonfinite) atomicAdd(out.nonfinite, 1u);
             }
-            if (bad && leader && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+            row[u] += step_row;
+            seg[u] += step_seg;
+            if (seg[u] >= segs) { seg[u] -= segs; ++row[u]; }
         }
     }
 }
@@ -335,11 +374,18 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
     exps += (int64_t)blockIdx.y * ps.exp_batch;
     out += (int64_t)blockIdx.y * ps.out_batch;
     const int64_t chunks_per_row = K >> 3;
-    const int64_t total = rows * chunks_per_row;
-    for (int64_t c = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; c < total;
-         c += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t row = c / chunks_per_row, kc = c - row * chunks_per_row;
-        const int ebyte = __ldg(exps + row * ps.exp_ld + (kc * 8) / block);
+    const int exp_shift = block == 16 ? 1 : 2;          // 8-element chunks per block, as a shift
+    // chunks are walked with a fixed stride: (row, chunk) advance by its quotient and remainder
+    const int64_t step = (int64_t)gridDim.x * blockDim.x;
+    const int64_t step_row = step / chunks_per_row, step_kc = step - step_row * chunks_per_row;
+    const int64_t first = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    int64_t row = first / chunks_per_row, kc = first - row * chunks_per_row;
+    for (; row < rows; row += step_row, kc += step_kc) {
+        if (kc >= chunks_per_row) {
+            kc -= chunks_per_row;
+            if (++row >= rows) break;
+        }
+        const int ebyte = __ldg(exps + row * ps.exp_ld + (kc >> exp_shift));
         int q[8];
         if (w <= 4) {
             const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant + row * ps.mant_ld + kc * 4));
@@ -390,21 +436,32 @@ __device__ __forceinline__ void decode_bf16_body(const uint8_t *__restrict__ man
     const int lane = threadIdx.x & 31;
     const int ipr = (int)(K >> 5);                      // 32-element items per row
     const int segs = (ipr + 31) >> 5;
-    const int64_t items = rows * segs;
     const bool b16 = block == 16;
     const int exp_shift = b16 ? 4 : 5;
     const int64_t nb_row = ps.exp_ld;
-    for (int64_t it0 = warp_id; it0 < items; it0 += n_warps * UNROLL) {
+    // items are walked with a fixed stride: (row, segment) advance by its quotient and remainder
+    const int64_t step = n_warps * UNROLL;
+    const int64_t step_row = step / segs;
+    const int step_seg = (int)(step - step_row * segs);
+    int64_t cur_row[UNROLL];
+    int cur_seg[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) {
+        const int64_t it = warp_id + u * n_warps;
+        cur_row[u] = it / segs;
+        cur_seg[u] = (int)(it - cur_row[u] * segs);
+    }
+    while (cur_row[0] < rows) {                         // warp-uniform: items ascend with u
         uint4 m[UNROLL][NIBBLE ? 1 : 2];
         uint32_t e[UNROLL];
         int64_t row[UNROLL], kc[UNROLL];
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
-            const int64_t it = it0 + u * n_warps;
-            const bool ok = it < items;
-            const int64_t r = ok ? it / segs : 0;
-            kc[u] = (ok ? it - r * segs : 0) * 32 + lane;
-            row[u] = (ok && kc[u] < ipr) ? r : -1;
+            kc[u] = cur_seg[u] * 32 + lane;
+            row[u] = (cur_row[u] < rows && kc[u] < ipr) ? cur_row[u] : -1;
+            cur_row[u] += step_row;
+            cur_seg[u] += step_seg;
+            if (cur_seg[u] >= segs) { cur_seg[u] -= segs; ++cur_row[u]; }
             if (row[u] >= 0) {
                 if (NIBBLE) {
                     m[u][0] = __ldcs(reinterpret_cast<const uint4 *>(mant + row[u] * ps.mant_ld + kc[u] * 16));

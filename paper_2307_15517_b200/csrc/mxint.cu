@@ -478,6 +478,53 @@ mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, Dev
     return MX_OK;
 }
 
+
+// Both operands of one layer in the tensor-core form: activations quantized straight to exact
+// bf16, packed weights decoded to bf16.  One launch when K % 32 == 0, else two.
+mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfloat16 *w_hat, DeviceInfo &d,
+                       cudaStream_t st)
+{
+    const int64_t M = a.M, N = a.N, K = a.K;
+    mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
+    if ((K % 32) != 0) {
+        mx_status_t s = quantize_rows_any(a.x, a.dt, M, K, a.ldx, a.fa, out, d, st);
+        if (s != MX_OK) return s;
+        return launch_dequant_bf16(a.w_mant, a.w_exp, N, K, a.fw, w_hat, K, d, st);
+    }
+    // CTAs are split between the two sides in proportion to the bytes each moves
+    mx::PrepJob job;
+    job.x = a.x; job.M = M; job.K = K; job.ldx = a.ldx; job.wa = a.fa.elem_bits; job.block = a.fa.block;
+    job.a_hat = a_hat;
+    job.w_mant = static_cast<const uint8_t *>(a.w_mant); job.w_exp = a.w_exp; job.N = N; job.ww = a.fw.elem_bits;
+    job.w_hat = w_hat;
+    const bool f32 = a.dt == MX_F32, nib = a.fw.elem_bits <= 4;
+    const double qb = (double)M * K * ((f32 ? 4.0 : 2.0) + 2.0);
+    const double db = (double)N * K * ((nib ? 0.5 : 1.0) + 1.0 / a.fw.block + 2.0);
+    const int need_q = grid_for((M * (K / 8) + 1) / 2, 256, 1 << 20, 1);
+    const int need_d = grid_for((N * (K / 32) + 1) / 2, 256, 1 << 20, 1);
+    const int per_sm = f32 ? (nib ? resident_ctas(mx::prep_operands_kernel<float, true>)
+                            : resident_ctas(mx::prep_operands_kernel<float, false>))
+                     : (nib ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
+                            : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>));
+    const int total = d.sm_count * per_sm;            // exactly one resident wave
+    int gq = (int)(total * qb / (qb + db) + 0.5);
+    gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
+    int gd = total - gq;
+    if (gq > need_q) gq = need_q;
+    if (gd > need_d) gd = need_d;
+    job.q_blocks = gq;
+    ProfScope prof(KIND_PREP, st);
+    if (f32) {
+        if (nib) mx::prep_operands_kernel<float, true><<<gq + gd, 256, 0, st>>>(job);
+        else mx::prep_operands_kernel<float, false><<<gq + gd, 256, 0, st>>>(job);
+    } else {
+        if (nib) mx::prep_operands_kernel<__nv_bfloat16, true><<<gq + gd, 256, 0, st>>>(job);
+        else mx::prep_operands_kernel<__nv_bfloat16, false><<<gq + gd, 256, 0, st>>>(job);
+    }
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 }  // namespace
 
 // =================================================================================================
@@ -704,46 +751,7 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
     }
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
-    if ((K % 32) == 0) {
-        // one launch prepares both operands: CTAs are split in proportion to the bytes each side moves
-        mx::PrepJob job;
-        job.x = x; job.M = M; job.K = K; job.ldx = ldx; job.wa = fa.elem_bits; job.block = fa.block;
-        job.a_hat = a_hat;
-        job.w_mant = static_cast<const uint8_t *>(w_mant); job.w_exp = w_exp; job.N = N; job.ww = fw.elem_bits;
-        job.w_hat = w_hat;
-        const double qb = (double)M * K * ((dt == MX_F32 ? 4.0 : 2.0) + 2.0);
-        const double db = (double)N * K * ((fw.elem_bits <= 4 ? 0.5 : 1.0) + 1.0 / fw.block + 2.0);
-        const int need_q = grid_for((M * (K / 8) + 1) / 2, 256, 1 << 20, 1);
-        const int need_d = grid_for((N * (K / 32) + 1) / 2, 256, 1 << 20, 1);
-        const bool nibw = fw.elem_bits <= 4;
-        const int per_sm = dt == MX_F32 ? (nibw ? resident_ctas(mx::prep_operands_kernel<float, true>)
-                                                : resident_ctas(mx::prep_operands_kernel<float, false>))
-                                        : (nibw ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
-                                                : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>));
-        const int total = d->sm_count * per_sm;           // exactly one resident wave
-        int gq = (int)(total * qb / (qb + db) + 0.5);
-        gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
-        int gd = total - gq;
-        if (gq > need_q) gq = need_q;
-        if (gd > need_d) gd = need_d;
-        job.q_blocks = gq;
-        {
-            ProfScope prof(KIND_PREP, st);
-            const bool nib = fw.elem_bits <= 4;
-            if (dt == MX_F32) {
-                if (nib) mx::prep_operands_kernel<float, true><<<gq + gd, 256, 0, st>>>(job);
-                else mx::prep_operands_kernel<float, false><<<gq + gd, 256, 0, st>>>(job);
-            } else {
-                if (nib) mx::prep_operands_kernel<__nv_bfloat16, true><<<gq + gd, 256, 0, st>>>(job);
-                else mx::prep_operands_kernel<__nv_bfloat16, false><<<gq + gd, 256, 0, st>>>(job);
-            }
-            MX_CUDA(cudaGetLastError());
-        }
-        return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
-    }
-    s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
-    if (s != MX_OK) return s;
-    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    s = tc_prepare(one, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }

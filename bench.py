@@ -169,14 +169,18 @@ def decode_sweep(mxb, synth, torch, hbm_gbs, iters=10):
             mxb.mx_linear_grouped(args, ws)
         torch.cuda.synchronize()
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        mxb.mx_profile_begin()
         a.record()
         for _ in range(iters):
             mxb.mx_linear_grouped(args, ws)
         b.record()
         torch.cuda.synchronize()
-        prof = mxb.mx_profile_end()
         ms_call = a.elapsed_time(b) / iters
+        # the same calls again with the library's per-kernel events (they add gaps between launches)
+        mxb.mx_profile_begin()
+        for _ in range(iters):
+            mxb.mx_linear_grouped(args, ws)
+        torch.cuda.synchronize()
+        prof = mxb.mx_profile_end()
         ms_kernel = prof["gemm_stream"][0] / iters
         out["tokens_%d" % T] = {
             "ms_per_call": ms_call, "gbs_call": wbytes / ms_call / 1e6,

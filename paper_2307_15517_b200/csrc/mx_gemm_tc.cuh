@@ -122,6 +122,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     __syncthreads();
     ptx::tc_fence_after_sync();
     const uint32_t tmem_base = *tmem_slot;
+    // Everything above is private to this CTA; from here on global memory is read and written.
+    ptx::dep_wait();
+    if (threadIdx.x == 0) ptx::dep_trigger();
 
     const int num_tiles = p.tiles_m * p.tiles_n;
     const int kblocks = (p.K + TC_BK - 1) / TC_BK;

@@ -177,6 +177,8 @@ gemv_stream_kernel(const StreamParams p)
         __syncthreads();
     }
 
+    ptx::dep_wait();                          // the quantized tokens come from the previous launch
+    if (threadIdx.x == 0) ptx::dep_trigger();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int g = lane >> 2, t = lane & 3;
     const int S = p.split, TPR = WARPS / S;                      // row tiles per round of the CTA

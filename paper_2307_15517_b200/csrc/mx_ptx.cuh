@@ -19,6 +19,15 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
     return t;
 }
 
+// ---- programmatic dependent launch ---------------------------------------------------------------
+// A kernel launched with the programmatic-stream-serialization attribute may become resident while
+// its predecessor in the stream still runs.  dep_wait() blocks until every predecessor grid has
+// completed and its memory is visible (a no-op for an ordinary launch): nothing before it may touch
+// global memory that another kernel writes or reads.  dep_trigger() lets the next kernel of the
+// stream be scheduled once every CTA of this grid has called it or exited.
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void dep_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---- mbarrier -----------------------------------------------------------------------------
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
 {

@@ -5,6 +5,7 @@
 // cover one block exchange their largest magnitude with warp shuffles, so the shared exponent
 // costs no shared memory and no second pass over the data.
 #pragma once
+#include "mx_ptx.cuh"
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -299,6 +300,8 @@ __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w,
                      QuantOut out)
 {
+    ptx::dep_wait();
+    ptx::dep_trigger();
     quantize_rows_body<InT, BLOCK, UNROLL>(x, rows, K, ldx, w, out,
                                            (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5),
                                            (int64_t)gridDim.x * (blockDim.x >> 5));
@@ -317,6 +320,8 @@ template <typename InT, int DT>
 __global__ void __launch_bounds__(256)
 quantize_multi_kernel(const QuantJob *__restrict__ jobs)
 {
+    ptx::dep_wait();
+    ptx::dep_trigger();
     const QuantJob j = jobs[blockIdx.y];
     if (j.dt != DT) return;
     const int64_t warp_id = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -536,6 +541,8 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
                    int64_t K, int block, int w, __nv_bfloat16 *__restrict__ out, int64_t ld_out,
                    PackedStrides ps)
 {
+    ptx::dep_wait();
+    ptx::dep_trigger();
     // blockIdx.y = batch item; rows of the packed source may be wider than K (a column slice)
     decode_bf16_body<NIBBLE, UNROLL>(mant + (int64_t)blockIdx.y * ps.mant_batch,
                                      exps + (int64_t)blockIdx.y * ps.exp_batch, rows, K, block, w,
@@ -563,6 +570,8 @@ template <typename InT, bool NIBBLE>
 __global__ void __launch_bounds__(256)
 prep_operands_kernel(const PrepJob j)
 {
+    ptx::dep_wait();
+    ptx::dep_trigger();
     const int warps = blockDim.x >> 5;
     if ((int)blockIdx.x < j.q_blocks) {
         QuantOut out{nullptr, nullptr, j.a_hat, j.K, nullptr};

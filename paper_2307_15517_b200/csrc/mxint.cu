@@ -149,6 +149,27 @@ int grid_for(int64_t work_items, int threads, int sm_count, int ctas_per_sm)
     return (int)g;
 }
 
+// Launch that may overlap the tail of the previous kernel in the stream (programmatic dependent
+// launch): the kernel becomes resident early, sets up, and blocks in ptx::dep_wait() until its
+// predecessor has completed.  Only for kernels that call dep_wait() before touching global memory.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dep(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                       Args &&...args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    // the launch profile records events between kernels, which serialises them anyway: launch plainly
+    cfg.numAttrs = g_prof.on ? 0 : 1;
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- quantize launchers ---------------------------------------------------------------------
 template <typename InT>
 mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t ldx,
@@ -164,9 +185,9 @@ mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t 
     const int grid = grid_for((chunks + UNROLL - 1) / UNROLL, 256, d.sm_count, per_sm);
     ProfScope prof(KIND_QUANTIZE, st);
     if (f.block == 16)
-        mx::quantize_rows_kernel<InT, 16, UNROLL><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+        MX_CUDA(launch_dep(mx::quantize_rows_kernel<InT, 16, UNROLL>, dim3(grid), dim3(256), 0, st, x, rows, K, ldx, f.elem_bits, out));
     else
-        mx::quantize_rows_kernel<InT, 32, UNROLL><<<grid, 256, 0, st>>>(x, rows, K, ldx, f.elem_bits, out);
+        MX_CUDA(launch_dep(mx::quantize_rows_kernel<InT, 32, UNROLL>, dim3(grid), dim3(256), 0, st, x, rows, K, ldx, f.elem_bits, out));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -207,9 +228,9 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
                                             : resident_ctas(mx::decode_bf16_kernel<false, UNROLL>);
         const dim3 grid((unsigned)grid_for((items + UNROLL - 1) / UNROLL, 256, d.sm_count, per_sm), (unsigned)batch);
         if (f.elem_bits <= 4)
-            mx::decode_bf16_kernel<true, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
+            MX_CUDA(launch_dep(mx::decode_bf16_kernel<true, UNROLL>, dim3(grid), dim3(256), 0, st, m, exps, rows, K, f.block, f.elem_bits, out, ld, ps));
         else
-            mx::decode_bf16_kernel<false, UNROLL><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
+            MX_CUDA(launch_dep(mx::decode_bf16_kernel<false, UNROLL>, dim3(grid), dim3(256), 0, st, m, exps, rows, K, f.block, f.elem_bits, out, ld, ps));
     } else {
         const dim3 grid((unsigned)grid_for(chunks, 256, d.sm_count, 16), (unsigned)batch);
         mx::dequantize_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(m, exps, rows, K, f.block, f.elem_bits, out, ld, ps);
@@ -321,7 +342,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
     const int threads = mx::tc_threads(BN, WMODE);
     ProfScope prof(KIND_GEMM_TC, st);
-    mx::gemm_tc_kernel<BN, WMODE><<<grid, threads, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, tm_y, p);
+    MX_CUDA(launch_dep(mx::gemm_tc_kernel<BN, WMODE>, dim3(grid), dim3(threads), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -473,7 +494,7 @@ mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, Dev
         done = true;
     }
     ProfScope prof(KIND_GEMM_STREAM, st);
-    mx::gemv_stream_kernel<NT, BULK><<<grid, mx::StreamCfg<NT, BULK>::THREADS, smem, st>>>(sp);
+    MX_CUDA(launch_dep(mx::gemv_stream_kernel<NT, BULK>, dim3(grid), dim3(mx::StreamCfg<NT, BULK>::THREADS), smem, st, sp));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -515,11 +536,11 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     job.q_blocks = gq;
     ProfScope prof(KIND_PREP, st);
     if (f32) {
-        if (nib) mx::prep_operands_kernel<float, true><<<gq + gd, 256, 0, st>>>(job);
-        else mx::prep_operands_kernel<float, false><<<gq + gd, 256, 0, st>>>(job);
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<float, true>, dim3(gq + gd), dim3(256), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<float, false>, dim3(gq + gd), dim3(256), 0, st, job));
     } else {
-        if (nib) mx::prep_operands_kernel<__nv_bfloat16, true><<<gq + gd, 256, 0, st>>>(job);
-        else mx::prep_operands_kernel<__nv_bfloat16, false><<<gq + gd, 256, 0, st>>>(job);
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, true>, dim3(gq + gd), dim3(256), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, false>, dim3(gq + gd), dim3(256), 0, st, job));
     }
     MX_CUDA(cudaGetLastError());
     return MX_OK;
@@ -892,11 +913,11 @@ static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers
         const dim3 qgrid((unsigned)grid_for((max_chunks + 1) / 2, 256, d->sm_count, 8), (unsigned)jobs.size());
         if (any_dt[0]) {
             ProfScope prof(KIND_QUANTIZE, st);
-            mx::quantize_multi_kernel<float, 0><<<qgrid, 256, 0, st>>>(dj);
+            MX_CUDA(launch_dep(mx::quantize_multi_kernel<float, 0>, dim3(qgrid), dim3(256), 0, st, dj));
         }
         if (any_dt[1]) {
             ProfScope prof(KIND_QUANTIZE, st);
-            mx::quantize_multi_kernel<__nv_bfloat16, 1><<<qgrid, 256, 0, st>>>(dj);
+            MX_CUDA(launch_dep(mx::quantize_multi_kernel<__nv_bfloat16, 1>, dim3(qgrid), dim3(256), 0, st, dj));
         }
         MX_CUDA(cudaGetLastError());
     }

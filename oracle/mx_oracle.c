@@ -32,6 +32,7 @@
  */
 #include <math.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #define MXO_OK 0
@@ -223,6 +224,28 @@ int mxo_gemm_samples(const int8_t *qa, const uint8_t *ea, int wa, const int8_t *
                 S ? S + t : 0);
     }
     return MXO_OK;
+}
+
+/*
+ * The operator with an MXInt result (Sec. 3.2, software emulators: the floating-point result of
+ * an operation is quantized again to the output precision; Fig. 2: the LinearOp's result is
+ * itself MXInt-typed).  The fp32 product y_ref (block terms summed exactly, rounded once, bias
+ * included) is computed as in mxo_gemm, then each output row is quantized with mxo_quantize in
+ * blocks of By along the output-feature axis N, which is the reduction axis of the next layer.
+ * qy [M,N] int8, ey [M,N/By]; y_ref and S ([M,N], nullable) as in mxo_gemm.
+ */
+int mxo_gemm_requant(const int8_t *qa, const uint8_t *ea, int wa, const int8_t *qw,
+                     const uint8_t *ew, int ww, int64_t M, int64_t N, int64_t K, int B,
+                     const float *bias, int By, int wy, int8_t *qy, uint8_t *ey,
+                     uint32_t *nonfinite, float *y_ref, double *S)
+{
+    if (!qy || !ey || !mxo_args_ok(M, N, By, wy)) return -1;
+    float *y = y_ref ? y_ref : (float *)malloc((size_t)(M > 0 ? M : 1) * (size_t)(N > 0 ? N : 1) * sizeof(float));
+    if (!y) return -2;
+    int rc = mxo_gemm(qa, ea, wa, qw, ew, ww, M, N, K, B, bias, y, NULL, S);
+    if (rc == 0) rc = mxo_quantize(y, M, N, N, 1, By, wy, qy, ey, nonfinite);
+    if (!y_ref) free(y);
+    return rc;
 }
 
 /* Average bits per value, Eq. 1: p = e/prod(B) + m + 1 with m = w - 1. */

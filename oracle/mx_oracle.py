@@ -45,6 +45,8 @@ def lib():
         L.mxo_gemm.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, p, p, p]
         L.mxo_gemm_samples.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, p, p, i64,
                                        p, p, p]
+        L.mxo_gemm_requant.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, i32, i32, p, p,
+                                       p, p, p]
         L.mxo_format_bits.argtypes = [i32, i32, i32, i32]
         L.mxo_format_bits.restype = C.c_double
         L.mxo_threads.restype = i32
@@ -117,6 +119,29 @@ def gemm(qa, ea, wa: int, qw, ew, ww: int, block: int, bias=None):
     _check(lib().mxo_gemm(_ptr(qa), _ptr(ea), wa, _ptr(qw), _ptr(ew), ww, M, N, K, block,
                           _ptr(bias), _ptr(y_ref), _ptr(y_seq), _ptr(S)))
     return y_ref, y_seq, S
+
+
+def gemm_requant(qa, ea, wa: int, qw, ew, ww: int, block: int, block_y: int, wy: int, bias=None):
+    """The product with an MXInt result.  Returns (qy int8 [M,N], ey uint8 [M,N/By], nonfinite,
+    y_ref fp32 [M,N], S fp64 [M,N])."""
+    qa = np.ascontiguousarray(qa, np.int8)
+    qw = np.ascontiguousarray(qw, np.int8)
+    ea = np.ascontiguousarray(ea, np.uint8)
+    ew = np.ascontiguousarray(ew, np.uint8)
+    M, K = qa.shape
+    N = qw.shape[0]
+    assert qw.shape[1] == K
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, np.float32)
+    qy = np.zeros((M, N), np.int8)
+    ey = np.zeros((M, N // block_y), np.uint8)
+    y_ref = np.zeros((M, N), np.float32)
+    S = np.zeros((M, N), np.float64)
+    bad = C.c_uint32(0)
+    _check(lib().mxo_gemm_requant(_ptr(qa), _ptr(ea), wa, _ptr(qw), _ptr(ew), ww, M, N, K, block,
+                                  _ptr(bias), block_y, wy, _ptr(qy), _ptr(ey), C.addressof(bad),
+                                  _ptr(y_ref), _ptr(S)))
+    return qy, ey, int(bad.value), y_ref, S
 
 
 def gemm_samples(qa, ea, wa: int, qw, ew, ww: int, block: int, si, sj, bias=None):

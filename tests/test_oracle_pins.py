@@ -390,3 +390,76 @@ def test_attention_oracle_reduces_to_plain_matmul_on_representable_inputs():
     for h in range(H):
         want = p[h * seq:(h + 1) * seq].astype(np.float64) @ v[:, h * d:(h + 1) * d].astype(np.float64)
         assert np.array_equal(ctx[h][0].astype(np.float64), want)
+
+
+# ---------------------------------------------------------------- product with an MXInt result
+
+def _requant_fixture():
+    rows = golden_io.load()
+    K = N = 16
+    a = [r for r in rows if r["kind"] == "rq_a"]
+    w = [r for r in rows if r["kind"] == "rq_w"]
+    qa = np.zeros((len(a), K), np.int8)
+    ea = np.zeros((len(a), 1), np.uint8)
+    for r in a:
+        v = golden_io.ints(r["q"])
+        qa[int(r["row"]), :len(v)] = v
+        ea[int(r["row"]), 0] = int(r["ebyte"])
+    qw = np.zeros((N, K), np.int8)
+    ew = np.zeros((N, 1), np.uint8)
+    for r in w:
+        v = golden_io.ints(r["q"])
+        qw[int(r["row"]), :len(v)] = v
+        ew[int(r["row"]), 0] = int(r["ebyte"])
+    bias = np.zeros(N, np.float32)
+    for r in rows:
+        if r["kind"] == "rq_bias":
+            bias[int(r["col"])] = float(r["value"])
+    return rows, qa, ea, int(a[0]["w"]), qw, ew, int(w[0]["w"]), bias
+
+
+def test_requantized_product_hand_worked():
+    """The pencil-worked layer of tests/golden: exact fp32 outputs (bias included), then one block
+    of 16 along the output-feature axis per row, at two output widths."""
+    rows, qa, ea, wa, qw, ew, ww, bias = _requant_fixture()
+    want_y = {int(r["row"]): golden_io.floats(r["y"]) for r in rows if r["kind"] == "rq_y"}
+    for wy in (4, 8):
+        qy, ey, bad, y_ref, _ = orc.gemm_requant(qa, ea, wa, qw, ew, ww, 16, 16, wy, bias=bias)
+        assert bad == 0
+        for r in (r for r in rows if r["kind"] == "rq_q" and int(r["wy"]) == wy):
+            i = int(r["row"])
+            q = golden_io.ints(r["q"])
+            assert y_ref[i, :len(want_y[i])].tolist() == want_y[i]
+            assert (y_ref[i, len(want_y[i]):] == 0).all()
+            assert ey[i, 0] == int(r["ebyte"])
+            assert qy[i, :len(q)].tolist() == q and (qy[i, len(q):] == 0).all()
+
+
+@pytest.mark.parametrize("By,wy", [(16, 4), (32, 8), (16, 2), (32, 5)])
+def test_requantized_product_invariants(By, wy):
+    """Whatever the widths: the result's exponent is that of the largest |y| of its block of the
+    exact fp32 product, every code is within half a step of y (one step where it saturates), and
+    an MXInt result that is fed back as an input is reproduced exactly by a second quantization."""
+    rng = np.random.default_rng(By + wy)
+    M, N, K, B, wa, ww = 5, 64, 96, 32, 8, 4
+    qa = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    qw = rng.integers(-7, 8, (N, K)).astype(np.int8)
+    ea = rng.integers(120, 131, (M, K // B)).astype(np.uint8)
+    ew = rng.integers(115, 125, (N, K // B)).astype(np.uint8)
+    bias = rng.standard_normal(N).astype(np.float32)
+    qy, ey, bad, y_ref, _ = orc.gemm_requant(qa, ea, wa, qw, ew, ww, B, By, wy, bias=bias)
+    assert bad == 0
+    y = y_ref.astype(np.float64).reshape(M, N // By, By)
+    amax = np.abs(y).max(axis=2)
+    _, ex = np.frexp(amax)                                    # amax = f * 2^ex, f in [0.5, 1)
+    assert np.array_equal(ey.astype(np.int64), ex - 1 + 127)
+    step = np.ldexp(1.0, ey.astype(np.int64) - 127 - (wy - 2))[:, :, None]
+    q = qy.astype(np.float64).reshape(M, N // By, By)
+    qmax = 2 ** (wy - 1) - 1
+    err = np.abs(q * step - y)
+    free = np.abs(q) < qmax
+    assert (err[free] <= 0.5 * step.repeat(By, 2)[free]).all()
+    assert (err <= step).all()
+    # the MXInt result as the next layer's input: quantizing its decoded values changes nothing
+    again_q, again_e, _ = orc.quantize(orc.dequantize(qy, ey, By, wy).astype(np.float32), By, wy)
+    assert np.array_equal(again_q, qy) and np.array_equal(again_e, ey)

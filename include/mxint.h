@@ -244,6 +244,36 @@ MX_API mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t
  */
 MX_API mx_status_t mx_poll_status(void *stream);
 
+/* ---- the layer with an MXInt result ------------------------------------------------------------
+ *
+ * Sec. 3.2 (software emulators): an operator's floating-point result is quantized again to the
+ * output precision; Fig. 2: the LinearOp's result is itself MXInt-typed, and Sec. 3.2 ("No
+ * mixed-arithmetic but mixed-precision quantization") notes that going from one MXInt width to
+ * another is cheap.  These two calls are mx_gemm / mx_linear with that last step done in the
+ * product kernel's epilogue: instead of fp32 values they write Q_fy(A W^T + bias), quantized in
+ * blocks of fy.block along N -- the reduction axis of the layer that consumes the result -- with
+ * the same rule as mx_quantize (exponent of the block's largest magnitude, round to nearest even,
+ * symmetric clamp; a block holding Inf/NaN gets exponent byte 255 and zero mantissas).
+ *   y_mant : device, [M, N/2] bytes (fy.elem_bits <= 4) or [M, N] int8, dense rows, 16-byte aligned
+ *   y_exp  : device, uint8 [M, N/fy.block]
+ *   nonfinite_count : device, nullable; incremented once per non-finite block (not cleared here)
+ * N % fy.block must be 0 (MX_ERR_SHAPE); fy.block may differ from fa.block.  Always the
+ * tensor-core kernel; workspace as for MX_ALGO_TCGEN05.  The fp32 accumulation order is the
+ * tensor pipe's, so a value within the product's tolerance of a rounding boundary may take either
+ * neighbouring code.  Other arguments, ownership and errors as for mx_gemm / mx_linear.
+ */
+MX_API mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                      const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t M,
+                      int64_t N, int64_t K, const float *bias, mx_format_t fy, void *y_mant,
+                      uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
+                      size_t workspace_bytes, void *stream);
+
+MX_API mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
+                        mx_format_t fa, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                        int64_t N, const float *bias, mx_format_t fy, void *y_mant,
+                        uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
+                        size_t workspace_bytes, void *stream);
+
 /* ---- product for callers that cannot allocate (the paper has no counterpart) -----------------
  *
  * Some callers of this library have no way to obtain device memory at the point where they

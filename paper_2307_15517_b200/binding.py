@@ -79,6 +79,10 @@ def _load() -> C.CDLL:
     L.mx_gemm_ex.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
     L.mx_linear_ex.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, i32, vp]
+    L.mx_gemm_q.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, F, vp, vp, vp, vp, sz, vp]
+    L.mx_linear_q.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, F, vp, vp, vp, vp, sz, vp]
+    L.mx_gemm_q.restype = i32
+    L.mx_linear_q.restype = i32
     L.mx_poll_status.argtypes = [vp]
     L.mx_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64]
     L.mx_gemm_batched_workspace_bytes.restype = sz
@@ -225,6 +229,46 @@ def mx_linear(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int
                             _ptr(w_exp), fw, N, _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace),
                             workspace.numel(), algo, _stream(stream)), "mx_linear")
     return y
+
+
+def _quantized_out(M: int, N: int, fy: MxFormat, device, y_mant, y_exp):
+    if y_mant is None:
+        y_mant = torch.empty((M, N // 2 if fy.elem_bits <= 4 else N), dtype=torch.uint8, device=device)
+    if y_exp is None:
+        y_exp = torch.empty((M, N // fy.block), dtype=torch.uint8, device=device)
+    return y_mant, y_exp
+
+
+def mx_gemm_q(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: int, N: int, K: int,
+              fy: MxFormat, bias: Optional[torch.Tensor] = None, y_mant=None, y_exp=None,
+              nonfinite_count: Optional[torch.Tensor] = None,
+              workspace: Optional[torch.Tensor] = None, stream=None):
+    """mx_gemm with the result quantized to format ``fy`` along N.  Returns (y_mant, y_exp)."""
+    _need_cuda(a_mant, a_exp, w_mant, w_exp, bias, y_mant, y_exp, nonfinite_count, workspace)
+    y_mant, y_exp = _quantized_out(M, N, fy, a_mant.device, y_mant, y_exp)
+    if workspace is None:
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_TCGEN05), a_mant.device)
+    _check(lib.mx_gemm_q(_ptr(a_mant), _ptr(a_exp), fa, _ptr(w_mant), _ptr(w_exp), fw, M, N, K,
+                         _ptr(bias), fy, _ptr(y_mant), _ptr(y_exp), _ptr(nonfinite_count),
+                         _ptr(workspace), workspace.numel(), _stream(stream)), "mx_gemm_q")
+    return y_mant, y_exp
+
+
+def mx_linear_q(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int, fy: MxFormat,
+                bias: Optional[torch.Tensor] = None, y_mant=None, y_exp=None,
+                nonfinite_count: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None):
+    """mx_linear with the result quantized to format ``fy`` along N.  Returns (y_mant, y_exp)."""
+    _need_cuda(x, w_mant, w_exp, bias, y_mant, y_exp, nonfinite_count, workspace)
+    M, K = x.shape
+    assert x.stride(1) == 1
+    y_mant, y_exp = _quantized_out(M, N, fy, x.device, y_mant, y_exp)
+    if workspace is None:
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_TCGEN05), x.device)
+    _check(lib.mx_linear_q(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant), _ptr(w_exp),
+                           fw, N, _ptr(bias), fy, _ptr(y_mant), _ptr(y_exp), _ptr(nonfinite_count),
+                           _ptr(workspace), workspace.numel(), _stream(stream)), "mx_linear_q")
+    return y_mant, y_exp
 
 
 def make_linear_args(layers):

@@ -157,6 +157,52 @@ __device__ __forceinline__ float absmax_nan(float m, float x)
     return d;
 }
 
+// Eight values of one block (exponent byte `ebyte`, width w) -> their packed mantissas: one word of
+// two's-complement nibbles (w <= 4, returned in p.x) or two words of int8.  Same arithmetic as
+// quantize_rows_body below (add-only rounding with the block-scaled magic constant, the
+// multiply-based form for blocks near the top of the range or holding Inf/NaN).
+__device__ __forceinline__ uint2 encode8_packed(const float (&v)[8], int ebyte, int w)
+{
+    const bool nibble = w <= 4;
+    const int qmax = (1 << (w - 1)) - 1;
+    const uint32_t off = nibble ? 8u : 128u;
+    const bool bad = ebyte == 255;
+    uint32_t f[8], corr;
+    if (ebyte <= 229 + w) {
+        const uint32_t mb = ((uint32_t)(ebyte + 25 - w) << 23) | 0x00400000u;
+        const float M = __uint_as_float(mb);
+        const float lo = __uint_as_float(mb - (uint32_t)qmax), hi = __uint_as_float(mb + (uint32_t)qmax);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = __float_as_uint(fminf(fmaxf(v[i] + M, lo), hi));
+        corr = mb - off;
+    } else {
+        const float qmaxf = (float)qmax, pow2_wm2 = (float)(1 << (w - 2));
+        const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float s = (v[i] * inv_pow2_E) * pow2_wm2;
+            const float t = fminf(fmaxf(s, -qmaxf), qmaxf) + 12582912.f;
+            f[i] = bad ? off : __float_as_uint(t) - 0x4B400000u + off;
+        }
+        corr = 0;
+    }
+    uint2 p = make_uint2(0, 0);
+    if (nibble) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) p.x += f[i] << (4 * i);
+        p.x = (p.x - corr * 0x11111111u) ^ 0x88888888u;
+    } else {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            p.x += f[i] << (8 * i);
+            p.y += f[4 + i] << (8 * i);
+        }
+        p.x = (p.x - corr * 0x01010101u) ^ 0x80808080u;
+        p.y = (p.y - corr * 0x01010101u) ^ 0x80808080u;
+    }
+    return p;
+}
+
 // rows x K, rows contiguous along K with leading dimension ldx.  BLOCK in {16, 32}.
 //
 // Work item of a warp = (row, segment of 256 elements): lane l owns the 8 elements starting at

@@ -274,6 +274,13 @@ mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, in
     return MX_OK;
 }
 
+struct QuantizedOut {            // MXInt result of the tensor-core product (see TcParams::yq_mant)
+    uint8_t *mant = nullptr;
+    uint8_t *exps = nullptr;
+    uint32_t *nonfinite = nullptr;
+    mx_format_t f{};
+};
+
 struct PackedW {                 // weight operand of the fused kernels (unused for W_BF16)
     const uint8_t *mant = nullptr;
     const uint8_t *exps = nullptr;
@@ -299,7 +306,7 @@ mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int6
 template <int BN, int WMODE>
 mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
                       int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
-                      DeviceInfo &d, cudaStream_t st)
+                      const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
 {
     using Cfg = mx::TcCfg<BN>;
     CUtensorMap tm_a, tm_w;
@@ -312,7 +319,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         tm_w = tm_a;                     // not read by the fused kernels
     }
     CUtensorMap tm_y = tm_a;             // placeholder when the epilogue stores directly
-    const bool tma_store = (ldy % 4) == 0;
+    const bool tma_store = !yq && (ldy % 4) == 0;
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
@@ -338,6 +345,11 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     p.w_exp = pw.exps;
     p.w_bits = pw.bits;
     p.block = pw.block;
+    p.yq_mant = yq ? yq->mant : nullptr;
+    p.yq_exp = yq ? yq->exps : nullptr;
+    p.yq_nonfinite = yq ? yq->nonfinite : nullptr;
+    p.yq_bits = yq ? yq->f.elem_bits : 0;
+    p.yq_block = yq ? yq->f.block : 0;
     const int tiles = p.tiles_m * p.tiles_n;
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
     const int threads = mx::tc_threads(BN, WMODE);
@@ -355,12 +367,13 @@ bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
 
 // Pre-decoded bf16 weights (both operands fetched by TMA).
 mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
-                   int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+                   int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st,
+                   const QuantizedOut *yq = nullptr)
 {
     const PackedW none;
     if (wide_tile(M, N, d))
-        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, d, st);
-    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, d, st);
+        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st);
+    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st);
 }
 
 // Packed weights decoded inside the kernel.
@@ -375,11 +388,11 @@ mx_status_t run_tc_fused(const __nv_bfloat16 *a_hat, const void *w_mant, const u
     pw.block = fw.block;
     const bool wide = wide_tile(M, N, d);
     if (fw.elem_bits <= 4) {
-        if (wide) return launch_tc<256, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
-        return launch_tc<128, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+        if (wide) return launch_tc<256, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
+        return launch_tc<128, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
     }
-    if (wide) return launch_tc<256, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
-    return launch_tc<128, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, d, st);
+    if (wide) return launch_tc<256, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
+    return launch_tc<128, mx::W_INT8>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
 }
 
 // The fused kernels read weight rows with 16-byte loads and exponent pairs with 2-byte loads.
@@ -786,6 +799,84 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
                         workspace_bytes, MX_ALGO_AUTO, stream);
 }
 
+// ---- the layer with an MXInt result -------------------------------------------------------------
+static mx_status_t check_quantized_out(mx_format_t fy, int64_t N, const void *y_mant, const uint8_t *y_exp)
+{
+    if (!y_mant || !y_exp) return MX_ERR_NULL;
+    if (!format_ok(fy)) return MX_ERR_FORMAT;
+    if ((N % fy.block) != 0) return MX_ERR_SHAPE;
+    if (!aligned16(y_mant)) return MX_ERR_ALIGN;
+    return MX_OK;
+}
+
+mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                      const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                      const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
+                      uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+{
+    // the output pointer checks (non-null, 16-byte aligned) apply to the mantissa array here
+    mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias,
+                                    static_cast<const float *>(y_mant), N);
+    if (s != MX_OK) return s;
+    if (!a_exp) return MX_ERR_NULL;
+    s = check_quantized_out(fy, N, y_mant, y_exp);
+    if (s != MX_OK) return s;
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    if (!workspace || workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
+                                                             round256((size_t)M * K * 2));
+    s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    if (s != MX_OK) return s;
+    QuantizedOut yq;
+    yq.mant = static_cast<uint8_t *>(y_mant);
+    yq.exps = y_exp;
+    yq.nonfinite = nonfinite_count;
+    yq.f = fy;
+    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq);
+}
+
+mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
+                        const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
+                        const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
+                        uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+{
+    mx_status_t s = check_gemm_args(x, nullptr, fa, w_mant, w_exp, fw, M, N, K, bias,
+                                    static_cast<const float *>(y_mant), N);
+    if (s != MX_OK) return s;
+    if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
+    if (ldx < K) return MX_ERR_SHAPE;
+    if ((ldx % 8) != 0) return MX_ERR_ALIGN;
+    s = check_quantized_out(fy, N, y_mant, y_exp);
+    if (s != MX_OK) return s;
+    DeviceInfo *d = nullptr;
+    s = device_info(&d);
+    if (s != MX_OK) return s;
+    if (!workspace || workspace_bytes < tc_workspace(M, N, K)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
+    mx_linear_args_t one;
+    one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
+    one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = nullptr; one.ldy = N;
+    s = tc_prepare(one, a_hat, w_hat, *d, st);
+    if (s != MX_OK) return s;
+    QuantizedOut yq;
+    yq.mant = static_cast<uint8_t *>(y_mant);
+    yq.exps = y_exp;
+    yq.nonfinite = nonfinite_count;
+    yq.f = fy;
+    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq);
+}
+
 // ---- decode: few tokens, weights streamed once ------------------------------------------------
 size_t mx_linear_grouped_workspace_bytes(const mx_linear_args_t *layers, int32_t n_layers)
 {
@@ -1136,6 +1227,11 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     p.w_exp = nullptr;
     p.w_bits = 0;
     p.block = 0;
+    p.yq_mant = nullptr;
+    p.yq_exp = nullptr;
+    p.yq_nonfinite = nullptr;
+    p.yq_bits = 0;
+    p.yq_block = 0;
     const int tiles = p.tiles_m * p.tiles_n;
     mx::gemm_tc_kernel<BN, mx::W_BF16><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
         tm_a, tm_w, tm_a, p);

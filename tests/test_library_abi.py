@@ -88,6 +88,12 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     assert g(y=odd) == -4
     assert g(algo=9) == -3
     assert L.mx_linear_ex(fake, 0, 8, 64, 60, f, fake, fake, f, 8, None, fake, 8, None, 0, 2, None) == -2
+    # the calls with an MXInt result: N must hold whole output blocks, outputs must be there
+    q = lambda **kw: L.mx_linear_q(fake, 0, 8, 64, 64, f, fake, fake, f, kw.get("N", 32), None, kw.get("fy", f),
+                                   kw.get("ym", fake), kw.get("ye", fake), None, None, 0, None)
+    assert q(N=40) == -2                                     # 40 is not a multiple of the output block
+    assert q(fy=mxb.MxFormat(8, 4)) == -3
+    assert q(ym=None) == -1 and q(ye=None) == -1
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")

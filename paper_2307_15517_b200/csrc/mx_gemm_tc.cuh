@@ -33,7 +33,12 @@ namespace mx {
 //   W_BF16   : already decoded to bf16 in global memory, fetched by TMA (192 threads)
 //   W_NIBBLE : packed 4-bit mantissas + exponent bytes, decoded in the kernel by 8 extra warps
 //   W_INT8   : int8 mantissas + exponent bytes, decoded in the kernel by 8 extra warps
-enum WMode { W_BF16 = 0, W_NIBBLE = 1, W_INT8 = 2 };
+//   W_NIBBLE_PERM : as W_NIBBLE for K % 64 == 0, with the cheapest possible decode: inside every
+//              group of 8 consecutive k the operand tile holds k in the order 0,4,1,5,2,6,3,7 (the
+//              order in which a shift and a mask pull pairs of nibbles out of a packed word), and
+//              the activation operand must have been written in the same order.  A dot product
+//              does not care in which order its terms are visited.
+enum WMode { W_BF16 = 0, W_NIBBLE = 1, W_INT8 = 2, W_NIBBLE_PERM = 3 };
 
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                                  // bf16 elements per 128-byte row
@@ -110,7 +115,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     if (threadIdx.x == 0) {
         for (int s = 0; s < STAGES; ++s) {
             // full: the TMA lane's expect_tx arrival (+ one arrival per decode warp in the fused modes)
-            ptx::mbar_init(full_bar(s), FUSED ? 1 + (2 * BN) / 32 : 1);
+            // (the lean decode publishes a K step with one of its four groups only)
+            ptx::mbar_init(full_bar(s), WMODE == W_NIBBLE_PERM ? 1 + BN / 64 : FUSED ? 1 + (2 * BN) / 32 : 1);
             ptx::mbar_init(empty_bar(s), 1);
         }
         for (int a = 0; a < 2; ++a) {
@@ -195,7 +201,103 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
         }
         __syncwarp();
-    } else if (FUSED && warp >= TC_THREADS / 32) {
+    } else if (WMODE == W_NIBBLE_PERM && warp >= TC_THREADS / 32) {
+        // ---- lean weight decode (see W_NIBBLE_PERM) ----
+        // The 2 * BN decode threads form four groups; group g fills the operand tile of K steps
+        // g, g + 4, g + 8, ...  A thread fetches the raw bytes of its next step right after it has
+        // published the current one, so no global load of its own is in flight when it reaches the
+        // proxy fence that precedes the publication (such a fence waits for them: with loads in
+        // flight every K step pays a full L2 round trip), and the fetch has three K steps to land.
+        // An item = 16 packed bytes (32 of the 64 k of a K step) of one tile row; a thread owns
+        // four items per step, 32 rows apart (BN = 128) or 64 (BN = 256).  Rows past N read row
+        // N - 1: their products land in columns that the epilogue never stores.
+        constexpr int GSIZE = BN / 2;                      // threads per group
+        constexpr int ITEMS = 4;
+        const int dt = threadIdx.x - TC_THREADS;
+        const int grp = dt / GSIZE, dl = dt % GSIZE;
+        const int h = dl & 1, trow0 = dl >> 1;             // item q: tile row trow0 + q * GSIZE / 2
+        const int my_tiles = blockIdx.x < num_tiles ? (num_tiles - 1 - blockIdx.x) / gridDim.x + 1 : 0;
+        const int total = my_tiles * kblocks;
+        const bool b16 = p.block == 16;
+        const int64_t mant_ld = p.K >> 1, nb_row = p.K / p.block;
+        const uint32_t row_off = (uint32_t)((trow0 >> 3) * 1024 + (trow0 & 7) * 128) + Cfg::A_BYTES;
+        uint32_t chunk_off[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) chunk_off[j] = row_off + (uint32_t)(((h * 4 + j) ^ (trow0 & 7)) << 4);
+        const int wsub = p.w_bits - 2;
+
+        struct Raw { uint4 m; uint32_t e; };
+        Raw raw[ITEMS];
+        auto load = [&](int i) {
+            if (i >= total) return;
+            const int ti = i / kblocks, kb = i - ti * kblocks;
+            const int n0 = ((blockIdx.x + ti * (int)gridDim.x) / p.tiles_m) * BN;
+#pragma unroll
+            for (int q = 0; q < ITEMS; ++q) {
+                const int n = min(n0 + trow0 + q * (GSIZE / 2), p.N - 1);
+                raw[q].m = __ldg(reinterpret_cast<const uint4 *>(p.w_mant + (int64_t)n * mant_ld + h * 16 + (int64_t)kb * 32));
+                const uint8_t *ep = p.w_exp + (int64_t)n * nb_row;
+                raw[q].e = b16 ? (uint32_t)__ldg(reinterpret_cast<const uint16_t *>(ep + h * 2 + kb * 4))
+                               : (uint32_t)__ldg(ep + h + kb * 2);
+            }
+        };
+        auto decode_store = [&](uint32_t stage, const Raw &r) {
+            const int e0 = (int)(r.e & 0xFF), e1 = b16 ? (int)(r.e >> 8) : e0;
+            const int f0 = e0 - wsub, f1 = e1 - wsub;
+            const uint32_t w4[4] = {r.m.x, r.m.y, r.m.z, r.m.w};
+            if ((unsigned)(f0 - 1) < 240u && (unsigned)(f1 - 1) < 240u) {
+                // scale 2^(E-(w-2)) as bf16 in both halves; c = -136 * scale
+                const uint32_t sb[2] = {(uint32_t)(f0 << 7) * 0x00010001u, (uint32_t)(f1 << 7) * 0x00010001u};
+                const __nv_bfloat162 m136 = as_bf162(0xC308C308u);
+                const __nv_bfloat162 cb[2] = {__hmul2(as_bf162(sb[0]), m136), __hmul2(as_bf162(sb[1]), m136)};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    // (w >> 4i) & 0x000F000F = nibbles i and i+4; ^ 0x43084308 turns each into the bf16
+                    // number 128 + (q + 8); one fma gives (136 + q) * s - 136 * s = q * s exactly
+                    uint32_t v[4];
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        const uint32_t x = ((w4[j] >> (4 * i)) & 0x000F000Fu) ^ 0x43084308u;
+                        v[i] = as_u32(__hfma2(as_bf162(x), as_bf162(sb[j >> 1]), cb[j >> 1]));
+                    }
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + chunk_off[j]), "r"(v[0]),
+                                 "r"(v[1]), "r"(v[2]), "r"(v[3])
+                                 : "memory");
+                }
+            } else {                                        // zero / subnormal / top-of-range / non-finite scale
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    int q[8];
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) q[i] = ((int)(w4[j] << (28 - 4 * i))) >> 28;
+                    uint32_t o[4];
+                    decode8_safe(q, j < 2 ? e0 : e1, p.w_bits, o);      // (k0,k1) (k2,k3) (k4,k5) (k6,k7)
+                    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(stage + chunk_off[j]),
+                                 "r"(__byte_perm(o[0], o[2], 0x5410)), "r"(__byte_perm(o[0], o[2], 0x7632)),
+                                 "r"(__byte_perm(o[1], o[3], 0x5410)), "r"(__byte_perm(o[1], o[3], 0x7632))
+                                 : "memory");
+                }
+            }
+        };
+        load(grp);
+        for (int i = grp; i < total; i += 4) {
+            const int s = i % STAGES;
+            const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+            bool ok = true;
+            if (lane == 0) ok = ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS);
+            if (!__shfl_sync(0xFFFFFFFFu, ok, 0)) {
+                timed_out = true;
+                break;
+            }
+            const uint32_t stage = smem_base + s * Cfg::STAGE_BYTES;
+#pragma unroll
+            for (int q = 0; q < ITEMS; ++q) decode_store(stage + (uint32_t)(q * GSIZE * 64), raw[q]);
+            ptx::fence_proxy_async_smem();          // generic-proxy stores -> visible to the MMA
+            __syncwarp();
+            if (lane == 0) ptx::mbar_arrive(full_bar(s));
+            load(i + 4);
+        }
+    } else if (FUSED && WMODE != W_NIBBLE_PERM && warp >= TC_THREADS / 32) {
         // ---- weight decode: packed mantissas + exponent bytes -> swizzled bf16 operand tile ----
         // Thread d owns half h = d & 1 (32 of the 64 k of a K step) of tile row d >> 1.  Raw
         // bytes are fetched three K steps ahead.

@@ -124,6 +124,8 @@ struct QuantOut {
     __nv_bfloat16 *xhat;  // decoded values as bf16, [rows, ld_xhat] (nullable)
     int64_t ld_xhat;
     uint32_t *nonfinite;  // nullable
+    int xhat_perm;        // 1: inside every group of 8 consecutive k, xhat holds k in the order
+                          // 0,4,1,5,2,6,3,7 (the operand order of the W_NIBBLE_PERM product kernel)
 };
 
 template <typename InT> struct Load8;
@@ -328,7 +330,9 @@ __device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, in
                     // q * 2^(E-127-(w-2)) as bf16 (exact: <= 7 significant bits)
                     uint32_t h[4];
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) h[i] = as_u32(__floats2bfloat162_rn(xh[2 * i], xh[2 * i + 1]));
+                    for (int i = 0; i < 4; ++i)
+                        h[i] = out.xhat_perm ? as_u32(__floats2bfloat162_rn(xh[i], xh[i + 4]))
+                                             : as_u32(__floats2bfloat162_rn(xh[2 * i], xh[2 * i + 1]));
                     *reinterpret_cast<uint4 *>(out.xhat + row[u] * out.ld_xhat + (int64_t)kc[u] * 8) =
                         make_uint4(h[0], h[1], h[2], h[3]);
                 }

@@ -33,7 +33,7 @@ struct DeviceInfo {
     bool is_sm100 = false;
     int sm_count = SM_COUNT_FALLBACK;
     uint32_t *status = nullptr;
-    bool tc_attr_set[2][3] = {{false, false, false}, {false, false, false}};
+    bool tc_attr_set[2][4] = {{false, false, false, false}, {false, false, false, false}};
     bool stream_attr_set[4] = {false, false, false, false};
 };
 DeviceInfo g_dev[MAX_DEVICES];
@@ -379,7 +379,7 @@ mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64
 // Packed weights decoded inside the kernel.
 mx_status_t run_tc_fused(const __nv_bfloat16 *a_hat, const void *w_mant, const uint8_t *w_exp,
                          const mx_format_t &fw, int64_t M, int64_t N, int64_t K, const float *bias,
-                         float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+                         float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st, bool perm_a = false)
 {
     PackedW pw;
     pw.mant = static_cast<const uint8_t *>(w_mant);
@@ -387,6 +387,10 @@ mx_status_t run_tc_fused(const __nv_bfloat16 *a_hat, const void *w_mant, const u
     pw.bits = fw.elem_bits;
     pw.block = fw.block;
     const bool wide = wide_tile(M, N, d);
+    if (perm_a) {                       // a_hat was written in the permuted K order: nibbles, K % 64 == 0
+        if (wide) return launch_tc<256, mx::W_NIBBLE_PERM>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
+        return launch_tc<128, mx::W_NIBBLE_PERM>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
+    }
     if (fw.elem_bits <= 4) {
         if (wide) return launch_tc<256, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
         return launch_tc<128, mx::W_NIBBLE>(a_hat, nullptr, pw, M, N, K, bias, y, ldy, nullptr, d, st);
@@ -780,9 +784,13 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     // the activations' mantissas and exponents go straight to the MMA operand form (exact bf16)
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
     if (fused) {
+        // 4-bit weights and whole K steps: the lean in-kernel decode, which wants both operands in
+        // its own K order inside every group of 8
+        const bool perm = fw.elem_bits <= 4 && (K % 64) == 0;
+        out.xhat_perm = perm ? 1 : 0;
         s = quantize_rows_any(x, dt, M, K, ldx, fa, out, *d, st);
         if (s != MX_OK) return s;
-        return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+        return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st, perm);
     }
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     s = tc_prepare(one, a_hat, w_hat, *d, st);

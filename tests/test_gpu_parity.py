@@ -286,6 +286,33 @@ def test_linear_single_layer_config(mxb):
     _check_tol(y_fused, y_ref, S)
 
 
+@pytest.mark.parametrize("case", [(16, 8, 4, 300, 1152, 520), (32, 4, 2, 130, 256, 72), (16, 6, 3, 257, 2048, 1000),
+                                  (32, 8, 4, 2048, 512, 2304)])
+def test_linear_in_kernel_weight_decode(mxb, case):
+    """mx_linear with MX_ALGO_TCGEN05_FUSED and 4-bit-container weights, K % 64 == 0: the product
+    kernel decodes the packed weights itself and both operand tiles hold k in a permuted order
+    inside every group of 8.  Includes all-zero weight blocks, a non-finite weight block and
+    weight exponents near both ends of the range (the decode's slow path)."""
+    B, wa, ww, M, K, N = case
+    x = synth.student_t_activations(M, K, seed=wa + 1)
+    wt = synth.gaussian_weights(N, K, seed=ww + 1).numpy()
+    wt[5, :B] = 0.0                                           # a zero block
+    wt[7, B:2 * B] *= np.float32(2.0 ** -120)                 # scale below the bf16 normal range
+    wt[9 % N, :B] *= np.float32(2.0 ** 100)                   # scale near the top
+    qa, ea, _ = orc.quantize(x.numpy(), B, wa)
+    qw, ew, _ = orc.quantize(wt, B, ww)
+    ew[11, 1] = 255                                           # a non-finite block: column 11 is NaN
+    fa, fw = mxb.MxFormat(B, wa), mxb.MxFormat(B, ww)
+    y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
+    y = mxb.mx_linear(x.cuda(), fa, _dev(orc.pack(qw, ww)), _dev(ew), fw, N, algo=mxb.MX_ALGO_TCGEN05_FUSED)
+    assert mxb.mx_poll_status() == 0
+    y = y.cpu().numpy()
+    assert np.array_equal(np.isnan(y), np.isnan(y_ref)) and np.isnan(y[:, 11]).all()
+    ok = ~np.isnan(y_ref)
+    err = np.abs(y.astype(np.float64) - y_ref.astype(np.float64))
+    assert (err[ok] <= (TOL * S + 1e-37)[ok]).all()
+
+
 @pytest.mark.parametrize("case", [(16, 8, 4), (32, 4, 4), (32, 6, 3), (16, 2, 8)])
 def test_linear_mixed_precision(mxb, case):
     B, wa, ww = case

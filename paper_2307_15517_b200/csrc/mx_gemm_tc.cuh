@@ -67,6 +67,11 @@ struct TcParams {
     int M, N, K;
     int tiles_m, tiles_n;
     int tma_store;   // 1: the epilogue writes Y with tiled TMA stores (needs ldy % 4 == 0)
+    // batch > 1 (W_BF16 kernels, fp32 result, no bias): `batch` independent products of the same
+    // shape in one launch; the three tensor maps are rank 3 (z = item) and item b writes to
+    // y + b * y_batch.  Tiles are numbered item-major.
+    int batch;
+    int64_t y_batch;
     uint32_t *status;
     // fused modes only: the packed weight operand
     const uint8_t *w_mant;
@@ -140,7 +145,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     ptx::dep_wait();
     if (threadIdx.x == 0) ptx::dep_trigger();
 
-    const int num_tiles = p.tiles_m * p.tiles_n;
+    const int tiles_item = p.tiles_m * p.tiles_n;
+    const int num_tiles = tiles_item * p.batch;
     const int kblocks = (p.K + TC_BK - 1) / TC_BK;
     bool timed_out = false;
 
@@ -149,7 +155,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             int s = 0;
             uint32_t ph = 0;
             for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x) {
-                const int m0 = (t % p.tiles_m) * TC_BM, n0 = (t / p.tiles_m) * BN;
+                const int tb = t / tiles_item, tt = t - tb * tiles_item;
+                const int m0 = (tt % p.tiles_m) * TC_BM, n0 = (tt / p.tiles_m) * BN;
                 for (int kb = 0; kb < kblocks; ++kb) {
                     if (!ptx::mbar_wait_bounded(empty_bar(s), ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS)) {
                         timed_out = true;
@@ -157,8 +164,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     }
                     ptx::mbar_arrive_expect_tx(full_bar(s), FUSED ? Cfg::A_BYTES : Cfg::STAGE_BYTES);
                     const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
-                    ptx::tma_load_2d(sa, &tmap_a, kb * TC_BK, m0, full_bar(s));
-                    if (!FUSED) ptx::tma_load_2d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, full_bar(s));
+                    if (!FUSED && p.batch > 1) {
+                        ptx::tma_load_3d(sa, &tmap_a, kb * TC_BK, m0, tb, full_bar(s));
+                        ptx::tma_load_3d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, tb, full_bar(s));
+                    } else {
+                        ptx::tma_load_2d(sa, &tmap_a, kb * TC_BK, m0, full_bar(s));
+                        if (!FUSED) ptx::tma_load_2d(sa + Cfg::A_BYTES, &tmap_w, kb * TC_BK, n0, full_bar(s));
+                    }
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
                 }
             }
@@ -435,7 +447,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
-            const int m0 = (t % p.tiles_m) * TC_BM, n0 = (t / p.tiles_m) * BN;
+            const int tb = t / tiles_item, tt = t - tb * tiles_item;
+            const int m0 = (tt % p.tiles_m) * TC_BM, n0 = (tt / p.tiles_m) * BN;
             // every lane waits (acquire), then the warp agrees on the outcome so that the
             // warp-collective TMEM loads below are never executed by a partial warp
             const bool ok = ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
@@ -445,7 +458,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             ptx::tc_fence_after_sync();
             const int row = m0 + quad * 32 + lane;
-            float *yrow = p.y + (int64_t)row * p.ldy;
+            float *yrow = p.y + (int64_t)tb * p.y_batch + (int64_t)row * p.ldy;
             const bool vec_ok = ((p.ldy & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
@@ -527,7 +540,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                         ptx::fence_proxy_async_smem();
                         __syncwarp();
                         if (lane == 0) {
-                            ptx::tma_store_2d(&tmap_y, n, m0 + quad * 32, buf);
+                            if (p.batch > 1) ptx::tma_store_3d(&tmap_y, n, m0 + quad * 32, tb, buf);
+                            else ptx::tma_store_2d(&tmap_y, n, m0 + quad * 32, buf);
                             ptx::bulk_commit_group();
                         }
                         ++epi_buf;

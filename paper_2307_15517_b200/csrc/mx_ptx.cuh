@@ -108,6 +108,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void *tmap,
         : "memory");
 }
 
+// The same for a rank-3 tensor map (z = batch item).
+__device__ __forceinline__ void tma_load_3d(uint32_t dst_smem, const void *tmap, int32_t x, int32_t y,
+                                            int32_t z, uint32_t bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        :
+        : "r"(dst_smem), "l"((uint64_t)tmap), "r"(bar), "r"(x), "r"(y), "r"(z)
+        : "memory");
+}
+__device__ __forceinline__ void tma_store_3d(const void *tmap, int32_t x, int32_t y, int32_t z, uint32_t src_smem)
+{
+    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.bulk_group [%0, {%2, %3, %4}], [%1];"
+                 :
+                 : "l"((uint64_t)tmap), "r"(src_smem), "r"(x), "r"(y), "r"(z)
+                 : "memory");
+}
+
 // 2-D tiled store shared -> global (bulk async group); elements outside the tensor are clipped.
 __device__ __forceinline__ void tma_store_2d(const void *tmap, int32_t x, int32_t y, uint32_t src_smem)
 {

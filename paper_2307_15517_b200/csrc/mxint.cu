@@ -247,7 +247,9 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
 }
 
 // ---- tensor-core GEMM launcher ----------------------------------------------------------------
-mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, int64_t K, int box_rows)
+// bf16 [rows, K] (dense rows); batch > 1: `batch` such items `item_bytes` apart, as a rank-3 map.
+mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, int64_t K, int box_rows,
+                             int64_t batch = 1, size_t item_bytes = 0)
 {
     if (!g_encode_tiled) {
         void *fn = nullptr;
@@ -259,11 +261,11 @@ mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, in
         }
         g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)K * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)mx::TC_BK, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base),
+    const cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
+    const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)item_bytes};
+    const cuuint32_t box[3] = {(cuuint32_t)mx::TC_BK, (cuuint32_t)box_rows, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, batch > 1 ? 3 : 2, const_cast<void *>(base),
                                       dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                                       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -281,19 +283,26 @@ struct QuantizedOut {            // MXInt result of the tensor-core product (see
     mx_format_t f{};
 };
 
+struct TcBatch {                 // several products of one shape in one launch (W_BF16 kernels)
+    int64_t count = 1;
+    size_t a_item = 0, w_item = 0;   // bytes between the items' bf16 operands
+    int64_t y_batch = 0;             // floats between the items' outputs
+};
+
 struct PackedW {                 // weight operand of the fused kernels (unused for W_BF16)
     const uint8_t *mant = nullptr;
     const uint8_t *exps = nullptr;
     int bits = 0, block = 0;
 };
 
-mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int64_t ldy)
+mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int64_t ldy, int64_t batch = 1,
+                           int64_t y_batch = 0)
 {
-    const cuuint64_t dims[2] = {(cuuint64_t)N, (cuuint64_t)M};
-    const cuuint64_t strides[1] = {(cuuint64_t)ldy * 4};
-    const cuuint32_t box[2] = {32, 32};
-    const cuuint32_t estr[2] = {1, 1};
-    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, y, dims, strides, box, estr,
+    const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)batch};
+    const cuuint64_t strides[2] = {(cuuint64_t)ldy * 4, (cuuint64_t)y_batch * 4};
+    const cuuint32_t box[3] = {32, 32, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, batch > 1 ? 3 : 2, y, dims, strides, box, estr,
                                       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                       CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -306,22 +315,22 @@ mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int6
 template <int BN, int WMODE>
 mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
                       int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
-                      const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
+                      const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st, const TcBatch &tb = TcBatch())
 {
     using Cfg = mx::TcCfg<BN>;
     CUtensorMap tm_a, tm_w;
-    mx_status_t s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
+    mx_status_t s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM, tb.count, tb.a_item);
     if (s != MX_OK) return s;
     if (WMODE == mx::W_BF16) {
-        s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
+        s = encode_bf16_rows(&tm_w, w_hat, N, K, BN, tb.count, tb.w_item);
         if (s != MX_OK) return s;
     } else {
         tm_w = tm_a;                     // not read by the fused kernels
     }
     CUtensorMap tm_y = tm_a;             // placeholder when the epilogue stores directly
-    const bool tma_store = !yq && (ldy % 4) == 0;
+    const bool tma_store = !yq && (ldy % 4) == 0 && (tb.y_batch % 4) == 0;
     if (tma_store) {
-        s = encode_f32_out(&tm_y, y, M, N, ldy);
+        s = encode_f32_out(&tm_y, y, M, N, ldy, tb.count, tb.y_batch);
         if (s != MX_OK) return s;
     }
     constexpr int slot = BN == 256 ? 0 : 1;
@@ -350,7 +359,11 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     p.yq_nonfinite = yq ? yq->nonfinite : nullptr;
     p.yq_bits = yq ? yq->f.elem_bits : 0;
     p.yq_block = yq ? yq->f.block : 0;
-    const int tiles = p.tiles_m * p.tiles_n;
+    p.batch = (int)tb.count;
+    p.y_batch = tb.y_batch;
+    const int64_t tiles64 = (int64_t)p.tiles_m * p.tiles_n * tb.count;
+    if (tiles64 > INT32_MAX / 2) return MX_ERR_SHAPE;
+    const int tiles = (int)tiles64;
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
     const int threads = mx::tc_threads(BN, WMODE);
     ProfScope prof(KIND_GEMM_TC, st);
@@ -368,12 +381,13 @@ bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
 // Pre-decoded bf16 weights (both operands fetched by TMA).
 mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
                    int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st,
-                   const QuantizedOut *yq = nullptr)
+                   const QuantizedOut *yq = nullptr, const TcBatch &tb = TcBatch())
 {
     const PackedW none;
-    if (wide_tile(M, N, d))
-        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st);
-    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st);
+    const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256) * tb.count;
+    if (N > 128 && tiles256 >= (int64_t)d.sm_count * 3 / 4)
+        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb);
+    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb);
 }
 
 // Packed weights decoded inside the kernel.
@@ -1091,17 +1105,17 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
         ps.out_batch = (int64_t)(out_item / 2);
         return ps;
     };
-    // one decode launch per operand covers every batch item, then one product launch per item
+    // one decode launch per operand and one product launch cover every batch item
     s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, strides(fa, lda, stride_a, a_item), batch, *d, st);
     if (s != MX_OK) return s;
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, strides(fw, ldw, stride_w, w_item), batch, *d, st);
     if (s != MX_OK) return s;
-    for (int64_t b = 0; b < batch; ++b) {
-        s = run_tc(a_hat + b * (int64_t)(a_item / 2), w_hat + b * (int64_t)(w_item / 2), M, N, K, nullptr,
-                   y + b * stride_y, ldy, *d, st);
-        if (s != MX_OK) return s;
-    }
-    return MX_OK;
+    TcBatch tb;
+    tb.count = batch;
+    tb.a_item = a_item;
+    tb.w_item = w_item;
+    tb.y_batch = stride_y;
+    return run_tc(a_hat, w_hat, M, N, K, nullptr, y, ldy, *d, st, nullptr, tb);
 }
 
 // ---- fp32 glue of the transformer block ---------------------------------------------------------
@@ -1240,6 +1254,8 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     p.yq_nonfinite = nullptr;
     p.yq_bits = 0;
     p.yq_block = 0;
+    p.batch = 1;
+    p.y_batch = 0;
     const int tiles = p.tiles_m * p.tiles_n;
     mx::gemm_tc_kernel<BN, mx::W_BF16><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
         tm_a, tm_w, tm_a, p);

@@ -248,6 +248,60 @@ int mxo_gemm_requant(const int8_t *qa, const uint8_t *ea, int wa, const int8_t *
     return rc;
 }
 
+/*
+ * Two-dimensional blocks (Sec. 4.1: a block has a shape; the paper's unified shape is (16, 2),
+ * "block size 32", as in MXInt((16,2),8,7) of Fig. 2 and the worked 8.25-bit example after
+ * Eq. 1).  Reading: B consecutive elements along the reduction axis k times BR adjacent rows
+ * share one exponent, the exponent of the largest magnitude among the B*BR values.  rows must be
+ * a multiple of BR.  q [rows,K] int8; ebyte [rows/BR, K/B].  Everything else as mxo_quantize.
+ */
+int mxo_quantize_2d(const float *x, int64_t rows, int64_t K, int64_t stride_row, int64_t stride_k,
+                    int B, int BR, int w, int8_t *q, uint8_t *ebyte, uint32_t *nonfinite)
+{
+    if (!mxo_args_ok(rows, K, B, w) || BR < 1 || (rows % BR) != 0) return MXO_BAD_ARG;
+    const int64_t nb = K / B;
+    const double qmax = (double)((1 << (w - 1)) - 1);
+    uint32_t bad = 0;
+    for (int64_t r0 = 0; r0 < rows; r0 += BR) {
+        for (int64_t b = 0; b < nb; ++b) {
+            float amax = 0.0f;
+            int any_nonfinite = 0;
+            for (int dr = 0; dr < BR; ++dr)
+                for (int k = 0; k < B; ++k) {
+                    float v = x[(r0 + dr) * stride_row + (b * B + k) * stride_k];
+                    if (isnan(v) || isinf(v)) any_nonfinite = 1;
+                    float a = fabsf(v);
+                    if (a > amax) amax = a;
+                }
+            const int eb = any_nonfinite ? 255 : mxo_exponent_byte(amax);
+            ebyte[(r0 / BR) * nb + b] = (uint8_t)eb;
+            if (any_nonfinite) ++bad;
+            const double s = ldexp(1.0, (eb - 127) - (w - 2));
+            for (int dr = 0; dr < BR; ++dr)
+                for (int k = 0; k < B; ++k) {
+                    double n = 0.0;
+                    if (!any_nonfinite) {
+                        n = nearbyint((double)x[(r0 + dr) * stride_row + (b * B + k) * stride_k] / s);
+                        if (n > qmax) n = qmax;
+                        if (n < -qmax) n = -qmax;
+                    }
+                    q[(r0 + dr) * K + b * B + k] = (int8_t)n;
+                }
+        }
+    }
+    if (nonfinite) *nonfinite = bad;
+    return MXO_OK;
+}
+
+/* Exponent bytes of a tensor with (B, BR) blocks written out per row: out[r][b] = ebyte[r/BR][b]. */
+int mxo_expand_exponent_rows(const uint8_t *ebyte, int64_t rows, int64_t nb, int BR, uint8_t *out)
+{
+    if (rows < 0 || nb < 0 || BR < 1 || (rows % BR) != 0) return MXO_BAD_ARG;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < nb; ++b) out[r * nb + b] = ebyte[(r / BR) * nb + b];
+    return MXO_OK;
+}
+
 /* Average bits per value, Eq. 1: p = e/prod(B) + m + 1 with m = w - 1. */
 double mxo_format_bits(int block, int block_rows, int exp_bits, int w)
 {

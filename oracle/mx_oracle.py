@@ -47,6 +47,8 @@ def lib():
                                        p, p, p]
         L.mxo_gemm_requant.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, i32, i32, p, p,
                                        p, p, p]
+        L.mxo_quantize_2d.argtypes = [p, i64, i64, i64, i64, i32, i32, i32, p, p, p]
+        L.mxo_expand_exponent_rows.argtypes = [p, i64, i64, i32, p]
         L.mxo_format_bits.argtypes = [i32, i32, i32, i32]
         L.mxo_format_bits.restype = C.c_double
         L.mxo_threads.restype = i32
@@ -75,6 +77,29 @@ def quantize(x, block: int, w: int, axis_strided: bool = False):
     _check(lib().mxo_quantize(_ptr(x), rows, K, sr, sk, block, w, _ptr(q), _ptr(e),
                               C.addressof(bad)))
     return q, e, int(bad.value)
+
+
+def quantize_2d(x, block: int, block_rows: int, w: int):
+    """Blocks of `block` along K times `block_rows` adjacent rows.  Returns (q int8 [rows,K],
+    ebyte uint8 [rows/block_rows, K/block], nonfinite)."""
+    x = np.asarray(x)
+    assert x.dtype == np.float32 and x.ndim == 2
+    rows, K = x.shape
+    sr, sk = x.strides[0] // 4, x.strides[1] // 4
+    q = np.zeros((rows, K), np.int8)
+    e = np.zeros((rows // block_rows, K // block), np.uint8)
+    bad = C.c_uint32(0)
+    _check(lib().mxo_quantize_2d(_ptr(x), rows, K, sr, sk, block, block_rows, w, _ptr(q), _ptr(e),
+                                 C.addressof(bad)))
+    return q, e, int(bad.value)
+
+
+def expand_exponent_rows(e, block_rows: int):
+    """Exponent bytes of a (block, block_rows) tensor written out once per row."""
+    e = np.ascontiguousarray(e, np.uint8)
+    out = np.zeros((e.shape[0] * block_rows, e.shape[1]), np.uint8)
+    _check(lib().mxo_expand_exponent_rows(_ptr(e), out.shape[0], e.shape[1], block_rows, _ptr(out)))
+    return out
 
 
 def dequantize(q, e, block: int, w: int):

@@ -463,3 +463,52 @@ def test_requantized_product_invariants(By, wy):
     # the MXInt result as the next layer's input: quantizing its decoded values changes nothing
     again_q, again_e, _ = orc.quantize(orc.dequantize(qy, ey, By, wy).astype(np.float32), By, wy)
     assert np.array_equal(again_q, qy) and np.array_equal(again_e, ey)
+
+
+# ---------------------------------------------------------------- two-dimensional blocks
+
+def test_two_row_blocks_hand_worked():
+    for r in (r for r in golden_io.load() if r["kind"] == "block2d"):
+        w = int(r["w"])
+        x = np.zeros((2, 16), np.float32)
+        for i, key in enumerate(("x0", "x1")):
+            v = golden_io.floats(r[key])
+            x[i, :len(v)] = v
+        q, e, bad = orc.quantize_2d(x, 16, 2, w)
+        assert e.shape == (1, 1) and e[0, 0] == int(r["ebyte"]) and bad == 0
+        for i, key in enumerate(("q0", "q1")):
+            want = golden_io.ints(r[key])
+            assert q[i, :len(want)].tolist() == want and (q[i, len(want):] == 0).all()
+
+
+@pytest.mark.parametrize("B,w", [(16, 4), (16, 8), (32, 3)])
+def test_two_row_blocks_reduce_to_known_cases(B, w):
+    """(B, 1) blocks are the one-dimensional quantizer; a (B, 2) block is the one-dimensional block
+    of 2B values obtained by laying the two rows side by side; the shared exponent is the larger of
+    the two rows' own exponents; the paper's storage figure follows (8.25 bits at (16,2), m = 7)."""
+    rng = np.random.default_rng(B + w)
+    x = (rng.standard_t(3, (6, 4 * B)) * np.exp(rng.uniform(-3, 3, (6, 1)))).astype(np.float32)
+    q1, e1, _ = orc.quantize(x, B, w)
+    qa, ea, _ = orc.quantize_2d(x, B, 1, w)
+    assert np.array_equal(qa, q1) and np.array_equal(ea, e1)
+    q2, e2, _ = orc.quantize_2d(x, B, 2, w)
+    assert np.array_equal(e2, np.maximum(e1[0::2], e1[1::2]))
+    side = np.concatenate([x[0::2].reshape(3, 4, B), x[1::2].reshape(3, 4, B)], axis=2).reshape(3, 8 * B)
+    qs, es, _ = orc.quantize(side, 2 * B, w) if 2 * B <= 32 else (None, None, None)
+    if qs is not None:
+        assert np.array_equal(es, e2)
+        assert np.array_equal(qs.reshape(3, 4, 2, B)[:, :, 0].reshape(3, 4 * B), q2[0::2])
+        assert np.array_equal(qs.reshape(3, 4, 2, B)[:, :, 1].reshape(3, 4 * B), q2[1::2])
+    full = orc.expand_exponent_rows(e2, 2)
+    assert np.array_equal(full[0::2], e2) and np.array_equal(full[1::2], e2)
+    # decoded values obey the one-dimensional bounds with the shared exponent
+    xhat = orc.dequantize(q2, full, B, w)
+    step = np.repeat(np.ldexp(1.0, full.astype(np.int64) - 127 - (w - 2)), B, axis=1)
+    qmax = 2 ** (w - 1) - 1
+    free = np.abs(q2) < qmax
+    assert (np.abs(xhat - x)[free] <= 0.5 * step[free]).all() and (np.abs(xhat - x) <= step).all()
+    # nonfinite: one NaN poisons the pair of rows' block
+    x[1, 3] = np.nan
+    q3, e3, bad = orc.quantize_2d(x, B, 2, w)
+    assert bad == 1 and e3[0, 0] == 255 and (q3[0:2, :B] == 0).all()
+    assert orc.lib().mxo_format_bits(16, 2, 8, 8) == 8.25

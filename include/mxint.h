@@ -80,8 +80,17 @@ typedef struct {
     int32_t block;      /* 16 or 32 elements along K share one exponent                        */
     int32_t elem_bits;  /* w = 2..8, sign included (paper m = w - 1)                           */
     int32_t exp_bits;   /* 8 (the paper fixes the shared exponent to 8 bits)                   */
-    int32_t block_rows; /* 1 (the paper's 2-D block shape (16,2) would be 2; not supported)    */
+    int32_t block_rows; /* 1, or 2: two adjacent rows share their exponents, the paper's (16,2) */
 } mx_format_t;
+
+/* Two-row blocks (block_rows == 2; Sec. 4.1 and Fig. 2: the paper's unified block shape is
+ * (16,2), "block size 32"): `block` consecutive elements along K times two adjacent rows (2r and
+ * 2r+1) share one exponent, that of the largest magnitude among them.  The exponent array of a
+ * [rows, K] tensor is then uint8 [rows/2, K/block] and rows must be even (MX_ERR_SHAPE).
+ * Accepted by mx_quantize (stride_k == 1), mx_dequantize, mx_gemm / mx_linear and their _q forms
+ * for either operand with MX_ALGO_AUTO, MX_ALGO_TCGEN05 and MX_ALGO_SIMT; the streaming, in-kernel
+ * decode, batched, grouped and static entry points and the output format fy take one-row blocks
+ * only (MX_ERR_FORMAT). */
 
 /* ---- size helpers (host only, no CUDA call) ------------------------------------------- */
 

@@ -33,7 +33,7 @@ class MxFormat(C.Structure):
         super().__init__(block, elem_bits, exp_bits, block_rows)
 
     def __repr__(self):
-        return "MxFormat(block=%d, elem_bits=%d)" % (self.block, self.elem_bits)
+        return "MxFormat(block=%d, elem_bits=%d, block_rows=%d)" % (self.block, self.elem_bits, self.block_rows)
 
 
 class MxLinearArgs(C.Structure):
@@ -181,9 +181,9 @@ def mx_quantize(x: torch.Tensor, f: MxFormat, mant_out: Optional[torch.Tensor] =
     assert x.dim() == 2
     rows, K = x.shape
     if mant_out is None:
-        mant_out = torch.empty((rows, mx_mant_bytes(1, K, f)), dtype=torch.uint8, device=x.device)
-    if exp_out is None:
-        exp_out = torch.empty((rows, mx_exp_bytes(1, K, f)), dtype=torch.uint8, device=x.device)
+        mant_out = torch.empty((rows, K // 2 if f.elem_bits <= 4 else K), dtype=torch.uint8, device=x.device)
+    if exp_out is None:          # two-row blocks: one row of exponent bytes per pair of rows
+        exp_out = torch.empty((rows // max(f.block_rows, 1), K // f.block), dtype=torch.uint8, device=x.device)
     _check(lib.mx_quantize(_ptr(x), _dtype_code(x), rows, K, x.stride(0), x.stride(1), f,
                            _ptr(mant_out), _ptr(exp_out), _ptr(nonfinite_count), _stream(stream)),
            "mx_quantize")

@@ -32,7 +32,7 @@ __global__ void __launch_bounds__(256)
 gemm_simt_kernel(const uint8_t *__restrict__ a_mant, const uint8_t *__restrict__ a_exp, int wa,
                  const uint8_t *__restrict__ w_mant, const uint8_t *__restrict__ w_exp, int ww,
                  int64_t M, int64_t N, int64_t K, int block, const float *__restrict__ bias,
-                 float *__restrict__ y, int64_t ldy)
+                 float *__restrict__ y, int64_t ldy, int a_row_shift, int w_row_shift)
 {
     const int64_t j = (int64_t)blockIdx.x * 16 + (threadIdx.x & 15);
     const int64_t i = (int64_t)blockIdx.y * 16 + (threadIdx.x >> 4);
@@ -51,7 +51,7 @@ gemm_simt_kernel(const uint8_t *__restrict__ a_mant, const uint8_t *__restrict__
             P = __dp4a((int)al, (int)wl, P);
             P = __dp4a((int)ah, (int)wh, P);
         }
-        const int ea = a_exp[i * nb + b], ew = w_exp[j * nb + b];
+        const int ea = a_exp[(i >> a_row_shift) * nb + b], ew = w_exp[(j >> w_row_shift) * nb + b];   // shifts: two-row blocks
         poisoned |= (ea == 255) | (ew == 255);
         acc = acc + ldexpf((float)P, ea + ew + shift0);   // |P| < 2^24: exact before the add
     }

@@ -116,6 +116,7 @@ struct PackedStrides {
     int64_t mant_ld, exp_ld;          // bytes between rows of the mantissa / exponent arrays
     int64_t mant_batch, exp_batch;    // bytes between batch items
     int64_t out_batch;                // elements between batch items of the output
+    int exp_row_shift;                // 1: two adjacent rows share one row of exponent bytes (two-row blocks)
 };
 
 struct QuantOut {
@@ -160,10 +161,11 @@ __device__ __forceinline__ float absmax_nan(float m, float x)
 }
 
 // Eight values of one block (exponent byte `ebyte`, width w) -> their packed mantissas: one word of
-// two's-complement nibbles (w <= 4, returned in p.x) or two words of int8.  Same arithmetic as
+// two's-complement nibbles (w <= 4, returned in p.x) or two words of int8; xh receives the decoded
+// values.  Same arithmetic as
 // quantize_rows_body below (add-only rounding with the block-scaled magic constant, the
 // multiply-based form for blocks near the top of the range or holding Inf/NaN).
-__device__ __forceinline__ uint2 encode8_packed(const float (&v)[8], int ebyte, int w)
+__device__ __forceinline__ uint2 encode8_full(const float (&v)[8], int ebyte, int w, float (&xh)[8])
 {
     const bool nibble = w <= 4;
     const int qmax = (1 << (w - 1)) - 1;
@@ -175,16 +177,22 @@ __device__ __forceinline__ uint2 encode8_packed(const float (&v)[8], int ebyte, 
         const float M = __uint_as_float(mb);
         const float lo = __uint_as_float(mb - (uint32_t)qmax), hi = __uint_as_float(mb + (uint32_t)qmax);
 #pragma unroll
-        for (int i = 0; i < 8; ++i) f[i] = __float_as_uint(fminf(fmaxf(v[i] + M, lo), hi));
+        for (int i = 0; i < 8; ++i) {
+            const float t = fminf(fmaxf(v[i] + M, lo), hi);
+            f[i] = __float_as_uint(t);
+            xh[i] = t - M;                                   // the decoded value q * s, exactly
+        }
         corr = mb - off;
     } else {
         const float qmaxf = (float)qmax, pow2_wm2 = (float)(1 << (w - 2));
         const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
+        const float dec_small = small_neg_pow2(w), dec_big = pow2_from_biased(bad ? 127 : ebyte);
 #pragma unroll
         for (int i = 0; i < 8; ++i) {
             const float s = (v[i] * inv_pow2_E) * pow2_wm2;
             const float t = fminf(fmaxf(s, -qmaxf), qmaxf) + 12582912.f;
             f[i] = bad ? off : __float_as_uint(t) - 0x4B400000u + off;
+            xh[i] = bad ? __uint_as_float(0x7FC00000u) : ((t - 12582912.f) * dec_small) * dec_big;
         }
         corr = 0;
     }
@@ -203,6 +211,11 @@ __device__ __forceinline__ uint2 encode8_packed(const float (&v)[8], int ebyte, 
         p.y = (p.y - corr * 0x01010101u) ^ 0x80808080u;
     }
     return p;
+}
+__device__ __forceinline__ uint2 encode8_packed(const float (&v)[8], int ebyte, int w)
+{
+    float unused[8];
+    return encode8_full(v, ebyte, w, unused);
 }
 
 // rows x K, rows contiguous along K with leading dimension ldx.  BLOCK in {16, 32}.
@@ -357,6 +370,70 @@ quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t
                                            (int64_t)gridDim.x * (blockDim.x >> 5));
 }
 
+// Two-row blocks (the paper's (16,2) block shape, Sec. 4.1 / Fig. 2): BLOCK elements along K times
+// two adjacent rows share one exponent.  Work item of a warp = (pair of rows, segment of 256
+// elements); a lane owns 8 elements of each row, so the block maximum is a maximum over 16
+// registers and one or two shuffles.  Same rounding arithmetic as the one-row kernel; exponent
+// bytes [rows/2, K/BLOCK].  rows must be even.
+template <typename InT, int BLOCK>
+__global__ void __launch_bounds__(256)
+quantize_rows2_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w, QuantOut out)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    constexpr int LANES = BLOCK / 8;
+    constexpr int LANE_SHIFT = BLOCK == 16 ? 1 : 2;
+    const int lane = threadIdx.x & 31;
+    const int64_t cpr = K >> 3, segs = (cpr + 31) >> 5, n_items = (rows >> 1) * segs;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const bool nibble = w <= 4, leader = (lane & (LANES - 1)) == 0;
+    const int64_t nb_row = K / BLOCK, mant_ld = nibble ? (K >> 1) : K;
+    for (int64_t it = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < n_items; it += n_warps) {
+        const int64_t pr = it / segs, kc = (it - pr * segs) * 32 + lane;
+        const bool live = kc < cpr;
+        float v[2][8];
+        float am = 0.f;
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            if (live) {
+                Load8<InT>::run(x + (2 * pr + r) * ldx + kc * 8, v[r]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[r][i] = 0.f;
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) am = absmax_nan(am, v[r][i]);
+        }
+        uint32_t amax = __float_as_uint(am);
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+        if (!live) continue;
+        const int ebyte = (int)(amax >> 23);                // 255 <=> an Inf or NaN in the block
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const int64_t row = 2 * pr + r;
+            float xh[8];
+            const uint2 pk = encode8_full(v[r], ebyte, w, xh);
+            if (out.mant) {
+                if (nibble) *reinterpret_cast<uint32_t *>(out.mant + row * mant_ld + kc * 4) = pk.x;
+                else *reinterpret_cast<uint2 *>(out.mant + row * mant_ld + kc * 8) = pk;
+            }
+            if (out.xhat) {
+                uint32_t h[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i)
+                    h[i] = out.xhat_perm ? as_u32(__floats2bfloat162_rn(xh[i], xh[i + 4]))
+                                         : as_u32(__floats2bfloat162_rn(xh[2 * i], xh[2 * i + 1]));
+                *reinterpret_cast<uint4 *>(out.xhat + row * out.ld_xhat + kc * 8) = make_uint4(h[0], h[1], h[2], h[3]);
+            }
+        }
+        if (leader) {
+            if (out.mant) out.exps[pr * nb_row + (kc >> LANE_SHIFT)] = (uint8_t)ebyte;
+            if (ebyte == 255 && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+        }
+    }
+}
+
 // Several tensors in one launch (the distinct activation tensors of a grouped decode call):
 // blockIdx.y selects the tensor, blockIdx.x strides over its rows.
 struct QuantJob {
@@ -440,7 +517,7 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
             kc -= chunks_per_row;
             if (++row >= rows) break;
         }
-        const int ebyte = __ldg(exps + row * ps.exp_ld + (kc >> exp_shift));
+        const int ebyte = __ldg(exps + (row >> ps.exp_row_shift) * ps.exp_ld + (kc >> exp_shift));
         int q[8];
         if (w <= 4) {
             const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant + row * ps.mant_ld + kc * 4));
@@ -525,7 +602,7 @@ __device__ __forceinline__ void decode_bf16_body(const uint8_t *__restrict__ man
                     m[u][0] = __ldcs(src);
                     m[u][NIBBLE ? 0 : 1] = __ldcs(src + 1);
                 }
-                const uint8_t *ep = exps + row[u] * nb_row + ((kc[u] * 32) >> exp_shift);
+                const uint8_t *ep = exps + (row[u] >> ps.exp_row_shift) * nb_row + ((kc[u] * 32) >> exp_shift);
                 e[u] = b16 ? (uint32_t)ep[0] | ((uint32_t)ep[1] << 8) : (uint32_t)ep[0];
             }
         }
@@ -614,6 +691,7 @@ struct PrepJob {
     int ww;
     __nv_bfloat16 *w_hat;     // [N, K]
     int q_blocks;
+    int w_row_shift;          // 1: the weights have two-row blocks
 };
 
 template <typename InT, bool NIBBLE>
@@ -633,6 +711,7 @@ prep_operands_kernel(const PrepJob j)
         ps.mant_ld = NIBBLE ? j.K / 2 : j.K;
         ps.exp_ld = j.K / j.block;
         ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+        ps.exp_row_shift = j.w_row_shift;
         const int64_t wid = (int64_t)(blockIdx.x - j.q_blocks) * warps + (threadIdx.x >> 5);
         const int64_t nw = (int64_t)(gridDim.x - j.q_blocks) * warps;
         decode_bf16_body<NIBBLE, 2>(j.w_mant, j.w_exp, j.N, j.K, j.block, j.ww, j.w_hat, j.K, ps, wid, nw);

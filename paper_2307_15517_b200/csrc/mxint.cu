@@ -117,11 +117,13 @@ mx_status_t device_info(DeviceInfo **out)
     return d.is_sm100 ? MX_OK : MX_ERR_ARCH;
 }
 
+// block_rows == 2: two adjacent rows share the exponents (the paper's (16,2) block shape).
 bool format_ok(const mx_format_t &f)
 {
     return (f.block == 16 || f.block == 32) && f.elem_bits >= 2 && f.elem_bits <= 8 &&
-           f.exp_bits == 8 && f.block_rows == 1;
+           f.exp_bits == 8 && (f.block_rows == 1 || f.block_rows == 2);
 }
+bool format_1d(const mx_format_t &f) { return format_ok(f) && f.block_rows == 1; }
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 size_t round256(size_t n) { return (n + 255u) & ~size_t(255); }
 
@@ -178,6 +180,15 @@ mx_status_t launch_quantize_rows(const InT *x, int64_t rows, int64_t K, int64_t 
 {
     const int64_t chunks = rows * (K / 8);
     if (chunks == 0) return MX_OK;
+    if (f.block_rows == 2) {
+        const int grid = grid_for((chunks + 1) / 2, 256, d.sm_count, 4);
+        ProfScope prof(KIND_QUANTIZE, st);
+        if (f.block == 16)
+            MX_CUDA(launch_dep(mx::quantize_rows2_kernel<InT, 16>, dim3(grid), dim3(256), 0, st, x, rows, K, ldx, f.elem_bits, out));
+        else
+            MX_CUDA(launch_dep(mx::quantize_rows2_kernel<InT, 32>, dim3(grid), dim3(256), 0, st, x, rows, K, ldx, f.elem_bits, out));
+        return MX_OK;
+    }
     constexpr int UNROLL = 2;
     // at most one resident wave of CTAs: the grid-stride loop does the rest without a ragged second wave
     const int per_sm = f.block == 16 ? resident_ctas(mx::quantize_rows_kernel<InT, 16, UNROLL>)
@@ -207,6 +218,7 @@ mx::PackedStrides dense_strides(int64_t K, const mx_format_t &f)
     ps.mant_ld = f.elem_bits <= 4 ? K / 2 : K;
     ps.exp_ld = K / f.block;
     ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+    ps.exp_row_shift = f.block_rows == 2 ? 1 : 0;
     return ps;
 }
 
@@ -437,6 +449,7 @@ mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t 
     (void)a_exp;
     if (!format_ok(fa) || !format_ok(fw) || fa.block != fw.block) return MX_ERR_FORMAT;
     if (M <= 0 || N <= 0 || K <= 0 || (K % fa.block) != 0 || ldy < N) return MX_ERR_SHAPE;
+    if ((M % fa.block_rows) != 0 || (N % fw.block_rows) != 0) return MX_ERR_SHAPE;     // whole two-row blocks
     if (M > INT32_MAX / 2 || N > INT32_MAX / 2 || K > INT32_MAX / 2) return MX_ERR_SHAPE;
     if (!aligned16(a) || !aligned16(w) || !aligned16(y) || (bias && !aligned16(bias))) return MX_ERR_ALIGN;
     return MX_OK;
@@ -501,7 +514,7 @@ size_t stream_table_bytes(int32_t n_layers)
 bool stream_layer_ok(const mx_linear_args_t &a)
 {
     return a.M >= 1 && a.M <= 16 && a.fw.block == 32 && a.fa.block == 32 && a.fw.elem_bits <= 4 &&
-           (a.K % 128) == 0;
+           (a.K % 128) == 0 && a.fa.block_rows == 1 && a.fw.block_rows == 1;
 }
 
 size_t stream_act_bytes(const mx_linear_args_t &a)
@@ -538,7 +551,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
 {
     const int64_t M = a.M, N = a.N, K = a.K;
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
-    if ((K % 32) != 0) {
+    if ((K % 32) != 0 || a.fa.block_rows == 2) {
         mx_status_t s = quantize_rows_any(a.x, a.dt, M, K, a.ldx, a.fa, out, d, st);
         if (s != MX_OK) return s;
         return launch_dequant_bf16(a.w_mant, a.w_exp, N, K, a.fw, w_hat, K, d, st);
@@ -549,6 +562,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     job.a_hat = a_hat;
     job.w_mant = static_cast<const uint8_t *>(a.w_mant); job.w_exp = a.w_exp; job.N = N; job.ww = a.fw.elem_bits;
     job.w_hat = w_hat;
+    job.w_row_shift = a.fw.block_rows == 2 ? 1 : 0;
     const bool f32 = a.dt == MX_F32, nib = a.fw.elem_bits <= 4;
     const double qb = (double)M * K * ((f32 ? 4.0 : 2.0) + 2.0);
     const double db = (double)N * K * ((nib ? 0.5 : 1.0) + 1.0 / a.fw.block + 2.0);
@@ -594,8 +608,8 @@ size_t mx_mant_bytes(int64_t rows, int64_t K, mx_format_t f)
 
 size_t mx_exp_bytes(int64_t rows, int64_t K, mx_format_t f)
 {
-    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
-    return (size_t)rows * (size_t)(K / f.block);
+    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0 || (rows % f.block_rows) != 0) return 0;
+    return (size_t)(rows / f.block_rows) * (size_t)(K / f.block);
 }
 
 double mx_format_bits(mx_format_t f)
@@ -652,8 +666,9 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
                         uint32_t *nonfinite_count, void *stream)
 {
     if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
-    if (rows < 0 || K < 0 || (K % f.block) != 0) return MX_ERR_SHAPE;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || (rows % f.block_rows) != 0) return MX_ERR_SHAPE;
     if (rows == 0 || K == 0) return MX_OK;               // empty tensor: nothing to do
+    if (f.block_rows != 1 && stride_k != 1) return MX_ERR_FORMAT;   // two-row blocks: rows contiguous along K only
     if (!x || !mant_out || !exp_out) return MX_ERR_NULL;
     if (stride_k == 0 || (stride_k == 1 && stride_row < K)) return MX_ERR_SHAPE;
     if (!aligned16(x) || !aligned16(mant_out)) return MX_ERR_ALIGN;
@@ -681,7 +696,7 @@ mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, i
 {
     if (!mant || !exps || !out) return MX_ERR_NULL;
     if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
-    if (rows < 0 || K < 0 || (K % f.block) != 0 || ld_out < K) return MX_ERR_SHAPE;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || ld_out < K || (rows % f.block_rows) != 0) return MX_ERR_SHAPE;
     if (!aligned16(mant) || !aligned16(out) || (ld_out % 8) != 0) return MX_ERR_ALIGN;
     if (rows == 0 || K == 0) return MX_OK;
     DeviceInfo *d = nullptr;
@@ -726,11 +741,12 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         ProfScope prof(KIND_GEMM_SIMT, st);
         mx::gemm_simt_kernel<<<grid, 256, 0, st>>>(static_cast<const uint8_t *>(a_mant), a_exp,
                                                    fa.elem_bits, static_cast<const uint8_t *>(w_mant),
-                                                   w_exp, fw.elem_bits, M, N, K, fa.block, bias, y, ldy);
+                                                   w_exp, fw.elem_bits, M, N, K, fa.block, bias, y, ldy,
+                                                   fa.block_rows == 2 ? 1 : 0, fw.block_rows == 2 ? 1 : 0);
         MX_CUDA(cudaGetLastError());
         return MX_OK;
     }
-    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0;
+    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0 && fw.block_rows == 1;
     if (fused && !fused_ok(K, w_exp)) return MX_ERR_ALIGN;
     if (!workspace || workspace_bytes < (fused ? fused_workspace(M, K) : tc_workspace(M, N, K)))
         return MX_ERR_WORKSPACE;
@@ -791,7 +807,7 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         return mx_gemm_ex(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, nullptr, 0,
                           MX_ALGO_SIMT, stream);
     }
-    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0;
+    const bool fused = algo == MX_ALGO_TCGEN05_FUSED && (K % 32) == 0 && fw.block_rows == 1;
     if (fused && !fused_ok(K, w_exp)) return MX_ERR_ALIGN;
     if (workspace_bytes < (fused ? fused_workspace(M, K) : tc_workspace(M, N, K))) return MX_ERR_WORKSPACE;
     __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
@@ -825,7 +841,7 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
 static mx_status_t check_quantized_out(mx_format_t fy, int64_t N, const void *y_mant, const uint8_t *y_exp)
 {
     if (!y_mant || !y_exp) return MX_ERR_NULL;
-    if (!format_ok(fy)) return MX_ERR_FORMAT;
+    if (!format_1d(fy)) return MX_ERR_FORMAT;
     if ((N % fy.block) != 0) return MX_ERR_SHAPE;
     if (!aligned16(y_mant)) return MX_ERR_ALIGN;
     return MX_OK;
@@ -1082,6 +1098,7 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, nullptr, y, ldy);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
+    if (fa.block_rows != 1 || fw.block_rows != 1) return MX_ERR_FORMAT;     // slices of packed tensors: one-row blocks
     if (batch <= 0 || lda < K || ldw < K || stride_a < 0 || stride_w < 0 || stride_y < 0) return MX_ERR_SHAPE;
     // row and batch strides must keep whole blocks and whole container bytes together
     if ((lda % fa.block) || (ldw % fw.block) || (stride_a % fa.block) || (stride_w % fw.block) ||
@@ -1103,6 +1120,7 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
         ps.mant_batch = f.elem_bits <= 4 ? bstride / 2 : bstride;
         ps.exp_batch = bstride / f.block;
         ps.out_batch = (int64_t)(out_item / 2);
+        ps.exp_row_shift = 0;
         return ps;
     };
     // one decode launch per operand and one product launch cover every batch item
@@ -1192,6 +1210,7 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
+    if (fa.block_rows != 1 || fw.block_rows != 1) return MX_ERR_FORMAT;
     const size_t need = tc_workspace(M, N, K);
     if (need > (size_t)MX_STATIC_SCRATCH_BYTES) {
         snprintf(t_cuda_error, sizeof(t_cuda_error),

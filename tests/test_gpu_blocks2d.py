@@ -1,0 +1,102 @@
+"""GPU parity for two-row blocks (the paper's (16,2) block shape): quantizer bit-exact against
+the oracle's ``quantize_2d``, products against the oracle's product on the per-row expansion of
+the shared exponents."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import mx_oracle as orc
+from paper_2307_15517_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def mxb():
+    from paper_2307_15517_b200 import binding
+    return binding
+
+
+def _dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+@pytest.mark.parametrize("B", (16, 32))
+@pytest.mark.parametrize("w", (2, 4, 5, 8))
+def test_quantize_two_row_blocks_bit_exact(mxb, B, w):
+    F = mxb.MxFormat(B, w, 8, 2)
+    rng = np.random.default_rng(10 * B + w)
+    x = (rng.standard_t(3, (130, 2080)) * np.exp(rng.uniform(-6, 6, (130, 1)))).astype(np.float32)
+    x[4, :B] = 0.0
+    x[5, :B] = 0.0                                    # an all-zero pair block
+    x[6, 40] = np.inf                                 # a non-finite pair block
+    x[9, :] = np.ldexp(x[9, :], 110).astype(np.float32)   # near the top: the multiply-based rounding path
+    x[10, ::3] = (rng.integers(-7, 8, x[10, ::3].shape) * 0.5).astype(np.float32)   # ties
+    for data in (x, x[:2, :64].copy(), np.zeros((0, 64), np.float32)):
+        q, e, bad = orc.quantize_2d(data, B, 2, w)
+        cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+        mant, exps = mxb.mx_quantize(_dev(data), F, nonfinite_count=cnt)
+        assert exps.shape == e.shape and np.array_equal(exps.cpu().numpy(), e)
+        assert np.array_equal(mant.cpu().numpy(), orc.pack(q, w))
+        assert int(cnt.item()) == bad
+        if data.shape[0]:
+            want = orc.dequantize(q, orc.expand_exponent_rows(e, 2), B, w)
+            for dtype in (torch.float32, torch.bfloat16):
+                got = mxb.mx_dequantize(mant, exps, data.shape[1], F, dtype=dtype).float().cpu().numpy()
+                ok = ~np.isnan(want)
+                assert np.array_equal(np.isnan(got), np.isnan(want))
+                assert np.array_equal(got[ok].astype(np.float64), want[ok])
+    xb = torch.from_numpy(x).to(torch.bfloat16)
+    q, e, _ = orc.quantize_2d(xb.float().numpy(), B, 2, w)
+    mant, exps = mxb.mx_quantize(xb.cuda(), F)
+    assert np.array_equal(mant.cpu().numpy(), orc.pack(q, w)) and np.array_equal(exps.cpu().numpy(), e)
+
+
+@pytest.mark.parametrize("case", [(16, 8, 4, 2, 2), (16, 8, 4, 2, 1), (32, 4, 4, 1, 2), (16, 6, 3, 2, 2)])
+def test_products_with_two_row_blocks(mxb, case):
+    """The paper's layer: activations MXInt((16,2),8,7), weights MXInt((16,2),8,3) -- and the mixed
+    cases where only one operand has two-row blocks."""
+    B, wa, ww, ra, rw = case
+    M, K, N = 300, 1152, 528
+    x = synth.student_t_activations(M, K, seed=wa).numpy()
+    wt = synth.gaussian_weights(N, K, seed=ww).numpy()
+    bias = synth.gaussian_weights(1, N, seed=5, std=1.0)[0].numpy()
+    qa, ea, _ = orc.quantize_2d(x, B, ra, wa)
+    qw, ew, _ = orc.quantize_2d(wt, B, rw, ww)
+    y_ref, y_seq, S = orc.gemm(qa, orc.expand_exponent_rows(ea, ra), wa, qw, orc.expand_exponent_rows(ew, rw), ww, B,
+                               bias=bias)
+    fa, fw = mxb.MxFormat(B, wa, 8, ra), mxb.MxFormat(B, ww, 8, rw)
+    w_mant, w_exp = mxb.mx_quantize(_dev(wt), fw)
+    assert np.array_equal(w_exp.cpu().numpy(), ew)
+    y = mxb.mx_linear(_dev(x), fa, w_mant, w_exp, fw, N, bias=_dev(bias))
+    assert mxb.mx_poll_status() == 0
+    err = np.abs(y.cpu().numpy().astype(np.float64) - y_ref)
+    assert (err <= TOL * S + 1e-37).all()
+    a_mant, a_exp = mxb.mx_quantize(_dev(x), fa)
+    y2 = mxb.mx_gemm(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias=_dev(bias), algo=mxb.MX_ALGO_TCGEN05)
+    assert np.array_equal(y2.cpu().numpy(), y.cpu().numpy())
+    y3 = mxb.mx_gemm(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias=_dev(bias), algo=mxb.MX_ALGO_SIMT)
+    assert np.array_equal(y3.cpu().numpy(), y_seq)
+    # the MXInt-result form accepts two-row inputs as well
+    qo, eo, _, _, _ = orc.gemm_requant(qa, orc.expand_exponent_rows(ea, ra), wa, qw, orc.expand_exponent_rows(ew, rw),
+                                       ww, B, 16, 8, bias=bias)
+    ym, ye = mxb.mx_gemm_q(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, mxb.MxFormat(16, 8), bias=_dev(bias))
+    assert (ye.cpu().numpy() == eo).mean() > 0.99
+    assert (orc.unpack(ym.cpu().numpy(), N, 8) == qo).mean() > 0.99
+
+
+def test_two_row_blocks_are_refused_where_unsupported(mxb):
+    F2 = mxb.MxFormat(32, 4, 8, 2)
+    F1 = mxb.MxFormat(32, 4)
+    x = torch.randn(4, 256, device="cuda")
+    with pytest.raises(mxb.MxError):
+        mxb.mx_quantize(torch.randn(3, 64, device="cuda"), mxb.MxFormat(16, 4, 8, 2))      # odd row count
+    with pytest.raises(mxb.MxError):
+        mxb.mx_quantize(torch.randn(64, 4, device="cuda").t(), mxb.MxFormat(16, 4, 8, 2))  # strided axis
+    wm, we = mxb.mx_quantize(torch.randn(64, 256, device="cuda"), F2)
+    with pytest.raises(mxb.MxError):
+        mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64, algo=mxb.MX_ALGO_STREAM)
+    y = mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64)       # AUTO falls back to the tensor-core kernel
+    assert torch.isfinite(y).all() and mxb.mx_poll_status() == 0
+    del F1

@@ -50,6 +50,8 @@ def test_size_helpers_match_eq1(mxb):
     assert total == int(4096 * 4096 * 0.53125)
     assert mxb.mx_mant_bytes(4, 40, F(16, 4)) == 0             # K not a multiple of the block
     assert mxb.mx_mant_bytes(4, 64, F(8, 4)) == 0              # unsupported block
+    assert mxb.mx_exp_bytes(128, 768, F(16, 8, 8, 2)) == 64 * 48   # (16,2) blocks: one exponent row per pair of rows
+    assert mxb.mx_exp_bytes(127, 768, F(16, 8, 8, 2)) == 0
     f4 = F(16, 4)
     assert mxb.mx_workspace_bytes(128, 768, 768, f4, f4) >= 2 * (128 + 768) * 768   # both operands as bf16
     fused = mxb.mx_workspace_bytes_ex(128, 768, 768, f4, f4, mxb.MX_ALGO_TCGEN05_FUSED)
@@ -74,7 +76,9 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     assert L.mx_quantize(fake, 0, 4, 64, 32, 1, f, fake, fake, None, None) == -2   # ld < K
     assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 9), fake, fake, None, None) == -3
     assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4, 5), fake, fake, None, None) == -3
-    assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4, 8, 2), fake, fake, None, None) == -3
+    assert L.mx_quantize(fake, 0, 4, 64, 64, 1, F(16, 4, 8, 3), fake, fake, None, None) == -3   # block_rows 1 or 2
+    assert L.mx_quantize(fake, 0, 3, 64, 64, 1, F(16, 4, 8, 2), fake, fake, None, None) == -2   # odd rows, two-row blocks
+    assert L.mx_quantize(fake, 0, 4, 64, 1, 4, F(16, 4, 8, 2), fake, fake, None, None) == -3    # two-row blocks, strided axis
     assert L.mx_quantize(fake, 7, 4, 64, 64, 1, f, fake, fake, None, None) == -3
     assert L.mx_quantize(odd, 0, 4, 64, 64, 1, f, fake, fake, None, None) == -4
     assert L.mx_quantize(fake, 0, 4, 64, 68, 1, f, fake, fake, None, None) == -4   # ld % 8

@@ -150,6 +150,7 @@ GEMM_SHAPES = [
     (1, 256, 128, 32, 8, 4),          # a single row
     (257, 513, 2048, 32, 5, 2),
     (1536, 2560, 256, 16, 8, 4),      # 120 tiles of 128x256: the wide-tile kernel, multi-wave
+    (2100, 2330, 192, 32, 8, 4),      # 90 tiles of 256x256, ragged both ways: the CTA-pair kernel
 ]
 
 

@@ -230,6 +230,48 @@ def decode_sweep(mxb, synth, torch, hbm_gbs, iters=10):
     return out
 
 
+def llama7b_rate(mxb, synth, torch, iters=10):
+    """The seven LLaMA-7B-shaped linears at 4096 tokens with the per-layer widths and block sizes drawn
+    for seed 0 (mean width about 4 bits), Student-t activations: one pass = seven mx_linear calls.
+    Inputs, weights and outputs of a pass take ~1.2 GB, far beyond the L2."""
+    layers = []
+    for li, spec in enumerate(synth.llama7b_mixed_layers(0)):
+        x, w = synth.llama7b_inputs(spec, li, seed=0)
+        fa, fw = mxb.MxFormat(spec.block, spec.w_act), mxb.MxFormat(spec.block, spec.w_wgt)
+        wm, we = mxb.mx_quantize(w.cuda(), fw)
+        M = x.shape[0]
+        layers.append(dict(spec=spec, fa=fa, fw=fw, x=x.cuda(), wm=wm, we=we,
+                           y=torch.empty((M, spec.N), dtype=torch.float32, device="cuda"),
+                           ws=mxb.alloc_workspace(mxb.mx_workspace_bytes(M, spec.N, spec.K, fa, fw))))
+        del x, w
+
+    def one_pass():
+        for L in layers:
+            mxb.mx_linear(L["x"], L["fa"], L["wm"], L["we"], L["fw"], L["spec"].N, y=L["y"], workspace=L["ws"])
+
+    for _ in range(2):
+        one_pass()
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        one_pass()
+    b.record()
+    torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / iters
+    mxb.mx_profile_begin()
+    for _ in range(iters):
+        one_pass()
+    torch.cuda.synchronize()
+    prof = mxb.mx_profile_end()
+    flops = sum(2.0 * L["x"].shape[0] * L["spec"].N * L["spec"].K for L in layers)
+    gemm_ms = prof["gemm_tc"][0] / iters
+    return {"ms_per_pass": ms, "tops": flops / ms / 1e9, "flops": flops,
+            "gemm_ms_per_pass": gemm_ms, "gemm_tflops": flops / gemm_ms / 1e9,
+            "layers": [[L["spec"].name, L["spec"].K, L["spec"].N, L["spec"].block, L["spec"].w_act, L["spec"].w_wgt]
+                       for L in layers]}
+
+
 def quantize_rate(mxb, torch, hbm_gbs, iters=20):
     """Quantizer throughput on activation-sized tensors (fp32 in, packed MXInt4/B16 out):
     algorithmic bytes = 4 read + 0.5 + 1/16 written per element."""
@@ -508,6 +550,7 @@ def run_ours(args):
         secondary = {"linear_q": linear_q, "block_16x2": block_16x2,
                      "decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
                      "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
+                     "llama7b_mixed": llama7b_rate(mxb, synth, torch),
                      "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
         assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"

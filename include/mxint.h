@@ -253,6 +253,15 @@ MX_API mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t
  */
 MX_API mx_status_t mx_poll_status(void *stream);
 
+/*
+ * Self-test of that mechanism: launches one warp that waits, with the same bounded wait the
+ * product kernels use, on a barrier nobody arrives on.  The wait gives up after `limit_us`
+ * microseconds (1 .. 100000, else MX_ERR_SHAPE), the kernel records the expiry and returns
+ * normally; the next mx_poll_status on that stream then reports MX_ERR_TIMEOUT (and clears it).
+ * Nothing faults or hangs; the device and the context stay usable.
+ */
+MX_API mx_status_t mx_selftest_wait_expiry(uint32_t limit_us, void *stream);
+
 /* ---- the layer with an MXInt result ------------------------------------------------------------
  *
  * Sec. 3.2 (software emulators): an operator's floating-point result is quantized again to the

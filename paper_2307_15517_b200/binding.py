@@ -84,6 +84,8 @@ def _load() -> C.CDLL:
     L.mx_gemm_q.restype = i32
     L.mx_linear_q.restype = i32
     L.mx_poll_status.argtypes = [vp]
+    L.mx_selftest_wait_expiry.argtypes = [C.c_uint32, vp]
+    L.mx_selftest_wait_expiry.restype = i32
     L.mx_gemm_batched_workspace_bytes.argtypes = [i64, i64, i64, i64]
     L.mx_gemm_batched_workspace_bytes.restype = sz
     L.mx_gemm_batched.argtypes = [vp, vp, F, i64, i64, vp, vp, F, i64, i64, i64, i64, i64, i64, vp, i64, i64,
@@ -368,6 +370,11 @@ def mx_gemm_static(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: 
 def mx_poll_status(stream=None) -> int:
     """Synchronises the stream and returns the library's device status (0 = MX_OK)."""
     return int(lib.mx_poll_status(_stream(stream)))
+
+
+def mx_selftest_wait_expiry(limit_us: int = 2000, stream=None) -> None:
+    """Launches the library's bounded-wait self-test (a wait nobody satisfies, given up after limit_us)."""
+    _check(lib.mx_selftest_wait_expiry(limit_us, _stream(stream)), "mx_selftest_wait_expiry")
 
 
 KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream", "prep")

@@ -1364,6 +1364,32 @@ mx_status_t mx_profile_end(double *ms_per_kind, int64_t *launches_per_kind)
     return rc;
 }
 
+// One warp waits, with the library's bounded wait, on a barrier that nothing ever arrives on.
+__global__ void wait_probe_kernel(uint32_t *status, uint64_t limit_ns)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_flag;
+    if (threadIdx.x == 0) {
+        mx::ptx::mbar_init(mx::ptx::smem_u32(&bar), 1);
+        abort_flag = 0;
+        mx::ptx::fence_mbar_init();
+    }
+    __syncthreads();
+    const bool ok = mx::ptx::mbar_wait_bounded(mx::ptx::smem_u32(&bar), 0u, &abort_flag, limit_ns);
+    if (!ok && threadIdx.x == 0) atomicOr(status, mx::STATUS_TIMEOUT_BIT);
+}
+
+mx_status_t mx_selftest_wait_expiry(uint32_t limit_us, void *stream)
+{
+    if (limit_us == 0 || limit_us > 100000u) return MX_ERR_SHAPE;       // at most 0.1 s
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    wait_probe_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>(d->status, (uint64_t)limit_us * 1000ull);
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 mx_status_t mx_poll_status(void *stream)
 {
     DeviceInfo *d = nullptr;

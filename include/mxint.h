@@ -217,7 +217,7 @@ MX_API mx_status_t mx_linear_grouped(const mx_linear_args_t *layers, int32_t n_l
  * for W with ldw / stride_w; Y_b = y + b*stride_y with leading dimension ldy.  The attention
  * matmuls of Fig. 1 (tensors "A" = Q K^T and "B" = P V) are this call: heads side by side in a
  * [tokens, heads*d] tensor give lda = heads*d, stride_a = d.  lda, ldw, stride_a, stride_w must be
- * multiples of the block size and of 8.  Tensor-core kernel, one launch per batch item after one
+ * multiples of the block size and of 8.  Tensor-core kernel, one launch for all items after one
  * decode launch per operand; workspace from mx_gemm_batched_workspace_bytes.
  */
 MX_API size_t mx_gemm_batched_workspace_bytes(int64_t M, int64_t N, int64_t K, int64_t batch);
@@ -241,6 +241,16 @@ MX_API mx_status_t mx_softmax(float *s, int64_t ld, int64_t rows, int64_t cols, 
                               int causal, int64_t rows_per_batch, void *stream);
 MX_API mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int relu,
                                void *stream);
+
+/* mx_softmax followed by mx_quantize of its result, in one pass and without the fp32 probabilities
+ * ever reaching memory (Fig. 1(d): the probabilities are an MXInt operand of the P V product):
+ * p = Q_fp(softmax(scale * s)) with blocks of fp.block along the columns (the key/token axis, the
+ * reduction axis of P V).  s: device fp32 [rows, ld] (read only, ld % 4 == 0); p_mant: device,
+ * [rows, cols/2] bytes (fp.elem_bits <= 4) or [rows, cols] int8; p_exp: device uint8
+ * [rows, cols/fp.block]; cols <= 8192, cols % fp.block == 0 (MX_ERR_SHAPE); one-row blocks only. */
+MX_API mx_status_t mx_softmax_q(const float *s, int64_t ld, int64_t rows, int64_t cols, float scale,
+                                int causal, int64_t rows_per_batch, mx_format_t fp, void *p_mant,
+                                uint8_t *p_exp, void *stream);
 
 /* ---- device status --------------------------------------------------------------------- */
 

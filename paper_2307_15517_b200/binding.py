@@ -93,6 +93,8 @@ def _load() -> C.CDLL:
     L.mx_layernorm.argtypes = [vp, i64, vp, vp, C.c_float, i64, i64, vp, i64, vp]
     L.mx_softmax.argtypes = [vp, i64, i64, i64, C.c_float, i32, i64, vp]
     L.mx_relu_add.argtypes = [vp, vp, vp, i64, i32, vp]
+    L.mx_softmax_q.argtypes = [vp, i64, i64, i64, C.c_float, i32, i64, F, vp, vp, vp]
+    L.mx_softmax_q.restype = i32
     for name in ("mx_gemm_batched", "mx_layernorm", "mx_softmax", "mx_relu_add"):
         getattr(L, name).restype = i32
     L.mx_linear_grouped_workspace_bytes.argtypes = [C.POINTER(MxLinearArgs), i32]
@@ -333,6 +335,19 @@ def mx_softmax(s: torch.Tensor, scale: float = 1.0, causal: bool = False, rows_p
     _check(lib.mx_softmax(_ptr(s), s.stride(0), s.shape[0], s.shape[1], scale, 1 if causal else 0,
                           rows_per_batch, _stream(stream)), "mx_softmax")
     return s
+
+
+def mx_softmax_q(s: torch.Tensor, fp: MxFormat, scale: float = 1.0, causal: bool = False, rows_per_batch: int = 0,
+                 stream=None):
+    """Softmax over the rows of the 2-D fp32 tensor s, returned quantized to format fp: (mant, exps)."""
+    _need_cuda(s)
+    assert s.dim() == 2 and s.stride(1) == 1 and s.dtype == torch.float32
+    rows, cols = s.shape
+    mant = torch.empty((rows, cols // 2 if fp.elem_bits <= 4 else cols), dtype=torch.uint8, device=s.device)
+    exps = torch.empty((rows, cols // fp.block), dtype=torch.uint8, device=s.device)
+    _check(lib.mx_softmax_q(_ptr(s), s.stride(0), rows, cols, scale, 1 if causal else 0, rows_per_batch, fp,
+                            _ptr(mant), _ptr(exps), _stream(stream)), "mx_softmax_q")
+    return mant, exps
 
 
 def mx_relu_add(a: torch.Tensor, b: Optional[torch.Tensor], y: Optional[torch.Tensor] = None,

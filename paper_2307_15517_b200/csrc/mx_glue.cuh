@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "mx_quantize.cuh"
+
 namespace mx {
 
 constexpr int GLUE_THREADS = 256;
@@ -97,6 +99,73 @@ softmax_kernel(float *__restrict__ s, int64_t ld, int cols, float scale, int cau
     for (int i = 0; i < PER; ++i) {
         const int c = threadIdx.x + i * GLUE_THREADS;
         if (c < cols) row[c] = v[i] * inv;
+    }
+}
+
+// The same softmax with an MXInt result (the probabilities are the quantized left operand of the
+// P V product, Fig. 1(d)): p[r, :] = Q(softmax(scale * s[r, :])) with blocks of BLOCK along the
+// columns, written as packed mantissas [rows, cols/2 or cols] and exponent bytes [rows, cols/BLOCK];
+// no fp32 probabilities are written.  A thread holds 8 consecutive columns per chunk, so a block
+// is 2 or 4 neighbouring lanes; rounding as in the quantizer.  cols % 8 == 0, cols % BLOCK == 0.
+template <int PER8, int BLOCK>
+__global__ void __launch_bounds__(GLUE_THREADS)
+softmax_q_kernel(const float *__restrict__ s, int64_t ld, int cols, float scale, int causal, int64_t rows_per_batch,
+                 int w, uint8_t *__restrict__ p_mant, uint8_t *__restrict__ p_exp)
+{
+    __shared__ float scratch[GLUE_THREADS / 32];
+    constexpr int LANES = BLOCK / 8, LANE_SHIFT = BLOCK == 16 ? 1 : 2;
+    const float *row = s + (int64_t)blockIdx.x * ld;
+    const int limit = causal ? (int)((int64_t)blockIdx.x % rows_per_batch) + 1 : cols;
+    const int chunks = cols >> 3;
+    float v[PER8][8];
+    float m = -INFINITY;
+#pragma unroll
+    for (int i = 0; i < PER8; ++i) {
+        const int ch = threadIdx.x + i * GLUE_THREADS;
+        if (ch < chunks) {
+            const float4 a = *reinterpret_cast<const float4 *>(row + ch * 8);
+            const float4 b = *reinterpret_cast<const float4 *>(row + ch * 8 + 4);
+            const float t[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[i][j] = (ch * 8 + j < limit) ? t[j] * scale : -INFINITY;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[i][j] = -INFINITY;
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) m = fmaxf(m, v[i][j]);
+    }
+    m = block_max(m, scratch);
+    float sum = 0.f;
+#pragma unroll
+    for (int i = 0; i < PER8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            v[i][j] = v[i][j] == -INFINITY ? 0.f : expf(v[i][j] - m);
+            sum += v[i][j];
+        }
+    const float inv = 1.0f / block_sum(sum, scratch);
+    const bool nibble = w <= 4;
+    const int64_t mant_ld = nibble ? (cols >> 1) : cols, nb_row = cols / BLOCK;
+#pragma unroll
+    for (int i = 0; i < PER8; ++i) {
+        const int ch = threadIdx.x + i * GLUE_THREADS;
+        float am = 0.f;
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            v[i][j] *= inv;
+            am = absmax_nan(am, v[i][j]);
+        }
+        uint32_t amax = __float_as_uint(am);
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+        if (ch < chunks) {
+            const int ebyte = (int)(amax >> 23);
+            const uint2 pk = encode8_packed(v[i], ebyte, w);
+            if (nibble) *reinterpret_cast<uint32_t *>(p_mant + (int64_t)blockIdx.x * mant_ld + ch * 4) = pk.x;
+            else *reinterpret_cast<uint2 *>(p_mant + (int64_t)blockIdx.x * mant_ld + ch * 8) = pk;
+            if ((threadIdx.x & (LANES - 1)) == 0) p_exp[(int64_t)blockIdx.x * nb_row + (ch >> LANE_SHIFT)] = (uint8_t)ebyte;
+        }
     }
 }
 

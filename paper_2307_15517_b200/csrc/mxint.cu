@@ -1228,6 +1228,40 @@ mx_status_t mx_softmax(float *s_inout, int64_t ld, int64_t rows, int64_t cols, f
     return MX_OK;
 }
 
+mx_status_t mx_softmax_q(const float *s_in, int64_t ld, int64_t rows, int64_t cols, float scale, int causal,
+                         int64_t rows_per_batch, mx_format_t fp, void *p_mant, uint8_t *p_exp, void *stream)
+{
+    if (!s_in || !p_mant || !p_exp) return MX_ERR_NULL;
+    if (!format_1d(fp)) return MX_ERR_FORMAT;
+    if (rows < 0 || cols <= 0 || ld < cols || cols > mx::GLUE_THREADS * mx::GLUE_MAX_PER_THREAD ||
+        (cols % fp.block) != 0 || (causal && rows_per_batch <= 0))
+        return MX_ERR_SHAPE;
+    if (!aligned16(s_in) || !aligned16(p_mant) || (ld % 4) != 0) return MX_ERR_ALIGN;
+    if (rows == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t st_ = device_info(&d);
+    if (st_ != MX_OK) return st_;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int per8 = (int)((cols / 8 + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);      // 1..4
+    const unsigned g = (unsigned)rows;
+    uint8_t *pm = static_cast<uint8_t *>(p_mant);
+#define MX_SOFTMAX_Q(P8)                                                                                         \
+    do {                                                                                                         \
+        if (fp.block == 16)                                                                                      \
+            mx::softmax_q_kernel<P8, 16><<<g, mx::GLUE_THREADS, 0, st>>>(s_in, ld, (int)cols, scale, causal,     \
+                                                                         rows_per_batch, fp.elem_bits, pm, p_exp); \
+        else                                                                                                     \
+            mx::softmax_q_kernel<P8, 32><<<g, mx::GLUE_THREADS, 0, st>>>(s_in, ld, (int)cols, scale, causal,     \
+                                                                         rows_per_batch, fp.elem_bits, pm, p_exp); \
+    } while (0)
+    if (per8 <= 1) MX_SOFTMAX_Q(1);
+    else if (per8 <= 2) MX_SOFTMAX_Q(2);
+    else MX_SOFTMAX_Q(4);
+#undef MX_SOFTMAX_Q
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int relu, void *stream)
 {
     if (!a || !y) return MX_ERR_NULL;

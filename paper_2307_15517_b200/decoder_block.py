@@ -60,9 +60,13 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
     s = torch.empty((H * seq, seq), dtype=torch.float32, device=x.device)
     mxb.mx_gemm_batched(qm, qe, fa, hid, d, km, ke, fa, hid, d, seq, seq, d, H, s, seq, seq * seq)
     rec("scores", s.clone() if keep is not None else s)
-    p = rec("probs", mxb.mx_softmax(s, 1.0 / math.sqrt(d), causal=True, rows_per_batch=seq))
     # context per head: probabilities and values MXInt, blocks along the key/token axis
-    pm, pe = mxb.mx_quantize(p, fa)
+    if keep is None:
+        # softmax and quantization in one pass: the fp32 probabilities are never written
+        pm, pe = mxb.mx_softmax_q(s, fa, 1.0 / math.sqrt(d), causal=True, rows_per_batch=seq)
+    else:
+        p = rec("probs", mxb.mx_softmax(s, 1.0 / math.sqrt(d), causal=True, rows_per_batch=seq))
+        pm, pe = mxb.mx_quantize(p, fa)
     vm, ve = mxb.mx_quantize(v.t(), fa)                      # [hidden, seq]: blocks along tokens
     ctx = torch.empty((seq, hid), dtype=torch.float32, device=x.device)
     mxb.mx_gemm_batched(pm, pe, fa, seq, seq * seq, vm, ve, fa, seq, d * seq, seq, d, seq, H, ctx, hid, d)

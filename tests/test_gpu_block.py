@@ -116,3 +116,52 @@ def test_decoder_block_stage_by_stage(mods):
     _mx_close(T["ffn_out"], blk.linear(T["ffn_act"], *Wq["w2"], B, wa, ww, bias=p["b2"]))
     assert np.array_equal(out.cpu().numpy(), T["ffn_out"] + T["x1"])
     assert np.isfinite(out.cpu().numpy()).all()
+
+
+@pytest.mark.parametrize("fmt", [(16, 8), (32, 4), (16, 6)])
+def test_softmax_with_mxint_result(mods, fmt):
+    """mx_softmax_q against the oracle's softmax (fp64) quantized by the oracle: every code is a
+    rounding of the exact probability up to the fp32 softmax's own error, nearly all codes and
+    exponent bytes are the oracle's, and masked positions are exact zeros."""
+    mxb, _ = mods
+    B, w = fmt
+    g = torch.Generator().manual_seed(B + w)
+    for heads, seq in ((2, 160), (1, 2048), (3, 96)):
+        s = torch.randn(heads * seq, seq, generator=g) * 5
+        want = blk.softmax_causal(s.numpy(), 0.3, seq)
+        q, e, _ = orc.quantize(want.astype(np.float32), B, w)
+        pm, pe = mxb.mx_softmax_q(s.cuda(), mxb.MxFormat(B, w), 0.3, causal=True, rows_per_batch=seq)
+        eg = pe.cpu().numpy()
+        qg = orc.unpack(pm.cpu().numpy(), seq, w)
+        assert (eg == e).mean() > 0.995 and np.abs(eg.astype(int) - e.astype(int)).max() <= 1
+        assert (qg == q).mean() > 0.99
+        step = np.repeat(np.ldexp(1.0, eg.astype(np.int64) - 127 - (w - 2)), B, axis=1)
+        qmax = 2 ** (w - 1) - 1
+        tol = 2e-5 * want + 1e-9                       # fp32 exp and row sum
+        free = np.abs(qg) < qmax
+        assert (np.abs(qg * step - want)[free] <= (0.5 * step + tol)[free]).all()
+        assert (want[~free] >= ((qmax - 0.5) * step - tol)[~free]).all()
+        assert (qg[want == 0] == 0).all()
+        # the two-step path of the library gives the same codes up to the last-bit differences of its row sums
+        p2 = mxb.mx_softmax(s.clone().cuda(), 0.3, causal=True, rows_per_batch=seq)
+        pm2, pe2 = mxb.mx_quantize(p2, mxb.MxFormat(B, w))
+        assert (pm2 == pm).float().mean().item() > 0.995 and (pe2 == pe).float().mean().item() > 0.999
+
+
+def test_decoder_block_fused_softmax_matches_staged_run(mods):
+    mxb, db = mods
+    cfg = db.BlockConfig(hidden=256, heads=2, head_dim=128, ffn=512)
+    seq = 160
+    g = torch.Generator().manual_seed(12)
+    x = synth.outlier_activations(seq, cfg.hidden, 6, 2, 40.0).cuda()
+    W = {n: synth.gaussian_weights(o, i, 30 + j).cuda() for j, (n, o, i) in enumerate(
+        [("wq", 256, 256), ("wk", 256, 256), ("wv", 256, 256), ("wo", 256, 256), ("w1", 512, 256), ("w2", 256, 512)])}
+    P = {n: (torch.randn(sz, generator=g) * 0.1).cuda() for n, sz in
+         [("bq", 256), ("bk", 256), ("bv", 256), ("bo", 256), ("b1", 512), ("b2", 256), ("ln1_b", 256), ("ln2_b", 256)]}
+    P["ln1_g"] = torch.ones(256, device="cuda")
+    P["ln2_g"] = torch.ones(256, device="cuda")
+    qw = db.quantize_weights(cfg, W)
+    staged = db.run(cfg, x, qw, P, keep={}).cpu().numpy()
+    fused = db.run(cfg, x, qw, P).cpu().numpy()
+    assert mxb.mx_poll_status() == 0
+    assert np.abs(fused - staged).max() <= 2e-3 * np.abs(staged).max()

@@ -302,6 +302,30 @@ int mxo_expand_exponent_rows(const uint8_t *ebyte, int64_t rows, int64_t nb, int
     return MXO_OK;
 }
 
+/*
+ * Cast between MXInt precisions (Sec. 3.2, "No mixed-arithmetic but mixed-precision quantization":
+ * going from one mantissa width of the same format to another is an extension or a shortening of
+ * the mantissas plus a shift of the exponent).  Reading: the cast is the quantizer applied to the
+ * exactly decoded values -- shortening rounds to nearest even like every other rounding here, the
+ * exponent is re-derived from the block's largest decoded magnitude, widening loses nothing.
+ * Block sizes may differ between the two sides.
+ */
+int mxo_cast(const int8_t *q_in, const uint8_t *e_in, int64_t rows, int64_t K, int B_in, int w_in,
+             int B_out, int w_out, int8_t *q_out, uint8_t *e_out, uint32_t *nonfinite)
+{
+    if (!mxo_args_ok(rows, K, B_in, w_in) || !mxo_args_ok(rows, K, B_out, w_out)) return MXO_BAD_ARG;
+    const int64_t n = rows * K;
+    double *xd = (double *)malloc((size_t)(n > 0 ? n : 1) * sizeof(double));
+    float *xf = (float *)malloc((size_t)(n > 0 ? n : 1) * sizeof(float));
+    if (!xd || !xf) { free(xd); free(xf); return -2; }
+    int rc = mxo_dequantize(q_in, e_in, rows, K, B_in, w_in, xd);
+    for (int64_t i = 0; i < n; ++i) xf[i] = (float)xd[i];      /* exact: <= 7 bits times a power of two */
+    if (rc == 0) rc = mxo_quantize(xf, rows, K, K, 1, B_out, w_out, q_out, e_out, nonfinite);
+    free(xd);
+    free(xf);
+    return rc;
+}
+
 /* Average bits per value, Eq. 1: p = e/prod(B) + m + 1 with m = w - 1. */
 double mxo_format_bits(int block, int block_rows, int exp_bits, int w)
 {

@@ -49,6 +49,7 @@ def lib():
                                        p, p, p]
         L.mxo_quantize_2d.argtypes = [p, i64, i64, i64, i64, i32, i32, i32, p, p, p]
         L.mxo_expand_exponent_rows.argtypes = [p, i64, i64, i32, p]
+        L.mxo_cast.argtypes = [p, p, i64, i64, i32, i32, i32, i32, p, p, p]
         L.mxo_format_bits.argtypes = [i32, i32, i32, i32]
         L.mxo_format_bits.restype = C.c_double
         L.mxo_threads.restype = i32
@@ -100,6 +101,19 @@ def expand_exponent_rows(e, block_rows: int):
     out = np.zeros((e.shape[0] * block_rows, e.shape[1]), np.uint8)
     _check(lib().mxo_expand_exponent_rows(_ptr(e), out.shape[0], e.shape[1], block_rows, _ptr(out)))
     return out
+
+
+def cast(q, e, block_in: int, w_in: int, block_out: int, w_out: int):
+    """MXInt -> MXInt of another width (and block size).  Returns (q int8, ebyte uint8, nonfinite)."""
+    q = np.ascontiguousarray(q, np.int8)
+    e = np.ascontiguousarray(e, np.uint8)
+    rows, K = q.shape
+    qo = np.zeros((rows, K), np.int8)
+    eo = np.zeros((rows, K // block_out), np.uint8)
+    bad = C.c_uint32(0)
+    _check(lib().mxo_cast(_ptr(q), _ptr(e), rows, K, block_in, w_in, block_out, w_out, _ptr(qo), _ptr(eo),
+                          C.addressof(bad)))
+    return qo, eo, int(bad.value)
 
 
 def dequantize(q, e, block: int, w: int):

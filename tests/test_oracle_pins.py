@@ -512,3 +512,50 @@ def test_two_row_blocks_reduce_to_known_cases(B, w):
     q3, e3, bad = orc.quantize_2d(x, B, 2, w)
     assert bad == 1 and e3[0, 0] == 255 and (q3[0:2, :B] == 0).all()
     assert orc.lib().mxo_format_bits(16, 2, 8, 8) == 8.25
+
+
+# ---------------------------------------------------------------- casts between widths
+
+def test_casts_hand_worked():
+    rows = golden_io.load()
+    blocks = {r["id"]: r for r in rows if r["kind"] == "block"}
+    for r in (r for r in rows if r["kind"] == "cast"):
+        src = blocks[r["from"]]
+        assert int(src["w"]) == int(r["w_in"])
+        q = np.zeros((1, 16), np.int8)
+        v = golden_io.ints(src["q"])
+        q[0, :len(v)] = v
+        e = np.array([[int(src["ebyte"])]], np.uint8)
+        qo, eo, bad = orc.cast(q, e, 16, int(r["w_in"]), 16, int(r["w_out"]))
+        want = golden_io.ints(r["q"])
+        assert bad == 0 and eo[0, 0] == int(r["ebyte"])
+        assert qo[0, :len(want)].tolist() == want and (qo[0, len(want):] == 0).all()
+
+
+@pytest.mark.parametrize("w_in,w_out", [(4, 8), (3, 6), (8, 8), (2, 5)])
+def test_widening_casts_lose_nothing(w_in, w_out):
+    rng = np.random.default_rng(w_in * 10 + w_out)
+    x = (rng.standard_t(3, (9, 128)) * np.exp(rng.uniform(-5, 5, (9, 1)))).astype(np.float32)
+    q, e, _ = orc.quantize(x, 32, w_in)
+    for b_out in (16, 32):
+        qo, eo, bad = orc.cast(q, e, 32, w_in, b_out, w_out)
+        assert bad == 0
+        assert np.array_equal(orc.dequantize(qo, eo, b_out, w_out), orc.dequantize(q, e, 32, w_in))
+    q2, e2, _ = orc.cast(q, e, 32, w_in, 32, w_in)                 # same format: identity
+    assert np.array_equal(q2, q) and np.array_equal(e2, e)
+
+
+def test_narrowing_cast_error_bound_and_nonfinite():
+    rng = np.random.default_rng(77)
+    x = rng.standard_normal((5, 64)).astype(np.float32)
+    q, e, _ = orc.quantize(x, 16, 8)
+    e[2, 1] = 255
+    qo, eo, bad = orc.cast(q, e, 16, 8, 32, 3)
+    assert bad == 1 and eo[2, 0] == 255 and (qo[2, :32] == 0).all()
+    xin = orc.dequantize(q, e, 16, 8)
+    xout = orc.dequantize(qo, eo, 32, 3)
+    ok = ~np.isnan(xout)
+    step = np.repeat(np.ldexp(1.0, eo.astype(np.int64) - 127 - 1), 32, axis=1)
+    assert (np.abs(xout - xin)[ok] <= step[ok]).all()
+    free = ok & (np.abs(qo) < 3)
+    assert (np.abs(xout - xin)[free] <= 0.5 * step[free]).all()

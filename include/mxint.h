@@ -137,6 +137,18 @@ MX_API mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64
 MX_API mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
                           mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream);
 
+/*
+ * Cast an MXInt tensor to another MXInt format (Sec. 3.2, "No mixed-arithmetic but mixed-precision
+ * quantization": another mantissa width of the same format costs an extension or shortening of
+ * the mantissas and an exponent shift).  Defined as mx_quantize applied to the exactly decoded
+ * values: shortening rounds to nearest even and re-derives the block exponent, widening is exact,
+ * a cast to the same format is the identity.  Block sizes may differ; one-row blocks only.
+ * Arrays as for mx_quantize (dense rows); nonfinite_count as there.
+ */
+MX_API mx_status_t mx_cast(const void *mant_in, const uint8_t *exp_in, mx_format_t f_in, int64_t rows,
+                           int64_t K, mx_format_t f_out, void *mant_out, uint8_t *exp_out,
+                           uint32_t *nonfinite_count, void *stream);
+
 /* ---- block-scaled product (Sec. 3.2, MXInt dot-product operator, Fig. 3 right) --------- */
 
 /*

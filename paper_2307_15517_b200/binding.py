@@ -75,6 +75,8 @@ def _load() -> C.CDLL:
     L.mx_last_cuda_error.restype = C.c_char_p
     L.mx_quantize.argtypes = [vp, i32, i64, i64, i64, i64, F, vp, vp, vp, vp]
     L.mx_dequantize.argtypes = [vp, vp, i64, i64, F, vp, i32, i64, vp]
+    L.mx_cast.argtypes = [vp, vp, F, i64, i64, F, vp, vp, vp, vp]
+    L.mx_cast.restype = i32
     L.mx_gemm.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, vp]
     L.mx_gemm_ex.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, i32, vp]
     L.mx_linear.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, vp, i64, vp, sz, vp]
@@ -191,6 +193,18 @@ def mx_quantize(x: torch.Tensor, f: MxFormat, mant_out: Optional[torch.Tensor] =
     _check(lib.mx_quantize(_ptr(x), _dtype_code(x), rows, K, x.stride(0), x.stride(1), f,
                            _ptr(mant_out), _ptr(exp_out), _ptr(nonfinite_count), _stream(stream)),
            "mx_quantize")
+    return mant_out, exp_out
+
+
+def mx_cast(mant: torch.Tensor, exps: torch.Tensor, K: int, f_in: MxFormat, f_out: MxFormat,
+            nonfinite_count: Optional[torch.Tensor] = None, stream=None):
+    """MXInt tensor -> MXInt tensor of another width / block size.  Returns (mant, exps)."""
+    _need_cuda(mant, exps, nonfinite_count)
+    rows = mant.shape[0]
+    mant_out = torch.empty((rows, K // 2 if f_out.elem_bits <= 4 else K), dtype=torch.uint8, device=mant.device)
+    exp_out = torch.empty((rows, K // f_out.block), dtype=torch.uint8, device=mant.device)
+    _check(lib.mx_cast(_ptr(mant), _ptr(exps), f_in, rows, K, f_out, _ptr(mant_out), _ptr(exp_out),
+                       _ptr(nonfinite_count), _stream(stream)), "mx_cast")
     return mant_out, exp_out
 
 

@@ -434,6 +434,67 @@ quantize_rows2_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_
     }
 }
 
+// Cast between MXInt formats (Sec. 3.2: a different mantissa width of the same format): the
+// quantizer on the exactly decoded values of an MXInt tensor, without the fp32 copy in between.
+// Warp item = (row, segment of 256 elements), 8 elements per lane; one-row blocks on both sides.
+template <int BLOCK_OUT>
+__global__ void __launch_bounds__(256)
+cast_rows_kernel(const uint8_t *__restrict__ mant_in, const uint8_t *__restrict__ exp_in, int block_in, int w_in,
+                 int64_t rows, int64_t K, int w_out, QuantOut out)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    constexpr int LANES = BLOCK_OUT / 8;
+    constexpr int LANE_SHIFT = BLOCK_OUT == 16 ? 1 : 2;
+    const int lane = threadIdx.x & 31;
+    const int64_t cpr = K >> 3, segs = (cpr + 31) >> 5, n_items = rows * segs;
+    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    const bool nib_in = w_in <= 4, nib_out = w_out <= 4, leader = (lane & (LANES - 1)) == 0;
+    const int in_shift = block_in == 16 ? 1 : 2;                    // 8-element chunks per input block, as a shift
+    const int64_t nb_in = K / block_in, nb_out = K / BLOCK_OUT;
+    const int64_t ld_in = nib_in ? (K >> 1) : K, ld_out = nib_out ? (K >> 1) : K;
+    for (int64_t it = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < n_items; it += n_warps) {
+        const int64_t row = it / segs, kc = (it - row * segs) * 32 + lane;
+        const bool live = kc < cpr;
+        float v[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = 0.f;
+        if (live) {
+            const int eb = __ldg(exp_in + row * nb_in + (kc >> in_shift));
+            int q[8];
+            if (nib_in) {
+                const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant_in + row * ld_in + kc * 4));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) q[i] = ((int)(p << (28 - 4 * i))) >> 28;
+            } else {
+                const uint2 p = __ldg(reinterpret_cast<const uint2 *>(mant_in + row * ld_in + kc * 8));
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    q[i] = ((int)(p.x << (24 - 8 * i))) >> 24;
+                    q[4 + i] = ((int)(p.y << (24 - 8 * i))) >> 24;
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < 8; ++i) v[i] = decode_value(q[i], eb, w_in);      // exact in fp32
+        }
+        float am = 0.f;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) am = absmax_nan(am, v[i]);
+        uint32_t amax = __float_as_uint(am);
+#pragma unroll
+        for (int d = 1; d < LANES; d <<= 1) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+        if (!live) continue;
+        const int ebyte = (int)(amax >> 23);
+        const uint2 pk = encode8_packed(v, ebyte, w_out);
+        if (nib_out) *reinterpret_cast<uint32_t *>(out.mant + row * ld_out + kc * 4) = pk.x;
+        else *reinterpret_cast<uint2 *>(out.mant + row * ld_out + kc * 8) = pk;
+        if (leader) {
+            out.exps[row * nb_out + (kc >> LANE_SHIFT)] = (uint8_t)ebyte;
+            if (ebyte == 255 && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+        }
+    }
+}
+
 // Several tensors in one launch (the distinct activation tensors of a grouped decode call):
 // blockIdx.y selects the tensor, blockIdx.x strides over its rows.
 struct QuantJob {

@@ -739,6 +739,32 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
     return MX_OK;
 }
 
+mx_status_t mx_cast(const void *mant_in, const uint8_t *exp_in, mx_format_t f_in, int64_t rows, int64_t K,
+                    mx_format_t f_out, void *mant_out, uint8_t *exp_out, uint32_t *nonfinite_count, void *stream)
+{
+    if (!format_1d(f_in) || !format_1d(f_out)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f_in.block) != 0 || (K % f_out.block) != 0) return MX_ERR_SHAPE;
+    if (rows == 0 || K == 0) return MX_OK;
+    if (!mant_in || !exp_in || !mant_out || !exp_out) return MX_ERR_NULL;
+    if (!aligned16(mant_in) || !aligned16(mant_out)) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    mx::QuantOut out{static_cast<uint8_t *>(mant_out), exp_out, nullptr, 0, nonfinite_count};
+    const int grid = grid_for(rows * (K / 8), 256, d->sm_count, 8);
+    const uint8_t *mi = static_cast<const uint8_t *>(mant_in);
+    ProfScope prof(KIND_QUANTIZE, st);
+    if (f_out.block == 16)
+        MX_CUDA(launch_dep(mx::cast_rows_kernel<16>, dim3(grid), dim3(256), 0, st, mi, exp_in, (int)f_in.block,
+                           (int)f_in.elem_bits, rows, K, (int)f_out.elem_bits, out));
+    else
+        MX_CUDA(launch_dep(mx::cast_rows_kernel<32>, dim3(grid), dim3(256), 0, st, mi, exp_in, (int)f_in.block,
+                           (int)f_in.elem_bits, rows, K, (int)f_out.elem_bits, out));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
                           mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream)
 {

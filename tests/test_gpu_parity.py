@@ -333,3 +333,23 @@ def test_linear_mixed_precision(mxb, case):
     qa, ea, _ = orc.quantize(x.to(torch.bfloat16).float().numpy(), B, wa)
     y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias.numpy())
     _check_tol(yb, y_ref, S)
+
+
+# ------------------------------------------------------------------------------ casts
+
+@pytest.mark.parametrize("case", [(16, 8, 16, 4), (32, 4, 32, 8), (16, 6, 32, 3), (32, 8, 16, 2), (16, 3, 16, 3)])
+def test_cast_between_widths_bit_exact(mxb, case):
+    """mx_cast against the oracle's cast (the quantizer on the decoded values): integer work, bit for
+    bit, including zero, subnormal-scale, top-of-range and non-finite blocks."""
+    b_in, w_in, b_out, w_out = case
+    rng = np.random.default_rng(b_in + 7 * w_in + w_out)
+    x = np.concatenate([(rng.standard_t(3, (131, 2080)) * np.exp(rng.uniform(-8, 8, (131, 1)))).astype(np.float32),
+                        _edge_case_rows(2080)[:12]])
+    q, e, _ = orc.quantize(x, b_in, w_in)
+    qo, eo, bad = orc.cast(q, e, b_in, w_in, b_out, w_out)
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mant, exps = mxb.mx_cast(_dev(orc.pack(q, w_in)), _dev(e), 2080, mxb.MxFormat(b_in, w_in), mxb.MxFormat(b_out, w_out),
+                             nonfinite_count=cnt)
+    assert np.array_equal(exps.cpu().numpy(), eo)
+    assert np.array_equal(mant.cpu().numpy(), orc.pack(qo, w_out))
+    assert int(cnt.item()) == bad

@@ -88,6 +88,48 @@ struct TcParams {
     int yq_bits, yq_block;
 };
 
+// MXInt-result epilogue of one lane: r holds 32 consecutive fp32 outputs (columns n .. n + 31) of
+// row `row`, i.e. one block of 32 or two blocks of 16 along N; no exchange between lanes is needed.
+// Adds the bias, derives the exponent byte(s), rounds like the quantizer and stores 16 or 32
+// mantissa bytes and one or two exponent bytes.
+__device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, int n, uint32_t (&r)[32])
+{
+    if (row >= p.M || n >= p.N) return;
+    const int64_t nb_row = p.N / p.yq_block;
+    uint32_t amax[2] = {0u, 0u};
+#pragma unroll
+    for (int v = 0; v < 32; ++v) {
+        float x = __uint_as_float(r[v]);
+        if (p.bias && n + v < p.N) x += __ldg(p.bias + n + v);
+        r[v] = __float_as_uint(x);
+        amax[v >> 4] = max(amax[v >> 4], r[v] & 0x7FFFFFFFu);
+    }
+    if (p.yq_block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        if (n + 16 * h >= p.N) break;            // N % yq_block == 0: a half is all in or all out
+        const int ebyte = (int)(amax[h] >> 23);   // 255 <=> an Inf or NaN in the block
+        if (p.yq_block == 16 || h == 0) {
+            p.yq_exp[(int64_t)row * nb_row + (n + 16 * h) / p.yq_block] = (uint8_t)ebyte;
+            if (ebyte == 255 && p.yq_nonfinite) atomicAdd(p.yq_nonfinite, 1u);
+        }
+        uint2 pk[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            float v8[8];
+#pragma unroll
+            for (int v = 0; v < 8; ++v) v8[v] = __uint_as_float(r[16 * h + 8 * u + v]);
+            pk[u] = encode8_packed(v8, ebyte, p.yq_bits);
+        }
+        if (p.yq_bits <= 4)
+            *reinterpret_cast<uint2 *>(p.yq_mant + (int64_t)row * (p.N >> 1) + ((n + 16 * h) >> 1)) =
+                make_uint2(pk[0].x, pk[1].x);
+        else
+            *reinterpret_cast<uint4 *>(p.yq_mant + (int64_t)row * p.N + n + 16 * h) =
+                make_uint4(pk[0].x, pk[0].y, pk[1].x, pk[1].y);
+    }
+}
+
 // Raw bytes of one (row, half K-step) item: 32 mantissas and their exponent bytes.
 template <int WMODE> struct RawItem {
     uint4 m[WMODE == W_INT8 ? 2 : 1];
@@ -467,43 +509,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
                 if (!FUSED && p.yq_mant) {
-                    // ---- MXInt result: this lane holds 32 consecutive outputs of its row, i.e. one
-                    // block of 32 or two blocks of 16; no exchange between lanes is needed ----
-                    if (row < p.M && n < p.N) {
-                        const int64_t nb_row = p.N / p.yq_block;
-                        uint32_t amax[2] = {0u, 0u};
-#pragma unroll
-                        for (int v = 0; v < 32; ++v) {
-                            float x = __uint_as_float(r[v]);
-                            if (p.bias && n + v < p.N) x += __ldg(p.bias + n + v);
-                            r[v] = __float_as_uint(x);
-                            amax[v >> 4] = max(amax[v >> 4], r[v] & 0x7FFFFFFFu);
-                        }
-                        if (p.yq_block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
-#pragma unroll
-                        for (int h = 0; h < 2; ++h) {
-                            if (n + 16 * h >= p.N) break;            // N % yq_block == 0: a half is all in or all out
-                            const int ebyte = (int)(amax[h] >> 23);   // 255 <=> an Inf or NaN in the block
-                            if (p.yq_block == 16 || h == 0) {
-                                p.yq_exp[(int64_t)row * nb_row + (n + 16 * h) / p.yq_block] = (uint8_t)ebyte;
-                                if (ebyte == 255 && p.yq_nonfinite) atomicAdd(p.yq_nonfinite, 1u);
-                            }
-                            uint2 pk[2];
-#pragma unroll
-                            for (int u = 0; u < 2; ++u) {
-                                float v8[8];
-#pragma unroll
-                                for (int v = 0; v < 8; ++v) v8[v] = __uint_as_float(r[16 * h + 8 * u + v]);
-                                pk[u] = encode8_packed(v8, ebyte, p.yq_bits);
-                            }
-                            if (p.yq_bits <= 4)
-                                *reinterpret_cast<uint2 *>(p.yq_mant + (int64_t)row * (p.N >> 1) + ((n + 16 * h) >> 1)) =
-                                    make_uint2(pk[0].x, pk[1].x);
-                            else
-                                *reinterpret_cast<uint4 *>(p.yq_mant + (int64_t)row * p.N + n + 16 * h) =
-                                    make_uint4(pk[0].x, pk[0].y, pk[1].x, pk[1].y);
-                        }
-                    }
+                    store_mxint_chunk(p, row, n, r);
                     continue;
                 }
                 if (p.tma_store) {

@@ -10,7 +10,7 @@
 //
 //   warp 0      : TMA producer (one lane, in both CTAs; bytes are counted on the leader's barrier)
 //   warp 1      : tensor-memory allocation (both CTAs), MMA issue (leader only)
-//   warps 2..5  : epilogue of the CTA's own 128 rows
+//   warps 2..5  : epilogue of the CTA's own 128 rows (fp32, or MXInt as in the one-CTA kernel)
 // Barriers: full[s] lives in the leader (one arrival + the bytes of both CTAs), empty[s] and
 // tfull[a] in both (the MMA thread's commits are multicast to the pair), tempty[a] in the leader
 // (eight arrivals: the four epilogue warps of both CTAs).  No TMA load is multicast.  Every wait
@@ -172,6 +172,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
+                if (p.yq_mant) {
+                    store_mxint_chunk(p, row, n, r);
+                    continue;
+                }
                 if (p.tma_store) {
                     if (n < p.N && m0 + quad * 32 < p.M) {          // warp-uniform
                         const uint32_t buf = epi_base + (uint32_t)((warp - 2) * 2 + (epi_buf & 1)) * 4096u;

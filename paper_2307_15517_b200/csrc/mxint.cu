@@ -388,7 +388,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
 
 // The CTA-pair kernel: 256 x 256 tiles, fp32 result, one product per launch.
 mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N, int64_t K,
-                       const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+                       const float *bias, float *y, int64_t ldy, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
 {
     using Cfg = mx::Tc2Cfg;
     CUtensorMap tm_a, tm_w;
@@ -397,7 +397,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     s = encode_bf16_rows(&tm_w, w_hat, N, K, Cfg::BN / 2);
     if (s != MX_OK) return s;
     CUtensorMap tm_y = tm_a;
-    const bool tma_store = (ldy % 4) == 0;
+    const bool tma_store = !yq && (ldy % 4) == 0;
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
@@ -418,6 +418,11 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     p.status = d.status;
     p.tma_store = tma_store ? 1 : 0;
     p.batch = 1;
+    p.yq_mant = yq ? yq->mant : nullptr;
+    p.yq_exp = yq ? yq->exps : nullptr;
+    p.yq_nonfinite = yq ? yq->nonfinite : nullptr;
+    p.yq_bits = yq ? yq->f.elem_bits : 0;
+    p.yq_block = yq ? yq->f.block : 0;
     const int tiles = p.tiles_m * p.tiles_n;
     const int pairs = tiles < d.sm_count / 2 ? tiles : d.sm_count / 2;
     ProfScope prof(KIND_GEMM_TC, st);
@@ -442,8 +447,8 @@ mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64
     // +2 % on 2048 x 6144 x 2048 to +14 % on 8192^3).  With at most one tile per pair the one-CTA kernel
     // starts faster and wins.
     const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
-    if (!yq && tb.count == 1 && M > 128 && pair_tiles > d.sm_count / 2)
-        return launch_tc2(a_hat, w_hat, M, N, K, bias, y, ldy, d, st);
+    if (tb.count == 1 && M > 128 && pair_tiles > d.sm_count / 2)
+        return launch_tc2(a_hat, w_hat, M, N, K, bias, y, ldy, yq, d, st);
     const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256) * tb.count;
     if (N > 128 && tiles256 >= (int64_t)d.sm_count * 3 / 4)
         return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb);

@@ -46,6 +46,7 @@ EXACT_CASES = [
     (130, 208, 256, 32, 16, 2),       # N % 32 == 16: the last 32-column chunk is half outside
     (2048, 1024, 320, 16, 32, 6),     # wide tiles, several per CTA
     (1, 64, 64, 32, 32, 5),
+    (2100, 2336, 128, 16, 16, 8),     # 90 tiles of 256x256, ragged rows: the CTA-pair kernel's epilogue
 ]
 
 

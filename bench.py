@@ -314,6 +314,7 @@ def decoder_block_rate(mxb, synth, torch, iters=5):
                                               ("b2", hid), ("ln1_b", hid), ("ln2_b", hid))}
     params["ln1_g"] = torch.ones(hid, device="cuda")
     params["ln2_g"] = torch.ones(hid, device="cuda")
+    params = db.prepare_params(params)
     x = synth.outlier_activations(seq, hid, 4, -(-hid * 5 // 1000), 40.0).cuda()
     for _ in range(2):
         db.run(cfg, x, qw, params)

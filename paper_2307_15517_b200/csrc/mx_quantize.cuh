@@ -557,6 +557,77 @@ quantize_strided_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int6
     }
 }
 
+// Blocks along the slow axis of a row-major tensor (stride_row == 1: x[r, k] = base[k * stride_k + r],
+// e.g. V of attention quantized along the token axis).  A CTA owns 32 rows r and walks k in tiles of
+// 256: every warp reads 128 contiguous bytes per k (coalesced), the tile is transposed through
+// shared memory, then 8 lanes cover the 256 k of one row -- 32 consecutive k each, i.e. two blocks
+// of 16 or one of 32 -- so that they write 128 (nibbles) or 256 contiguous bytes per row.
+// Tile element (r, k) sits at r * 264 + k + k / 32: with this padding both the transposing store
+// and the per-lane reads are (nearly) free of bank conflicts.
+template <typename InT>
+__global__ void __launch_bounds__(256)
+quantize_transposed_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t stride_k, int block, int w,
+                           QuantOut out)
+{
+    __shared__ float tile[32 * 264];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const bool nibble = w <= 4;
+    const int64_t nb_row = K / block, mant_ld = nibble ? (K >> 1) : K;
+    const int64_t row_tiles = (rows + 31) >> 5, k_tiles = (K + 255) >> 8;
+    for (int64_t tix = blockIdx.x; tix < row_tiles * k_tiles; tix += gridDim.x) {
+        const int64_t r0 = (tix % row_tiles) * 32, k0 = (tix / row_tiles) * 256;
+        __syncthreads();                                    // the previous tile has been consumed
+#pragma unroll 4
+        for (int kk = warp; kk < 256; kk += 8) {
+            const int64_t k = k0 + kk;
+            float v = 0.f;
+            if (k < K && r0 + lane < rows) v = (float)x[k * stride_k + r0 + lane];
+            tile[lane * 264 + kk + (kk >> 5)] = v;
+        }
+        __syncthreads();
+        const int r = threadIdx.x >> 3, kg = threadIdx.x & 7;       // 32 k starting at k0 + 32 * kg of row r0 + r
+        const int64_t row = r0 + r, kb = k0 + 32 * kg;
+        if (row < rows && kb < K) {                                  // K % block == 0 and 32 % block == 0: whole blocks
+            const float *src = tile + r * 264 + kg * 33;
+            float v[4][8];
+            uint32_t amax[2] = {0u, 0u};
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float am = 0.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    v[c][i] = src[c * 8 + i];
+                    am = absmax_nan(am, v[c][i]);
+                }
+                amax[c >> 1] = max(amax[c >> 1], __float_as_uint(am));
+            }
+            if (block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
+            uint2 pk[4];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) pk[c] = encode8_packed(v[c], (int)(amax[c >> 1] >> 23), w);
+            if (nibble)
+                *reinterpret_cast<uint4 *>(out.mant + row * mant_ld + (kb >> 1)) = make_uint4(pk[0].x, pk[1].x, pk[2].x, pk[3].x);
+            else {
+                uint4 *dst = reinterpret_cast<uint4 *>(out.mant + row * mant_ld + kb);
+                dst[0] = make_uint4(pk[0].x, pk[0].y, pk[1].x, pk[1].y);
+                dst[1] = make_uint4(pk[2].x, pk[2].y, pk[3].x, pk[3].y);
+            }
+            const int e0 = (int)(amax[0] >> 23), e1 = (int)(amax[1] >> 23);
+            if (block == 32) {
+                out.exps[row * nb_row + (kb >> 5)] = (uint8_t)e0;
+                if (e0 == 255 && out.nonfinite) atomicAdd(out.nonfinite, 1u);
+            } else {
+                out.exps[row * nb_row + (kb >> 4)] = (uint8_t)e0;
+                out.exps[row * nb_row + (kb >> 4) + 1] = (uint8_t)e1;
+                if (out.nonfinite) {
+                    if (e0 == 255) atomicAdd(out.nonfinite, 1u);
+                    if (e1 == 255) atomicAdd(out.nonfinite, 1u);
+                }
+            }
+        }
+    }
+}
+
 // (mant, exps) -> decoded values, 8 elements per thread.
 template <typename OutT>
 __global__ void __launch_bounds__(256)

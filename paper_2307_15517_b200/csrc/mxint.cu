@@ -732,6 +732,20 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     mx::QuantOut out{static_cast<uint8_t *>(mant_out), exp_out, nullptr, 0, nonfinite_count};
     if (stride_k == 1) return quantize_rows_any(x, dt, rows, K, stride_row, f, out, *d, st);
+    if (stride_row == 1 && (K % 32) == 0 && (reinterpret_cast<uintptr_t>(mant_out) & 15u) == 0) {
+        // a transposed view: blocks along the slow axis of a row-major tensor
+        const int64_t tiles = ((rows + 31) / 32) * ((K + 255) / 256);
+        const int tgrid = (int)(tiles < (int64_t)d->sm_count * 4 ? tiles : (int64_t)d->sm_count * 4);
+        ProfScope prof(KIND_QUANTIZE, st);
+        if (dt == MX_F32)
+            mx::quantize_transposed_kernel<float><<<tgrid, 256, 0, st>>>(static_cast<const float *>(x), rows, K, stride_k,
+                                                                         f.block, f.elem_bits, out);
+        else
+            mx::quantize_transposed_kernel<__nv_bfloat16><<<tgrid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(x), rows, K,
+                                                                                 stride_k, f.block, f.elem_bits, out);
+        MX_CUDA(cudaGetLastError());
+        return MX_OK;
+    }
     const int grid = grid_for(rows * (K / f.block), 256, d->sm_count, 8);
     ProfScope prof(KIND_QUANTIZE, st);
     if (dt == MX_F32)

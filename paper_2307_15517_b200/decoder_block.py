@@ -29,9 +29,21 @@ class BlockConfig:
 
 
 def quantize_weights(cfg: BlockConfig, weights: Dict[str, torch.Tensor]):
-    """weights: fp32 CUDA tensors wq, wk, wv, wo [hidden, hidden], w1 [ffn, hidden], w2 [hidden, ffn]."""
+    """weights: fp32 CUDA tensors wq, wk, wv, wo [hidden, hidden], w1 [ffn, hidden], w2 [hidden, ffn].
+    The three projections of the block input are stored as one [3 * hidden, hidden] matrix (rows of wq, then
+    wk, then wv): one layer call then quantizes the input once and produces q, k and v side by side."""
     fw = mxb.MxFormat(cfg.block, cfg.w_wgt)
-    return {k: mxb.mx_quantize(v, fw) for k, v in weights.items()}
+    out = {k: mxb.mx_quantize(v, fw) for k, v in weights.items() if k not in ("wq", "wk", "wv")}
+    parts = [mxb.mx_quantize(weights[k], fw) for k in ("wq", "wk", "wv")]      # rows are quantized independently
+    out["wqkv"] = (torch.cat([p[0] for p in parts]), torch.cat([p[1] for p in parts]))
+    return out
+
+
+def prepare_params(params: Dict[str, torch.Tensor]) -> Dict[str, torch.Tensor]:
+    """Adds the concatenated bias of the fused q/k/v projection."""
+    out = dict(params)
+    out["bqkv"] = torch.cat([params["bq"], params["bk"], params["bv"]])
+    return out
 
 
 def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Tensor],
@@ -50,10 +62,11 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
         wm, we = qweights[name]
         return mxb.mx_linear(inp, fa, wm, we, fw, n_out, bias=bias)
 
+    if "bqkv" not in params:
+        params = prepare_params(params)
     h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
-    q = rec("q", linear(h1, "wq", params["bq"], hid))
-    k = rec("k", linear(h1, "wk", params["bk"], hid))
-    v = rec("v", linear(h1, "wv", params["bv"], hid))
+    qkv = linear(h1, "wqkv", params["bqkv"], 3 * hid)           # [seq, 3 * hidden]: q | k | v
+    q, k, v = rec("q", qkv[:, :hid]), rec("k", qkv[:, hid:2 * hid]), rec("v", qkv[:, 2 * hid:])
     # attention scores per head: both operands MXInt, blocks along the head dimension
     qm, qe = mxb.mx_quantize(q, fa)
     km, ke = mxb.mx_quantize(k, fa)

@@ -119,6 +119,26 @@ def test_quantize_along_a_strided_axis(mxb):
         assert np.array_equal(mant.cpu().numpy(), packed) and np.array_equal(exps.cpu().numpy(), e)
 
 
+@pytest.mark.parametrize("B,w", [(16, 4), (32, 8), (16, 6), (32, 2)])
+def test_quantize_transposed_view_bit_exact(mxb, B, w):
+    """Blocks along the slow axis of a row-major tensor (the transposing kernel): ragged row and k
+    tiles, edge-case values, non-finite count."""
+    rng = np.random.default_rng(B + w)
+    base = (rng.standard_t(3, (608, 77)) * np.exp(rng.uniform(-6, 6, (1, 77)))).astype(np.float32)   # [k, r]
+    edge = _edge_case_rows(608)                                                                     # [12, 608]
+    base[:, :12] = edge.T
+    q, e, bad = orc.quantize(np.ascontiguousarray(base.T), B, w)
+    cnt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    mant, exps = mxb.mx_quantize(_dev(base).t(), mxb.MxFormat(B, w), nonfinite_count=cnt)
+    assert np.array_equal(exps.cpu().numpy(), e)
+    assert np.array_equal(mant.cpu().numpy(), orc.pack(q, w))
+    assert int(cnt.item()) == bad and bad > 0
+    xb = torch.from_numpy(base).to(torch.bfloat16)
+    q, e, _ = orc.quantize(np.ascontiguousarray(xb.float().numpy().T), B, w)
+    mant, exps = mxb.mx_quantize(xb.cuda().t(), mxb.MxFormat(B, w))
+    assert np.array_equal(mant.cpu().numpy(), orc.pack(q, w)) and np.array_equal(exps.cpu().numpy(), e)
+
+
 def test_quantize_single_layer_config(mxb):
     x, wt, spec = synth.single_layer(0)
     F = mxb.MxFormat(spec.block, spec.w_act)

@@ -126,7 +126,7 @@ def test_softmax_with_mxint_result(mods, fmt):
     mxb, _ = mods
     B, w = fmt
     g = torch.Generator().manual_seed(B + w)
-    for heads, seq in ((2, 160), (1, 2048), (3, 96)):
+    for heads, seq in ((2, 160), (1, 2048), (3, 96), (1, 4096)):
         s = torch.randn(heads * seq, seq, generator=g) * 5
         want = blk.softmax_causal(s.numpy(), 0.3, seq)
         q, e, _ = orc.quantize(want.astype(np.float32), B, w)

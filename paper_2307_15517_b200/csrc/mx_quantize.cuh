@@ -376,19 +376,16 @@ quantize_rows_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t
 // registers and one or two shuffles.  Same rounding arithmetic as the one-row kernel; exponent
 // bytes [rows/2, K/BLOCK].  rows must be even.
 template <typename InT, int BLOCK>
-__global__ void __launch_bounds__(256)
-quantize_rows2_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w, QuantOut out)
+__device__ __forceinline__ void quantize_rows2_body(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx,
+                                                    int w, const QuantOut &out, int64_t warp_id, int64_t n_warps)
 {
-    ptx::dep_wait();
-    ptx::dep_trigger();
     constexpr int LANES = BLOCK / 8;
     constexpr int LANE_SHIFT = BLOCK == 16 ? 1 : 2;
     const int lane = threadIdx.x & 31;
     const int64_t cpr = K >> 3, segs = (cpr + 31) >> 5, n_items = (rows >> 1) * segs;
-    const int64_t n_warps = (int64_t)gridDim.x * (blockDim.x >> 5);
     const bool nibble = w <= 4, leader = (lane & (LANES - 1)) == 0;
     const int64_t nb_row = K / BLOCK, mant_ld = nibble ? (K >> 1) : K;
-    for (int64_t it = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); it < n_items; it += n_warps) {
+    for (int64_t it = warp_id; it < n_items; it += n_warps) {
         const int64_t pr = it / segs, kc = (it - pr * segs) * 32 + lane;
         const bool live = kc < cpr;
         float v[2][8];
@@ -432,6 +429,16 @@ quantize_rows2_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_
             if (ebyte == 255 && out.nonfinite) atomicAdd(out.nonfinite, 1u);
         }
     }
+}
+
+template <typename InT, int BLOCK>
+__global__ void __launch_bounds__(256)
+quantize_rows2_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t ldx, int w, QuantOut out)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    quantize_rows2_body<InT, BLOCK>(x, rows, K, ldx, w, out, (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5),
+                                    (int64_t)gridDim.x * (blockDim.x >> 5));
 }
 
 // Cast between MXInt formats (Sec. 3.2: a different mantissa width of the same format): the
@@ -824,6 +831,7 @@ struct PrepJob {
     __nv_bfloat16 *w_hat;     // [N, K]
     int q_blocks;
     int w_row_shift;          // 1: the weights have two-row blocks
+    int a_rows2;              // 1: the activations get two-row blocks
 };
 
 template <typename InT, bool NIBBLE>
@@ -836,7 +844,10 @@ prep_operands_kernel(const PrepJob j)
     if ((int)blockIdx.x < j.q_blocks) {
         QuantOut out{nullptr, nullptr, j.a_hat, j.K, nullptr};
         const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)j.q_blocks * warps;
-        if (j.block == 16) quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
+        if (j.a_rows2) {
+            if (j.block == 16) quantize_rows2_body<InT, 16>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
+            else quantize_rows2_body<InT, 32>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
+        } else if (j.block == 16) quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
         else quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
     } else {
         PackedStrides ps;

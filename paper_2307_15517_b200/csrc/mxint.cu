@@ -604,7 +604,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
 {
     const int64_t M = a.M, N = a.N, K = a.K;
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
-    if ((K % 32) != 0 || a.fa.block_rows == 2) {
+    if ((K % 32) != 0) {
         mx_status_t s = quantize_rows_any(a.x, a.dt, M, K, a.ldx, a.fa, out, d, st);
         if (s != MX_OK) return s;
         return launch_dequant_bf16(a.w_mant, a.w_exp, N, K, a.fw, w_hat, K, d, st);
@@ -616,6 +616,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     job.w_mant = static_cast<const uint8_t *>(a.w_mant); job.w_exp = a.w_exp; job.N = N; job.ww = a.fw.elem_bits;
     job.w_hat = w_hat;
     job.w_row_shift = a.fw.block_rows == 2 ? 1 : 0;
+    job.a_rows2 = a.fa.block_rows == 2 ? 1 : 0;
     const bool f32 = a.dt == MX_F32, nib = a.fw.elem_bits <= 4;
     const double qb = (double)M * K * ((f32 ? 4.0 : 2.0) + 2.0);
     const double db = (double)N * K * ((nib ? 0.5 : 1.0) + 1.0 / a.fw.block + 2.0);

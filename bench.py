@@ -272,6 +272,28 @@ def llama7b_rate(mxb, synth, torch, iters=10):
                        for L in layers]}
 
 
+def single_layer_latency(mxb, synth, torch, iters=200):
+    """The single 128 x 768 x 768 MXInt4/B16 layer (151 MFLOP: latency-bound, two launches)."""
+    x, w, spec = synth.single_layer(0)
+    fa, fw = mxb.MxFormat(spec.block, spec.w_act), mxb.MxFormat(spec.block, spec.w_wgt)
+    xd = x.cuda()
+    wm, we = mxb.mx_quantize(w.cuda(), fw)
+    y = torch.empty((x.shape[0], spec.N), dtype=torch.float32, device="cuda")
+    ws = mxb.alloc_workspace(mxb.mx_workspace_bytes(x.shape[0], spec.N, spec.K, fa, fw))
+    for _ in range(10):
+        mxb.mx_linear(xd, fa, wm, we, fw, spec.N, y=y, workspace=ws)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(iters):
+        mxb.mx_linear(xd, fa, wm, we, fw, spec.N, y=y, workspace=ws)
+    b.record()
+    torch.cuda.synchronize()
+    us = a.elapsed_time(b) * 1e3 / iters
+    return {"us_per_call": us, "tops": 2.0 * x.shape[0] * spec.N * spec.K / us / 1e6,
+            "note": "back-to-back calls on one stream, operands L2-resident; a roofline fraction is not meaningful here"}
+
+
 def quantize_rate(mxb, torch, hbm_gbs, iters=20):
     """Quantizer throughput on activation-sized tensors (fp32 in, packed MXInt4/B16 out):
     algorithmic bytes = 4 read + 0.5 + 1/16 written per element."""
@@ -551,6 +573,7 @@ def run_ours(args):
         secondary = {"linear_q": linear_q, "block_16x2": block_16x2,
                      "decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
                      "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
+                     "single_layer": single_layer_latency(mxb, synth, torch),
                      "llama7b_mixed": llama7b_rate(mxb, synth, torch),
                      "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}

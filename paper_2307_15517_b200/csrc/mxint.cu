@@ -261,6 +261,25 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
 }
 
 // ---- tensor-core GEMM launcher ----------------------------------------------------------------
+// Encoded tensor maps by (kind, base, extents): pure functions of their key, so entries never go stale.
+typedef std::tuple<int, const void *, int64_t, int64_t, int64_t, int64_t, int64_t> MapKey;
+std::map<MapKey, CUtensorMap> g_map_cache;
+std::mutex g_map_mu;
+bool cached_map(const MapKey &key, CUtensorMap *out)
+{
+    std::lock_guard<std::mutex> lk(g_map_mu);
+    auto it = g_map_cache.find(key);
+    if (it == g_map_cache.end()) return false;
+    *out = it->second;
+    return true;
+}
+void remember_map(const MapKey &key, const CUtensorMap &tm)
+{
+    std::lock_guard<std::mutex> lk(g_map_mu);
+    if (g_map_cache.size() > 8192) g_map_cache.clear();
+    g_map_cache[key] = tm;
+}
+
 // bf16 [rows, K] (dense rows); batch > 1: `batch` such items `item_bytes` apart, as a rank-3 map.
 mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, int64_t K, int box_rows,
                              int64_t batch = 1, size_t item_bytes = 0)
@@ -275,6 +294,10 @@ mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, in
         }
         g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
     }
+    // A map depends only on these seven numbers; a layer called again with the same workspace finds
+    // its maps here instead of paying a driver call each (a few microseconds per product for small layers).
+    const MapKey key = std::make_tuple(0, base, rows, K, (int64_t)box_rows, batch, (int64_t)item_bytes);
+    if (cached_map(key, tm)) return MX_OK;
     const cuuint64_t dims[3] = {(cuuint64_t)K, (cuuint64_t)rows, (cuuint64_t)batch};
     const cuuint64_t strides[2] = {(cuuint64_t)K * 2, (cuuint64_t)item_bytes};
     const cuuint32_t box[3] = {(cuuint32_t)mx::TC_BK, (cuuint32_t)box_rows, 1};
@@ -287,6 +310,7 @@ mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, in
         snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled failed (%d)", (int)r);
         return MX_ERR_CUDA;
     }
+    remember_map(key, *tm);
     return MX_OK;
 }
 
@@ -312,6 +336,8 @@ struct PackedW {                 // weight operand of the fused kernels (unused 
 mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int64_t ldy, int64_t batch = 1,
                            int64_t y_batch = 0)
 {
+    const MapKey key = std::make_tuple(1, static_cast<const void *>(y), M, N, ldy, batch, y_batch);
+    if (cached_map(key, tm)) return MX_OK;
     const cuuint64_t dims[3] = {(cuuint64_t)N, (cuuint64_t)M, (cuuint64_t)batch};
     const cuuint64_t strides[2] = {(cuuint64_t)ldy * 4, (cuuint64_t)y_batch * 4};
     const cuuint32_t box[3] = {32, 32, 1};
@@ -323,6 +349,7 @@ mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int6
         snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled (output) failed (%d)", (int)r);
         return MX_ERR_CUDA;
     }
+    remember_map(key, *tm);
     return MX_OK;
 }
 

@@ -98,6 +98,21 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     assert q(N=40) == -2                                     # 40 is not a multiple of the output block
     assert q(fy=mxb.MxFormat(8, 4)) == -3
     assert q(ym=None) == -1 and q(ye=None) == -1
+    assert q(fy=F(16, 4, 8, 2)) == -3                        # the result format takes one-row blocks only
+    # casts and the softmax with an MXInt result
+    c = lambda **kw: L.mx_cast(kw.get("m", fake), fake, kw.get("fi", f), kw.get("rows", 4), kw.get("K", 64),
+                               kw.get("fo", F(32, 8)), kw.get("mo", fake), fake, None, None)
+    assert c(K=48) == -2                                     # 48 is not a multiple of the output block 32
+    assert c(fi=F(16, 4, 8, 2)) == -3 and c(fo=F(16, 9)) == -3
+    assert c(m=None) == -1 and c(mo=odd) == -4
+    assert c(rows=0) == 0                                    # empty tensor: nothing to do
+    sq = lambda **kw: L.mx_softmax_q(kw.get("s", fake), kw.get("ld", 64), 4, kw.get("cols", 64), C.c_float(1.0),
+                                     kw.get("causal", 0), kw.get("rpb", 0), kw.get("fp", F(16, 8)), fake, fake, None)
+    assert sq(cols=40) == -2 and sq(cols=16384, ld=16384) == -2 and sq(ld=32) == -2
+    assert sq(causal=1, rpb=0) == -2
+    assert sq(fp=F(16, 8, 8, 2)) == -3
+    assert sq(s=None) == -1 and sq(ld=66) == -4
+    assert L.mx_selftest_wait_expiry(0, None) == -2
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")

@@ -21,6 +21,9 @@
  * Conventions for every entry point:
  *   - All data pointers are DEVICE pointers owned by the caller.  The library neither
  *     allocates, frees nor keeps them.  Base pointers must be 16-byte aligned.
+ *   - Every call works on the CURRENT CUDA device of the calling thread: all pointers must belong
+ *     to it, `stream` must be one of its streams, and the library's per-device state (status
+ *     word, tensor-map cache, the built-in scratch of mx_gemm_static) is that device's.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls are
  *     asynchronous on it and never synchronise the host, except mx_poll_status.
  *   - Arguments are validated on the host before anything is launched; a negative
@@ -332,6 +335,7 @@ MX_API mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t 
  *  - The call creates no buffer, event or handle: no cudaMalloc/cudaFree, no allocating library
  *    routine.  The first call on a device looks up the array's device address and sets a kernel
  *    attribute; make that first call before any stream capture begins.
+ *  - The array used is the CURRENT device's copy; the operands must live on that device.
  *  - All calls on a device share the one array.  It keeps the previous call's bytes; the call
  *    rewrites every byte it later reads, so nothing has to be cleared.  Two calls whose kernels
  *    can overlap on the GPU (different streams, or different host threads) race on it: issue

@@ -140,9 +140,19 @@ def _dtype_code(t: torch.Tensor) -> int:
 
 
 def _need_cuda(*tensors):
+    """Every tensor must live on the CURRENT CUDA device: the library launches on the current device
+    and keeps its per-device state (status word, built-in scratch) by that device's index."""
+    cur = None
     for t in tensors:
-        if t is not None and not t.is_cuda:
+        if t is None:
+            continue
+        if not t.is_cuda:
             raise ValueError("device tensors required (this library has no host path)")
+        if cur is None:
+            cur = torch.cuda.current_device()
+        if t.device.index != cur:
+            raise ValueError("tensor on cuda:%d but the current device is cuda:%d; select the device first "
+                             "(torch.cuda.set_device / torch.cuda.device)" % (t.device.index, cur))
 
 
 # ---- size helpers ---------------------------------------------------------------------------

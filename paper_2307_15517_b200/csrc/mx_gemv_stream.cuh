@@ -7,12 +7,14 @@
 // scale per block, blocks added in ascending order in fp32 -- bit-identical to the CUDA-core
 // kernel when a row's blocks are not split over warps.
 //
-//  * weights  : packed 4-bit mantissas [N, K/2] + exponent bytes [N, K/32] (block 32), read with
-//               coalesced 32-bit loads, four blocks (and their four exponent bytes) per step,
-//               the next step's ten registers prefetched while the current one is consumed.
+//  * weights  : packed 4-bit mantissas [N, K/2] + exponent bytes [N, K/32] (block 32).  TMA
+//               variant: every warp owns a two-stage ring of shared-memory stages, each filled by
+//               three tiled TMA loads (16 rows x 256 mantissa bytes as two 128-byte swizzled boxes,
+//               16 rows x 16 exponent bytes).  Register variant: coalesced 32-bit loads, four blocks
+//               and their four exponent bytes per step, two register sets alternating.
 //  * tokens   : already quantized (int8 or nibble container); each CTA stages them once per
-//               layer into shared memory in the operand order of the integer MMA below, with
-//               their float block scales and the per-block sums needed to undo the +8 offset.
+//               layer into shared memory in the operand order of the integer MMA below, together
+//               with their float block scales.
 //  * per block: a two's-complement nibble moved into the HIGH half of a byte is the signed byte
 //               16*q, so one shift/AND pair turns a packed word into the A operand of
 //               mma.sync.m16n8k32 (s8 x s8 -> s32) with no sign extension; the accumulator starts
@@ -324,7 +326,9 @@ gemv_stream_kernel(const StreamParams p)
                     const CUtensorMap *tm_m = p.tmaps + 2 * li, *tm_e = tm_m + 1;
                     const int nblk = b_hi - b_lo;                       // multiple of 16
                     auto issue = [&](int step, int st) {              // step: CH-block chunk index from b_lo
-                        if (lane == 0) {
+                        // after an expired wait (this warp's or, through the flag, another's) nothing new
+                        // is put in flight: the CTA is about to return
+                        if (lane == 0 && !timed_out && *abort_flag == 0) {
                             const uint32_t bar = my_bar + 8 * st;
                             const uint32_t dst = ptx::smem_u32(my_stage + st * Cfg::MANT_BYTES);
                             const int b = b_lo + step * CH;
@@ -342,7 +346,11 @@ gemv_stream_kernel(const StreamParams p)
                     for (int step = 0; step < nsteps && !timed_out; ++step) {
                         const bool ok = ptx::mbar_wait_bounded(my_bar + 8 * st, (phase_bits >> st) & 1u, abort_flag,
                                                                STREAM_WAIT_LIMIT_NS);
-                        if (!__all_sync(0xFFFFFFFFu, ok)) { timed_out = true; break; }
+                        if (!__all_sync(0xFFFFFFFFu, ok)) {
+                            timed_out = true;
+                            *abort_flag = 1;                          // the other warps stop issuing as well
+                            break;
+                        }
                         phase_bits ^= 1u << st;
                         const uint8_t *sm = my_stage + st * Cfg::MANT_BYTES;
                         const uint8_t *se = my_exps + st * (16 * CH);
@@ -414,7 +422,11 @@ gemv_stream_kernel(const StreamParams p)
     if (BULK && timed_out) {
         *abort_flag = 1;
         atomicOr(p.status, 1u);
+        // copies already in flight get time to land before the CTA's shared memory is released
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 100000ull) __nanosleep(1000);
     }
+    if (BULK) __syncthreads();                // no warp leaves while another may still be waiting out its copies
 }
 
 }  // namespace mx

@@ -39,6 +39,7 @@ struct DeviceInfo {
     bool tc2_attr_set = false;
 };
 DeviceInfo g_dev[MAX_DEVICES];
+std::mutex g_init_mu;        // guards every lazily initialised field above and below (calls may come from several host threads)
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *,
                                   const cuuint64_t *, const cuuint64_t *, const cuuint32_t *,
@@ -102,6 +103,7 @@ mx_status_t device_info(DeviceInfo **out)
     MX_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= MAX_DEVICES) return MX_ERR_CUDA;
     DeviceInfo &d = g_dev[dev];
+    std::lock_guard<std::mutex> lk(g_init_mu);
     if (!d.probed) {
         int major = 0, sms = 0;
         MX_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev));
@@ -280,19 +282,39 @@ void remember_map(const MapKey &key, const CUtensorMap &tm)
     g_map_cache[key] = tm;
 }
 
+// The driver's tensor-map encoder, looked up once.
+mx_status_t ensure_encoder()
+{
+    std::lock_guard<std::mutex> lk(g_init_mu);
+    if (g_encode_tiled) return MX_OK;
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
+    if (q != cudaDriverEntryPointSuccess || !fn) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled not available");
+        return MX_ERR_CUDA;
+    }
+    g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    return MX_OK;
+}
+
+// Sets a kernel's dynamic shared-memory limit the first time the kernel is used on a device.
+template <typename K> mx_status_t smem_attr_once(bool &done, K kernel, int bytes)
+{
+    std::lock_guard<std::mutex> lk(g_init_mu);
+    if (done) return MX_OK;
+    MX_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes));
+    done = true;
+    return MX_OK;
+}
+
 // bf16 [rows, K] (dense rows); batch > 1: `batch` such items `item_bytes` apart, as a rank-3 map.
 mx_status_t encode_bf16_rows(CUtensorMap *tm, const void *base, int64_t rows, int64_t K, int box_rows,
                              int64_t batch = 1, size_t item_bytes = 0)
 {
-    if (!g_encode_tiled) {
-        void *fn = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-        if (q != cudaDriverEntryPointSuccess || !fn) {
-            snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled not available");
-            return MX_ERR_CUDA;
-        }
-        g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
+    {
+        const mx_status_t es = ensure_encoder();
+        if (es != MX_OK) return es;
     }
     // A map depends only on these seven numbers; a layer called again with the same workspace finds
     // its maps here instead of paying a driver call each (a few microseconds per product for small layers).
@@ -325,6 +347,7 @@ struct TcBatch {                 // several products of one shape in one launch 
     int64_t count = 1;
     size_t a_item = 0, w_item = 0;   // bytes between the items' bf16 operands
     int64_t y_batch = 0;             // floats between the items' outputs
+    bool no_events = false;          // never bracket the launch with profile events (mx_gemm_static)
 };
 
 struct PackedW {                 // weight operand of the fused kernels (unused for W_BF16)
@@ -375,11 +398,8 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         if (s != MX_OK) return s;
     }
     constexpr int slot = BN == 256 ? 0 : 1;
-    if (!d.tc_attr_set[slot][WMODE]) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN, WMODE>,
-                                     cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES));
-        d.tc_attr_set[slot][WMODE] = true;
-    }
+    s = smem_attr_once(d.tc_attr_set[slot][WMODE], mx::gemm_tc_kernel<BN, WMODE>, (int)Cfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
     mx::TcParams p;
     p.y = y;
     p.bias = bias;
@@ -407,6 +427,11 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     const int tiles = (int)tiles64;
     const int grid = tiles < d.sm_count ? tiles : d.sm_count;
     const int threads = mx::tc_threads(BN, WMODE);
+    if (tb.no_events) {
+        mx::gemm_tc_kernel<BN, WMODE><<<grid, threads, Cfg::SMEM_BYTES, st>>>(tm_a, tm_w, tm_y, p);
+        MX_CUDA(cudaGetLastError());
+        return MX_OK;
+    }
     ProfScope prof(KIND_GEMM_TC, st);
     MX_CUDA(launch_dep(mx::gemm_tc_kernel<BN, WMODE>, dim3(grid), dim3(threads), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
@@ -429,10 +454,8 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
     }
-    if (!d.tc2_attr_set) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)Cfg::SMEM_BYTES));
-        d.tc2_attr_set = true;
-    }
+    s = smem_attr_once(d.tc2_attr_set, mx::gemm_tc2_kernel, (int)Cfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
     mx::TcParams p{};
     p.y = y;
     p.bias = bias;
@@ -565,13 +588,8 @@ mx_status_t packed_weight_maps(const void *w_mant, const void *w_exp, int64_t N,
     const auto key = std::make_tuple(w_mant, w_exp, N, K);
     auto it = g_wmap_cache.find(key);
     if (it == g_wmap_cache.end()) {
-        if (!g_encode_tiled) {
-            void *fn = nullptr;
-            cudaDriverEntryPointQueryResult q;
-            MX_CUDA(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q));
-            if (q != cudaDriverEntryPointSuccess || !fn) return MX_ERR_CUDA;
-            g_encode_tiled = reinterpret_cast<EncodeTiledFn>(fn);
-        }
+        const mx_status_t es = ensure_encoder();
+        if (es != MX_OK) return es;
         WeightMaps wm;
         mx_status_t s = encode_u8_rows(&wm.mant, w_mant, N, K / 2, 128, CU_TENSOR_MAP_SWIZZLE_128B);
         if (s != MX_OK) return s;
@@ -611,12 +629,9 @@ bool same_activation(const mx_linear_args_t &a, const mx_linear_args_t &b)
 template <int NT, bool BULK>
 mx_status_t launch_stream(const mx::StreamParams &sp, size_t smem, int grid, DeviceInfo &d, cudaStream_t st)
 {
-    bool &done = d.stream_attr_set[(NT - 1) * 2 + (BULK ? 1 : 0)];
-    if (!done) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemv_stream_kernel<NT, BULK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     227 * 1024));
-        done = true;
-    }
+    const mx_status_t as = smem_attr_once(d.stream_attr_set[(NT - 1) * 2 + (BULK ? 1 : 0)],
+                                          mx::gemv_stream_kernel<NT, BULK>, 227 * 1024);
+    if (as != MX_OK) return as;
     ProfScope prof(KIND_GEMM_STREAM, st);
     MX_CUDA(launch_dep(mx::gemv_stream_kernel<NT, BULK>, dim3(grid), dim3(mx::StreamCfg<NT, BULK>::THREADS), smem, st, sp));
     MX_CUDA(cudaGetLastError());
@@ -1378,10 +1393,13 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     if (s != MX_OK) return s;
     int dev = 0;
     MX_CUDA(cudaGetDevice(&dev));
-    if (!g_static_scratch_addr[dev]) {              // set-up: first call on this device
-        void *p = nullptr;
-        MX_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
-        g_static_scratch_addr[dev] = p;
+    {
+        std::lock_guard<std::mutex> lk(g_init_mu);
+        if (!g_static_scratch_addr[dev]) {          // set-up: first call on this device
+            void *p = nullptr;
+            MX_CUDA(cudaGetSymbolAddress(&p, g_static_scratch));
+            g_static_scratch_addr[dev] = p;
+        }
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint8_t *scratch = static_cast<uint8_t *>(g_static_scratch_addr[dev]);
@@ -1396,45 +1414,9 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     mx::dequantize_kernel<__nv_bfloat16><<<grid_for(N * (K / 8), 256, d->sm_count, 16), 256, 0, st>>>(
         static_cast<const uint8_t *>(w_mant), w_exp, N, K, fw.block, fw.elem_bits, w_hat, K, dense_strides(K, fw));
     MX_CUDA(cudaGetLastError());
-    constexpr int BN = 128;
-    using Cfg = mx::TcCfg<BN>;
-    CUtensorMap tm_a, tm_w;
-    s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
-    if (s != MX_OK) return s;
-    s = encode_bf16_rows(&tm_w, w_hat, N, K, BN);
-    if (s != MX_OK) return s;
-    if (!d->tc_attr_set[1][mx::W_BF16]) {
-        MX_CUDA(cudaFuncSetAttribute(mx::gemm_tc_kernel<BN, mx::W_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Cfg::SMEM_BYTES));
-        d->tc_attr_set[1][mx::W_BF16] = true;
-    }
-    mx::TcParams p;
-    p.y = y;
-    p.bias = bias;
-    p.ldy = ldy;
-    p.M = (int)M;
-    p.N = (int)N;
-    p.K = (int)K;
-    p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
-    p.tiles_n = (int)((N + BN - 1) / BN);
-    p.status = d->status;
-    p.tma_store = 0;
-    p.w_mant = nullptr;
-    p.w_exp = nullptr;
-    p.w_bits = 0;
-    p.block = 0;
-    p.yq_mant = nullptr;
-    p.yq_exp = nullptr;
-    p.yq_nonfinite = nullptr;
-    p.yq_bits = 0;
-    p.yq_block = 0;
-    p.batch = 1;
-    p.y_batch = 0;
-    const int tiles = p.tiles_m * p.tiles_n;
-    mx::gemm_tc_kernel<BN, mx::W_BF16><<<tiles < d->sm_count ? tiles : d->sm_count, mx::TC_THREADS, Cfg::SMEM_BYTES, st>>>(
-        tm_a, tm_w, tm_a, p);
-    MX_CUDA(cudaGetLastError());
-    return MX_OK;
+    TcBatch opt;
+    opt.no_events = true;
+    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, PackedW(), M, N, K, bias, y, ldy, nullptr, *d, st, opt);
 }
 
 mx_status_t mx_profile_begin(void)

@@ -1,0 +1,158 @@
+"""Full-size parity of the decoder block (Fig. 1(d)) at OPT-6.7B shapes -- hidden 4096, 32 heads of
+128, FFN 16384, sequence 2048 -- in the launch configuration bench.py times, and of the batched
+tensor-core kernel when every CTA walks several tiles of several batch items.
+
+A block cannot be compared end to end with a CPU run (quantization is discontinuous), so every
+stage of ONE GPU run is checked against the oracle applied to the GPU's own input of that stage:
+MXInt products on sampled outputs within 1e-5 * S, the transposing quantizer bit for bit on sampled
+rows, the fp32 glue within a few fp32 ulps."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import block_oracle as blk
+from oracle import mx_oracle as orc
+from paper_2307_15517_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def mods():
+    from paper_2307_15517_b200 import binding, decoder_block
+    return binding, decoder_block
+
+
+def _close(got, ref, S, what):
+    err = np.abs(np.asarray(got, np.float64) - np.asarray(ref, np.float64))
+    assert (err <= TOL * S + 1e-30).all(), "%s: max |d|/S = %.3e" % (what, float((err / np.maximum(S, 1e-300)).max()))
+
+
+@pytest.mark.parametrize("case", [
+    # batch, M, N, K, B, w : tiles per launch
+    (80, 384, 512, 64, 16, 8),      # 480 tiles of 128x256 over 148 CTAs: three to four tiles of different items per CTA
+    (100, 300, 100, 96, 32, 8),     # 300 tiles of 128x128, ragged M and N, K tail
+    (40, 130, 260, 256, 16, 4),     # nibble operands, 4 K steps, 160 tiles
+])
+def test_batched_product_many_tiles_per_cta(mods, case):
+    """Every output of every item against the oracle: the persistent loop with more than one tile
+    per CTA and more than one batch item (item-major tile numbering, rank-3 tensor maps)."""
+    mxb, _ = mods
+    batch, M, N, K, B, w = case
+    qmax = 2 ** (w - 1) - 1
+    qa = synth.random_ints((M, batch * K), -qmax, qmax, 900 + batch).numpy()
+    qw = synth.random_ints((N, batch * K), -qmax, qmax, 901 + batch).numpy()
+    ea = synth.random_bytes((M, batch * K // B), 124, 130, 902 + batch).numpy()
+    ew = synth.random_bytes((N, batch * K // B), 120, 126, 903 + batch).numpy()
+    f = mxb.MxFormat(B, w)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    y = torch.full((batch * M, N), 5.0, device="cuda")
+    mxb.mx_gemm_batched(dev(orc.pack(qa, w)), dev(ea), f, batch * K, K, dev(orc.pack(qw, w)), dev(ew), f,
+                        batch * K, K, M, N, K, batch, y, N, M * N)
+    assert mxb.mx_poll_status() == 0
+    got = y.cpu().numpy()
+    nb = K // B
+    for b in range(batch):
+        y_ref, _, S = orc.gemm(qa[:, b * K:(b + 1) * K], ea[:, b * nb:(b + 1) * nb], w,
+                               qw[:, b * K:(b + 1) * K], ew[:, b * nb:(b + 1) * nb], w, B)
+        _close(got[b * M:(b + 1) * M], y_ref, S, "item %d" % b)
+
+
+def _sampled_linear(rng, x_gpu_np, w_cpu, bias, B, wa, ww, got, what, n=768):
+    """got[i, j] against the oracle's product of the quantized rows of x (the GPU's own stage input)
+    and the quantized weights, at n random positions."""
+    qa, ea, _ = orc.quantize(np.ascontiguousarray(x_gpu_np, np.float32), B, wa)
+    qw, ew, _ = orc.quantize(w_cpu, B, ww)
+    M, N = got.shape
+    si, sj = rng.integers(0, M, n), rng.integers(0, N, n)
+    y_ref, _, S = orc.gemm_samples(qa, ea, wa, qw, ew, ww, B, si, sj, bias=bias)
+    _close(got[si, sj], y_ref, S, what)
+
+
+def test_decoder_block_opt67b_shapes_stage_by_stage(mods):
+    mxb, db = mods
+    sh = synth.decoder_block_shapes()
+    cfg = db.BlockConfig(hidden=sh["hidden"], heads=sh["heads"], head_dim=sh["head_dim"], ffn=sh["ffn"],
+                         block=sh["block"], w_act=sh["w_act"], w_wgt=sh["w_wgt"])
+    seq, hid, ffn, H, d = sh["seq"], cfg.hidden, cfg.ffn, cfg.heads, cfg.head_dim
+    B, wa, ww = cfg.block, cfg.w_act, cfg.w_wgt
+    assert (hid, H, d, ffn, seq) == (4096, 32, 128, 16384, 2048)
+    rng = np.random.default_rng(67)
+    g = torch.Generator().manual_seed(67)
+    x = synth.outlier_activations(seq, hid, 4, -(-hid * 5 // 1000), 40.0)
+    W = {n: synth.gaussian_weights(o, i, 670 + j) for j, (n, o, i) in enumerate(
+        [("wq", hid, hid), ("wk", hid, hid), ("wv", hid, hid), ("wo", hid, hid), ("w1", ffn, hid), ("w2", hid, ffn)])}
+    P = {n: torch.randn(sz, generator=g) * 0.02 for n, sz in
+         [("bq", hid), ("bk", hid), ("bv", hid), ("bo", hid), ("b1", ffn), ("b2", hid), ("ln1_b", hid), ("ln2_b", hid)]}
+    P["ln1_g"] = 1 + 0.1 * torch.randn(hid, generator=g)
+    P["ln2_g"] = 1 + 0.1 * torch.randn(hid, generator=g)
+    qw = db.quantize_weights(cfg, {k: v.cuda() for k, v in W.items()})
+    keep = {}
+    out = db.run(cfg, x.cuda(), qw, {k: v.cuda() for k, v in P.items()}, keep=keep)
+    assert mxb.mx_poll_status() == 0
+    p = {k: v.numpy() for k, v in P.items()}
+    T = lambda name: keep[name].cpu().numpy()
+
+    # ---- fp32 glue on sampled rows -------------------------------------------------------------
+    rows = rng.choice(seq, 48, replace=False)
+    ln1 = T("ln1")
+    assert np.allclose(ln1[rows], blk.layernorm(x.numpy()[rows], p["ln1_g"], p["ln1_b"], cfg.eps), rtol=1e-5, atol=1e-5)
+
+    # ---- q, k, v: one 12288-wide layer call on row-concatenated weights ---------------------------
+    for name, wn, bn in (("q", "wq", "bq"), ("k", "wk", "bk"), ("v", "wv", "bv")):
+        _sampled_linear(rng, ln1, W[wn].numpy(), p[bn], B, wa, ww, T(name), name)
+    q, k, v = T("q"), T("k"), T("v")
+
+    # ---- scores: all 32 heads, 64 sampled outputs each (batched kernel, 4096 tiles) ---------------
+    scores = T("scores")
+    for h in range(H):
+        qa, ea, _ = orc.quantize(np.ascontiguousarray(q[:, h * d:(h + 1) * d]), B, wa)
+        qk, ek, _ = orc.quantize(np.ascontiguousarray(k[:, h * d:(h + 1) * d]), B, wa)
+        si, sj = rng.integers(0, seq, 64), rng.integers(0, seq, 64)
+        y_ref, _, S = orc.gemm_samples(qa, ea, wa, qk, ek, wa, B, si, sj)
+        _close(scores[h * seq + si, sj], y_ref, S, "scores head %d" % h)
+
+    # ---- causal softmax: three whole heads --------------------------------------------------------
+    probs = T("probs")
+    for h in (0, 13, H - 1):
+        want = blk.softmax_causal(scores[h * seq:(h + 1) * seq], 1 / math.sqrt(d), seq)
+        got = probs[h * seq:(h + 1) * seq]
+        assert np.allclose(got, want, rtol=1e-5, atol=1e-7), "softmax head %d" % h
+        assert (got[want == 0] == 0).all()
+
+    # ---- V quantized along the token axis (transposing quantizer at 4096 x 2048): sampled rows ----
+    fa = mxb.MxFormat(B, wa)
+    vm, ve = mxb.mx_quantize(keep["v"].t(), fa)
+    vrows = rng.choice(hid, 64, replace=False)
+    qv, ev, _ = orc.quantize(np.ascontiguousarray(v.T[vrows]), B, wa)
+    assert np.array_equal(vm.cpu().numpy()[vrows], orc.pack(qv, wa))
+    assert np.array_equal(ve.cpu().numpy()[vrows], ev)
+
+    # ---- context: per head 16 rows of P against all 128 columns of V ------------------------------
+    ctx = T("ctx")
+    for h in range(H):
+        prow = rng.choice(seq, 16, replace=False)
+        qa, ea, _ = orc.quantize(np.ascontiguousarray(probs[h * seq + prow]), B, wa)
+        qv, ev, _ = orc.quantize(np.ascontiguousarray(v[:, h * d:(h + 1) * d].T), B, wa)
+        y_ref, _, S = orc.gemm(qa, ea, wa, qv, ev, wa, B)
+        _close(ctx[prow][:, h * d:(h + 1) * d], y_ref, S, "ctx head %d" % h)
+
+    # ---- out projection, residual, second LayerNorm, FFN ------------------------------------------
+    attn_out = T("attn_out")
+    _sampled_linear(rng, ctx, W["wo"].numpy(), p["bo"], B, wa, ww, attn_out, "attn_out")
+    x1 = T("x1")
+    assert np.array_equal(x1, attn_out + x.numpy())
+    ln2 = T("ln2")
+    assert np.allclose(ln2[rows], blk.layernorm(x1[rows], p["ln2_g"], p["ln2_b"], cfg.eps), rtol=1e-5, atol=1e-5)
+    ffn_pre = T("ffn_pre")
+    _sampled_linear(rng, ln2, W["w1"].numpy(), p["b1"], B, wa, ww, ffn_pre, "ffn_pre")
+    ffn_act = T("ffn_act")
+    assert np.array_equal(ffn_act, np.maximum(ffn_pre, 0))
+    ffn_out = T("ffn_out")
+    _sampled_linear(rng, ffn_act, W["w2"].numpy(), p["b2"], B, wa, ww, ffn_out, "ffn_out")
+    res = out.cpu().numpy()
+    assert np.array_equal(res, ffn_out + x1)
+    assert np.isfinite(res).all()

@@ -130,6 +130,78 @@ __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, in
     }
 }
 
+// fp32 epilogue of one lane: r holds 32 consecutive outputs (columns n .. n + 31) of row `row`; the
+// warp's 32 rows start at `rows0`.  Adds the bias and writes the 32 x 32 block either through one of
+// the warp's two 4 KB shared-memory buffers (`warp_bufs`, 128-byte swizzled box layout) and a tiled
+// TMA store -- whole 128-byte lines reach L2, rows >= M and columns >= N are clipped by the store --
+// or, when ldy % 4 != 0, with plain stores.  `epi_buf` counts the warp's TMA blocks (buffer parity).
+// Shared by the one-CTA, the CTA-pair and the chunked kernel.
+__device__ __forceinline__ void store_f32_chunk(const TcParams &p, const CUtensorMap *tmap_y, uint32_t (&r)[32], int row,
+                                                int rows0, int n, int tb, uint32_t warp_bufs, uint32_t &epi_buf, int lane)
+{
+    if (p.tma_store) {
+        if (n < p.N && rows0 < p.M) {                      // warp-uniform
+            const uint32_t buf = warp_bufs + (epi_buf & 1u) * 4096u;
+            if (lane == 0) ptx::bulk_wait_group_read<1>();   // the buffer used two blocks ago is free
+            __syncwarp();
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                float4 o;
+                o.x = __uint_as_float(r[4 * v + 0]);
+                o.y = __uint_as_float(r[4 * v + 1]);
+                o.z = __uint_as_float(r[4 * v + 2]);
+                o.w = __uint_as_float(r[4 * v + 3]);
+                if (p.bias) {
+                    const int c = n + 4 * v;
+                    if (c + 4 <= p.N) {
+                        const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + c));
+                        o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                    } else {
+                        if (c + 0 < p.N) o.x += __ldg(p.bias + c + 0);
+                        if (c + 1 < p.N) o.y += __ldg(p.bias + c + 1);
+                        if (c + 2 < p.N) o.z += __ldg(p.bias + c + 2);
+                    }
+                }
+                const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
+                asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y),
+                             "f"(o.z), "f"(o.w)
+                             : "memory");
+            }
+            ptx::fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0) {
+                if (p.batch > 1) ptx::tma_store_3d(tmap_y, n, rows0, tb, buf);
+                else ptx::tma_store_2d(tmap_y, n, rows0, buf);
+                ptx::bulk_commit_group();
+            }
+            ++epi_buf;
+        }
+    } else if (row < p.M && n < p.N) {
+        float *yrow = p.y + (int64_t)tb * p.y_batch + (int64_t)row * p.ldy;
+        const bool vec_ok = ((p.ldy & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0) && ((p.y_batch & 3) == 0);
+        if (vec_ok && n + 32 <= p.N) {
+#pragma unroll
+            for (int v = 0; v < 8; ++v) {
+                float4 o;
+                o.x = __uint_as_float(r[4 * v + 0]);
+                o.y = __uint_as_float(r[4 * v + 1]);
+                o.z = __uint_as_float(r[4 * v + 2]);
+                o.w = __uint_as_float(r[4 * v + 3]);
+                if (p.bias) {
+                    const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + n) + v);
+                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
+                }
+                reinterpret_cast<float4 *>(yrow + n)[v] = o;
+            }
+        } else {
+#pragma unroll
+            for (int v = 0; v < 32; ++v)
+                if (n + v < p.N)
+                    yrow[n + v] = p.bias ? __uint_as_float(r[v]) + __ldg(p.bias + n + v) : __uint_as_float(r[v]);
+        }
+    }
+}
+
 // Raw bytes of one (row, half K-step) item: 32 mantissas and their exponent bytes.
 template <int WMODE> struct RawItem {
     uint4 m[WMODE == W_INT8 ? 2 : 1];
@@ -500,8 +572,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             ptx::tc_fence_after_sync();
             const int row = m0 + quad * 32 + lane;
-            float *yrow = p.y + (int64_t)tb * p.y_batch + (int64_t)row * p.ldy;
-            const bool vec_ok = ((p.ldy & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
@@ -512,69 +582,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     store_mxint_chunk(p, row, n, r);
                     continue;
                 }
-                if (p.tma_store) {
-                    // Stage the 32x32 block in shared memory in the 128-byte swizzled box layout and let
-                    // one lane hand it to a tiled TMA store: full 128-byte lines reach L2, the store
-                    // clips rows >= M and columns >= N by itself.
-                    if (n < p.N && m0 + quad * 32 < p.M) {          // warp-uniform
-                        const uint32_t buf = epi_base + (uint32_t)((warp - 2) * 2 + (epi_buf & 1)) * 4096u;
-                        if (lane == 0) ptx::bulk_wait_group_read<1>();   // the buffer used two blocks ago is free
-                        __syncwarp();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o;
-                            o.x = __uint_as_float(r[4 * v + 0]);
-                            o.y = __uint_as_float(r[4 * v + 1]);
-                            o.z = __uint_as_float(r[4 * v + 2]);
-                            o.w = __uint_as_float(r[4 * v + 3]);
-                            if (p.bias) {
-                                const int c = n + 4 * v;
-                                if (c + 4 <= p.N) {
-                                    const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + c));
-                                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
-                                } else {
-                                    if (c + 0 < p.N) o.x += __ldg(p.bias + c + 0);
-                                    if (c + 1 < p.N) o.y += __ldg(p.bias + c + 1);
-                                    if (c + 2 < p.N) o.z += __ldg(p.bias + c + 2);
-                                }
-                            }
-                            const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
-                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y),
-                                         "f"(o.z), "f"(o.w)
-                                         : "memory");
-                        }
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            if (p.batch > 1) ptx::tma_store_3d(&tmap_y, n, m0 + quad * 32, tb, buf);
-                            else ptx::tma_store_2d(&tmap_y, n, m0 + quad * 32, buf);
-                            ptx::bulk_commit_group();
-                        }
-                        ++epi_buf;
-                    }
-                } else if (row < p.M && n < p.N) {
-                    if (vec_ok && n + 32 <= p.N) {
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o;
-                            o.x = __uint_as_float(r[4 * v + 0]);
-                            o.y = __uint_as_float(r[4 * v + 1]);
-                            o.z = __uint_as_float(r[4 * v + 2]);
-                            o.w = __uint_as_float(r[4 * v + 3]);
-                            if (p.bias) {
-                                const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + n) + v);
-                                o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
-                            }
-                            reinterpret_cast<float4 *>(yrow + n)[v] = o;
-                        }
-                    } else {
-#pragma unroll
-                        for (int v = 0; v < 32; ++v)
-                            if (n + v < p.N)
-                                yrow[n + v] = p.bias ? __uint_as_float(r[v]) + __ldg(p.bias + n + v)
-                                                     : __uint_as_float(r[v]);
-                    }
-                }
+                store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

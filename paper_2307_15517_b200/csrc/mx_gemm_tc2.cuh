@@ -164,8 +164,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             }
             ptx::tc_fence_after_sync();
             const int row = m0 + quad * 32 + lane;
-            float *yrow = p.y + (int64_t)row * p.ldy;
-            const bool vec_ok = ((p.ldy & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.y) & 15) == 0);
 #pragma unroll 1
             for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
@@ -176,65 +174,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                     store_mxint_chunk(p, row, n, r);
                     continue;
                 }
-                if (p.tma_store) {
-                    if (n < p.N && m0 + quad * 32 < p.M) {          // warp-uniform
-                        const uint32_t buf = epi_base + (uint32_t)((warp - 2) * 2 + (epi_buf & 1)) * 4096u;
-                        if (lane == 0) ptx::bulk_wait_group_read<1>();
-                        __syncwarp();
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o;
-                            o.x = __uint_as_float(r[4 * v + 0]);
-                            o.y = __uint_as_float(r[4 * v + 1]);
-                            o.z = __uint_as_float(r[4 * v + 2]);
-                            o.w = __uint_as_float(r[4 * v + 3]);
-                            if (p.bias) {
-                                const int c = n + 4 * v;
-                                if (c + 4 <= p.N) {
-                                    const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + c));
-                                    o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
-                                } else {
-                                    if (c + 0 < p.N) o.x += __ldg(p.bias + c + 0);
-                                    if (c + 1 < p.N) o.y += __ldg(p.bias + c + 1);
-                                    if (c + 2 < p.N) o.z += __ldg(p.bias + c + 2);
-                                }
-                            }
-                            const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((v ^ (lane & 7)) << 4);
-                            asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "f"(o.x), "f"(o.y),
-                                         "f"(o.z), "f"(o.w)
-                                         : "memory");
-                        }
-                        ptx::fence_proxy_async_smem();
-                        __syncwarp();
-                        if (lane == 0) {
-                            ptx::tma_store_2d(&tmap_y, n, m0 + quad * 32, buf);
-                            ptx::bulk_commit_group();
-                        }
-                        ++epi_buf;
-                    }
-                } else if (row < p.M && n < p.N) {
-                    if (vec_ok && n + 32 <= p.N) {
-#pragma unroll
-                        for (int v = 0; v < 8; ++v) {
-                            float4 o;
-                            o.x = __uint_as_float(r[4 * v + 0]);
-                            o.y = __uint_as_float(r[4 * v + 1]);
-                            o.z = __uint_as_float(r[4 * v + 2]);
-                            o.w = __uint_as_float(r[4 * v + 3]);
-                            if (p.bias) {
-                                const float4 b = __ldg(reinterpret_cast<const float4 *>(p.bias + n) + v);
-                                o.x += b.x; o.y += b.y; o.z += b.z; o.w += b.w;
-                            }
-                            reinterpret_cast<float4 *>(yrow + n)[v] = o;
-                        }
-                    } else {
-#pragma unroll
-                        for (int v = 0; v < 32; ++v)
-                            if (n + v < p.N)
-                                yrow[n + v] = p.bias ? __uint_as_float(r[v]) + __ldg(p.bias + n + v)
-                                                     : __uint_as_float(r[v]);
-                    }
-                }
+                store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, 0, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -16,6 +16,7 @@
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
 #include "mx_gemm_tc2.cuh"
+#include "mx_gemm_tcx.cuh"
 #include "mx_gemv_stream.cuh"
 #include "mx_glue.cuh"
 #include "mx_quantize.cuh"
@@ -37,6 +38,7 @@ struct DeviceInfo {
     bool tc_attr_set[2][4] = {{false, false, false, false}, {false, false, false, false}};
     bool stream_attr_set[4] = {false, false, false, false};
     bool tc2_attr_set = false;
+    bool tcx_attr_set = false;
 };
 DeviceInfo g_dev[MAX_DEVICES];
 std::mutex g_init_mu;        // guards every lazily initialised field above and below (calls may come from several host threads)
@@ -481,6 +483,45 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     return MX_OK;
 }
 
+// The chunked kernel (two-level accumulation): 128 x 128 tiles, fp32 result, one product per launch.
+mx_status_t launch_tcx(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N, int64_t K,
+                       const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+{
+    using Cfg = mx::TcxCfg;
+    CUtensorMap tm_a, tm_w;
+    mx_status_t s = encode_bf16_rows(&tm_a, a_hat, M, K, mx::TC_BM);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_w, w_hat, N, K, Cfg::BN);
+    if (s != MX_OK) return s;
+    CUtensorMap tm_y = tm_a;
+    const bool tma_store = (ldy % 4) == 0;
+    if (tma_store) {
+        s = encode_f32_out(&tm_y, y, M, N, ldy);
+        if (s != MX_OK) return s;
+    }
+    s = smem_attr_once(d.tcx_attr_set, mx::gemm_tcx_kernel, (int)Cfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
+    mx::TcParams p{};
+    p.y = y;
+    p.bias = bias;
+    p.ldy = ldy;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.tiles_m = (int)((M + mx::TC_BM - 1) / mx::TC_BM);
+    p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
+    p.status = d.status;
+    p.tma_store = tma_store ? 1 : 0;
+    p.batch = 1;
+    const int64_t tiles64 = (int64_t)p.tiles_m * p.tiles_n;
+    if (tiles64 > INT32_MAX / 2) return MX_ERR_SHAPE;
+    const int grid = tiles64 < d.sm_count ? (int)tiles64 : d.sm_count;
+    ProfScope prof(KIND_GEMM_TC, st);
+    MX_CUDA(launch_dep(mx::gemm_tcx_kernel, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
 {
     const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256);
@@ -728,7 +769,8 @@ size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx
         const size_t tc = tc_workspace(M, N, K);
         return st > tc ? st : tc;
     }
-    case MX_ALGO_TCGEN05: return tc_workspace(M, N, K);
+    case MX_ALGO_TCGEN05:
+    case MX_ALGO_TCGEN05_CHUNKED: return tc_workspace(M, N, K);
     case MX_ALGO_TCGEN05_FUSED: return (K % 32) == 0 ? fused_workspace(M, K) : tc_workspace(M, N, K);
     default: return 0;
     }
@@ -866,7 +908,8 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         if (algo == MX_ALGO_AUTO) algo = can_stream ? MX_ALGO_STREAM : MX_ALGO_TCGEN05;
         if (algo == MX_ALGO_STREAM) return grouped_impl(&one, 1, &a_exp, workspace, workspace_bytes, stream);
     }
-    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
+        algo != MX_ALGO_TCGEN05_CHUNKED)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -895,6 +938,7 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
                                                              round256((size_t)M * K * 2));
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
+    if (algo == MX_ALGO_TCGEN05_CHUNKED) return launch_tcx(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }
 
@@ -924,7 +968,8 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         algo = (stream_layer_ok(one) && (reinterpret_cast<uintptr_t>(w_exp) & 3u) == 0) ? MX_ALGO_STREAM
                                                                                      : MX_ALGO_TCGEN05;
     if (algo == MX_ALGO_STREAM) return mx_linear_grouped(&one, 1, workspace, workspace_bytes, stream);
-    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05)
+    if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
+        algo != MX_ALGO_TCGEN05_CHUNKED)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -961,6 +1006,7 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     s = tc_prepare(one, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
+    if (algo == MX_ALGO_TCGEN05_CHUNKED) return launch_tcx(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }
 

@@ -187,11 +187,12 @@ def test_gemm_simt_matches_sequential_oracle_exactly(mxb, shape):
 
 
 TC_ALGOS = ("MX_ALGO_TCGEN05", "MX_ALGO_TCGEN05_FUSED")
+TC_ALGOS_ALL = TC_ALGOS + ("MX_ALGO_TCGEN05_CHUNKED",)
 
 
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
 @pytest.mark.parametrize("with_bias", (False, True))
-@pytest.mark.parametrize("algo", TC_ALGOS)
+@pytest.mark.parametrize("algo", TC_ALGOS_ALL)
 def test_gemm_tensor_core_within_tolerance(mxb, shape, with_bias, algo):
     """Block exponents spread over 2^+-3 per operand (2^+-6 per product term), wider than any of
     the paper-shaped workloads produce within one row."""
@@ -229,7 +230,68 @@ def test_gemm_tensor_core_adversarial_exponent_spread(mxb):
     _check_tol(y, y_ref, S)
 
 
-@pytest.mark.parametrize("algo", TC_ALGOS)
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+def test_gemm_chunked_accumulation_meets_tolerance_on_any_exponent_spread(mxb, shape):
+    """Block exponents drawn uniformly over 2^+-8 per operand (terms 2^+-16 apart), where the
+    single-accumulator kernels only meet their derived bound: with the accumulator drained every K
+    step and the partial sums added in fp32 registers, the stated 1e-5 * S holds on every shape."""
+    M, N, K, B, wa, ww = shape
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=31 * M + N, spread=8)
+    bias = np.random.default_rng(3).standard_normal(N).astype(np.float32) if (M + N) % 2 else None
+    y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
+    ypad = torch.full((M, N + 8), -77.0, device="cuda")
+    y = mxb.mx_gemm(_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)),
+                    _dev(ew), mxb.MxFormat(B, ww), M, N, K, bias=None if bias is None else _dev(bias),
+                    y=ypad[:, :N], algo=mxb.MX_ALGO_TCGEN05_CHUNKED)
+    assert mxb.mx_poll_status() == 0
+    _check_tol(y, y_ref, S)
+    assert (ypad[:, N:] == -77.0).all()
+
+
+@pytest.mark.parametrize("K", (11008, 16384))
+def test_gemm_long_reductions_with_wide_exponent_spread(mxb, K):
+    """The longest reductions of the paper-shaped workloads (LLaMA-7B down projection, OPT-6.7B FFN)
+    with the adversarial +-8 exponent spread: the chunked kernel inside 1e-5 * S, the default kernel
+    inside its derived bound ceil(K/16) * 17 * 2^-23 * S (asserted at these K, not only at K = 320)."""
+    M, N, B, wa, ww = 160, 200, 16, 8, 4
+    qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=K, spread=8)
+    y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
+    args = (_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)), _dev(ew),
+            mxb.MxFormat(B, ww), M, N, K)
+    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05_CHUNKED)
+    assert mxb.mx_poll_status() == 0
+    _check_tol(y, y_ref, S)
+    worst_chunked = float((np.abs(y.cpu().numpy().astype(np.float64) - y_ref) / S).max())
+    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05).cpu().numpy().astype(np.float64)
+    assert mxb.mx_poll_status() == 0
+    assert (np.abs(y - y_ref) <= -(-K // 16) * 17 * 2.0 ** -23 * S).all()
+    worst_default = float((np.abs(y - y_ref) / S).max())
+    print("K=%d spread +-8: max |dY|/S chunked %.2e, single accumulator %.2e" % (K, worst_chunked, worst_default))
+    assert worst_chunked <= 1e-5
+
+
+def test_linear_student_t_full_reduction_length_default_kernel(mxb):
+    """Heavy-tailed (Student-t, nu = 3) activations over the full K = 11008 of the LLaMA-7B down
+    projection through mx_linear with the default kernel: every output (not a sample) inside
+    1e-5 * S, and the measured worst ratio is reported."""
+    M, N, K, B, wa, ww = 256, 384, 11008, 16, 8, 4
+    x = synth.student_t_activations(M, K, 5)
+    w = synth.gaussian_weights(N, K, 6)
+    qa, ea, _ = orc.quantize(x.numpy(), B, wa)
+    qw, ew, _ = orc.quantize(w.numpy(), B, ww)
+    y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
+    fw = mxb.MxFormat(B, ww)
+    wm, we = mxb.mx_quantize(w.cuda(), fw)
+    worst = {}
+    for name in ("MX_ALGO_AUTO", "MX_ALGO_TCGEN05_CHUNKED"):
+        y = mxb.mx_linear(x.cuda(), mxb.MxFormat(B, wa), wm, we, fw, N, algo=getattr(mxb, name))
+        assert mxb.mx_poll_status() == 0
+        _check_tol(y, y_ref, S)
+        worst[name] = float((np.abs(y.cpu().numpy().astype(np.float64) - y_ref) / np.maximum(S, 1e-300)).max())
+    print("Student-t K=11008: max |dY|/S", worst)
+
+
+@pytest.mark.parametrize("algo", TC_ALGOS_ALL)
 @pytest.mark.parametrize("ww,B", [(4, 16), (4, 32), (3, 16), (8, 16), (6, 32)])
 def test_gemm_one_hot_rows_expose_the_operand_layout(mxb, algo, ww, B):
     """A = identity-like rows: Y must be the decoded weights, element for element (catches any

@@ -502,6 +502,14 @@ cast_rows_kernel(const uint8_t *__restrict__ mant_in, const uint8_t *__restrict_
     }
 }
 
+// Zeroes `n` words (the progress counters of the product kernel that prepares its own operands).
+__global__ void __launch_bounds__(1024) clear_words_kernel(uint32_t *__restrict__ words, int n)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) words[i] = 0u;
+}
+
 // Several tensors in one launch (the distinct activation tensors of a grouped decode call):
 // blockIdx.y selects the tensor, blockIdx.x strides over its rows.
 struct QuantJob {
@@ -693,6 +701,57 @@ dequantize_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__ 
 }
 
 
+// 32 consecutive elements of a row (one 16-byte word of nibbles, or two of int8) and their exponent
+// byte(s) `e` (block 16: low byte = first half, next byte = second half; block 32: one byte) ->
+// 32 exact bf16 values, o[j] = elements 8j .. 8j + 7.
+template <bool NIBBLE>
+__device__ __forceinline__ void decode32(const uint4 (&m)[NIBBLE ? 1 : 2], uint32_t e, bool b16, int w, uint32_t (&o)[4][4])
+{
+    const int e0 = (int)(e & 0xFF), e1 = b16 ? (int)((e >> 8) & 0xFF) : e0;
+    const uint32_t w8[8] = {m[0].x, m[0].y, m[0].z, m[0].w,
+                            m[NIBBLE ? 0 : 1].x, m[NIBBLE ? 0 : 1].y, m[NIBBLE ? 0 : 1].z, m[NIBBLE ? 0 : 1].w};
+    if (NIBBLE) {
+        if (nibble_fast_ok(e0, w) && nibble_fast_ok(e1, w)) {
+            const __nv_bfloat162 m136 = as_bf162(0xC308C308u);       // -136
+            const __nv_bfloat162 s0 = as_bf162(bf16x2_scale_bits(e0, w));
+            const __nv_bfloat162 s1 = as_bf162(bf16x2_scale_bits(e1, w));
+            const __nv_bfloat162 c0 = __hmul2(s0, m136), c1 = __hmul2(s1, m136);
+            decode8_nibbles(w8[0], s0, c0, o[0]);
+            decode8_nibbles(w8[1], s0, c0, o[1]);
+            decode8_nibbles(w8[2], s1, c1, o[2]);
+            decode8_nibbles(w8[3], s1, c1, o[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int q[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) q[i] = ((int)(w8[j] << (28 - 4 * i))) >> 28;
+                decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
+            }
+        }
+    } else {
+        if (byte_fast_ok(e0, w) && byte_fast_ok(e1, w)) {
+            const float s0 = f32_scale(e0, w), s1 = f32_scale(e1, w);
+            const float c0 = -8388736.0f * s0, c1 = -8388736.0f * s1;   // -(2^23+128)*s, exact
+            decode8_bytes(w8[0], w8[1], s0, c0, o[0]);
+            decode8_bytes(w8[2], w8[3], s0, c0, o[1]);
+            decode8_bytes(w8[4], w8[5], s1, c1, o[2]);
+            decode8_bytes(w8[6], w8[7], s1, c1, o[3]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                int q[8];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    q[i] = ((int)(w8[2 * j] << (24 - 8 * i))) >> 24;
+                    q[4 + i] = ((int)(w8[2 * j + 1] << (24 - 8 * i))) >> 24;
+                }
+                decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
+            }
+        }
+    }
+}
+
 // (mant, exps) -> bf16 operand, 32 elements per thread: one 16-byte (nibbles) or two 16-byte
 // (int8) loads, four 16-byte stores.  Work item of a warp = (row, segment of 1024 elements);
 // UNROLL items per warp are loaded before any is decoded so that several loads are in flight.
@@ -748,51 +807,8 @@ __device__ __forceinline__ void decode_bf16_body(const uint8_t *__restrict__ man
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             if (row[u] < 0) continue;
-            const int e0 = (int)(e[u] & 0xFF), e1 = b16 ? (int)((e[u] >> 8) & 0xFF) : e0;
-            const uint32_t w8[8] = {m[u][0].x, m[u][0].y, m[u][0].z, m[u][0].w,
-                                    m[u][NIBBLE ? 0 : 1].x, m[u][NIBBLE ? 0 : 1].y,
-                                    m[u][NIBBLE ? 0 : 1].z, m[u][NIBBLE ? 0 : 1].w};
             uint32_t o[4][4];
-            if (NIBBLE) {
-                if (nibble_fast_ok(e0, w) && nibble_fast_ok(e1, w)) {
-                    const __nv_bfloat162 m136 = as_bf162(0xC308C308u);       // -136
-                    const __nv_bfloat162 s0 = as_bf162(bf16x2_scale_bits(e0, w));
-                    const __nv_bfloat162 s1 = as_bf162(bf16x2_scale_bits(e1, w));
-                    const __nv_bfloat162 c0 = __hmul2(s0, m136), c1 = __hmul2(s1, m136);
-                    decode8_nibbles(w8[0], s0, c0, o[0]);
-                    decode8_nibbles(w8[1], s0, c0, o[1]);
-                    decode8_nibbles(w8[2], s1, c1, o[2]);
-                    decode8_nibbles(w8[3], s1, c1, o[3]);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        int q[8];
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) q[i] = ((int)(w8[j] << (28 - 4 * i))) >> 28;
-                        decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
-                    }
-                }
-            } else {
-                if (byte_fast_ok(e0, w) && byte_fast_ok(e1, w)) {
-                    const float s0 = f32_scale(e0, w), s1 = f32_scale(e1, w);
-                    const float c0 = -8388736.0f * s0, c1 = -8388736.0f * s1;
-                    decode8_bytes(w8[0], w8[1], s0, c0, o[0]);
-                    decode8_bytes(w8[2], w8[3], s0, c0, o[1]);
-                    decode8_bytes(w8[4], w8[5], s1, c1, o[2]);
-                    decode8_bytes(w8[6], w8[7], s1, c1, o[3]);
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        int q[8];
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            q[i] = ((int)(w8[2 * j] << (24 - 8 * i))) >> 24;
-                            q[4 + i] = ((int)(w8[2 * j + 1] << (24 - 8 * i))) >> 24;
-                        }
-                        decode8_safe(q, j < 2 ? e0 : e1, w, o[j]);
-                    }
-                }
-            }
+            decode32<NIBBLE>(m[u], e[u], b16, w, o);
             uint4 *dst = reinterpret_cast<uint4 *>(out + row[u] * ld_out + kc[u] * 32);
 #pragma unroll
             for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[j][0], o[j][1], o[j][2], o[j][3]);

@@ -39,14 +39,20 @@ def _close(got, ref, S, what):
 ])
 def test_batched_product_many_tiles_per_cta(mods, case):
     """Every output of every item against the oracle: the persistent loop with more than one tile
-    per CTA and more than one batch item (item-major tile numbering, rank-3 tensor maps)."""
+    per CTA and more than one batch item (item-major tile numbering, rank-3 tensor maps).  The block
+    exponents differ from row to row and from item to item but not along K inside an item, so every
+    partial sum is an integer below 2^24 times one power of two: any order of accumulation gives the
+    exactly summed result and the comparison is bit for bit -- a tile, item or row taken from the
+    wrong place cannot hide inside a tolerance."""
     mxb, _ = mods
     batch, M, N, K, B, w = case
     qmax = 2 ** (w - 1) - 1
+    nb = K // B
+    assert K * qmax * qmax < 2 ** 24
     qa = synth.random_ints((M, batch * K), -qmax, qmax, 900 + batch).numpy()
     qw = synth.random_ints((N, batch * K), -qmax, qmax, 901 + batch).numpy()
-    ea = synth.random_bytes((M, batch * K // B), 124, 130, 902 + batch).numpy()
-    ew = synth.random_bytes((N, batch * K // B), 120, 126, 903 + batch).numpy()
+    ea = np.repeat(synth.random_bytes((M, batch), 121, 133, 902 + batch).numpy(), nb, axis=1)
+    ew = np.repeat(synth.random_bytes((N, batch), 115, 127, 903 + batch).numpy(), nb, axis=1)
     f = mxb.MxFormat(B, w)
     dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
     y = torch.full((batch * M, N), 5.0, device="cuda")
@@ -54,7 +60,31 @@ def test_batched_product_many_tiles_per_cta(mods, case):
                         batch * K, K, M, N, K, batch, y, N, M * N)
     assert mxb.mx_poll_status() == 0
     got = y.cpu().numpy()
+    for b in range(batch):
+        y_ref, y_seq, S = orc.gemm(qa[:, b * K:(b + 1) * K], ea[:, b * nb:(b + 1) * nb], w,
+                                   qw[:, b * K:(b + 1) * K], ew[:, b * nb:(b + 1) * nb], w, B)
+        assert np.array_equal(y_ref, y_seq)                 # order-independent by construction
+        assert np.array_equal(got[b * M:(b + 1) * M], y_ref), "item %d" % b
+
+
+def test_batched_product_exponents_varying_along_k(mods):
+    """The same launch shape with block exponents that also change along K (within 2^+-1 per operand,
+    as the rows of attention operands do): every output within 1e-5 * S."""
+    mxb, _ = mods
+    batch, M, N, K, B, w = 48, 300, 260, 128, 16, 8
+    qmax = 2 ** (w - 1) - 1
     nb = K // B
+    qa = synth.random_ints((M, batch * K), -qmax, qmax, 910).numpy()
+    qw = synth.random_ints((N, batch * K), -qmax, qmax, 911).numpy()
+    ea = synth.random_bytes((M, batch * nb), 126, 128, 912).numpy()
+    ew = synth.random_bytes((N, batch * nb), 120, 122, 913).numpy()
+    f = mxb.MxFormat(B, w)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    y = torch.full((batch * M, N), 5.0, device="cuda")
+    mxb.mx_gemm_batched(dev(orc.pack(qa, w)), dev(ea), f, batch * K, K, dev(orc.pack(qw, w)), dev(ew), f,
+                        batch * K, K, M, N, K, batch, y, N, M * N)
+    assert mxb.mx_poll_status() == 0
+    got = y.cpu().numpy()
     for b in range(batch):
         y_ref, _, S = orc.gemm(qa[:, b * K:(b + 1) * K], ea[:, b * nb:(b + 1) * nb], w,
                                qw[:, b * K:(b + 1) * K], ew[:, b * nb:(b + 1) * nb], w, B)

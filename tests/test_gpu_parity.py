@@ -396,6 +396,51 @@ def test_linear_in_kernel_weight_decode(mxb, case):
     assert (err[ok] <= (TOL * S + 1e-37)[ok]).all()
 
 
+@pytest.mark.parametrize("case", [
+    # B, wa, ww, M, K, N, bf16 input
+    (16, 8, 4, 700, 768, 1100, False),      # ragged M and N: partly filled panels and tiles
+    (32, 4, 8, 300, 1024, 520, True),       # int8 weight container, bf16 activations, block 32
+    (16, 6, 3, 1500, 256, 2600, False),     # a single K group, more tiles than CTA pairs
+    (32, 8, 4, 2304, 2048, 640, False),     # more activation panels than the first wave covers
+])
+def test_linear_with_operands_prepared_inside_the_product_kernel(mxb, case):
+    """mx_linear with MX_ALGO_TCGEN05 on shapes the pair kernel can prepare for itself (K % 256 == 0,
+    M, N >= 256): extra warps quantize the activations and decode the weights while the tiles run;
+    every output against the oracle, with zero, tiny, huge and non-finite weight blocks, a bias and
+    canary columns."""
+    B, wa, ww, M, K, N, bf16 = case
+    x = synth.student_t_activations(M, K, seed=wa + 3)
+    if bf16:
+        x = x.to(torch.bfloat16)
+    wt = synth.gaussian_weights(N, K, seed=ww + 3).numpy()
+    wt[5, :B] = 0.0
+    wt[7, B:2 * B] *= np.float32(2.0 ** -120)
+    wt[9, :B] *= np.float32(2.0 ** 100)
+    qa, ea, _ = orc.quantize(x.float().numpy(), B, wa)
+    qw, ew, _ = orc.quantize(wt, B, ww)
+    ew[11, 1] = 255
+    bias = np.random.default_rng(4).standard_normal(N).astype(np.float32)
+    fa, fw = mxb.MxFormat(B, wa), mxb.MxFormat(B, ww)
+    y_ref, _, S = orc.gemm(qa, ea, wa, qw, ew, ww, B, bias=bias)
+    ypad = torch.full((M, N + 8), -77.0, device="cuda")
+    mxb.mx_linear(x.cuda(), fa, _dev(orc.pack(qw, ww)), _dev(ew), fw, N, bias=_dev(bias), y=ypad[:, :N],
+                  algo=mxb.MX_ALGO_TCGEN05)
+    assert mxb.mx_poll_status() == 0
+    y = ypad[:, :N].cpu().numpy()
+    assert np.array_equal(np.isnan(y), np.isnan(y_ref)) and np.isnan(y[:, 11]).all()
+    ok = ~np.isnan(y_ref)
+    err = np.abs(y.astype(np.float64) - y_ref.astype(np.float64))
+    assert (err[ok] <= (TOL * S + 1e-37)[ok]).all(), float((err[ok] / np.maximum(S[ok], 1e-300)).max())
+    assert (ypad[:, N:] == -77.0).all()
+    # a second call into the same workspace-sized buffers (counters cleared again) gives the same bits
+    ws = mxb.alloc_workspace(mxb.mx_workspace_bytes(M, N, K, fa, fw))
+    wm, we = _dev(orc.pack(qw, ww)), _dev(ew)
+    y1 = mxb.mx_linear(x.cuda(), fa, wm, we, fw, N, bias=_dev(bias), workspace=ws, algo=mxb.MX_ALGO_TCGEN05).clone()
+    y2 = mxb.mx_linear(x.cuda(), fa, wm, we, fw, N, bias=_dev(bias), workspace=ws, algo=mxb.MX_ALGO_TCGEN05)
+    assert mxb.mx_poll_status() == 0
+    assert torch.equal(torch.nan_to_num(y1), torch.nan_to_num(y2)) and np.array_equal(y1.cpu().numpy()[ok], y[ok])
+
+
 @pytest.mark.parametrize("case", [(16, 8, 4), (32, 4, 4), (32, 6, 3), (16, 2, 8)])
 def test_linear_mixed_precision(mxb, case):
     B, wa, ww = case

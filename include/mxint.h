@@ -76,11 +76,13 @@ typedef enum {
                             only; needs K % 32 == 0 and a 2-byte aligned w_exp, else it falls back to
                             the separate pass).  Saves memory, but the decode costs more issue slots
                             than the MMA leaves free, so it is slower than MX_ALGO_TCGEN05.          */
-    MX_ALGO_TCGEN05_CHUNKED = 5 /* tensor-core kernel with two-level accumulation: the tensor pipe sums one
-                            K step of 64 elements at a time, the partial sums are added in fp32 registers
-                            with round-to-nearest in ascending K order.  Meets 1e-5 * S (S = sum of the
-                            magnitudes of the block terms) for any spread of the block exponents and any K;
-                            costs about half the throughput of MX_ALGO_TCGEN05.  fp32 result only.      */
+    MX_ALGO_TCGEN05_BLOCKWISE = 5 /* tensor-core kernel that gives every block its own accumulator: the tensor
+                            pipe sums one block (exactly: all addends share one scale), the block terms
+                            are added in fp32 registers with round-to-nearest in ascending block order --
+                            the same bits as MX_ALGO_SIMT while every block term is a normal fp32 number.
+                            Meets 1e-5 * S for any spread of the block exponents and any K; a fraction of
+                            the throughput of MX_ALGO_TCGEN05 (a tensor-memory read per block).  fp32
+                            result only.                                                                  */
 } mx_algo_t;
 
 /* Accuracy of the product kernels against the exactly summed result (Sec. 3.2 leaves the accumulator
@@ -96,8 +98,9 @@ typedef enum {
  *                                  workload measured: N(0, sigma) weights, outlier-channel or
  *                                  Student-t activations, K up to 16384) the error stays below
  *                                  1e-5 * S, typically below 1e-6 * S.
- *   MX_ALGO_TCGEN05_CHUNKED      : < 48 * 2^-23 * S from the tensor pipe plus the rounding of K/64
- *                                  fp32 additions: below 1e-5 * S whatever the operands. */
+ *   MX_ALGO_TCGEN05_BLOCKWISE    : exact block sums out of the tensor pipe, one fp32 rounding per block,
+ *                                  ascending blocks: the result of MX_ALGO_SIMT, bit for bit, whatever
+ *                                  the operands (block terms inside the fp32 normal range). */
 
 /* The (B, e, m) tuple of Sec. 4.1. */
 typedef struct {

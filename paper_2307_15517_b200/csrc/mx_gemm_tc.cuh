@@ -135,7 +135,7 @@ __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, in
 // the warp's two 4 KB shared-memory buffers (`warp_bufs`, 128-byte swizzled box layout) and a tiled
 // TMA store -- whole 128-byte lines reach L2, rows >= M and columns >= N are clipped by the store --
 // or, when ldy % 4 != 0, with plain stores.  `epi_buf` counts the warp's TMA blocks (buffer parity).
-// Shared by the one-CTA, the CTA-pair and the chunked kernel.
+// Shared by the one-CTA, the CTA-pair and the block-wise kernel.
 __device__ __forceinline__ void store_f32_chunk(const TcParams &p, const CUtensorMap *tmap_y, uint32_t (&r)[32], int row,
                                                 int rows0, int n, int tb, uint32_t warp_bufs, uint32_t &epi_buf, int lane)
 {

@@ -1,27 +1,28 @@
-// Tensor-core MXInt product with two-level accumulation (Sec. 3.2 MXInt dot-product operator: the
-// paper fixes the integer block sums and the one shared scale per block, not the width of the
-// accumulator across blocks).
+// Tensor-core MXInt product that follows the operator of Sec. 3.2 to the letter: exact integer sums
+// inside each block, one shared scale per block, and the blocks added in fp32 in ascending order.
 //
-// The tensor pipe adds the 16 products of an MMA step and the running accumulator after aligning
-// all 17 addends to the largest and cutting the rest off (no rounding).  With block scales that
-// differ by many binades inside one row, a large running sum therefore eats the low bits of every
-// later small block, once per step, for the whole reduction.  Here the pipe only ever sums ONE
-// K step of 64 elements (four MMA steps, the first overwriting the accumulator): a chunk's loss is
-// at most 3 * 16 cut-offs of one ulp of the chunk's own largest term, i.e. < 48 * 2^-23 * S_chunk,
-// and the chunks are then added by the CUDA cores in fp32 registers with round-to-nearest, in
-// ascending K order.  Summed over a row: |dY| < 48 * 2^-23 * S (= 5.7e-6 * S) from the pipe plus the
-// ordinary rounding of K/64 fp32 additions, whatever the exponent spread and whatever K.
+// The tensor pipe adds the 16 products of an MMA step and the running accumulator after aligning all
+// addends to the largest and cutting the rest off (no rounding).  With block scales that differ by
+// many binades inside one row, a large running sum therefore eats the low bits of every later small
+// block.  Here the pipe only ever sums ONE block (one MMA step for blocks of 16, two for blocks of
+// 32, the first overwriting the accumulator): all its addends are integers (< 2^14) times the same
+// power of two and their sum stays below 2^19 times it, so nothing is cut off and the block term
+// q-sum * 2^(Ea+Ew-(wa-2)-(ww-2)) arrives in tensor memory exactly.  The CUDA cores then add the block
+// terms in fp32 registers with round-to-nearest, in ascending block order: bit for bit the
+// sequential fp32 accumulation of the definition (as long as no block term leaves the fp32 normal
+// range), and within (K/B) roundings of the exactly summed result whatever the exponent spread.
 //
-// Kernel: persistent, one CTA per SM, 128 x 128 tile, K step 64, four TMA stages, FOUR chunk
-// accumulators of 128 columns in tensor memory (all 512 columns) so the MMA thread runs up to four
-// chunks ahead of the drain.
+// Kernel: persistent, one CTA per SM, 128 x 128 tile, K step 64 per TMA stage, four stages, FOUR
+// block accumulators of 128 columns in tensor memory (all 512 columns) so the MMA thread runs up
+// to four blocks ahead of the drain.
 //   warp 0      : TMA producer (one lane)
 //   warp 1      : tensor-memory allocation, MMA issue (one lane)
 //   warps 2..9  : drain: warp w reads TMEM lanes 32 * (w % 4) .. + 31 (the hardware's lane window of a
-//                 warp), columns 64 * ((w - 2) / 4) .. + 63, of every chunk and adds them to 64 fp32
-//                 registers per lane; after the tile's last chunk it writes its 32 x 64 piece of Y
+//                 warp), columns 64 * ((w - 2) / 4) .. + 63, of every block term and adds them to 64
+//                 fp32 registers per lane (packed pairs); after the tile's last block it writes its
+//                 32 x 64 piece of Y
 // Costs against the single-accumulator kernels: the 128 x 128 tile moves twice the shared-memory
-// bytes per flop of the 256-wide tiles, and every K step pays a TMEM read and 64 additions per lane.
+// bytes per flop of the 256-wide tiles, and every block pays a TMEM read and 64 additions per lane.
 #pragma once
 #include <cuda.h>
 #include <cuda_runtime.h>
@@ -32,10 +33,18 @@
 
 namespace mx {
 
+// (lo, hi) pair of fp32 sums += (a, b); each half rounds to nearest like a scalar add.
+__device__ __forceinline__ uint64_t add2_rn(uint64_t acc, uint32_t a, uint32_t b)
+{
+    uint64_t d;
+    asm("{\n\t.reg .b64 t;\n\tmov.b64 t, {%2, %3};\n\tadd.rn.f32x2 %0, %1, t;\n\t}" : "=l"(d) : "l"(acc), "r"(a), "r"(b));
+    return d;
+}
+
 struct TcxCfg {
     static constexpr int BN = 128;
     static constexpr int STAGES = 4;
-    static constexpr int ACCS = 4;                                   // chunk accumulators in tensor memory
+    static constexpr int ACCS = 4;                                   // block accumulators in tensor memory
     static constexpr int DRAIN_WARPS = 8;
     static constexpr int THREADS = 64 + 32 * DRAIN_WARPS;            // 320
     static constexpr uint32_t A_BYTES = TC_BM * TC_BK * 2;
@@ -95,7 +104,8 @@ gemm_tcx_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
     if (threadIdx.x == 0) ptx::dep_trigger();
 
     const int num_tiles = p.tiles_m * p.tiles_n;
-    const int kblocks = (p.K + TC_BK - 1) / TC_BK;           // one chunk per K step
+    const int kblocks = (p.K + TC_BK - 1) / TC_BK;           // TMA stages per tile
+    const int steps_blk = p.block / 16;                      // MMA steps per block: 1 or 2
     bool timed_out = false;
 
     if (warp == 0) {
@@ -124,24 +134,33 @@ gemm_tcx_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             int s = 0, a = 0;
             uint32_t ph = 0, aph = 0;
             for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x) {
-                for (int kb = 0; kb < kblocks; ++kb) {
-                    if (!ptx::mbar_wait_bounded(tempty_bar(a), aph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS) ||
-                        !ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, TC_WAIT_LIMIT_NS)) {
+                for (int kb = 0; kb < kblocks && !timed_out; ++kb) {
+                    if (!ptx::mbar_wait_bounded(full_bar(s), ph, abort_flag, TC_WAIT_LIMIT_NS)) {
                         timed_out = true;
                         break;
                     }
                     ptx::tc_fence_after_sync();
-                    const uint32_t d_tmem = tmem_base + (uint32_t)(a * BN);
                     const uint32_t sa = smem_base + s * Cfg::STAGE_BYTES;
                     const uint32_t sw = sa + Cfg::A_BYTES;
-#pragma unroll
-                    for (int j = 0; j < TC_BK / 16; ++j)       // the chunk starts from zero: j == 0 overwrites
-                        ptx::mma_bf16_ss(d_tmem, ptx::smem_desc_k_sw128(sa, j * 32), ptx::smem_desc_k_sw128(sw, j * 32),
-                                         idesc, j != 0 ? 1u : 0u);
-                    ptx::mma_commit(empty_bar(s));             // stage free once these MMAs retire
-                    ptx::mma_commit(tfull_bar(a));             // ... and the chunk's sum is complete
+                    const int steps = min(TC_BK, p.K - kb * TC_BK) / 16;      // K % block == 0: whole blocks
+                    for (int j = 0; j < steps; ++j) {
+                        const bool first = (j % steps_blk) == 0, last = ((j + 1) % steps_blk) == 0;
+                        if (first) {
+                            if (!ptx::mbar_wait_bounded(tempty_bar(a), aph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS)) {
+                                timed_out = true;
+                                break;
+                            }
+                            ptx::tc_fence_after_sync();
+                        }
+                        ptx::mma_bf16_ss(tmem_base + (uint32_t)(a * BN), ptx::smem_desc_k_sw128(sa, j * 32),
+                                         ptx::smem_desc_k_sw128(sw, j * 32), idesc, first ? 0u : 1u);   // a block starts from zero
+                        if (last) {
+                            ptx::mma_commit(tfull_bar(a));             // the block's sum is complete
+                            if (++a == ACCS) { a = 0; aph ^= 1u; }
+                        }
+                    }
+                    ptx::mma_commit(empty_bar(s));                 // stage free once these MMAs retire
                     if (++s == STAGES) { s = 0; ph ^= 1u; }
-                    if (++a == ACCS) { a = 0; aph ^= 1u; }
                 }
             }
         }
@@ -153,10 +172,11 @@ gemm_tcx_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         uint32_t aph = 0, epi_buf = 0;
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x) {
             const int m0 = (t % p.tiles_m) * TC_BM, n0 = (t / p.tiles_m) * BN;
-            float acc[64];
+            uint64_t acc[32];                                   // 64 fp32 sums as packed pairs
 #pragma unroll
-            for (int v = 0; v < 64; ++v) acc[v] = 0.f;
-            for (int kb = 0; kb < kblocks; ++kb) {
+            for (int v = 0; v < 32; ++v) acc[v] = 0ull;
+            const int nblocks = p.K / p.block;
+            for (int b = 0; b < nblocks; ++b) {
                 const bool ok = ptx::mbar_wait_bounded(tfull_bar(a), aph, abort_flag, TC_WAIT_LIMIT_NS);
                 if (!__all_sync(0xFFFFFFFFu, ok)) {
                     timed_out = true;
@@ -172,9 +192,9 @@ gemm_tcx_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 __syncwarp();
                 if (lane == 0) ptx::mbar_arrive(tempty_bar(a));    // the values are in registers: the accumulator is free
 #pragma unroll
-                for (int v = 0; v < 32; ++v) {
-                    acc[v] += __uint_as_float(r0[v]);              // ascending chunks, round to nearest
-                    acc[32 + v] += __uint_as_float(r1[v]);
+                for (int v = 0; v < 16; ++v) {                     // ascending blocks, one rounding per block and output
+                    acc[v] = add2_rn(acc[v], r0[2 * v], r0[2 * v + 1]);
+                    acc[16 + v] = add2_rn(acc[16 + v], r1[2 * v], r1[2 * v + 1]);
                 }
                 if (++a == ACCS) { a = 0; aph ^= 1u; }
             }
@@ -184,7 +204,10 @@ gemm_tcx_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             for (int c = 0; c < 2; ++c) {
                 uint32_t r[32];
 #pragma unroll
-                for (int v = 0; v < 32; ++v) r[v] = __float_as_uint(acc[32 * c + v]);
+                for (int v = 0; v < 16; ++v) {
+                    r[2 * v] = (uint32_t)acc[16 * c + v];
+                    r[2 * v + 1] = (uint32_t)(acc[16 * c + v] >> 32);
+                }
                 store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n0 + half * 64 + 32 * c, 0,
                                 epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
             }

@@ -509,9 +509,10 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     return MX_OK;
 }
 
-// The chunked kernel (two-level accumulation): 128 x 128 tiles, fp32 result, one product per launch.
+// The block-wise kernel (one tensor-memory accumulator per block, blocks added in fp32 registers):
+// 128 x 128 tiles, fp32 result, one product per launch.
 mx_status_t launch_tcx(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N, int64_t K,
-                       const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
+                       int block, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st)
 {
     using Cfg = mx::TcxCfg;
     CUtensorMap tm_a, tm_w;
@@ -539,6 +540,7 @@ mx_status_t launch_tcx(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     p.status = d.status;
     p.tma_store = tma_store ? 1 : 0;
     p.batch = 1;
+    p.block = block;
     const int64_t tiles64 = (int64_t)p.tiles_m * p.tiles_n;
     if (tiles64 > INT32_MAX / 2) return MX_ERR_SHAPE;
     const int grid = tiles64 < d.sm_count ? (int)tiles64 : d.sm_count;
@@ -831,7 +833,7 @@ size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx
         return st > tc ? st : tc;
     }
     case MX_ALGO_TCGEN05:
-    case MX_ALGO_TCGEN05_CHUNKED: return tc_workspace(M, N, K);
+    case MX_ALGO_TCGEN05_BLOCKWISE: return tc_workspace(M, N, K);
     case MX_ALGO_TCGEN05_FUSED: return (K % 32) == 0 ? fused_workspace(M, K) : tc_workspace(M, N, K);
     default: return 0;
     }
@@ -970,7 +972,7 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         if (algo == MX_ALGO_STREAM) return grouped_impl(&one, 1, &a_exp, workspace, workspace_bytes, stream);
     }
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
-        algo != MX_ALGO_TCGEN05_CHUNKED)
+        algo != MX_ALGO_TCGEN05_BLOCKWISE)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -999,7 +1001,7 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
                                                              round256((size_t)M * K * 2));
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
-    if (algo == MX_ALGO_TCGEN05_CHUNKED) return launch_tcx(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
+    if (algo == MX_ALGO_TCGEN05_BLOCKWISE) return launch_tcx(a_hat, w_hat, M, N, K, fa.block, bias, y, ldy, *d, st);
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }
 
@@ -1031,7 +1033,7 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
                                                                                      : MX_ALGO_TCGEN05;
     if (algo == MX_ALGO_STREAM) return mx_linear_grouped(&one, 1, workspace, workspace_bytes, stream);
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
-        algo != MX_ALGO_TCGEN05_CHUNKED)
+        algo != MX_ALGO_TCGEN05_BLOCKWISE)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -1070,7 +1072,7 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         return run_linear_fused(one, ws, nullptr, *d, st);
     s = tc_prepare(one, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
-    if (algo == MX_ALGO_TCGEN05_CHUNKED) return launch_tcx(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
+    if (algo == MX_ALGO_TCGEN05_BLOCKWISE) return launch_tcx(a_hat, w_hat, M, N, K, fa.block, bias, y, ldy, *d, st);
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }
 

@@ -187,7 +187,7 @@ def test_gemm_simt_matches_sequential_oracle_exactly(mxb, shape):
 
 
 TC_ALGOS = ("MX_ALGO_TCGEN05", "MX_ALGO_TCGEN05_FUSED")
-TC_ALGOS_ALL = TC_ALGOS + ("MX_ALGO_TCGEN05_CHUNKED",)
+TC_ALGOS_ALL = TC_ALGOS + ("MX_ALGO_TCGEN05_BLOCKWISE",)
 
 
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
@@ -231,10 +231,11 @@ def test_gemm_tensor_core_adversarial_exponent_spread(mxb):
 
 
 @pytest.mark.parametrize("shape", GEMM_SHAPES)
-def test_gemm_chunked_accumulation_meets_tolerance_on_any_exponent_spread(mxb, shape):
+def test_gemm_blockwise_accumulation_is_the_sequential_fp32_sum(mxb, shape):
     """Block exponents drawn uniformly over 2^+-8 per operand (terms 2^+-16 apart), where the
-    single-accumulator kernels only meet their derived bound: with the accumulator drained every K
-    step and the partial sums added in fp32 registers, the stated 1e-5 * S holds on every shape."""
+    single-accumulator kernels only meet their derived bound: with one tensor-memory accumulator per
+    block and the block terms added in fp32 registers in ascending order, the result is the oracle's
+    sequential sum bit for bit, and the stated 1e-5 * S holds on every shape."""
     M, N, K, B, wa, ww = shape
     qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=31 * M + N, spread=8)
     bias = np.random.default_rng(3).standard_normal(N).astype(np.float32) if (M + N) % 2 else None
@@ -242,32 +243,35 @@ def test_gemm_chunked_accumulation_meets_tolerance_on_any_exponent_spread(mxb, s
     ypad = torch.full((M, N + 8), -77.0, device="cuda")
     y = mxb.mx_gemm(_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)),
                     _dev(ew), mxb.MxFormat(B, ww), M, N, K, bias=None if bias is None else _dev(bias),
-                    y=ypad[:, :N], algo=mxb.MX_ALGO_TCGEN05_CHUNKED)
+                    y=ypad[:, :N], algo=mxb.MX_ALGO_TCGEN05_BLOCKWISE)
     assert mxb.mx_poll_status() == 0
     _check_tol(y, y_ref, S)
+    assert np.array_equal(y.cpu().numpy(), y_seq)
     assert (ypad[:, N:] == -77.0).all()
 
 
 @pytest.mark.parametrize("K", (11008, 16384))
 def test_gemm_long_reductions_with_wide_exponent_spread(mxb, K):
     """The longest reductions of the paper-shaped workloads (LLaMA-7B down projection, OPT-6.7B FFN)
-    with the adversarial +-8 exponent spread: the chunked kernel inside 1e-5 * S, the default kernel
+    with the adversarial +-8 exponent spread: the block-wise kernel equal to the sequential fp32 sum
+    and inside 1e-5 * S, the default kernel
     inside its derived bound ceil(K/16) * 17 * 2^-23 * S (asserted at these K, not only at K = 320)."""
     M, N, B, wa, ww = 160, 200, 16, 8, 4
     qa, ea, qw, ew = _random_operands(M, N, K, B, wa, ww, seed=K, spread=8)
     y_ref, y_seq, S = orc.gemm(qa, ea, wa, qw, ew, ww, B)
     args = (_dev(orc.pack(qa, wa)), _dev(ea), mxb.MxFormat(B, wa), _dev(orc.pack(qw, ww)), _dev(ew),
             mxb.MxFormat(B, ww), M, N, K)
-    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05_CHUNKED)
+    y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05_BLOCKWISE)
     assert mxb.mx_poll_status() == 0
     _check_tol(y, y_ref, S)
-    worst_chunked = float((np.abs(y.cpu().numpy().astype(np.float64) - y_ref) / S).max())
+    assert np.array_equal(y.cpu().numpy(), y_seq)
+    worst_blockwise = float((np.abs(y.cpu().numpy().astype(np.float64) - y_ref) / S).max())
     y = mxb.mx_gemm(*args, algo=mxb.MX_ALGO_TCGEN05).cpu().numpy().astype(np.float64)
     assert mxb.mx_poll_status() == 0
     assert (np.abs(y - y_ref) <= -(-K // 16) * 17 * 2.0 ** -23 * S).all()
     worst_default = float((np.abs(y - y_ref) / S).max())
-    print("K=%d spread +-8: max |dY|/S chunked %.2e, single accumulator %.2e" % (K, worst_chunked, worst_default))
-    assert worst_chunked <= 1e-5
+    print("K=%d spread +-8: max |dY|/S block-wise %.2e, single accumulator %.2e" % (K, worst_blockwise, worst_default))
+    assert worst_blockwise <= 1e-5
 
 
 def test_linear_student_t_full_reduction_length_default_kernel(mxb):
@@ -283,7 +287,7 @@ def test_linear_student_t_full_reduction_length_default_kernel(mxb):
     fw = mxb.MxFormat(B, ww)
     wm, we = mxb.mx_quantize(w.cuda(), fw)
     worst = {}
-    for name in ("MX_ALGO_AUTO", "MX_ALGO_TCGEN05_CHUNKED"):
+    for name in ("MX_ALGO_AUTO", "MX_ALGO_TCGEN05_BLOCKWISE"):
         y = mxb.mx_linear(x.cuda(), mxb.MxFormat(B, wa), wm, we, fw, N, algo=getattr(mxb, name))
         assert mxb.mx_poll_status() == 0
         _check_tol(y, y_ref, S)

@@ -31,9 +31,14 @@ METRIC = "mx_linear_effective_tops"
 UNIT = "TOPS"
 WORKLOAD = "opt-1.3b prefill linears, 2048 tokens, MXInt4 block 16 (4 layers per step)"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of gemm_tc_kernel<256,0>, averaged over the
-# four launches of a step, from the ncu capture summarised in profiles/gemm_tc_kernel_opt13b_prefill.md
-GEMM_TC_DRAM_BYTES_PER_LAUNCH = 46.8e6   # dram read + write per launch, ncu capture in profiles/gemm_tc_kernel_opt13b_prefill.md
+# dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the four launches of a step, from the
+# ncu captures summarised under profiles/ (gemm_tc_kernel_opt13b_prefill.md, prep_operands_kernel_opt13b_prefill.md)
+GEMM_TC_DRAM_BYTES_PER_LAUNCH = 46.8e6
+PREP_DRAM_BYTES_PER_LAUNCH = None        # filled in from the capture of the operand-preparation kernel
+# Dense bf16 tensor throughput of one SM per clock (tcgen05, 128x256x16 per 128 clocks): 8192 flop.
+# SMs x this x the SM clock sampled during the timed region = the hardware bound the fractions below use
+# beside the measured rate of the vendor's GEMM (which itself runs power-capped near 1.35 GHz).
+TENSOR_FLOP_PER_CLK_PER_SM = 8192
 
 
 def load_peaks():
@@ -119,9 +124,16 @@ def build_device_workload(mxb, synth, torch, seed):
         xd = x.cuda()
         y = torch.empty((x.shape[0], spec.N), dtype=torch.float32, device="cuda")
         ws = mxb.alloc_workspace(mxb.mx_workspace_bytes(x.shape[0], spec.N, spec.K, fa, fw))
+        M = x.shape[0]
         layers.append(dict(spec=spec, fa=fa, fw=fw, x=xd, x_host=x.pin_memory(), w_mant=w_mant,
                            w_exp=w_exp, y=y, ws=ws,
-                           y_host=torch.empty((x.shape[0], spec.N), dtype=torch.float32).pin_memory()))
+                           y_host=torch.empty((M, spec.N), dtype=torch.float32).pin_memory(),
+                           # the same layer with an MXInt8 result (blocks of `block` along N)
+                           fy=mxb.MxFormat(spec.block, 8),
+                           yq_mant=torch.empty((M, spec.N), dtype=torch.uint8, device="cuda"),
+                           yq_exp=torch.empty((M, spec.N // spec.block), dtype=torch.uint8, device="cuda"),
+                           yq_mant_host=torch.empty((M, spec.N), dtype=torch.uint8).pin_memory(),
+                           yq_exp_host=torch.empty((M, spec.N // spec.block), dtype=torch.uint8).pin_memory()))
     torch.cuda.synchronize()
     return layers
 
@@ -159,7 +171,8 @@ class E2EPipeline:
         for st in (self.s_in, self.s_run, self.s_out):
             cur.wait_stream(st)
 
-    def step(self, mxb, layers):
+    def step(self, mxb, layers, quantized=False):
+        """quantized: the layer returns MXInt8 (mx_linear_q) and only its packed bytes go back to the host."""
         torch = self.torch
         for L in layers:
             with torch.cuda.stream(self.s_in):
@@ -171,12 +184,20 @@ class E2EPipeline:
                 self.s_run.wait_event(L["ev_in"])
                 if "ev_out" in L:
                     self.s_run.wait_event(L["ev_out"])       # y's previous contents have reached the host
-                mxb.mx_linear(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, y=L["y"],
-                              workspace=L["ws"], stream=self.s_run)
+                if quantized:
+                    mxb.mx_linear_q(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, L["fy"],
+                                    y_mant=L["yq_mant"], y_exp=L["yq_exp"], workspace=L["ws"], stream=self.s_run)
+                else:
+                    mxb.mx_linear(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, y=L["y"],
+                                  workspace=L["ws"], stream=self.s_run)
                 L["ev_run"] = self.s_run.record_event()
             with torch.cuda.stream(self.s_out):
                 self.s_out.wait_event(L["ev_run"])
-                L["y_host"].copy_(L["y"], non_blocking=True)
+                if quantized:
+                    L["yq_mant_host"].copy_(L["yq_mant"], non_blocking=True)
+                    L["yq_exp_host"].copy_(L["yq_exp"], non_blocking=True)
+                else:
+                    L["y_host"].copy_(L["y"], non_blocking=True)
                 L["ev_out"] = self.s_out.record_event()
 
 
@@ -354,7 +375,7 @@ def decoder_block_rate(mxb, synth, torch, iters=5):
     return {"ms_per_block": ms, "tops": fl / ms / 1e9, "flops": fl,
             "kernels_ms": {k: v[0] / iters for k, v in prof.items() if v[1]},
             "launches": sum(v[1] for v in prof.values()) / iters,
-            "note": "includes torch allocations of the intermediates; glue kernels are not in kernels_ms"}
+            "note": "includes torch allocations of the intermediates"}
 
 
 # ------------------------------------------------------------------------------ oracle (CPU)
@@ -513,7 +534,7 @@ def run_ours(args):
     assert mxb.mx_poll_status() == 0, "device status after the timed region"
 
     # ---- end to end: pinned host inputs in, results out, every step ----
-    ms_e2e = float("nan")
+    ms_e2e = ms_e2e_q = float("nan")
     if not args.skip_e2e:
         pipe = E2EPipeline(torch)
         pipe.begin()
@@ -531,17 +552,29 @@ def run_ours(args):
         torch.cuda.synchronize()
         ms_e2e = a.elapsed_time(b)
         barrier()
+        # the same leg with the layer's own result type: MXInt8 mantissas + exponent bytes go back, not fp32
+        for L in (L for S in sets for L in S):
+            L.pop("ev_run", None), L.pop("ev_out", None), L.pop("ev_in", None)
+        pipe.begin()
+        for _ in range(2):
+            pipe.step(mxb, next_set(), quantized=True)
+        pipe.end()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        pipe.begin()
+        for _ in range(args.steps):
+            pipe.step(mxb, next_set(), quantized=True)
+        pipe.end()
+        b.record()
+        torch.cuda.synchronize()
+        ms_e2e_q = a.elapsed_time(b)
+        barrier()
 
     secondary = None
     linear_q = None
     if world == 1 and not args.skip_secondary:          # single-GPU runs only
         # the prefill step once more with MXInt8 results instead of fp32 (no fp32 Y is written)
-        for S in sets:
-            for L in S:
-                M, N = L["y"].shape
-                L["fy"] = mxb.MxFormat(L["spec"].block, 8)
-                L["yq_mant"] = torch.empty((M, N), dtype=torch.uint8, device="cuda")
-                L["yq_exp"] = torch.empty((M, N // L["spec"].block), dtype=torch.uint8, device="cuda")
         for _ in range(3):
             run_step_q(mxb, next_set())
         torch.cuda.synchronize()
@@ -577,17 +610,28 @@ def run_ours(args):
                      "llama7b_mixed": llama7b_rate(mxb, synth, torch),
                      "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
+        # every configuration's whole call against the vendor-GEMM rate (tensor-bound ones)
+        for key in ("linear_q", "block_16x2", "llama7b_mixed", "decoder_block"):
+            secondary[key]["frac_of_bf16_burst"] = secondary[key]["tops"] / peaks["bf16_tflops"]
+        secondary["llama7b_mixed"]["gemm_frac_of_bf16_burst"] = secondary["llama7b_mixed"]["gemm_tflops"] / peaks["bf16_tflops"]
         assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"
     barrier()
 
-    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], dist, device="cuda")
+    ms_total, ms_e2e, ms_e2e_q = max_over_ranks([ms_total, ms_e2e, ms_e2e_q], dist, device="cuda")
 
     if rank == 0:
         value = aggregate_tops(world, flops_step, args.steps, ms_total)
         e2e_value = aggregate_tops(world, flops_step, args.steps, ms_e2e)
+        e2e_q_value = aggregate_tops(world, flops_step, args.steps, ms_e2e_q)
+        d2h_q = sum(L["yq_mant_host"].numel() + L["yq_exp_host"].numel() for L in layers)
         gemm_ms, gemm_n = prof["gemm_tc"]
         achieved = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
         peak = peaks["bf16_tflops"]          # burst figure: the timed region lasts well under a second
+        # hardware bound at the clock this run actually had: SMs x 8192 flop per clock x sampled SM MHz
+        sms = torch.cuda.get_device_properties(local_rank).multi_processor_count
+        mhz = (clocks or {}).get("sm_mhz") or (clocks or {}).get("sm_max_mhz") or 1965.0
+        peak_clock = sms * TENSOR_FLOP_PER_CLK_PER_SM * mhz * 1e6 / 1e12
+        per_gpu = value / world
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
@@ -603,7 +647,11 @@ def run_ours(args):
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
                     "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / args.steps,
                     "note": "pinned host X in and fp32 Y out for every layer of every step; copies in both "
-                            "directions and the kernels run on three event-chained streams (PCIe-bound)"},
+                            "directions and the kernels run on three event-chained streams (PCIe-bound)",
+                    "mxint8_results": {"value": e2e_q_value, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                                       "d2h_bytes_per_step": d2h_q, "ms_per_step": ms_e2e_q / args.steps,
+                                       "note": "the same leg through mx_linear_q: the layer's MXInt8 result "
+                                               "(mantissas + exponent bytes) goes back instead of fp32"}},
             "gpu_launches": sum(n for _, n in prof.values()),
             "gpu_launches_note": "counted by the library over an instrumented repeat of the K timed steps",
             "kernels": {k: {"ms_per_step": ms / args.steps, "launches_per_step": n / args.steps}
@@ -612,10 +660,20 @@ def run_ours(args):
                             "(%.4f ms per step with the extra event records in the stream)" % (ms_instr / args.steps),
             "roofline": {"bound": "tensor", "kernel": "gemm_tc2_kernel / gemm_tc_kernel", "achieved": achieved,
                          "peak": peak, "unit": "TFLOP/s", "frac": achieved / peak,
-                         "peak_kind": "bf16 burst, %s" % peaks_kind,
+                         "peak_kind": "rate of the vendor's bf16 GEMM (burst), %s" % peaks_kind,
                          "frac_of_sustained_peak": achieved / peaks["bf16_tflops_sustained"],
+                         # the bound the silicon sets at the clock sampled during the timed region
+                         "peak_clock_derived": peak_clock, "frac_of_clock_derived_peak": achieved / peak_clock,
+                         "clock_derived_note": "%d SMs x %d flop/clk x %.0f MHz (median sampled under load)"
+                                               % (sms, TENSOR_FLOP_PER_CLK_PER_SM, mhz),
                          "traffic": GEMM_TC_DRAM_BYTES_PER_LAUNCH,
-                         "algorithmic_flops_per_launch": flops_step / 4.0},
+                         "algorithmic_flops_per_launch": flops_step / 4.0,
+                         # the whole call (operand preparation + product) against the same peaks
+                         "call": {"achieved": per_gpu, "frac": per_gpu / peak,
+                                  "frac_of_sustained_peak": per_gpu / peaks["bf16_tflops_sustained"],
+                                  "frac_of_clock_derived_peak": per_gpu / peak_clock,
+                                  "traffic_per_step": None if PREP_DRAM_BYTES_PER_LAUNCH is None else
+                                  4 * (GEMM_TC_DRAM_BYTES_PER_LAUNCH + PREP_DRAM_BYTES_PER_LAUNCH)}},
             "secondary": secondary,
             "cpu_baseline": None if args.skip_cpu_baseline else cpu_baseline(),
         }

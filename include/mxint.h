@@ -159,7 +159,8 @@ MX_API mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64
                         int64_t stride_row, int64_t stride_k, mx_format_t f, void *mant_out,
                         uint8_t *exp_out, uint32_t *nonfinite_count, void *stream);
 
-/* Inverse map (test helper): out[r*ld_out + k] = q * 2^(E-(w-2)) as `dt` (exact in both
+/* Inverse map (Sec. 3.2: the software emulator of a format converts between it and floating point in
+ * both directions; here a test helper): out[r*ld_out + k] = q * 2^(E-(w-2)) as `dt` (exact in both
  * fp32 and bf16); NaN for blocks with exponent byte 255. */
 MX_API mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, int64_t K,
                           mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream);
@@ -233,7 +234,9 @@ typedef struct {
 } mx_linear_args_t;
 
 /*
- * Runs n_layers independent MXInt linear layers with few tokens each (decode) in ONE kernel
+ * Sec. 1 and Sec. 6 motivate MX formats by the memory footprint of the parameters: at a few tokens per
+ * step a layer's time is the time to stream its packed weights once.  This call
+ * runs n_layers independent MXInt linear layers with few tokens each (decode) in ONE kernel
  * launch: every distinct activation tensor is quantized to its format once (layers that name
  * the same x, shape and format share it), then a single persistent kernel streams all weight
  * matrices from HBM exactly once.  Per output the integer block sums are exact and the blocks are
@@ -291,7 +294,7 @@ MX_API mx_status_t mx_softmax_q(const float *s, int64_t ld, int64_t rows, int64_
                                 int causal, int64_t rows_per_batch, mx_format_t fp, void *p_mant,
                                 uint8_t *p_exp, void *stream);
 
-/* ---- device status --------------------------------------------------------------------- */
+/* ---- device status (the paper has no counterpart: it describes no runtime) ---------------- */
 
 /*
  * Every device-side wait in this library (mbarrier polls of the tensor-core pipeline) gives up
@@ -375,9 +378,10 @@ MX_API mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_f
  * Between mx_profile_begin and mx_profile_end the library brackets each of its kernel launches
  * with a pair of CUDA events on the launch stream.  mx_profile_end waits for them and returns,
  * per kernel kind, the summed device time in milliseconds and the number of launches (arrays of
- * MX_KERNEL_KINDS entries, host memory).  Kinds: 0 quantize, 1 dequantize, 2 tensor-core GEMM,
- * 3 CUDA-core GEMM, 4 weight-streaming GEMM, 5 operand preparation of mx_linear (activation
- * quantize + weight decode in one launch).  Not thread-safe with respect to concurrent
+ * MX_KERNEL_KINDS entries, host memory).  Kinds: 0 quantize (incl. casts and the transposing
+ * quantizer), 1 dequantize, 2 tensor-core GEMM, 3 CUDA-core GEMM, 4 weight-streaming GEMM, 5 operand
+ * preparation of mx_linear (activation quantize + weight decode in one launch), 6 fp32 glue
+ * (LayerNorm, softmax with fp32 or MXInt result, ReLU/add).  Not thread-safe with respect to concurrent
  * compute calls on other host threads being attributed correctly; meant for one stream. */
 #define MX_KERNEL_KINDS 8
 MX_API mx_status_t mx_profile_begin(void);

@@ -417,7 +417,7 @@ def mx_selftest_wait_expiry(limit_us: int = 2000, stream=None) -> None:
     _check(lib.mx_selftest_wait_expiry(limit_us, _stream(stream)), "mx_selftest_wait_expiry")
 
 
-KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream", "prep")
+KERNEL_KINDS = ("quantize", "dequantize", "gemm_tc", "gemm_simt", "gemm_stream", "prep", "glue")
 
 
 def mx_profile_begin() -> None:

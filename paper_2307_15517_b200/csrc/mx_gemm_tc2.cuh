@@ -25,96 +25,6 @@
 
 namespace mx {
 
-// ---- operand preparation inside the product kernel (PREP > 0) ---------------------------------------
-// mx_linear has to turn fp32/bf16 activations into their quantized, exactly decoded bf16 operand and
-// packed weights into theirs before the tensor cores can use them.  Both passes are HBM-bound while
-// the product is tensor-bound, so with PREP extra warps per CTA they run INSIDE the product kernel,
-// ahead of the tiles that need them, instead of in a launch of their own in front of it:
-//   * work unit  = 256 consecutive k (one "K group" = four K steps) of 32 activation rows (quantize:
-//                  block maximum, shared exponent, rounding, exact bf16) or of 128 weight rows (decode);
-//                  32 warp items each, spread over the CTA's PREP warps
-//   * order      = K group by K group for all activation panels and for the weight panels of the first
-//                  wave of tiles, then the remaining weight panels in the order the tiles reach them;
-//                  unit i belongs to CTA i % gridDim.x, so all CTAs advance through the list together
-//   * hand-over  = one counter per (128-row panel, K group) in the workspace, zero at launch: every
-//                  prep warp adds 1 after a release fence when its share of a unit is written; the TMA
-//                  producer of a tile polls (acquire, bounded) the two counters of the K group it is
-//                  about to load, then orders its TMA loads behind them with a proxy fence
-// Prep warps never wait on anything, every CTA of the grid is resident (one per SM), so the consumers'
-// waits always end; they are bounded like every other wait of the library.
-struct FusedPrep {
-    const void *x;              // activations [M, K], fp32 or bf16, leading dimension ldx
-    int64_t ldx;
-    int x_bf16;                 // 1: x is bf16
-    int wa, ww;                 // mantissa widths of activations / weights
-    int block;                  // 16 or 32, both operands
-    __nv_bfloat16 *a_hat;       // [M, K] exact bf16 operand (written here)
-    const uint8_t *w_mant;      // packed weights [N, K/2] (ww <= 4) or [N, K]
-    const uint8_t *w_exp;       // [N, K/block]
-    __nv_bfloat16 *w_hat;       // [N, K] (written here)
-    uint32_t *flags;            // [(PA + PW) * G] progress counters, all zero at launch
-    int PA, PW;                 // 128-row panels of A / W covered by the tile grid
-    int G;                      // K groups = K / 256
-    int W0;                     // weight panels the first wave of tiles needs
-};
-constexpr int PREP_KG = 256;    // elements per K group
-
-__device__ __forceinline__ bool flag_wait_bounded(const uint32_t *flag, uint32_t target, volatile uint32_t *abort_flag,
-                                                  uint64_t limit_ns)
-{
-    uint64_t t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        uint32_t v;
-        asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
-        if (v >= target) return true;
-        if ((it & 0x7F) == 0) {
-            if (*abort_flag) return false;
-            const uint64_t now = ptx::globaltimer_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > limit_ns) return false;
-        }
-    }
-}
-
-// One decode unit: rows [r0, r0 + 128) x k [k0, k0 + 256) of the packed weights -> bf16.  A lane item
-// is 32 elements (one or two 16-byte loads, four 16-byte stores); 8 lanes cover the 256 k of a row,
-// so a warp item is 4 rows and the unit has 32 warp items.
-template <bool NIBBLE>
-__device__ __forceinline__ void decode_unit(const FusedPrep &fp, int N, int K, int r0, int k0, int pw, int n_pw, int lane)
-{
-    const bool b16 = fp.block == 16;
-    const int64_t mant_ld = NIBBLE ? (K >> 1) : K, nb_row = K / fp.block;
-    const int sub = lane >> 3, kc = lane & 7;                   // row within the warp item, 32-element chunk
-#pragma unroll 2
-    for (int wi = pw; wi < 32; wi += n_pw) {
-        const int row = r0 + wi * 4 + sub;
-        if (row < N) {
-            const int k = k0 + kc * 32;
-            uint4 m[NIBBLE ? 1 : 2];
-            const uint4 *src = reinterpret_cast<const uint4 *>(fp.w_mant + (int64_t)row * mant_ld + (NIBBLE ? (k >> 1) : k));
-            m[0] = __ldcs(src);
-            if (!NIBBLE) m[NIBBLE ? 0 : 1] = __ldcs(src + 1);
-            const uint8_t *ep = fp.w_exp + (int64_t)row * nb_row + k / fp.block;
-            const uint32_t e = b16 ? (uint32_t)__ldg(ep) | ((uint32_t)__ldg(ep + 1) << 8) : (uint32_t)__ldg(ep);
-            uint32_t o[4][4];
-            decode32<NIBBLE>(m, e, b16, fp.ww, o);
-            uint4 *dst = reinterpret_cast<uint4 *>(fp.w_hat + (int64_t)row * K + k);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) dst[j] = make_uint4(o[j][0], o[j][1], o[j][2], o[j][3]);
-        }
-    }
-}
-
-// One quantize unit: rows [r0, r0 + rows) x k [k0, k0 + 256) of the activations -> exact bf16.
-template <typename InT>
-__device__ __forceinline__ void quantize_unit(const FusedPrep &fp, int K, int r0, int rows, int k0, int pw, int n_pw)
-{
-    QuantOut out{nullptr, nullptr, fp.a_hat + (int64_t)r0 * K + k0, K, nullptr, 0};
-    const InT *x = static_cast<const InT *>(fp.x) + (int64_t)r0 * fp.ldx + k0;
-    if (fp.block == 16) quantize_rows_body<InT, 16, 2>(x, rows, PREP_KG, fp.ldx, fp.wa, out, pw, n_pw);
-    else quantize_rows_body<InT, 32, 2>(x, rows, PREP_KG, fp.ldx, fp.wa, out, pw, n_pw);
-}
-
 struct Tc2Cfg {
     static constexpr int BN = 256;                        // pair tile: 256 x 256
     static constexpr int STAGES = 6;
@@ -127,10 +37,9 @@ struct Tc2Cfg {
     static constexpr uint32_t TMEM_COLS = 512;            // two accumulators of 256 columns
 };
 
-template <int PREP>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS + 32 * PREP, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
-                const __grid_constant__ CUtensorMap tmap_y, const TcParams p, const FusedPrep fp)
+                const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
 {
     using Cfg = Tc2Cfg;
     constexpr int STAGES = Cfg::STAGES, BN = Cfg::BN;
@@ -190,19 +99,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
                 const int m0 = (t % p.tiles_m) * 256 + (int)rank * 128;
                 const int n0 = (t / p.tiles_m) * BN + (int)rank * (BN / 2);
                 for (int kb = 0; kb < kblocks; ++kb) {
-                    if (PREP > 0 && (kb & 3) == 0) {
-                        // this CTA's 128 rows of A and of W in K group kb / 4: written by prep warps somewhere
-                        // in the grid; their release/our acquire orders the data, the proxy fence orders the
-                        // TMA loads (async proxy) behind it
-                        const uint32_t *fa_ = fp.flags + (m0 >> 7) * fp.G + (kb >> 2);
-                        const uint32_t *fw_ = fp.flags + (fp.PA + (n0 >> 7)) * fp.G + (kb >> 2);
-                        if (!flag_wait_bounded(fa_, 4u * PREP, abort_flag, TC_WAIT_LIMIT_NS) ||
-                            !flag_wait_bounded(fw_, (uint32_t)PREP, abort_flag, TC_WAIT_LIMIT_NS)) {
-                            timed_out = true;
-                            break;
-                        }
-                        asm volatile("fence.proxy.async.global;" ::: "memory");
-                    }
                     if (!ptx::mbar_wait_bounded_cluster(empty_bar(s), ph ^ 1u, abort_flag, TC_WAIT_LIMIT_NS)) {
                         timed_out = true;
                         break;
@@ -253,43 +149,6 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             }
         }
         __syncwarp();
-    } else if (PREP > 0 && warp >= TC_THREADS / 32) {
-        // ---- operand preparation (see FusedPrep): never waits ----
-        const int pw = warp - TC_THREADS / 32;
-        const int c1 = fp.PA * 4 + fp.W0;                    // units per K group in the first part of the list
-        const int n1 = fp.G * c1;
-        const int total = n1 + (fp.PW - fp.W0) * fp.G;
-        for (int i = blockIdx.x; i < total; i += gridDim.x) {
-            int g, panel, sub = 0;
-            bool is_a = false;
-            if (i < n1) {
-                g = i / c1;
-                const int u = i - g * c1;
-                if (u < fp.PA * 4) { is_a = true; panel = u >> 2; sub = u & 3; }
-                else panel = u - fp.PA * 4;
-            } else {
-                const int j = i - n1;
-                panel = fp.W0 + j / fp.G;
-                g = j - (j / fp.G) * fp.G;
-            }
-            const int k0 = g * PREP_KG;
-            if (is_a) {
-                const int r0 = panel * 128 + sub * 32;
-                const int rows = min(32, p.M - r0);
-                if (rows > 0) {
-                    if (fp.x_bf16) quantize_unit<__nv_bfloat16>(fp, p.K, r0, rows, k0, pw, PREP);
-                    else quantize_unit<float>(fp, p.K, r0, rows, k0, pw, PREP);
-                }
-            } else {
-                if (fp.ww <= 4) decode_unit<true>(fp, p.N, p.K, panel * 128, k0, pw, PREP, lane);
-                else decode_unit<false>(fp, p.N, p.K, panel * 128, k0, pw, PREP, lane);
-            }
-            __syncwarp();
-            if (lane == 0) {
-                __threadfence();                                // release: the warp's stores before the count
-                atomicAdd(fp.flags + (is_a ? panel : fp.PA + panel) * fp.G + g, 1u);
-            }
-        }
     } else {
         const int quad = warp & 3;
         int it = 0;

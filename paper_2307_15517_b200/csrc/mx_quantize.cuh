@@ -502,14 +502,6 @@ cast_rows_kernel(const uint8_t *__restrict__ mant_in, const uint8_t *__restrict_
     }
 }
 
-// Zeroes `n` words (the progress counters of the product kernel that prepares its own operands).
-__global__ void __launch_bounds__(1024) clear_words_kernel(uint32_t *__restrict__ words, int n)
-{
-    ptx::dep_wait();
-    ptx::dep_trigger();
-    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) words[i] = 0u;
-}
-
 // Several tensors in one launch (the distinct activation tensors of a grouped decode call):
 // blockIdx.y selects the tensor, blockIdx.x strides over its rows.
 struct QuantJob {

@@ -38,7 +38,6 @@ struct DeviceInfo {
     bool tc_attr_set[2][4] = {{false, false, false, false}, {false, false, false, false}};
     bool stream_attr_set[4] = {false, false, false, false};
     bool tc2_attr_set = false;
-    bool tc2p_attr_set = false;
     bool tcx_attr_set = false;
 };
 DeviceInfo g_dev[MAX_DEVICES];
@@ -52,7 +51,7 @@ EncodeTiledFn g_encode_tiled = nullptr;
 
 // ---- launch profile: CUDA events around every kernel launch, summed per kernel kind ----------
 enum KernelKind { KIND_QUANTIZE = 0, KIND_DEQUANTIZE = 1, KIND_GEMM_TC = 2, KIND_GEMM_SIMT = 3,
-                  KIND_GEMM_STREAM = 4, KIND_PREP = 5, KIND_COUNT = MX_KERNEL_KINDS };
+                  KIND_GEMM_STREAM = 4, KIND_PREP = 5, KIND_GLUE = 6, KIND_COUNT = MX_KERNEL_KINDS };
 struct ProfEntry { cudaEvent_t a, b; int kind; };
 struct Profiler {
     bool on = false;
@@ -441,14 +440,9 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     return MX_OK;
 }
 
-// The CTA-pair kernel: 256 x 256 tiles, one product per launch.  With `prep` the kernel also
-// prepares its own operands (PREP_WARPS extra warps per CTA, see mx::FusedPrep) and the whole grid of
-// one CTA per SM is launched whatever the number of tiles; the progress counters are zeroed by a
-// small launch in front of it.
-constexpr int PREP_WARPS = 8;
+// The CTA-pair kernel: 256 x 256 tiles, one product per launch.
 mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N, int64_t K,
-                       const float *bias, float *y, int64_t ldy, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st,
-                       mx::FusedPrep *prep = nullptr)
+                       const float *bias, float *y, int64_t ldy, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
 {
     using Cfg = mx::Tc2Cfg;
     CUtensorMap tm_a, tm_w;
@@ -462,8 +456,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
     }
-    s = prep ? smem_attr_once(d.tc2p_attr_set, mx::gemm_tc2_kernel<PREP_WARPS>, (int)Cfg::SMEM_BYTES)
-             : smem_attr_once(d.tc2_attr_set, mx::gemm_tc2_kernel<0>, (int)Cfg::SMEM_BYTES);
+    s = smem_attr_once(d.tc2_attr_set, mx::gemm_tc2_kernel, (int)Cfg::SMEM_BYTES);
     if (s != MX_OK) return s;
     mx::TcParams p{};
     p.y = y;
@@ -483,28 +476,9 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     p.yq_bits = yq ? yq->f.elem_bits : 0;
     p.yq_block = yq ? yq->f.block : 0;
     const int tiles = p.tiles_m * p.tiles_n;
-    if (prep) {
-        const int pairs = d.sm_count / 2;
-        prep->PA = 2 * p.tiles_m;
-        prep->PW = 2 * p.tiles_n;
-        prep->G = (int)(K / mx::PREP_KG);
-        const int w0 = 2 * ((pairs - 1) / p.tiles_m + 1);
-        prep->W0 = w0 < prep->PW ? w0 : prep->PW;
-        const int n_flags = (prep->PA + prep->PW) * prep->G;
-        {
-            ProfScope prof(KIND_PREP, st);
-            MX_CUDA(launch_dep(mx::clear_words_kernel, dim3(1), dim3(1024), 0, st, prep->flags, n_flags));
-        }
-        ProfScope prof(KIND_GEMM_TC, st);
-        MX_CUDA(launch_dep(mx::gemm_tc2_kernel<PREP_WARPS>, dim3(2 * pairs), dim3(mx::TC_THREADS + 32 * PREP_WARPS),
-                           Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p, *prep));
-        MX_CUDA(cudaGetLastError());
-        return MX_OK;
-    }
     const int pairs = tiles < d.sm_count / 2 ? tiles : d.sm_count / 2;
-    const mx::FusedPrep none{};
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::gemm_tc2_kernel<0>, dim3(2 * pairs), dim3(mx::TC_THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p, none));
+    MX_CUDA(launch_dep(mx::gemm_tc2_kernel, dim3(2 * pairs), dim3(mx::TC_THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -562,11 +536,13 @@ mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64
                    const QuantizedOut *yq = nullptr, const TcBatch &tb = TcBatch())
 {
     const PackedW none;
-    // More than one wave of 256 x 256 tiles: CTA pairs (a third less shared-memory traffic per flop; from
-    // +2 % on 2048 x 6144 x 2048 to +14 % on 8192^3).  With at most one tile per pair the one-CTA kernel
-    // starts faster and wins.
+    // CTA pairs (a third less shared-memory traffic per flop) when there is more than one wave of 256 x 256
+    // tiles (+2 % on 2048 x 6144 x 2048, +14 % on 8192^3), or one nearly full wave of long tiles (K >= 4096:
+    // 2048 x 2048 x 8192 runs in 49.5 instead of 56.5 us); a short single wave starts faster on the one-CTA
+    // kernel (2048^3: 19.7 against 22.4 us).
     const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
-    if (tb.count == 1 && M > 128 && pair_tiles > d.sm_count / 2)
+    const int pairs = d.sm_count / 2;
+    if (tb.count == 1 && M > 128 && (pair_tiles > pairs || (K >= 4096 && 4 * pair_tiles >= 3 * pairs)))
         return launch_tc2(a_hat, w_hat, M, N, K, bias, y, ldy, yq, d, st);
     const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256) * tb.count;
     if (N > 128 && tiles256 >= (int64_t)d.sm_count * 3 / 4)
@@ -607,41 +583,8 @@ size_t tc_operand_bytes(int64_t M, int64_t N, int64_t K)
 {
     return round256((size_t)M * K * 2) + round256((size_t)N * K * 2);
 }
-// progress counters of the kernel that prepares its own operands: one per (128-row panel, 256 k)
-size_t prep_flag_bytes(int64_t M, int64_t N, int64_t K)
-{
-    return round256((size_t)(2 * ((M + 255) / 256) + 2 * ((N + 255) / 256)) * (size_t)((K + 255) / 256) * 4);
-}
-size_t tc_workspace(int64_t M, int64_t N, int64_t K) { return tc_operand_bytes(M, N, K) + prep_flag_bytes(M, N, K); }
+size_t tc_workspace(int64_t M, int64_t N, int64_t K) { return tc_operand_bytes(M, N, K); }
 
-// mx_linear's operands can be prepared inside the product kernel when the shape fits its unit grid
-// (whole K groups, one-row blocks, at least one pair tile each way) ...
-bool fused_prep_fits(const mx_linear_args_t &a)
-{
-    return (a.K % mx::PREP_KG) == 0 && a.M >= 256 && a.N >= 256 && a.fa.block_rows == 1 && a.fw.block_rows == 1;
-}
-// ... and MX_ALGO_AUTO does so when the layer is large enough for a full grid of CTAs to pay.
-bool fused_prep_pays(const mx_linear_args_t &a) { return a.M >= 512 && a.N >= 512 && (double)a.M * a.N * a.K >= 4e9; }
-
-// The product of one layer with the operand preparation inside the kernel.
-mx_status_t run_linear_fused(const mx_linear_args_t &a, uint8_t *ws, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
-{
-    __nv_bfloat16 *a_hat = reinterpret_cast<__nv_bfloat16 *>(ws);
-    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)a.M * a.K * 2));
-    mx::FusedPrep fp{};
-    fp.x = a.x;
-    fp.ldx = a.ldx;
-    fp.x_bf16 = a.dt == MX_BF16 ? 1 : 0;
-    fp.wa = a.fa.elem_bits;
-    fp.ww = a.fw.elem_bits;
-    fp.block = a.fa.block;
-    fp.a_hat = a_hat;
-    fp.w_mant = static_cast<const uint8_t *>(a.w_mant);
-    fp.w_exp = a.w_exp;
-    fp.w_hat = w_hat;
-    fp.flags = reinterpret_cast<uint32_t *>(ws + tc_operand_bytes(a.M, a.N, a.K));
-    return launch_tc2(a_hat, w_hat, a.M, a.N, a.K, a.bias, a.y, a.ldy, yq, d, st, &fp);
-}
 size_t fused_workspace(int64_t M, int64_t K) { return round256((size_t)M * K * 2); }
 size_t packed_workspace(int64_t M, int64_t K, const mx_format_t &fa)
 {
@@ -1027,7 +970,6 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     mx_linear_args_t one;
     one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
     one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = ldy;
-    const bool explicit_algo = algo != MX_ALGO_AUTO;
     if (algo == MX_ALGO_AUTO)
         algo = (stream_layer_ok(one) && (reinterpret_cast<uintptr_t>(w_exp) & 3u) == 0) ? MX_ALGO_STREAM
                                                                                      : MX_ALGO_TCGEN05;
@@ -1068,8 +1010,6 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
         return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st, perm);
     }
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
-    if (algo == MX_ALGO_TCGEN05 && fused_prep_fits(one) && (explicit_algo || fused_prep_pays(one)))
-        return run_linear_fused(one, ws, nullptr, *d, st);
     s = tc_prepare(one, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
     if (algo == MX_ALGO_TCGEN05_BLOCKWISE) return launch_tcx(a_hat, w_hat, M, N, K, fa.block, bias, y, ldy, *d, st);
@@ -1158,7 +1098,6 @@ mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int6
     yq.exps = y_exp;
     yq.nonfinite = nonfinite_count;
     yq.f = fy;
-    if (fused_prep_fits(one) && fused_prep_pays(one)) return run_linear_fused(one, ws, &yq, *d, st);
     s = tc_prepare(one, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
     return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq);
@@ -1399,6 +1338,7 @@ mx_status_t mx_layernorm(const float *x, int64_t ldx, const float *gamma, const 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int per = (int)((cols + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);
     const unsigned g = (unsigned)rows;
+    ProfScope prof(KIND_GLUE, st);
     if (per <= 4) mx::layernorm_kernel<4><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
     else if (per <= 8) mx::layernorm_kernel<8><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
     else if (per <= 16) mx::layernorm_kernel<16><<<g, mx::GLUE_THREADS, 0, st>>>(x, ldx, gamma, beta, eps, (int)cols, y, ldy);
@@ -1421,6 +1361,7 @@ mx_status_t mx_softmax(float *s_inout, int64_t ld, int64_t rows, int64_t cols, f
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int per = (int)((cols + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);
     const unsigned g = (unsigned)rows;
+    ProfScope prof(KIND_GLUE, st);
     if (per <= 4) mx::softmax_kernel<4><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
     else if (per <= 8) mx::softmax_kernel<8><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
     else if (per <= 16) mx::softmax_kernel<16><<<g, mx::GLUE_THREADS, 0, st>>>(s_inout, ld, (int)cols, scale, causal, rows_per_batch);
@@ -1446,6 +1387,7 @@ mx_status_t mx_softmax_q(const float *s_in, int64_t ld, int64_t rows, int64_t co
     const int per8 = (int)((cols / 8 + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);      // 1..4
     const unsigned g = (unsigned)rows;
     uint8_t *pm = static_cast<uint8_t *>(p_mant);
+    ProfScope prof(KIND_GLUE, st);
 #define MX_SOFTMAX_Q(P8)                                                                                         \
     do {                                                                                                         \
         if (fp.block == 16)                                                                                      \
@@ -1473,6 +1415,7 @@ mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int
     mx_status_t s = device_info(&d);
     if (s != MX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    ProfScope prof(KIND_GLUE, st);
     mx::relu_add_kernel<<<grid_for((n + 3) / 4, mx::GLUE_THREADS, d->sm_count, 8), mx::GLUE_THREADS, 0, st>>>(a, b, y, n, relu);
     MX_CUDA(cudaGetLastError());
     return MX_OK;

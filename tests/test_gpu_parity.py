@@ -403,15 +403,15 @@ def test_linear_in_kernel_weight_decode(mxb, case):
 @pytest.mark.parametrize("case", [
     # B, wa, ww, M, K, N, bf16 input
     (16, 8, 4, 700, 768, 1100, False),      # ragged M and N: partly filled panels and tiles
-    (32, 4, 8, 300, 1024, 520, True),       # int8 weight container, bf16 activations, block 32
+    (32, 4, 4, 300, 1024, 520, True),       # bf16 activations, block 32
+    (32, 4, 8, 300, 1024, 520, True),       # int8 weight container
     (16, 6, 3, 1500, 256, 2600, False),     # a single K group, more tiles than CTA pairs
     (32, 8, 4, 2304, 2048, 640, False),     # more activation panels than the first wave covers
 ])
-def test_linear_with_operands_prepared_inside_the_product_kernel(mxb, case):
-    """mx_linear with MX_ALGO_TCGEN05 on shapes the pair kernel can prepare for itself (K % 256 == 0,
-    M, N >= 256): extra warps quantize the activations and decode the weights while the tiles run;
-    every output against the oracle, with zero, tiny, huge and non-finite weight blocks, a bias and
-    canary columns."""
+def test_linear_tensor_core_ragged_shapes_and_edge_blocks(mxb, case):
+    """mx_linear with MX_ALGO_TCGEN05 on shapes with ragged tiles both ways (one-CTA and CTA-pair
+    kernels, both weight containers, bf16 and fp32 activations): every output against the oracle, with
+    zero, tiny, huge and non-finite weight blocks, a bias and canary columns."""
     B, wa, ww, M, K, N, bf16 = case
     x = synth.student_t_activations(M, K, seed=wa + 3)
     if bf16:
@@ -436,7 +436,7 @@ def test_linear_with_operands_prepared_inside_the_product_kernel(mxb, case):
     err = np.abs(y.astype(np.float64) - y_ref.astype(np.float64))
     assert (err[ok] <= (TOL * S + 1e-37)[ok]).all(), float((err[ok] / np.maximum(S[ok], 1e-300)).max())
     assert (ypad[:, N:] == -77.0).all()
-    # a second call into the same workspace-sized buffers (counters cleared again) gives the same bits
+    # a second call into a caller-provided workspace gives the same bits
     ws = mxb.alloc_workspace(mxb.mx_workspace_bytes(M, N, K, fa, fw))
     wm, we = _dev(orc.pack(qw, ww)), _dev(ew)
     y1 = mxb.mx_linear(x.cuda(), fa, wm, we, fw, N, bias=_dev(bias), workspace=ws, algo=mxb.MX_ALGO_TCGEN05).clone()

@@ -495,6 +495,7 @@ def run_ours(args):
     flops_step = sum(layer_flops(tokens, L["spec"]) for L in layers)
     h2d = sum(L["x_host"].numel() * 4 for L in layers)
     d2h = sum(L["y_host"].numel() * 4 for L in layers)
+    d2h_q = sum(L["yq_mant_host"].numel() + L["yq_exp_host"].numel() for L in layers)
     layer_list = [[L["spec"].name, L["spec"].K, L["spec"].N] for L in layers]
     counter = [0]
 
@@ -623,7 +624,6 @@ def run_ours(args):
         value = aggregate_tops(world, flops_step, args.steps, ms_total)
         e2e_value = aggregate_tops(world, flops_step, args.steps, ms_e2e)
         e2e_q_value = aggregate_tops(world, flops_step, args.steps, ms_e2e_q)
-        d2h_q = sum(L["yq_mant_host"].numel() + L["yq_exp_host"].numel() for L in layers)
         gemm_ms, gemm_n = prof["gemm_tc"]
         achieved = flops_step * args.steps / (gemm_ms * 1e-3) / 1e12 if gemm_ms > 0 else 0.0
         peak = peaks["bf16_tflops"]          # burst figure: the timed region lasts well under a second

@@ -338,3 +338,196 @@ int mxo_threads(void) { return omp_get_max_threads(); }
 #else
 int mxo_threads(void) { return 1; }
 #endif
+
+/* ==================================================================================================
+ * The two other MX formats of Sec. 2 "What are MX Formats?": Block Minifloat (BMF) and Block
+ * Logarithm (BL).  The paper describes them in words only -- BMF "shares the exponent bias in a
+ * block", BL "strips out the mantissa and shares the exponent bias, resulting in values that are
+ * always powers of two" -- and compares them with MXInt in Table 1 and Fig. 5.  Readings taken here
+ * (none is fixed by the paper: "parity unpinned" for all of them; pinned by the worked blocks and
+ * invariants in tests/test_oracle_pins.py):
+ *
+ *   element  = sign bit, ebits-bit exponent field F (0 .. Fmax = 2^ebits - 1), mbits-bit mantissa T
+ *              (BL: mbits = 0); one byte per element: code = sign << (ebits+mbits) | F << mbits | T
+ *   block    = B consecutive elements along k share one byte: the shared bias, stored as beta + 127
+ *              where 2^beta is the binade of the top exponent field (0: zero/subnormal block,
+ *              255: the block holds Inf/NaN and decodes to NaN) -- "sharing the exponent bias":
+ *              an element's exponent is F - (Fmax - beta)
+ *   BMF value: F >= 1: (-1)^s * 2^(beta - (Fmax - F)) * (1 + T / 2^mbits)
+ *              F == 0: (-1)^s * 2^(beta - (Fmax - 1)) * (T / 2^mbits)          (gradual underflow)
+ *              beta = floor(log2(max |x|)); rounding to nearest, ties to even on the element's own
+ *              grid, carries into the next binade, saturation at the largest code
+ *   BL value : F >= 1: (-1)^s * 2^(beta - (Fmax - F)); F == 0: zero
+ *              rounding in the log domain: |x| in [2^k, 2^(k+1)) goes to 2^(k+1) iff |x| >= sqrt(2) 2^k;
+ *              beta = that rounded exponent of max |x|; below half a binade under the smallest
+ *              power the value flushes to zero
+ *   tiny     : a block whose maximum is below 2^-95 (shared byte < 32) is stored as a zero block
+ *              (shared byte 0, which decodes to zeros whatever the codes): every decoded element of
+ *              every other block then lies inside the range of bf16, so the formats decode to bf16
+ *              exactly (at most 6 significant bits, exponent >= -133)
+ *   limits   : BMF 1 + ebits + mbits <= 8, ebits <= 5;  BL ebits <= 5
+ * ================================================================================================== */
+#define MXO_KIND_BMF 1
+#define MXO_KIND_BL 2
+
+static int mxo_alt_args_ok(int kind, int64_t rows, int64_t K, int B, int ebits, int mbits)
+{
+    if (rows < 0 || K < 0 || B <= 0 || (K % B) != 0) return 0;
+    if (kind == MXO_KIND_BMF) return ebits >= 1 && ebits <= 5 && mbits >= 1 && 1 + ebits + mbits <= 8;
+    if (kind == MXO_KIND_BL) return ebits >= 1 && ebits <= 5 && mbits == 0;
+    return 0;
+}
+
+/* round(log2(a)) for a finite a > 0: the exponent of the nearest power of two in the log domain. */
+static int mxo_round_log2(double a)
+{
+    int ex;
+    const double f = 2.0 * frexp(a, &ex);     /* a = f * 2^(ex-1), f in [1, 2) */
+    /* f >= sqrt(2)  <=>  f*f >= 2; f has at most 24 significant bits, so f*f is exact in double */
+    return (ex - 1) + (f * f >= 2.0 ? 1 : 0);
+}
+
+/* Magnitude code (F << mbits | T) of |x| = a on the BMF grid whose top field Fmax sits at 2^beta. */
+static int mxo_bmf_code(double a, int beta, int ebits, int mbits)
+{
+    const int fmax = (1 << ebits) - 1;
+    const int top = (fmax << mbits) | ((1 << mbits) - 1);
+    if (a == 0.0) return 0;
+    /* t = a in units of the subnormal step 2^(beta - (fmax - 1) - mbits): exact scaling */
+    const double t = ldexp(a, -(beta - (fmax - 1) - mbits));
+    double code;
+    if (t < (double)(1 << mbits)) {
+        code = nearbyint(t);                    /* F = 0 (a carry lands on F = 1, T = 0 by itself) */
+    } else {
+        int ex;
+        (void)frexp(t, &ex);                    /* t in [2^(ex-1), 2^ex) */
+        const int j = (ex - 1) - mbits;         /* binade above the subnormal range: F = j + 1 */
+        const double sig = nearbyint(ldexp(t, -j));            /* in [2^mbits, 2^(mbits+1)] */
+        code = (double)((j + 1) << mbits) + (sig - (double)(1 << mbits));  /* carry rolls into F */
+    }
+    if (code > (double)top) code = (double)top;
+    return (int)code;
+}
+
+/*
+ * x (rows x K, row stride ldx) -> one code byte per element, one shared byte per block of B along k.
+ * kind 1: BMF(ebits, mbits), kind 2: BL(ebits).  nonfinite (nullable) counts blocks holding Inf/NaN.
+ */
+int mxo_alt_quantize(const float *x, int64_t rows, int64_t K, int64_t ldx, int kind, int B, int ebits,
+                     int mbits, uint8_t *codes, uint8_t *shared, uint32_t *nonfinite)
+{
+    if (!mxo_alt_args_ok(kind, rows, K, B, ebits, mbits)) return MXO_BAD_ARG;
+    const int64_t nb = K / B;
+    const int fmax = (1 << ebits) - 1;
+    uint32_t bad = 0;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t b = 0; b < nb; ++b) {
+            const float *xb = x + r * ldx + b * B;
+            uint8_t *cb = codes + r * K + b * B;
+            float amax = 0.0f;
+            int any_nonfinite = 0;
+            for (int k = 0; k < B; ++k) {
+                if (isnan(xb[k]) || isinf(xb[k])) any_nonfinite = 1;
+                if (fabsf(xb[k]) > amax) amax = fabsf(xb[k]);
+            }
+            if (any_nonfinite) {
+                shared[r * nb + b] = 255;
+                memset(cb, 0, (size_t)B);
+                ++bad;
+                continue;
+            }
+            int sb = mxo_exponent_byte(amax);                  /* floor(log2 amax) + 127, 0 for zero/subnormal */
+            if (kind == MXO_KIND_BL && sb > 0) {
+                sb = mxo_round_log2((double)amax) + 127;
+                if (sb > 254) sb = 254;
+            }
+            if (sb < 32) {                                     /* zero, subnormal or tiny block */
+                shared[r * nb + b] = 0;
+                memset(cb, 0, (size_t)B);
+                continue;
+            }
+            shared[r * nb + b] = (uint8_t)sb;
+            const int beta = sb - 127;
+            for (int k = 0; k < B; ++k) {
+                const double a = fabs((double)xb[k]);
+                const int sign = signbit(xb[k]) ? 1 : 0;
+                int mag;
+                if (kind == MXO_KIND_BMF) {
+                    mag = mxo_bmf_code(a, beta, ebits, mbits);
+                } else if (a == 0.0) {
+                    mag = 0;
+                } else {
+                    int f = mxo_round_log2(a) - beta + fmax;
+                    mag = f > fmax ? fmax : (f < 1 ? 0 : f);
+                }
+                cb[k] = (uint8_t)((sign << (ebits + mbits)) | mag);
+            }
+        }
+    if (nonfinite) *nonfinite = bad;
+    return MXO_OK;
+}
+
+/* Decoded value of one code under a shared byte. */
+static double mxo_alt_value(int kind, int code, int sb, int ebits, int mbits)
+{
+    if (sb == 255) return (double)NAN;
+    if (sb == 0) return 0.0;
+    const int fmax = (1 << ebits) - 1, beta = sb - 127;
+    const int sign = (code >> (ebits + mbits)) & 1;
+    const int f = (code >> mbits) & fmax, t = code & ((1 << mbits) - 1);
+    double v;
+    if (kind == MXO_KIND_BMF)
+        v = f >= 1 ? ldexp(1.0 + ldexp((double)t, -mbits), beta - (fmax - f))
+                   : ldexp(ldexp((double)t, -mbits), beta - (fmax - 1));
+    else
+        v = f >= 1 ? ldexp(1.0, beta - (fmax - f)) : 0.0;
+    return sign ? -v : v;
+}
+
+int mxo_alt_dequantize(const uint8_t *codes, const uint8_t *shared, int64_t rows, int64_t K, int kind,
+                       int B, int ebits, int mbits, double *xhat)
+{
+    if (!mxo_alt_args_ok(kind, rows, K, B, ebits, mbits)) return MXO_BAD_ARG;
+    const int64_t nb = K / B;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k)
+            xhat[r * K + k] = mxo_alt_value(kind, codes[r * K + k], shared[r * nb + k / B], ebits, mbits);
+    return MXO_OK;
+}
+
+/*
+ * Y = A W^T (+ bias) for operands in BMF or BL (Sec. 3.2, software emulator: the plain floating-point
+ * operator on the dequantized values): every product of two decoded values is exact in double, the
+ * products are summed in long double and rounded to fp32 once.  S = sum of |products| (+ |bias|).
+ * An operand block with shared byte 255 makes the outputs it touches NaN.
+ */
+int mxo_alt_gemm(const uint8_t *ac, const uint8_t *as, int akind, int aeb, int amb, const uint8_t *wc,
+                 const uint8_t *ws, int wkind, int web, int wmb, int64_t M, int64_t N, int64_t K, int B,
+                 const float *bias, float *y_ref, double *S)
+{
+    if (!mxo_alt_args_ok(akind, M, K, B, aeb, amb) || !mxo_alt_args_ok(wkind, N, K, B, web, wmb))
+        return MXO_BAD_ARG;
+    const int64_t nb = K / B;
+#pragma omp parallel for schedule(static)
+    for (int64_t i = 0; i < M; ++i)
+        for (int64_t j = 0; j < N; ++j) {
+            long double wide = 0.0L;
+            double sabs = 0.0;
+            int poisoned = 0;
+            for (int64_t k = 0; k < K; ++k) {
+                const int sa = as[i * nb + k / B], sw = ws[j * nb + k / B];
+                if (sa == 255 || sw == 255) { poisoned = 1; continue; }
+                const double t = mxo_alt_value(akind, ac[i * K + k], sa, aeb, amb) *
+                                 mxo_alt_value(wkind, wc[j * K + k], sw, web, wmb);
+                wide += (long double)t;
+                sabs += fabs(t);
+            }
+            if (bias) {
+                wide += (long double)bias[j];
+                sabs += fabs((double)bias[j]);
+            }
+            y_ref[i * N + j] = poisoned ? NAN : (float)wide;
+            if (S) S[i * N + j] = poisoned ? (double)NAN : sabs;
+        }
+    return MXO_OK;
+}

@@ -50,6 +50,9 @@ def lib():
         L.mxo_quantize_2d.argtypes = [p, i64, i64, i64, i64, i32, i32, i32, p, p, p]
         L.mxo_expand_exponent_rows.argtypes = [p, i64, i64, i32, p]
         L.mxo_cast.argtypes = [p, p, i64, i64, i32, i32, i32, i32, p, p, p]
+        L.mxo_alt_quantize.argtypes = [p, i64, i64, i64, i32, i32, i32, i32, p, p, p]
+        L.mxo_alt_dequantize.argtypes = [p, p, i64, i64, i32, i32, i32, i32, p]
+        L.mxo_alt_gemm.argtypes = [p, p, i32, i32, i32, p, p, i32, i32, i32, i64, i64, i64, i32, p, p, p]
         L.mxo_format_bits.argtypes = [i32, i32, i32, i32]
         L.mxo_format_bits.restype = C.c_double
         L.mxo_threads.restype = i32
@@ -203,6 +206,48 @@ def gemm_samples(qa, ea, wa: int, qw, ew, ww: int, block: int, si, sj, bias=None
                                   block, _ptr(bias), _ptr(si), _ptr(sj), n, _ptr(y_ref),
                                   _ptr(y_seq), _ptr(S)))
     return y_ref, y_seq, S
+
+
+KIND_BMF, KIND_BL = 1, 2
+
+
+def alt_quantize(x, kind: int, block: int, ebits: int, mbits: int = 0):
+    """Block Minifloat (kind 1) / Block Logarithm (kind 2) quantizer.  x: float32 [rows, K].
+    Returns (codes uint8 [rows, K], shared bytes uint8 [rows, K/B], nonfinite)."""
+    x = np.ascontiguousarray(x, np.float32)
+    rows, K = x.shape
+    codes = np.zeros((rows, K), np.uint8)
+    shared = np.zeros((rows, K // block), np.uint8)
+    bad = C.c_uint32(0)
+    _check(lib().mxo_alt_quantize(_ptr(x), rows, K, K, kind, block, ebits, mbits, _ptr(codes), _ptr(shared),
+                                  C.addressof(bad)))
+    return codes, shared, int(bad.value)
+
+
+def alt_dequantize(codes, shared, kind: int, block: int, ebits: int, mbits: int = 0):
+    codes = np.ascontiguousarray(codes, np.uint8)
+    shared = np.ascontiguousarray(shared, np.uint8)
+    rows, K = codes.shape
+    out = np.zeros((rows, K), np.float64)
+    _check(lib().mxo_alt_dequantize(_ptr(codes), _ptr(shared), rows, K, kind, block, ebits, mbits, _ptr(out)))
+    return out
+
+
+def alt_gemm(ac, ash, afmt, wc, wsh, wfmt, block: int, bias=None):
+    """afmt / wfmt = (kind, ebits, mbits).  Returns (y_ref fp32 [M,N], S fp64 [M,N])."""
+    ac = np.ascontiguousarray(ac, np.uint8)
+    wc = np.ascontiguousarray(wc, np.uint8)
+    ash = np.ascontiguousarray(ash, np.uint8)
+    wsh = np.ascontiguousarray(wsh, np.uint8)
+    M, K = ac.shape
+    N = wc.shape[0]
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, np.float32)
+    y = np.zeros((M, N), np.float32)
+    S = np.zeros((M, N), np.float64)
+    _check(lib().mxo_alt_gemm(_ptr(ac), _ptr(ash), afmt[0], afmt[1], afmt[2], _ptr(wc), _ptr(wsh), wfmt[0],
+                              wfmt[1], wfmt[2], M, N, K, block, _ptr(bias), _ptr(y), _ptr(S)))
+    return y, S
 
 
 def format_bits(block: int, w: int, block_rows: int = 1, exp_bits: int = 8) -> float:

@@ -559,3 +559,134 @@ def test_narrowing_cast_error_bound_and_nonfinite():
     assert (np.abs(xout - xin)[ok] <= step[ok]).all()
     free = ok & (np.abs(qo) < 3)
     assert (np.abs(xout - xin)[free] <= 0.5 * step[free]).all()
+
+
+# ------------------------------------------------------------------------------ Block Minifloat / Block Logarithm
+
+ALT_FORMATS = [(orc.KIND_BMF, 4, 3), (orc.KIND_BMF, 2, 5), (orc.KIND_BMF, 5, 2), (orc.KIND_BMF, 3, 2),
+               (orc.KIND_BL, 4, 0), (orc.KIND_BL, 3, 0), (orc.KIND_BL, 5, 0)]
+
+
+def test_alt_formats_hand_worked_blocks():
+    """The pencil-worked BMF / BL blocks of the fixture: shared byte, code bytes and decoded values."""
+    rows = [r for r in golden_io.load() if r["kind"] == "alt"]
+    assert len(rows) == 4
+    for r in rows:
+        kind, eb, mb, B = (orc.KIND_BMF if r["fmt"] == "bmf" else orc.KIND_BL), int(r["ebits"]), int(r["mbits"]), int(r["block"])
+        x = np.zeros((1, B), np.float32)
+        vals = golden_io.floats(r["x"])
+        x[0, :len(vals)] = vals
+        codes, shared, bad = orc.alt_quantize(x, kind, B, eb, mb)
+        assert bad == 0 and shared[0, 0] == int(r["shared"]), r["id"]
+        want = [int(t, 16) for t in r["codes"].split(",")]
+        assert list(codes[0, :len(want)]) == want, r["id"]
+        assert (codes[0, len(want):] == 0).all()
+        xhat = orc.alt_dequantize(codes, shared, kind, B, eb, mb)
+        assert list(xhat[0, :len(want)]) == golden_io.floats(r["xhat"]), r["id"]
+
+
+@pytest.mark.parametrize("fmt", ALT_FORMATS)
+def test_alt_formats_invariants(fmt):
+    kind, eb, mb = fmt
+    B = 16
+    rng = np.random.default_rng(10 * eb + mb + kind)
+    x = (rng.standard_normal((40, 8 * B)) * np.exp2(rng.integers(-12, 12, (40, 1)))).astype(np.float32)
+    x[3, :B] = 0.0
+    x[4, 5] = np.inf
+    x[5, B + 2] = np.nan
+    x[6, :B] = (rng.standard_normal(B) * 2.0 ** -110).astype(np.float32)        # below 2^-95: a zero block
+    codes, shared, bad = orc.alt_quantize(x, kind, B, eb, mb)
+    xh = orc.alt_dequantize(codes, shared, kind, B, eb, mb)
+    fmax = 2 ** eb - 1
+    assert bad == 2 and shared[4, 0] == 255 and shared[5, 1] == 255 and np.isnan(xh[4, :B]).all()
+    assert shared[3, 0] == 0 and shared[6, 0] == 0 and (xh[3, :B] == 0).all() and (xh[6, :B] == 0).all()
+    assert (codes >> (1 + eb + mb) == 0).all()                      # unused high bits stay clear
+    ok = np.ones_like(x, bool)
+    ok[4, :B] = ok[5, B:2 * B] = ok[3, :B] = ok[6, :B] = False
+    amax = np.abs(np.where(ok, x, 0)).reshape(40, 8, B).max(axis=2)
+    live = amax > 0
+    live[4, 0] = live[5, 1] = False
+    # shared byte: exponent of the block maximum (BMF: frexp; BL: nearest power of two in the log domain)
+    mant, ex = np.frexp(amax[live].astype(np.float64))
+    if kind == orc.KIND_BMF:
+        assert (shared[live] == ex - 1 + 127).all()
+    else:
+        up = (2 * mant) ** 2 >= 2.0
+        assert (shared[live] == ex - 1 + up + 127).all()
+    beta = np.repeat(shared.astype(np.int64) - 127, B, axis=1)
+    a, ah = np.abs(x.astype(np.float64)), np.abs(xh)
+    assert (np.sign(xh[ok]) * np.sign(x[ok]) >= 0).all()            # signs survive (zero may appear)
+    assert (ah[ok] <= np.exp2(beta[ok] + 1.0)).all()                # the shared byte bounds the block's range
+    top = np.exp2(beta.astype(np.float64))
+    if kind == orc.KIND_BMF:
+        lo = top * 2.0 ** -(fmax - 1)                               # smallest normal binade of the block
+        normal = ok & (a >= lo) & (a < top * (2 - 2.0 ** -mb))      # not saturated, not subnormal
+        assert (np.abs(ah - a)[normal] <= a[normal] * 2.0 ** -(mb + 1)).all()      # half an ulp of mb+1 bits
+        sub = ok & (a < lo)
+        assert (np.abs(ah - a)[sub] <= (lo * 2.0 ** -(mb + 1))[sub]).all()          # half a subnormal step
+        # decoded values carry at most mb + 1 significant bits
+        m, _ = np.frexp(ah[ok])
+        assert (np.ldexp(m, mb + 1) % 1 == 0).all()
+    else:
+        kept = ok & (ah > 0) & (a < top)
+        ratio = ah[kept] / a[kept]
+        assert (ratio <= 2 ** 0.5 * (1 + 1e-12)).all() and (ratio >= 2 ** -0.5 * (1 - 1e-12)).all()
+        assert (np.log2(ah[ok & (ah > 0)]) % 1 == 0).all()          # always a power of two
+        flushed = ok & (ah == 0) & (a > 0)
+        assert (a[flushed] < (top * 2.0 ** -(fmax - 1) * 2 ** -0.5 * (1 + 1e-12))[flushed]).all()
+    # every decoded value is a bf16 number: its binary32 image has 16 zero low bits
+    f32 = xh[ok].astype(np.float32)
+    assert (f32.astype(np.float64) == xh[ok]).all() and (f32.view(np.uint32) & 0xFFFF == 0).all()
+    # idempotence: the decoded tensor quantizes to the same codes and shared bytes
+    c2, s2, _ = orc.alt_quantize(np.where(np.isnan(xh), 0, xh).astype(np.float32), kind, B, eb, mb)
+    good_rows = [r for r in range(40) if r not in (4, 5)]
+    assert np.array_equal(c2[good_rows], codes[good_rows]) and np.array_equal(s2[good_rows], shared[good_rows])
+    # sign symmetry
+    c3, s3, _ = orc.alt_quantize(np.where(np.isfinite(x), -x, x).astype(np.float32), kind, B, eb, mb)
+    assert np.array_equal(s3, shared) and np.array_equal(c3 & (2 ** (eb + mb) - 1), codes & (2 ** (eb + mb) - 1))
+
+
+@pytest.mark.parametrize("mb", (2, 3, 5))
+def test_bmf_top_binade_is_the_mxint_grid(mb):
+    """Inside the binade of the block maximum a minifloat with mb mantissa bits and MXInt of width
+    mb + 2 have the same grid (step 2^(E - mb)) and the same rounding: the two quantizers, pinned
+    separately, must decode to the same values there."""
+    B = 16
+    rng = np.random.default_rng(mb)
+    x = (rng.uniform(1.0, 2.0, (30, 4 * B)) * rng.choice([-1.0, 1.0], (30, 4 * B)) *
+         np.exp2(rng.integers(-6, 6, (30, 1)))).astype(np.float32)
+    codes, shared, _ = orc.alt_quantize(x, orc.KIND_BMF, B, 8 - 1 - mb if mb >= 3 else 4, mb)
+    eb = 8 - 1 - mb if mb >= 3 else 4
+    q, e, _ = orc.quantize(x, B, mb + 2)
+    assert np.array_equal(shared, e)
+    assert np.array_equal(orc.alt_dequantize(codes, shared, orc.KIND_BMF, B, eb, mb), orc.dequantize(q, e, B, mb + 2))
+
+
+def test_alt_gemm_is_the_fp64_matmul_of_the_decoded_values():
+    """Emulator form of Sec. 3.2 on BMF / BL operands: the product of the decoded tensors, summed exactly
+    (numpy float64 holds every product and every sum of these few terms exactly), rounded to fp32 once."""
+    B, M, N, K = 16, 9, 11, 64
+    rng = np.random.default_rng(5)
+    a = rng.standard_normal((M, K)).astype(np.float32)
+    w = (rng.standard_normal((N, K)) * 0.05).astype(np.float32)
+    bias = rng.standard_normal(N).astype(np.float32)
+    for afmt, wfmt in (((orc.KIND_BMF, 4, 3), (orc.KIND_BMF, 4, 3)), ((orc.KIND_BMF, 3, 4), (orc.KIND_BL, 4, 0)),
+                       ((orc.KIND_BL, 5, 0), (orc.KIND_BL, 3, 0))):
+        ac, ash, _ = orc.alt_quantize(a, afmt[0], B, afmt[1], afmt[2])
+        wc, wsh, _ = orc.alt_quantize(w, wfmt[0], B, wfmt[1], wfmt[2])
+        y, S = orc.alt_gemm(ac, ash, afmt, wc, wsh, wfmt, B, bias=bias)
+        ah = orc.alt_dequantize(ac, ash, afmt[0], B, afmt[1], afmt[2])
+        wh = orc.alt_dequantize(wc, wsh, wfmt[0], B, wfmt[1], wfmt[2])
+        # exact reference with Python fractions
+        from fractions import Fraction
+        for i in (0, 4, 8):
+            for j in (0, 5, 10):
+                exact = sum(Fraction(float(ah[i, k])) * Fraction(float(wh[j, k])) for k in range(K)) + Fraction(float(bias[j]))
+                assert abs(Fraction(float(y[i, j])) - exact) <= Fraction(float(np.spacing(np.float32(abs(float(exact)))))) / 2
+                assert abs(S[i, j] - float(sum(abs(Fraction(float(ah[i, k])) * Fraction(float(wh[j, k]))) for k in range(K))
+                                           + abs(Fraction(float(bias[j]))))) <= 1e-12 * S[i, j]
+        assert np.allclose(y, (ah @ wh.T + bias).astype(np.float32), rtol=1e-6, atol=1e-6)
+    wsh2 = wsh.copy()
+    wsh2[2, 1] = 255
+    y, S = orc.alt_gemm(ac, ash, afmt, wc, wsh2, wfmt, B)
+    assert np.isnan(y[:, 2]).all() and not np.isnan(np.delete(y, 2, axis=1)).any()

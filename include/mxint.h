@@ -344,6 +344,60 @@ MX_API mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t 
                         uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
                         size_t workspace_bytes, void *stream);
 
+/* ---- the other MX formats of the paper: Block Minifloat and Block Logarithm ---------------------
+ *
+ * Sec. 2 "What are MX Formats?" puts two more block formats beside MXInt and Table 1 / Fig. 5 compare
+ * them: Block Minifloat (BMF) "shares the exponent bias in a block" -- every element is a small
+ * floating-point number --, Block Logarithm (BL) "strips out the mantissa and shares the exponent
+ * bias", so every value is a power of two.  The paper gives no bit-level definition; this library's
+ * reading (stated in full because results depend on it):
+ *   element : one byte, sign << (elem_exp_bits + elem_man_bits) | F << elem_man_bits | T
+ *             (F = exponent field, 0 .. Fmax = 2^elem_exp_bits - 1; T = mantissa; BL: elem_man_bits = 0)
+ *   shared  : one byte per `block` consecutive elements along K = 127 + beta, 2^beta being the binade
+ *             of the top field Fmax; 0 = zero block (decodes to zeros whatever the codes),
+ *             255 = the block holds Inf/NaN (codes 0, decodes to NaN)
+ *   BMF     : F >= 1: (-1)^s 2^(beta-(Fmax-F)) (1 + T / 2^man);  F == 0: (-1)^s 2^(beta-(Fmax-1)) T / 2^man;
+ *             beta = floor(log2 max|x|); round to nearest even on the element's own grid, carries into
+ *             the next binade, saturation at the largest code
+ *   BL      : F >= 1: (-1)^s 2^(beta-(Fmax-F));  F == 0: zero;  rounding in the log domain (a value
+ *             goes to the next power of two iff its significand is >= sqrt(2)), beta = the rounded
+ *             exponent of max|x|; more than half a binade below the smallest power flushes to zero
+ *   a block whose maximum is below 2^-95 is stored as a zero block, so that every decoded element
+ *   is exactly a bf16 number and the formats can feed the bf16 tensor-core product without loss
+ *   limits  : block 16 or 32;  BMF 1 + exp + man <= 8, exp <= 5, man >= 1;  BL exp <= 5
+ * Average bits per value: 8 / block + 1 + elem_exp_bits + elem_man_bits (the analogue of Eq. 1).
+ */
+typedef enum { MX_ELEM_BMF = 1, MX_ELEM_BL = 2 } mx_elem_kind_t;
+typedef struct {
+    int32_t kind;           /* mx_elem_kind_t                                                  */
+    int32_t block;          /* 16 or 32 elements along K share one bias byte                   */
+    int32_t elem_exp_bits;  /* exponent bits of an element                                     */
+    int32_t elem_man_bits;  /* mantissa bits of an element (0 for MX_ELEM_BL)                  */
+} mx_alt_format_t;
+
+/* x ([rows, K] of `dt`, leading dimension ldx elements, ldx % 8 == 0, K % block == 0) -> codes (device,
+ * uint8 [rows, K], 16-byte aligned) and shared bytes (device, uint8 [rows, K/block]).
+ * nonfinite_count (device, nullable) is incremented once per block holding Inf/NaN. */
+MX_API mx_status_t mx_alt_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, int64_t ldx,
+                                   mx_alt_format_t f, uint8_t *codes, uint8_t *shared,
+                                   uint32_t *nonfinite_count, void *stream);
+
+/* Inverse map: out[r*ld_out + k] = decoded value as `dt` (exact in fp32 and in bf16); ld_out % 8 == 0. */
+MX_API mx_status_t mx_alt_dequantize(const uint8_t *codes, const uint8_t *shared, int64_t rows, int64_t K,
+                                     mx_alt_format_t f, void *out, mx_dtype_t dt, int64_t ld_out,
+                                     void *stream);
+
+/* Y[M,N] = A[M,K] W[N,K]^T (+ bias) on operands in BMF or BL (kinds and bit splits may differ, the
+ * block sizes must be equal): Sec. 3.2's emulated operator -- the floating-point product of the
+ * decoded values -- on the tensor-core kernels of mx_gemm, fp32 accumulation.  Workspace:
+ * mx_alt_gemm_workspace_bytes (both operands as bf16), 256-byte aligned.  Tolerance as for mx_gemm
+ * with S = sum_k |a_k w_k|.  Other conventions as for mx_gemm. */
+MX_API size_t mx_alt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+MX_API mx_status_t mx_alt_gemm(const uint8_t *a_codes, const uint8_t *a_shared, mx_alt_format_t fa,
+                               const uint8_t *w_codes, const uint8_t *w_shared, mx_alt_format_t fw,
+                               int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                               void *workspace, size_t workspace_bytes, void *stream);
+
 /* ---- product for callers that cannot allocate (the paper has no counterpart) -----------------
  *
  * Some callers of this library have no way to obtain device memory at the point where they

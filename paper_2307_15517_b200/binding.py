@@ -37,6 +37,18 @@ class MxFormat(C.Structure):
         return "MxFormat(block=%d, elem_bits=%d, block_rows=%d)" % (self.block, self.elem_bits, self.block_rows)
 
 
+class MxAltFormat(C.Structure):
+    """A Block Minifloat (kind 1) or Block Logarithm (kind 2) format: mirrors ``mx_alt_format_t``."""
+    _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("elem_exp_bits", C.c_int32),
+                ("elem_man_bits", C.c_int32)]
+
+    def __init__(self, kind: int, block: int, elem_exp_bits: int, elem_man_bits: int = 0):
+        super().__init__(kind, block, elem_exp_bits, elem_man_bits)
+
+
+MX_ELEM_BMF, MX_ELEM_BL = 1, 2
+
+
 class MxLinearArgs(C.Structure):
     """One layer of ``mx_linear_grouped`` (mirrors ``mx_linear_args_t``)."""
     _fields_ = [("x", C.c_void_p), ("dt", C.c_int), ("M", C.c_int64), ("K", C.c_int64),
@@ -106,6 +118,14 @@ def _load() -> C.CDLL:
     L.mx_linear_grouped.restype = i32
     L.mx_gemm_static.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp]
     L.mx_gemm_static.restype = i32
+    A = MxAltFormat
+    L.mx_alt_quantize.argtypes = [vp, i32, i64, i64, i64, A, vp, vp, vp, vp]
+    L.mx_alt_dequantize.argtypes = [vp, vp, i64, i64, A, vp, i32, i64, vp]
+    L.mx_alt_gemm_workspace_bytes.argtypes = [i64, i64, i64]
+    L.mx_alt_gemm_workspace_bytes.restype = sz
+    L.mx_alt_gemm.argtypes = [vp, vp, A, vp, vp, A, i64, i64, i64, vp, vp, i64, vp, sz, vp]
+    for name in ("mx_alt_quantize", "mx_alt_dequantize", "mx_alt_gemm"):
+        getattr(L, name).restype = i32
     L.mx_profile_begin.argtypes = []
     L.mx_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
@@ -384,6 +404,44 @@ def mx_relu_add(a: torch.Tensor, b: Optional[torch.Tensor], y: Optional[torch.Te
         y = torch.empty_like(a)
     _check(lib.mx_relu_add(_ptr(a), _ptr(b), _ptr(y), a.numel(), 1 if relu else 0, _stream(stream)),
            "mx_relu_add")
+    return y
+
+
+def mx_alt_quantize(x: torch.Tensor, f: MxAltFormat, nonfinite_count: Optional[torch.Tensor] = None, stream=None):
+    """x: [rows, K] fp32/bf16, rows contiguous.  Returns (codes uint8 [rows, K], shared uint8 [rows, K/block])."""
+    _need_cuda(x, nonfinite_count)
+    assert x.dim() == 2 and x.stride(1) == 1
+    rows, K = x.shape
+    codes = torch.empty((rows, K), dtype=torch.uint8, device=x.device)
+    shared = torch.empty((rows, K // f.block), dtype=torch.uint8, device=x.device)
+    _check(lib.mx_alt_quantize(_ptr(x), _dtype_code(x), rows, K, x.stride(0), f, _ptr(codes), _ptr(shared),
+                               _ptr(nonfinite_count), _stream(stream)), "mx_alt_quantize")
+    return codes, shared
+
+
+def mx_alt_dequantize(codes: torch.Tensor, shared: torch.Tensor, f: MxAltFormat, dtype=torch.float32, stream=None):
+    _need_cuda(codes, shared)
+    rows, K = codes.shape
+    out = torch.empty((rows, K), dtype=dtype, device=codes.device)
+    _check(lib.mx_alt_dequantize(_ptr(codes), _ptr(shared), rows, K, f, _ptr(out), _dtype_code(out), K,
+                                 _stream(stream)), "mx_alt_dequantize")
+    return out
+
+
+def mx_alt_gemm(a_codes, a_shared, fa: MxAltFormat, w_codes, w_shared, fw: MxAltFormat,
+                bias: Optional[torch.Tensor] = None, y: Optional[torch.Tensor] = None,
+                workspace: Optional[torch.Tensor] = None, stream=None):
+    """Y = A W^T on Block Minifloat / Block Logarithm operands (codes [M, K] and [N, K])."""
+    _need_cuda(a_codes, a_shared, w_codes, w_shared, bias, y, workspace)
+    M, K = a_codes.shape
+    N = w_codes.shape[0]
+    if y is None:
+        y = torch.empty((M, N), dtype=torch.float32, device=a_codes.device)
+    if workspace is None:
+        workspace = alloc_workspace(int(lib.mx_alt_gemm_workspace_bytes(M, N, K)), a_codes.device)
+    _check(lib.mx_alt_gemm(_ptr(a_codes), _ptr(a_shared), fa, _ptr(w_codes), _ptr(w_shared), fw, M, N, K,
+                           _ptr(bias), _ptr(y), y.stride(0), _ptr(workspace), workspace.numel(), _stream(stream)),
+           "mx_alt_gemm")
     return y
 
 

@@ -13,6 +13,7 @@
 #include <vector>
 
 #include "../../include/mxint.h"
+#include "mx_alt.cuh"
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
 #include "mx_gemm_tc2.cuh"
@@ -1419,6 +1420,111 @@ mx_status_t mx_relu_add(const float *a, const float *b, float *y, int64_t n, int
     mx::relu_add_kernel<<<grid_for((n + 3) / 4, mx::GLUE_THREADS, d->sm_count, 8), mx::GLUE_THREADS, 0, st>>>(a, b, y, n, relu);
     MX_CUDA(cudaGetLastError());
     return MX_OK;
+}
+
+// ---- Block Minifloat / Block Logarithm ---------------------------------------------------------
+static bool alt_format_ok(const mx_alt_format_t &f)
+{
+    if (f.block != 16 && f.block != 32) return false;
+    if (f.kind == MX_ELEM_BMF)
+        return f.elem_exp_bits >= 1 && f.elem_exp_bits <= 5 && f.elem_man_bits >= 1 &&
+               1 + f.elem_exp_bits + f.elem_man_bits <= 8;
+    if (f.kind == MX_ELEM_BL) return f.elem_exp_bits >= 1 && f.elem_exp_bits <= 5 && f.elem_man_bits == 0;
+    return false;
+}
+static mx::AltFormat alt_of(const mx_alt_format_t &f)
+{
+    return mx::AltFormat{f.kind, f.block, f.elem_exp_bits, f.elem_man_bits};
+}
+
+mx_status_t mx_alt_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, int64_t ldx, mx_alt_format_t f,
+                            uint8_t *codes, uint8_t *shared, uint32_t *nonfinite_count, void *stream)
+{
+    if (!alt_format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || ldx < K) return MX_ERR_SHAPE;
+    if (rows == 0 || K == 0) return MX_OK;
+    if (!x || !codes || !shared) return MX_ERR_NULL;
+    if (!aligned16(x) || !aligned16(codes) || (ldx % 8) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int64_t items = rows * ((K / 8 + 31) / 32);
+    const int grid = grid_for(items * 32, 256, d->sm_count, 8);
+    const mx::AltFormat af = alt_of(f);
+    ProfScope prof(KIND_QUANTIZE, st);
+    if (dt == MX_F32) {
+        const float *xf = static_cast<const float *>(x);
+        if (f.block == 16) MX_CUDA(launch_dep(mx::alt_quantize_kernel<float, 16>, dim3(grid), dim3(256), 0, st, xf, rows, K, ldx, af, codes, shared, nonfinite_count));
+        else MX_CUDA(launch_dep(mx::alt_quantize_kernel<float, 32>, dim3(grid), dim3(256), 0, st, xf, rows, K, ldx, af, codes, shared, nonfinite_count));
+    } else {
+        const __nv_bfloat16 *xb = static_cast<const __nv_bfloat16 *>(x);
+        if (f.block == 16) MX_CUDA(launch_dep(mx::alt_quantize_kernel<__nv_bfloat16, 16>, dim3(grid), dim3(256), 0, st, xb, rows, K, ldx, af, codes, shared, nonfinite_count));
+        else MX_CUDA(launch_dep(mx::alt_quantize_kernel<__nv_bfloat16, 32>, dim3(grid), dim3(256), 0, st, xb, rows, K, ldx, af, codes, shared, nonfinite_count));
+    }
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+static mx_status_t alt_decode_any(const uint8_t *codes, const uint8_t *shared, int64_t rows, int64_t K,
+                                  const mx_alt_format_t &f, void *out, mx_dtype_t dt, int64_t ld_out, DeviceInfo &d,
+                                  cudaStream_t st)
+{
+    const int grid = grid_for(rows * (K / 8), 256, d.sm_count, 8);
+    const mx::AltFormat af = alt_of(f);
+    ProfScope prof(KIND_DEQUANTIZE, st);
+    if (dt == MX_F32)
+        MX_CUDA(launch_dep(mx::alt_decode_kernel<float>, dim3(grid), dim3(256), 0, st, codes, shared, rows, K, af,
+                           static_cast<float *>(out), ld_out));
+    else
+        MX_CUDA(launch_dep(mx::alt_decode_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, codes, shared, rows, K, af,
+                           static_cast<__nv_bfloat16 *>(out), ld_out));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_alt_dequantize(const uint8_t *codes, const uint8_t *shared, int64_t rows, int64_t K, mx_alt_format_t f,
+                              void *out, mx_dtype_t dt, int64_t ld_out, void *stream)
+{
+    if (!codes || !shared || !out) return MX_ERR_NULL;
+    if (!alt_format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f.block) != 0 || ld_out < K) return MX_ERR_SHAPE;
+    if (!aligned16(codes) || !aligned16(out) || (ld_out % 8) != 0) return MX_ERR_ALIGN;
+    if (rows == 0 || K == 0) return MX_OK;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    return alt_decode_any(codes, shared, rows, K, f, out, dt, ld_out, *d, static_cast<cudaStream_t>(stream));
+}
+
+size_t mx_alt_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return 0;
+    return tc_operand_bytes(M, N, K);
+}
+
+mx_status_t mx_alt_gemm(const uint8_t *a_codes, const uint8_t *a_shared, mx_alt_format_t fa, const uint8_t *w_codes,
+                        const uint8_t *w_shared, mx_alt_format_t fw, int64_t M, int64_t N, int64_t K, const float *bias,
+                        float *y, int64_t ldy, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!a_codes || !a_shared || !w_codes || !w_shared || !y) return MX_ERR_NULL;
+    if (!alt_format_ok(fa) || !alt_format_ok(fw) || fa.block != fw.block) return MX_ERR_FORMAT;
+    if (M <= 0 || N <= 0 || K <= 0 || (K % fa.block) != 0 || ldy < N) return MX_ERR_SHAPE;
+    if (M > INT32_MAX / 2 || N > INT32_MAX / 2 || K > INT32_MAX / 2) return MX_ERR_SHAPE;
+    if (!aligned16(a_codes) || !aligned16(w_codes) || !aligned16(y) || (bias && !aligned16(bias))) return MX_ERR_ALIGN;
+    if (!workspace || workspace_bytes < tc_operand_bytes(M, N, K)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
+    __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + round256((size_t)M * K * 2));
+    s = alt_decode_any(a_codes, a_shared, M, K, fa, a_hat, MX_BF16, K, *d, st);
+    if (s != MX_OK) return s;
+    s = alt_decode_any(w_codes, w_shared, N, K, fw, w_hat, MX_BF16, K, *d, st);
+    if (s != MX_OK) return s;
+    return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
 }
 
 // ---- product without any allocation ---------------------------------------------------------

@@ -151,6 +151,45 @@ int mxo_unpack(const uint8_t *in, int64_t rows, int64_t K, int w, int8_t *q)
     return MXO_OK;
 }
 
+/*
+ * Dense storage (Eq. 1: a value costs its m mantissa bits plus the sign bit, nothing more): element k
+ * of a row occupies bits [k*w, (k+1)*w) of the row's bit stream, two's complement, bit b of the stream
+ * being bit (b % 8) of byte b / 8.  A row of K elements takes K*w/8 bytes (K % 8 == 0).
+ */
+int mxo_pack_dense(const int8_t *q, int64_t rows, int64_t K, int w, uint8_t *out)
+{
+    if (w < 2 || w > 8 || rows < 0 || K < 0 || (K % 8) != 0) return MXO_BAD_ARG;
+    const int64_t row_bytes = K * w / 8;
+    memset(out, 0, (size_t)(rows * row_bytes));
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            const unsigned field = (unsigned)q[r * K + k] & ((1u << w) - 1u);
+            for (int b = 0; b < w; ++b)
+                if ((field >> b) & 1u) {
+                    const int64_t bit = k * w + b;
+                    out[r * row_bytes + bit / 8] |= (uint8_t)(1u << (bit % 8));
+                }
+        }
+    return MXO_OK;
+}
+
+int mxo_unpack_dense(const uint8_t *in, int64_t rows, int64_t K, int w, int8_t *q)
+{
+    if (w < 2 || w > 8 || rows < 0 || K < 0 || (K % 8) != 0) return MXO_BAD_ARG;
+    const int64_t row_bytes = K * w / 8;
+    for (int64_t r = 0; r < rows; ++r)
+        for (int64_t k = 0; k < K; ++k) {
+            int field = 0;
+            for (int b = 0; b < w; ++b) {
+                const int64_t bit = k * w + b;
+                if ((in[r * row_bytes + bit / 8] >> (bit % 8)) & 1) field |= 1 << b;
+            }
+            if (field & (1 << (w - 1))) field -= 1 << w;      /* sign extension */
+            q[r * K + k] = (int8_t)field;
+        }
+    return MXO_OK;
+}
+
 /* One output element: wide reference, sequential-fp32 variant and condition scale. */
 static void mxo_dot(const int8_t *qa, const uint8_t *ea, int wa, const int8_t *qw,
                     const uint8_t *ew, int ww, int64_t K, int B, const float *bias_j,

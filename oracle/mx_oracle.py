@@ -42,6 +42,8 @@ def lib():
         L.mxo_dequantize.argtypes = [p, p, i64, i64, i32, i32, p]
         L.mxo_pack.argtypes = [p, i64, i64, i32, p]
         L.mxo_unpack.argtypes = [p, i64, i64, i32, p]
+        L.mxo_pack_dense.argtypes = [p, i64, i64, i32, p]
+        L.mxo_unpack_dense.argtypes = [p, i64, i64, i32, p]
         L.mxo_gemm.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, p, p, p]
         L.mxo_gemm_samples.argtypes = [p, p, i32, p, p, i32, i64, i64, i64, i32, p, p, p, i64,
                                        p, p, p]
@@ -134,6 +136,23 @@ def pack(q, w: int):
     out = np.zeros((rows, K // 2 if w <= 4 else K), np.uint8)
     _check(lib().mxo_pack(_ptr(q), rows, K, w, _ptr(out)))
     return out
+
+
+def pack_dense(q, w: int):
+    """w bits per element, K*w/8 bytes per row (the storage Eq. 1 counts)."""
+    q = np.ascontiguousarray(q, np.int8)
+    rows, K = q.shape
+    out = np.zeros((rows, K * w // 8), np.uint8)
+    _check(lib().mxo_pack_dense(_ptr(q), rows, K, w, _ptr(out)))
+    return out
+
+
+def unpack_dense(packed, K: int, w: int):
+    packed = np.ascontiguousarray(packed, np.uint8)
+    rows = packed.shape[0]
+    q = np.zeros((rows, K), np.int8)
+    _check(lib().mxo_unpack_dense(_ptr(packed), rows, K, w, _ptr(q)))
+    return q
 
 
 def unpack(packed, K: int, w: int):

@@ -690,3 +690,32 @@ def test_alt_gemm_is_the_fp64_matmul_of_the_decoded_values():
     wsh2[2, 1] = 255
     y, S = orc.alt_gemm(ac, ash, afmt, wc, wsh2, wfmt, B)
     assert np.isnan(y[:, 2]).all() and not np.isnan(np.delete(y, 2, axis=1)).any()
+
+
+# ------------------------------------------------------------------------------ dense storage
+
+def test_dense_packing_hand_worked_and_eq1():
+    rows = [r for r in golden_io.load() if r["kind"] == "dense"]
+    assert len(rows) == 4
+    for r in rows:
+        w, q = int(r["w"]), np.array([golden_io.ints(r["q"])], np.int8)
+        img = orc.pack_dense(q, w)
+        assert [int(t, 16) for t in r["bytes"].split(",")] == list(img[0]), r
+        assert np.array_equal(orc.unpack_dense(img, q.shape[1], w), q)
+    rng = np.random.default_rng(8)
+    for w in range(2, 9):
+        K, B = 96, 32
+        q = rng.integers(-(2 ** (w - 1)), 2 ** (w - 1), (7, K)).astype(np.int8)
+        img = orc.pack_dense(q, w)
+        # Eq. 1: bits per value = exponent share + m + 1; the mantissa part is exactly w = m + 1 bits
+        assert img.shape[1] * 8 == K * w
+        assert abs((img.shape[1] * 8 + 8 * (K // B)) / K - orc.format_bits(B, w)) < 1e-12
+        assert np.array_equal(orc.unpack_dense(img, K, w), q)
+        # an independent construction: numpy bit arrays, little-endian within bytes
+        bits = ((q.astype(np.int64)[:, :, None] >> np.arange(w)) & 1).reshape(7, K * w).astype(np.uint8)
+        assert np.array_equal(np.packbits(bits, axis=1, bitorder="little"), img)
+    # the 4- and 8-bit widths coincide with the containers
+    q4 = rng.integers(-8, 8, (3, 32)).astype(np.int8)
+    assert np.array_equal(orc.pack_dense(q4, 4), orc.pack(q4, 4))
+    q8 = rng.integers(-128, 128, (3, 32)).astype(np.int8)
+    assert np.array_equal(orc.pack_dense(q8, 8), orc.pack(q8, 8))

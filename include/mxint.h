@@ -108,7 +108,18 @@ typedef struct {
     int32_t elem_bits;  /* w = 2..8, sign included (paper m = w - 1)                           */
     int32_t exp_bits;   /* 8 (the paper fixes the shared exponent to 8 bits)                   */
     int32_t block_rows; /* 1, or 2: two adjacent rows share their exponents, the paper's (16,2) */
+    int32_t packing;    /* 0: container (below); 1: dense, elem_bits bits per element (Eq. 1)      */
 } mx_format_t;
+
+/* Dense storage (packing == 1): Eq. 1 charges a value m + 1 bits, so a row of K mantissas takes
+ * K * elem_bits / 8 bytes: element k sits in bits [k*w, (k+1)*w) of the row's bit stream, two's
+ * complement, stream bit b being bit b % 8 of byte b / 8 (for w = 4 and w = 8 this IS the container).
+ * It is the form for tensors at rest -- weights: mx_pack_dense converts a quantized tensor into it,
+ * mx_unpack_dense back, mx_mant_bytes gives its size, and mx_dequantize, mx_gemm(_ex) with the
+ * tensor-core kernels, mx_gemm_q and the weight operand of mx_linear(_ex) / mx_linear_q read it
+ * directly.  Everything else (the quantizer's output, casts, the CUDA-core, streaming, in-kernel
+ * decode, batched, grouped and static entry points, activation and result formats) takes the
+ * container only and answers MX_ERR_FORMAT to packing == 1. */
 
 /* Two-row blocks (block_rows == 2; Sec. 4.1 and Fig. 2: the paper's unified block shape is
  * (16,2), "block size 32"): `block` consecutive elements along K times two adjacent rows (2r and
@@ -137,6 +148,14 @@ MX_API size_t mx_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_format_t fa
 /* The same for an explicitly named kernel (0 for an unknown algo or a bad format). */
 MX_API size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw,
                                     mx_algo_t algo);
+
+/* Container <-> dense storage of the mantissas of a [rows, K] tensor (the exponent array is the same
+ * for both).  `f` names widths and block; its packing field is ignored.  Both arrays are device
+ * memory, the container 16-byte aligned. */
+MX_API mx_status_t mx_pack_dense(const void *mant, int64_t rows, int64_t K, mx_format_t f, void *dense_out,
+                                 void *stream);
+MX_API mx_status_t mx_unpack_dense(const void *dense, int64_t rows, int64_t K, mx_format_t f, void *mant_out,
+                                   void *stream);
 
 MX_API const char *mx_status_string(mx_status_t s);
 

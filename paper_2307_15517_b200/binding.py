@@ -28,13 +28,18 @@ STATUS_NAMES = {0: "MX_OK", -1: "MX_ERR_NULL", -2: "MX_ERR_SHAPE", -3: "MX_ERR_F
 class MxFormat(C.Structure):
     """The (B, e, m) tuple of the paper's Sec. 4.1 with w = m + 1 (sign included)."""
     _fields_ = [("block", C.c_int32), ("elem_bits", C.c_int32), ("exp_bits", C.c_int32),
-                ("block_rows", C.c_int32)]
+                ("block_rows", C.c_int32), ("packing", C.c_int32)]
 
-    def __init__(self, block: int = 16, elem_bits: int = 4, exp_bits: int = 8, block_rows: int = 1):
-        super().__init__(block, elem_bits, exp_bits, block_rows)
+    def __init__(self, block: int = 16, elem_bits: int = 4, exp_bits: int = 8, block_rows: int = 1, packing: int = 0):
+        super().__init__(block, elem_bits, exp_bits, block_rows, packing)
+
+    def dense(self) -> "MxFormat":
+        """The same format with dense storage of the mantissas (elem_bits bits per element)."""
+        return MxFormat(self.block, self.elem_bits, self.exp_bits, self.block_rows, 1)
 
     def __repr__(self):
-        return "MxFormat(block=%d, elem_bits=%d, block_rows=%d)" % (self.block, self.elem_bits, self.block_rows)
+        return "MxFormat(block=%d, elem_bits=%d, block_rows=%d, packing=%d)" % (self.block, self.elem_bits,
+                                                                                  self.block_rows, self.packing)
 
 
 class MxAltFormat(C.Structure):
@@ -88,6 +93,10 @@ def _load() -> C.CDLL:
     L.mx_last_cuda_error.restype = C.c_char_p
     L.mx_quantize.argtypes = [vp, i32, i64, i64, i64, i64, F, vp, vp, vp, vp]
     L.mx_dequantize.argtypes = [vp, vp, i64, i64, F, vp, i32, i64, vp]
+    L.mx_pack_dense.argtypes = [vp, i64, i64, F, vp, vp]
+    L.mx_unpack_dense.argtypes = [vp, i64, i64, F, vp, vp]
+    L.mx_pack_dense.restype = i32
+    L.mx_unpack_dense.restype = i32
     L.mx_cast.argtypes = [vp, vp, F, i64, i64, F, vp, vp, vp, vp]
     L.mx_cast.restype = i32
     L.mx_gemm.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, vp, vp, i64, vp, sz, vp]
@@ -225,6 +234,23 @@ def mx_quantize(x: torch.Tensor, f: MxFormat, mant_out: Optional[torch.Tensor] =
                            _ptr(mant_out), _ptr(exp_out), _ptr(nonfinite_count), _stream(stream)),
            "mx_quantize")
     return mant_out, exp_out
+
+
+def mx_pack_dense(mant: torch.Tensor, K: int, f: MxFormat, stream=None) -> torch.Tensor:
+    """Container mantissas [rows, K/2 or K] -> dense storage [rows, K * elem_bits / 8]."""
+    _need_cuda(mant)
+    rows = mant.shape[0]
+    out = torch.empty((rows, K * f.elem_bits // 8), dtype=torch.uint8, device=mant.device)
+    _check(lib.mx_pack_dense(_ptr(mant), rows, K, f, _ptr(out), _stream(stream)), "mx_pack_dense")
+    return out
+
+
+def mx_unpack_dense(dense: torch.Tensor, K: int, f: MxFormat, stream=None) -> torch.Tensor:
+    _need_cuda(dense)
+    rows = dense.shape[0]
+    out = torch.empty((rows, K // 2 if f.elem_bits <= 4 else K), dtype=torch.uint8, device=dense.device)
+    _check(lib.mx_unpack_dense(_ptr(dense), rows, K, f, _ptr(out), _stream(stream)), "mx_unpack_dense")
+    return out
 
 
 def mx_cast(mant: torch.Tensor, exps: torch.Tensor, K: int, f_in: MxFormat, f_out: MxFormat,

@@ -825,6 +825,112 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
                                      (int64_t)gridDim.x * (blockDim.x >> 5));
 }
 
+// ---- dense storage: w bits per element (Eq. 1 counts m + 1 bits per value) ---------------------
+// Element k of a row sits in bits [k*w, (k+1)*w) of the row's bit stream (two's complement; stream
+// bit b = bit b % 8 of byte b / 8); a row takes K*w/8 bytes.  Eight consecutive elements are exactly w
+// bytes, which is a thread's unit in the three kernels below (byte loads and stores: w = 3, 5, 6 leave
+// no wider alignment).
+
+// The 8*w bits of eight elements starting at byte address p.
+__device__ __forceinline__ uint64_t dense_load8(const uint8_t *p, int w)
+{
+    uint64_t v = 0;
+    for (int i = 0; i < w; ++i) v |= (uint64_t)__ldg(p + i) << (8 * i);
+    return v;
+}
+__device__ __forceinline__ int dense_field(uint64_t v, int i, int w)
+{
+    const int f = (int)((v >> (i * w)) & ((1u << w) - 1u));
+    return (f << (32 - w)) >> (32 - w);                         // sign extension
+}
+
+// container (nibbles for w <= 4, int8 above) -> dense
+__global__ void __launch_bounds__(256)
+dense_pack_kernel(const uint8_t *__restrict__ mant, int64_t rows, int64_t K, int w, uint8_t *__restrict__ dense)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int64_t cpr = K >> 3, total = rows * cpr;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = t / cpr, kc = t - row * cpr;
+        int q[8];
+        if (w <= 4) {
+            const uint32_t p = __ldg(reinterpret_cast<const uint32_t *>(mant + row * (K >> 1) + kc * 4));
+#pragma unroll
+            for (int i = 0; i < 8; ++i) q[i] = ((int)(p << (28 - 4 * i))) >> 28;
+        } else {
+            const uint2 p = __ldg(reinterpret_cast<const uint2 *>(mant + row * K + kc * 8));
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                q[i] = ((int)(p.x << (24 - 8 * i))) >> 24;
+                q[4 + i] = ((int)(p.y << (24 - 8 * i))) >> 24;
+            }
+        }
+        uint64_t v = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v |= (uint64_t)((uint32_t)q[i] & ((1u << w) - 1u)) << (i * w);
+        uint8_t *dst = dense + row * (K * w / 8) + kc * w;
+        for (int i = 0; i < w; ++i) dst[i] = (uint8_t)(v >> (8 * i));
+    }
+}
+
+// dense -> container
+__global__ void __launch_bounds__(256)
+dense_unpack_kernel(const uint8_t *__restrict__ dense, int64_t rows, int64_t K, int w, uint8_t *__restrict__ mant)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int64_t cpr = K >> 3, total = rows * cpr;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = t / cpr, kc = t - row * cpr;
+        const uint64_t v = dense_load8(dense + row * (K * w / 8) + kc * w, w);
+        if (w <= 4) {
+            uint32_t p = 0;
+#pragma unroll
+            for (int i = 0; i < 8; ++i) p |= ((uint32_t)dense_field(v, i, w) & 0xFu) << (4 * i);
+            *reinterpret_cast<uint32_t *>(mant + row * (K >> 1) + kc * 4) = p;
+        } else {
+            uint2 p = make_uint2(0, 0);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                p.x |= ((uint32_t)dense_field(v, i, w) & 0xFFu) << (8 * i);
+                p.y |= ((uint32_t)dense_field(v, 4 + i, w) & 0xFFu) << (8 * i);
+            }
+            *reinterpret_cast<uint2 *>(mant + row * K + kc * 8) = p;
+        }
+    }
+}
+
+// dense mantissas + exponent bytes -> decoded values (fp32, or bf16: the MMA operand form), 8 per thread
+template <typename OutT>
+__global__ void __launch_bounds__(256)
+dequantize_dense_kernel(const uint8_t *__restrict__ dense, const uint8_t *__restrict__ exps, int64_t rows, int64_t K,
+                        int block, int w, int exp_row_shift, OutT *__restrict__ out, int64_t ld_out)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int64_t cpr = K >> 3, total = rows * cpr, nb_row = K / block;
+    const int exp_shift = block == 16 ? 1 : 2;
+    for (int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; t < total; t += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t row = t / cpr, kc = t - row * cpr;
+        const uint64_t v = dense_load8(dense + row * (K * w / 8) + kc * w, w);
+        const int ebyte = __ldg(exps + (row >> exp_row_shift) * nb_row + (kc >> exp_shift));
+        float f[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) f[i] = decode_value(dense_field(v, i, w), ebyte, w);
+        OutT *o = out + row * ld_out + kc * 8;
+        if constexpr (sizeof(OutT) == 4) {
+            reinterpret_cast<float4 *>(o)[0] = make_float4(f[0], f[1], f[2], f[3]);
+            reinterpret_cast<float4 *>(o)[1] = make_float4(f[4], f[5], f[6], f[7]);
+        } else {
+            uint32_t h[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) h[i] = as_u32(__floats2bfloat162_rn(f[2 * i], f[2 * i + 1]));
+            *reinterpret_cast<uint4 *>(o) = make_uint4(h[0], h[1], h[2], h[3]);
+        }
+    }
+}
+
 // Both operands of the tensor-core product in one launch: the first `q_blocks` CTAs quantize the
 // activations straight to their exact bf16 operand form, the remaining CTAs decode the packed
 // weights to theirs.  Two HBM-bound passes overlap instead of queueing behind each other.

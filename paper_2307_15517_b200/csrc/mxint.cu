@@ -125,10 +125,17 @@ mx_status_t device_info(DeviceInfo **out)
 }
 
 // block_rows == 2: two adjacent rows share the exponents (the paper's (16,2) block shape).
-bool format_ok(const mx_format_t &f)
+// Either storage form of the mantissas ...
+bool format_ok_any(const mx_format_t &f)
 {
     return (f.block == 16 || f.block == 32) && f.elem_bits >= 2 && f.elem_bits <= 8 &&
-           f.exp_bits == 8 && (f.block_rows == 1 || f.block_rows == 2);
+           f.exp_bits == 8 && (f.block_rows == 1 || f.block_rows == 2) && (f.packing == 0 || f.packing == 1);
+}
+// ... the container form only (what most kernels read and every kernel writes).
+bool format_ok(const mx_format_t &f) { return format_ok_any(f) && f.packing == 0; }
+size_t mant_row_bytes(int64_t K, const mx_format_t &f)
+{
+    return f.packing ? (size_t)(K * f.elem_bits / 8) : (f.elem_bits <= 4 ? (size_t)(K / 2) : (size_t)K);
 }
 bool format_1d(const mx_format_t &f) { return format_ok(f) && f.block_rows == 1; }
 bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -262,6 +269,15 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
                                 const mx_format_t &f, __nv_bfloat16 *out, int64_t ld,
                                 const DeviceInfo &d, cudaStream_t st)
 {
+    if (f.packing) {                    // dense storage: w bits per element
+        if (rows == 0 || K == 0) return MX_OK;
+        ProfScope prof(KIND_DEQUANTIZE, st);
+        MX_CUDA(launch_dep(mx::dequantize_dense_kernel<__nv_bfloat16>, dim3(grid_for(rows * (K / 8), 256, d.sm_count, 8)),
+                           dim3(256), 0, st, static_cast<const uint8_t *>(mant), exps, rows, K, (int)f.block,
+                           (int)f.elem_bits, f.block_rows == 2 ? 1 : 0, out, ld));
+        MX_CUDA(cudaGetLastError());
+        return MX_OK;
+    }
     return launch_dequant_bf16(mant, exps, rows, K, f, out, ld, dense_strides(K, f), 1, d, st);
 }
 
@@ -598,7 +614,7 @@ mx_status_t check_gemm_args(const void *a, const void *a_exp, const mx_format_t 
 {
     if (!a || !w || !w_exp || !y) return MX_ERR_NULL;
     (void)a_exp;
-    if (!format_ok(fa) || !format_ok(fw) || fa.block != fw.block) return MX_ERR_FORMAT;
+    if (!format_ok_any(fa) || !format_ok_any(fw) || fa.block != fw.block) return MX_ERR_FORMAT;
     if (M <= 0 || N <= 0 || K <= 0 || (K % fa.block) != 0 || ldy < N) return MX_ERR_SHAPE;
     if ((M % fa.block_rows) != 0 || (N % fw.block_rows) != 0) return MX_ERR_SHAPE;     // whole two-row blocks
     if (M > INT32_MAX / 2 || N > INT32_MAX / 2 || K > INT32_MAX / 2) return MX_ERR_SHAPE;
@@ -660,7 +676,7 @@ size_t stream_table_bytes(int32_t n_layers)
 bool stream_layer_ok(const mx_linear_args_t &a)
 {
     return a.M >= 1 && a.M <= 16 && a.fw.block == 32 && a.fa.block == 32 && a.fw.elem_bits <= 4 &&
-           (a.K % 128) == 0 && a.fa.block_rows == 1 && a.fw.block_rows == 1;
+           (a.K % 128) == 0 && a.fa.block_rows == 1 && a.fw.block_rows == 1 && a.fa.packing == 0 && a.fw.packing == 0;
 }
 
 size_t stream_act_bytes(const mx_linear_args_t &a)
@@ -694,7 +710,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
 {
     const int64_t M = a.M, N = a.N, K = a.K;
     mx::QuantOut out{nullptr, nullptr, a_hat, K, nullptr};
-    if ((K % 32) != 0) {
+    if ((K % 32) != 0 || a.fw.packing) {
         mx_status_t s = quantize_rows_any(a.x, a.dt, M, K, a.ldx, a.fa, out, d, st);
         if (s != MX_OK) return s;
         return launch_dequant_bf16(a.w_mant, a.w_exp, N, K, a.fw, w_hat, K, d, st);
@@ -746,13 +762,13 @@ static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers
 
 size_t mx_mant_bytes(int64_t rows, int64_t K, mx_format_t f)
 {
-    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
-    return f.elem_bits <= 4 ? (size_t)rows * (size_t)(K / 2) : (size_t)rows * (size_t)K;
+    if (!format_ok_any(f) || rows < 0 || K < 0 || (K % f.block) != 0) return 0;
+    return (size_t)rows * mant_row_bytes(K, f);
 }
 
 size_t mx_exp_bytes(int64_t rows, int64_t K, mx_format_t f)
 {
-    if (!format_ok(f) || rows < 0 || K < 0 || (K % f.block) != 0 || (rows % f.block_rows) != 0) return 0;
+    if (!format_ok_any(f) || rows < 0 || K < 0 || (K % f.block) != 0 || (rows % f.block_rows) != 0) return 0;
     return (size_t)(rows / f.block_rows) * (size_t)(K / f.block);
 }
 
@@ -765,7 +781,7 @@ double mx_format_bits(mx_format_t f)
 size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx_format_t fw,
                              mx_algo_t algo)
 {
-    if (!format_ok(fa) || !format_ok(fw) || M <= 0 || N <= 0 || K <= 0) return 0;
+    if (!format_ok_any(fa) || !format_ok_any(fw) || M <= 0 || N <= 0 || K <= 0) return 0;
     const size_t pk = packed_workspace(M, K, fa);          // mx_linear with the CUDA-core kernel
     switch (algo) {
     case MX_ALGO_SIMT: return pk;
@@ -850,6 +866,40 @@ mx_status_t mx_quantize(const void *x, mx_dtype_t dt, int64_t rows, int64_t K, i
     return MX_OK;
 }
 
+static mx_status_t repack_impl(const void *src, int64_t rows, int64_t K, mx_format_t f, void *dst, bool to_dense, void *stream)
+{
+    f.packing = 0;
+    if (!format_ok(f)) return MX_ERR_FORMAT;
+    if (rows < 0 || K < 0 || (K % f.block) != 0) return MX_ERR_SHAPE;
+    if (rows == 0 || K == 0) return MX_OK;
+    if (!src || !dst) return MX_ERR_NULL;
+    if (!aligned16(to_dense ? src : dst)) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int grid = grid_for(rows * (K / 8), 256, d->sm_count, 8);
+    ProfScope prof(KIND_QUANTIZE, st);
+    if (to_dense)
+        MX_CUDA(launch_dep(mx::dense_pack_kernel, dim3(grid), dim3(256), 0, st, static_cast<const uint8_t *>(src), rows, K,
+                           (int)f.elem_bits, static_cast<uint8_t *>(dst)));
+    else
+        MX_CUDA(launch_dep(mx::dense_unpack_kernel, dim3(grid), dim3(256), 0, st, static_cast<const uint8_t *>(src), rows, K,
+                           (int)f.elem_bits, static_cast<uint8_t *>(dst)));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
+mx_status_t mx_pack_dense(const void *mant, int64_t rows, int64_t K, mx_format_t f, void *dense_out, void *stream)
+{
+    return repack_impl(mant, rows, K, f, dense_out, true, stream);
+}
+
+mx_status_t mx_unpack_dense(const void *dense, int64_t rows, int64_t K, mx_format_t f, void *mant_out, void *stream)
+{
+    return repack_impl(dense, rows, K, f, mant_out, false, stream);
+}
+
 mx_status_t mx_cast(const void *mant_in, const uint8_t *exp_in, mx_format_t f_in, int64_t rows, int64_t K,
                     mx_format_t f_out, void *mant_out, uint8_t *exp_out, uint32_t *nonfinite_count, void *stream)
 {
@@ -880,7 +930,7 @@ mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, i
                           mx_format_t f, void *out, mx_dtype_t dt, int64_t ld_out, void *stream)
 {
     if (!mant || !exps || !out) return MX_ERR_NULL;
-    if (!format_ok(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
+    if (!format_ok_any(f) || (dt != MX_F32 && dt != MX_BF16)) return MX_ERR_FORMAT;
     if (rows < 0 || K < 0 || (K % f.block) != 0 || ld_out < K || (rows % f.block_rows) != 0) return MX_ERR_SHAPE;
     if (!aligned16(mant) || !aligned16(out) || (ld_out % 8) != 0) return MX_ERR_ALIGN;
     if (rows == 0 || K == 0) return MX_OK;
@@ -888,6 +938,14 @@ mx_status_t mx_dequantize(const void *mant, const uint8_t *exps, int64_t rows, i
     mx_status_t s = device_info(&d);
     if (s != MX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (f.packing && dt == MX_F32) {
+        ProfScope prof(KIND_DEQUANTIZE, st);
+        MX_CUDA(launch_dep(mx::dequantize_dense_kernel<float>, dim3(grid_for(rows * (K / 8), 256, d->sm_count, 8)), dim3(256), 0,
+                           st, static_cast<const uint8_t *>(mant), exps, rows, K, (int)f.block, (int)f.elem_bits,
+                           f.block_rows == 2 ? 1 : 0, static_cast<float *>(out), ld_out));
+        MX_CUDA(cudaGetLastError());
+        return MX_OK;
+    }
     if (dt == MX_BF16)
         return launch_dequant_bf16(mant, exps, rows, K, f, static_cast<__nv_bfloat16 *>(out), ld_out, *d, st);
     ProfScope prof(KIND_DEQUANTIZE, st);
@@ -918,6 +976,8 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
         algo != MX_ALGO_TCGEN05_BLOCKWISE)
         return MX_ERR_FORMAT;
+    // dense storage is read by the decode pass in front of the tensor-core kernels only
+    if ((fa.packing || fw.packing) && algo != MX_ALGO_TCGEN05 && algo != MX_ALGO_TCGEN05_BLOCKWISE) return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
@@ -966,11 +1026,14 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
     mx_status_t s = check_gemm_args(x, nullptr, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
     if (s != MX_OK) return s;
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
+    if (fa.packing) return MX_ERR_FORMAT;                 // the activations are produced here: container form
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
     mx_linear_args_t one;
     one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
     one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = ldy;
+    if (fw.packing && algo != MX_ALGO_AUTO && algo != MX_ALGO_TCGEN05 && algo != MX_ALGO_TCGEN05_BLOCKWISE)
+        return MX_ERR_FORMAT;
     if (algo == MX_ALGO_AUTO)
         algo = (stream_layer_ok(one) && (reinterpret_cast<uintptr_t>(w_exp) & 3u) == 0) ? MX_ALGO_STREAM
                                                                                      : MX_ALGO_TCGEN05;
@@ -1078,6 +1141,7 @@ mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int6
                                     static_cast<const float *>(y_mant), N);
     if (s != MX_OK) return s;
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
+    if (fa.packing) return MX_ERR_FORMAT;
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
     s = check_quantized_out(fy, N, y_mant, y_exp);
@@ -1288,6 +1352,7 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
     if (fa.block_rows != 1 || fw.block_rows != 1) return MX_ERR_FORMAT;     // slices of packed tensors: one-row blocks
+    if (fa.packing || fw.packing) return MX_ERR_FORMAT;
     if (batch <= 0 || lda < K || ldw < K || stride_a < 0 || stride_w < 0 || stride_y < 0) return MX_ERR_SHAPE;
     // row and batch strides must keep whole blocks and whole container bytes together
     if ((lda % fa.block) || (ldw % fw.block) || (stride_a % fa.block) || (stride_w % fw.block) ||
@@ -1542,7 +1607,7 @@ mx_status_t mx_gemm_static(const void *a_mant, const uint8_t *a_exp, mx_format_t
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
-    if (fa.block_rows != 1 || fw.block_rows != 1) return MX_ERR_FORMAT;
+    if (fa.block_rows != 1 || fw.block_rows != 1 || fa.packing || fw.packing) return MX_ERR_FORMAT;
     const size_t need = tc_operand_bytes(M, N, K);
     if (need > (size_t)MX_STATIC_SCRATCH_BYTES) {
         snprintf(t_cuda_error, sizeof(t_cuda_error),

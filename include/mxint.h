@@ -126,9 +126,10 @@ typedef struct {
  * 2r+1) share one exponent, that of the largest magnitude among them.  The exponent array of a
  * [rows, K] tensor is then uint8 [rows/2, K/block] and rows must be even (MX_ERR_SHAPE).
  * Accepted by mx_quantize (stride_k == 1), mx_dequantize, mx_gemm / mx_linear and their _q forms
- * for either operand with MX_ALGO_AUTO, MX_ALGO_TCGEN05 and MX_ALGO_SIMT; the streaming, in-kernel
- * decode, batched, grouped and static entry points and the output format fy take one-row blocks
- * only (MX_ERR_FORMAT). */
+ * for either operand with MX_ALGO_AUTO, MX_ALGO_TCGEN05(_BLOCKWISE) and MX_ALGO_SIMT, as the result
+ * format fy of the _q forms (rows of Y pair up: exponent array [M/2, N/fy.block]) and by
+ * mx_gemm_batched (items must start on even rows); the streaming, in-kernel decode, grouped and
+ * static entry points take one-row blocks only (MX_ERR_FORMAT). */
 
 /* ---- size helpers (host only, no CUDA call) ------------------------------------------- */
 

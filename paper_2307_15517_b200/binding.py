@@ -310,7 +310,7 @@ def _quantized_out(M: int, N: int, fy: MxFormat, device, y_mant, y_exp):
     if y_mant is None:
         y_mant = torch.empty((M, N // 2 if fy.elem_bits <= 4 else N), dtype=torch.uint8, device=device)
     if y_exp is None:
-        y_exp = torch.empty((M, N // fy.block), dtype=torch.uint8, device=device)
+        y_exp = torch.empty((M // max(fy.block_rows, 1), N // fy.block), dtype=torch.uint8, device=device)
     return y_mant, y_exp
 
 

@@ -86,6 +86,7 @@ struct TcParams {
     uint8_t *yq_exp;
     uint32_t *yq_nonfinite;   // nullable: number of blocks that held Inf/NaN
     int yq_bits, yq_block;
+    int yq_rows2;             // 1: rows 2i and 2i+1 share the exponent bytes (two-row blocks); exponents [M/2, N/yq_block]
 };
 
 // MXInt-result epilogue of one lane: r holds 32 consecutive fp32 outputs (columns n .. n + 31) of
@@ -94,23 +95,32 @@ struct TcParams {
 // mantissa bytes and one or two exponent bytes.
 __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, int n, uint32_t (&r)[32])
 {
-    if (row >= p.M || n >= p.N) return;
+    // every lane of the warp runs the shuffle below; lanes outside the matrix contribute zeros
+    const bool live = row < p.M && n < p.N;
     const int64_t nb_row = p.N / p.yq_block;
     uint32_t amax[2] = {0u, 0u};
 #pragma unroll
     for (int v = 0; v < 32; ++v) {
         float x = __uint_as_float(r[v]);
-        if (p.bias && n + v < p.N) x += __ldg(p.bias + n + v);
+        if (p.bias && live && n + v < p.N) x += __ldg(p.bias + n + v);
         r[v] = __float_as_uint(x);
-        amax[v >> 4] = max(amax[v >> 4], r[v] & 0x7FFFFFFFu);
+        if (live && n + v < p.N) amax[v >> 4] = max(amax[v >> 4], r[v] & 0x7FFFFFFFu);
     }
     if (p.yq_block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
+    if (p.yq_rows2) {
+        // rows 2i and 2i+1 are neighbouring lanes (the warp's first row is a multiple of 32; M is even)
+        amax[0] = max(amax[0], __shfl_xor_sync(0xFFFFFFFFu, amax[0], 1));
+        amax[1] = max(amax[1], __shfl_xor_sync(0xFFFFFFFFu, amax[1], 1));
+    }
+    if (!live) return;
+    const bool writes_exp = !p.yq_rows2 || (row & 1) == 0;
+    const int64_t erow = p.yq_rows2 ? (row >> 1) : row;
 #pragma unroll
     for (int h = 0; h < 2; ++h) {
         if (n + 16 * h >= p.N) break;            // N % yq_block == 0: a half is all in or all out
         const int ebyte = (int)(amax[h] >> 23);   // 255 <=> an Inf or NaN in the block
-        if (p.yq_block == 16 || h == 0) {
-            p.yq_exp[(int64_t)row * nb_row + (n + 16 * h) / p.yq_block] = (uint8_t)ebyte;
+        if ((p.yq_block == 16 || h == 0) && writes_exp) {
+            p.yq_exp[erow * nb_row + (n + 16 * h) / p.yq_block] = (uint8_t)ebyte;
             if (ebyte == 255 && p.yq_nonfinite) atomicAdd(p.yq_nonfinite, 1u);
         }
         uint2 pk[2];

@@ -439,6 +439,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     p.yq_nonfinite = yq ? yq->nonfinite : nullptr;
     p.yq_bits = yq ? yq->f.elem_bits : 0;
     p.yq_block = yq ? yq->f.block : 0;
+    p.yq_rows2 = yq && yq->f.block_rows == 2 ? 1 : 0;
     p.batch = (int)tb.count;
     p.y_batch = tb.y_batch;
     const int64_t tiles64 = (int64_t)p.tiles_m * p.tiles_n * tb.count;
@@ -492,6 +493,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     p.yq_nonfinite = yq ? yq->nonfinite : nullptr;
     p.yq_bits = yq ? yq->f.elem_bits : 0;
     p.yq_block = yq ? yq->f.block : 0;
+    p.yq_rows2 = yq && yq->f.block_rows == 2 ? 1 : 0;
     const int tiles = p.tiles_m * p.tiles_n;
     const int pairs = tiles < d.sm_count / 2 ? tiles : d.sm_count / 2;
     ProfScope prof(KIND_GEMM_TC, st);
@@ -1090,11 +1092,11 @@ mx_status_t mx_linear(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_
 }
 
 // ---- the layer with an MXInt result -------------------------------------------------------------
-static mx_status_t check_quantized_out(mx_format_t fy, int64_t N, const void *y_mant, const uint8_t *y_exp)
+static mx_status_t check_quantized_out(mx_format_t fy, int64_t M, int64_t N, const void *y_mant, const uint8_t *y_exp)
 {
     if (!y_mant || !y_exp) return MX_ERR_NULL;
-    if (!format_1d(fy)) return MX_ERR_FORMAT;
-    if ((N % fy.block) != 0) return MX_ERR_SHAPE;
+    if (!format_ok(fy)) return MX_ERR_FORMAT;
+    if ((N % fy.block) != 0 || (M % fy.block_rows) != 0) return MX_ERR_SHAPE;
     if (!aligned16(y_mant)) return MX_ERR_ALIGN;
     return MX_OK;
 }
@@ -1109,7 +1111,7 @@ mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, 
                                     static_cast<const float *>(y_mant), N);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
-    s = check_quantized_out(fy, N, y_mant, y_exp);
+    s = check_quantized_out(fy, M, N, y_mant, y_exp);
     if (s != MX_OK) return s;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -1144,7 +1146,7 @@ mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int6
     if (fa.packing) return MX_ERR_FORMAT;
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
-    s = check_quantized_out(fy, N, y_mant, y_exp);
+    s = check_quantized_out(fy, M, N, y_mant, y_exp);
     if (s != MX_OK) return s;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -1351,7 +1353,6 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, nullptr, y, ldy);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
-    if (fa.block_rows != 1 || fw.block_rows != 1) return MX_ERR_FORMAT;     // slices of packed tensors: one-row blocks
     if (fa.packing || fw.packing) return MX_ERR_FORMAT;
     if (batch <= 0 || lda < K || ldw < K || stride_a < 0 || stride_w < 0 || stride_y < 0) return MX_ERR_SHAPE;
     // row and batch strides must keep whole blocks and whole container bytes together
@@ -1367,14 +1368,17 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
     const size_t a_item = round256((size_t)M * K * 2), w_item = round256((size_t)N * K * 2);
     __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) + (size_t)batch * a_item);
+    // two-row blocks: an item must start on an even row of the packed tensor
+    if ((fa.block_rows == 2 && ((stride_a / lda) & 1)) || (fw.block_rows == 2 && ((stride_w / ldw) & 1))) return MX_ERR_ALIGN;
     auto strides = [](const mx_format_t &f, int64_t ld, int64_t bstride, size_t out_item) {
         mx::PackedStrides ps;
         ps.mant_ld = f.elem_bits <= 4 ? ld / 2 : ld;
         ps.exp_ld = ld / f.block;
         ps.mant_batch = f.elem_bits <= 4 ? bstride / 2 : bstride;
-        ps.exp_batch = bstride / f.block;
+        ps.exp_row_shift = f.block_rows == 2 ? 1 : 0;   // rows 2i, 2i+1 read one row of exponent bytes
+        // an item starts (bstride / ld) rows down and (bstride % ld) elements into the row
+        ps.exp_batch = ((bstride / ld) >> ps.exp_row_shift) * (ld / f.block) + (bstride % ld) / f.block;
         ps.out_batch = (int64_t)(out_item / 2);
-        ps.exp_row_shift = 0;
         return ps;
     };
     // one decode launch per operand and one product launch cover every batch item

@@ -100,3 +100,51 @@ def test_two_row_blocks_are_refused_where_unsupported(mxb):
     y = mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64)       # AUTO falls back to the tensor-core kernel
     assert torch.isfinite(y).all() and mxb.mx_poll_status() == 0
     del F1
+
+
+@pytest.mark.parametrize("case", [(300, 544, 512, 16, 16, 4), (130, 208, 256, 32, 32, 8), (2100, 2336, 128, 16, 16, 8),
+                                  (2048, 1024, 320, 16, 32, 6)])
+def test_result_in_two_row_blocks_bit_exact_where_fp32_is_order_independent(mxb, case):
+    """mx_gemm_q with fy = (By, 2): the rows of Y pair up and share exponent bytes.  Operands whose partial
+    sums are all exactly representable, so the fp32 product is the oracle's whatever the order, and the
+    codes must be the oracle's two-row quantization of it, bit for bit (one-CTA and CTA-pair epilogues)."""
+    M, N, K, B, By, wy = case
+    qa = synth.random_ints((M, K), -7, 7, M + wy).numpy()
+    qw = synth.random_ints((N, K), -7, 7, N + wy).numpy()
+    ea = np.full((M, K // B), 129, np.uint8)
+    ew = np.full((N, K // B), 124, np.uint8)
+    scale = 2.0 ** ((129 - 127 - 2) + (124 - 127 - 2))
+    bias = (synth.random_ints((1, N), -1000, 1000, 7).numpy()[0] * scale).astype(np.float32)
+    y_ref, y_seq, _ = orc.gemm(qa, ea, 4, qw, ew, 4, B, bias=bias)
+    assert np.array_equal(y_ref, y_seq)
+    qy, ey, bad = orc.quantize_2d(y_ref, By, 2, wy)
+    f4 = mxb.MxFormat(B, 4)
+    ym, ye = mxb.mx_gemm_q(_dev(orc.pack(qa, 4)), _dev(ea), f4, _dev(orc.pack(qw, 4)), _dev(ew), f4, M, N, K,
+                           mxb.MxFormat(By, wy, 8, 2), bias=_dev(bias),
+                           y_exp=torch.empty((M // 2, N // By), dtype=torch.uint8, device="cuda"))
+    assert mxb.mx_poll_status() == 0 and bad == 0
+    assert np.array_equal(ye.cpu().numpy(), ey)
+    assert np.array_equal(ym.cpu().numpy(), orc.pack(qy, wy))
+
+
+def test_batched_product_on_two_row_blocks(mxb):
+    """Per-head products on slices of packed [tokens, heads*d] tensors quantized in (16,2) blocks, and
+    items stacked along the rows of the weight-side tensor: bit for bit on order-independent operands."""
+    H, M, N, d, B, w = 5, 200, 136, 64, 16, 8
+    qa = synth.random_ints((M, H * d), -127, 127, 70).numpy()
+    ea = np.repeat(np.repeat(synth.random_bytes((M // 2, H), 121, 133, 71).numpy(), d // B, axis=1), 1, axis=0)
+    qw = synth.random_ints((H * N, d), -127, 127, 72).numpy()              # items stacked along rows
+    ew = np.repeat(synth.random_bytes((H * N // 2, 1), 115, 127, 73).numpy(), d // B, axis=1)
+    f2 = mxb.MxFormat(B, w, 8, 2)
+    y = torch.full((H * M, N), 3.0, device="cuda")
+    mxb.mx_gemm_batched(_dev(orc.pack(qa, w)), _dev(ea), f2, H * d, d, _dev(orc.pack(qw, w)), _dev(ew), f2,
+                        d, N * d, M, N, d, H, y, N, M * N)
+    assert mxb.mx_poll_status() == 0
+    got = y.cpu().numpy()
+    ea_rows, ew_rows = orc.expand_exponent_rows(ea, 2), orc.expand_exponent_rows(ew, 2)
+    nb = d // B
+    for h in range(H):
+        y_ref, y_seq, _ = orc.gemm(qa[:, h * d:(h + 1) * d], ea_rows[:, h * nb:(h + 1) * nb], w,
+                                   qw[h * N:(h + 1) * N], ew_rows[h * N:(h + 1) * N], w, B)
+        assert np.array_equal(y_ref, y_seq)
+        assert np.array_equal(got[h * M:(h + 1) * M], y_ref), h

@@ -102,7 +102,7 @@ def test_two_row_blocks_are_refused_where_unsupported(mxb):
     del F1
 
 
-@pytest.mark.parametrize("case", [(300, 544, 512, 16, 16, 4), (130, 208, 256, 32, 32, 8), (2100, 2336, 128, 16, 16, 8),
+@pytest.mark.parametrize("case", [(300, 544, 512, 16, 16, 4), (130, 208, 256, 32, 16, 8), (2100, 2336, 128, 16, 16, 8),
                                   (2048, 1024, 320, 16, 32, 6)])
 def test_result_in_two_row_blocks_bit_exact_where_fp32_is_order_independent(mxb, case):
     """mx_gemm_q with fy = (By, 2): the rows of Y pair up and share exponent bytes.  Operands whose partial

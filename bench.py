@@ -602,9 +602,21 @@ def run_ours(args):
         ms_2d, _ = timed_steps(run_step_2d, args.steps, profile=False)
         block_16x2 = {"ms_per_step": ms_2d / args.steps, "tops": flops_step * args.steps / (ms_2d * 1e-3) / 1e12,
                       "formats": "activations MXInt((16,2),8,7), weights MXInt((16,2),8,3): two-row blocks"}
+        # ... and with one tensor-memory accumulator per block (bit-identical to the sequential fp32 sum)
+        def run_step_bw(mxb_, layers_):
+            for L in layers_:
+                mxb_.mx_linear(L["x"], L["fa"], L["w_mant"], L["w_exp"], L["fw"], L["spec"].N, y=L["y"],
+                               workspace=L["ws"], algo=mxb_.MX_ALGO_TCGEN05_BLOCKWISE)
+
+        for _ in range(3):
+            run_step_bw(mxb, next_set())
+        torch.cuda.synchronize()
+        ms_bw, _ = timed_steps(run_step_bw, args.steps, profile=False)
+        blockwise = {"ms_per_step": ms_bw / args.steps, "tops": flops_step * args.steps / (ms_bw * 1e-3) / 1e12,
+                     "algo": "MX_ALGO_TCGEN05_BLOCKWISE: exact block sums, fp32 block adds in ascending order"}
         del sets, layers
         torch.cuda.empty_cache()
-        secondary = {"linear_q": linear_q, "block_16x2": block_16x2,
+        secondary = {"linear_q": linear_q, "block_16x2": block_16x2, "blockwise": blockwise,
                      "decode_sweep": decode_sweep(mxb, synth, torch, peaks["hbm_gbs"]),
                      "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
                      "single_layer": single_layer_latency(mxb, synth, torch),
@@ -612,7 +624,7 @@ def run_ours(args):
                      "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
         # every configuration's whole call against the vendor-GEMM rate (tensor-bound ones)
-        for key in ("linear_q", "block_16x2", "llama7b_mixed", "decoder_block"):
+        for key in ("linear_q", "block_16x2", "blockwise", "llama7b_mixed", "decoder_block"):
             secondary[key]["frac_of_bf16_burst"] = secondary[key]["tops"] / peaks["bf16_tflops"]
         secondary["llama7b_mixed"]["gemm_frac_of_bf16_burst"] = secondary["llama7b_mixed"]["gemm_tflops"] / peaks["bf16_tflops"]
         assert mxb.mx_poll_status() == 0, "device status after the secondary metrics"

@@ -76,13 +76,20 @@ typedef enum {
                             only; needs K % 32 == 0 and a 2-byte aligned w_exp, else it falls back to
                             the separate pass).  Saves memory, but the decode costs more issue slots
                             than the MMA leaves free, so it is slower than MX_ALGO_TCGEN05.          */
-    MX_ALGO_TCGEN05_BLOCKWISE = 5 /* tensor-core kernel that gives every block its own accumulator: the tensor
+    MX_ALGO_TCGEN05_BLOCKWISE = 5, /* tensor-core kernel that gives every block its own accumulator: the tensor
                             pipe sums one block (exactly: all addends share one scale), the block terms
                             are added in fp32 registers with round-to-nearest in ascending block order --
                             the same bits as MX_ALGO_SIMT while every block term is a normal fp32 number.
                             Meets 1e-5 * S for any spread of the block exponents and any K; a fraction of
                             the throughput of MX_ALGO_TCGEN05 (a tensor-memory read per block).  fp32
                             result only.                                                                  */
+    MX_ALGO_TCGEN05_MXF8 = 6 /* the hardware's block-scaled tensor-core path (tcgen05.mma.kind::mxf8f6f4 with one
+                            E8M0 scale per 32 elements): the MXInt operator of Sec. 3.2 in silicon.  Exact for
+                            the formats it can hold: block 32 and elem_bits <= 5 on BOTH operands (an element
+                            q * 2^-(w-2) is an E4M3 number, the exponent byte is the E8M0 scale), K % 128 == 0,
+                            container storage; anything else answers MX_ERR_FORMAT.  Twice the tensor peak of
+                            the bf16 kernels; accumulation across blocks in fp32 as MX_ALGO_TCGEN05.  Workspace:
+                            mx_workspace_bytes_ex with this algo.  mx_gemm_ex and mx_linear_ex only.            */
 } mx_algo_t;
 
 /* Accuracy of the product kernels against the exactly summed result (Sec. 3.2 leaves the accumulator

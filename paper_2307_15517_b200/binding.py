@@ -19,6 +19,7 @@ LIB_PATH = os.path.join(_HERE, "libmxint.so")
 MX_F32, MX_BF16 = 0, 1
 MX_ALGO_AUTO, MX_ALGO_SIMT, MX_ALGO_TCGEN05, MX_ALGO_STREAM, MX_ALGO_TCGEN05_FUSED = 0, 1, 2, 3, 4
 MX_ALGO_TCGEN05_BLOCKWISE = 5
+MX_ALGO_TCGEN05_MXF8 = 6
 
 STATUS_NAMES = {0: "MX_OK", -1: "MX_ERR_NULL", -2: "MX_ERR_SHAPE", -3: "MX_ERR_FORMAT",
                 -4: "MX_ERR_ALIGN", -5: "MX_ERR_WORKSPACE", -6: "MX_ERR_CUDA",

@@ -17,6 +17,7 @@
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
 #include "mx_gemm_tc2.cuh"
+#include "mx_gemm_tc8.cuh"
 #include "mx_gemm_tcx.cuh"
 #include "mx_gemv_stream.cuh"
 #include "mx_glue.cuh"
@@ -40,6 +41,7 @@ struct DeviceInfo {
     bool stream_attr_set[4] = {false, false, false, false};
     bool tc2_attr_set = false;
     bool tcx_attr_set = false;
+    bool tc8_attr_set = false;
 };
 DeviceInfo g_dev[MAX_DEVICES];
 std::mutex g_init_mu;        // guards every lazily initialised field above and below (calls may come from several host threads)
@@ -543,6 +545,98 @@ mx_status_t launch_tcx(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     return MX_OK;
 }
 
+// ---- hardware block-scaled path (kind::mxf8f6f4): blocks of 32, widths <= 5 on both operands --------
+bool mxf8_fits(const mx_format_t &fa, const mx_format_t &fw, int64_t K)
+{
+    return fa.block == 32 && fw.block == 32 && fa.elem_bits <= 5 && fw.elem_bits <= 5 && (K % 128) == 0 &&
+           fa.packing == 0 && fw.packing == 0;
+}
+size_t mxf8_sf_bytes(int64_t rows, int64_t K) { return round256((size_t)((rows + 127) / 128) * (size_t)(K / 128) * 512); }
+// E4M3 elements and scale chunks of both operands
+size_t mxf8_operand_bytes(int64_t M, int64_t N, int64_t K)
+{
+    return round256((size_t)M * K) + mxf8_sf_bytes(M, K) + round256((size_t)N * K) + mxf8_sf_bytes(N, K);
+}
+
+mx_status_t encode_u8_sw128(CUtensorMap *tm, const void *base, int64_t rows, int64_t row_bytes, int box_rows)
+{
+    mx_status_t s = ensure_encoder();
+    if (s != MX_OK) return s;
+    const MapKey key = std::make_tuple(3, base, rows, row_bytes, (int64_t)box_rows, (int64_t)0, (int64_t)0);
+    if (cached_map(key, tm)) return MX_OK;
+    const cuuint64_t dims[2] = {(cuuint64_t)row_bytes, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {128, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = g_encode_tiled(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void *>(base), dims, strides, box, estr,
+                                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        snprintf(t_cuda_error, sizeof(t_cuda_error), "cuTensorMapEncodeTiled (8-bit operand) failed (%d)", (int)r);
+        return MX_ERR_CUDA;
+    }
+    remember_map(key, *tm);
+    return MX_OK;
+}
+
+// Packed MXInt operands -> E4M3 + scale chunks in `ws` (mxf8_operand_bytes), then the block-scaled product.
+mx_status_t run_tc8(const void *a_mant, const uint8_t *a_exp, const mx_format_t &fa, const void *w_mant, const uint8_t *w_exp,
+                    const mx_format_t &fw, int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
+                    uint8_t *ws, DeviceInfo &d, cudaStream_t st)
+{
+    using Cfg = mx::Tc8Cfg;
+    uint8_t *a8 = ws;
+    uint8_t *sfa = a8 + round256((size_t)M * K);
+    uint8_t *w8 = sfa + mxf8_sf_bytes(M, K);
+    uint8_t *sfw = w8 + round256((size_t)N * K);
+    const int64_t chunks_a = (M + 127) / 128, chunks_w = (N + 127) / 128;
+    {
+        ProfScope prof(KIND_DEQUANTIZE, st);
+        MX_CUDA(launch_dep(mx::pack_e4m3_kernel, dim3(grid_for(M * (K / 8), 256, d.sm_count, 8)), dim3(256), 0, st,
+                           static_cast<const uint8_t *>(a_mant), a_exp, M, K, (int)fa.elem_bits, fa.block_rows == 2 ? 1 : 0,
+                           a8, sfa, chunks_a));
+    }
+    {
+        ProfScope prof(KIND_DEQUANTIZE, st);
+        MX_CUDA(launch_dep(mx::pack_e4m3_kernel, dim3(grid_for(N * (K / 8), 256, d.sm_count, 8)), dim3(256), 0, st,
+                           static_cast<const uint8_t *>(w_mant), w_exp, N, K, (int)fw.elem_bits, fw.block_rows == 2 ? 1 : 0,
+                           w8, sfw, chunks_w));
+    }
+    CUtensorMap tm_a, tm_w;
+    mx_status_t s = encode_u8_sw128(&tm_a, a8, M, K, mx::TC_BM);
+    if (s != MX_OK) return s;
+    s = encode_u8_sw128(&tm_w, w8, N, K, Cfg::BN);
+    if (s != MX_OK) return s;
+    CUtensorMap tm_y = tm_a;
+    const bool tma_store = (ldy % 4) == 0;
+    if (tma_store) {
+        s = encode_f32_out(&tm_y, y, M, N, ldy);
+        if (s != MX_OK) return s;
+    }
+    s = smem_attr_once(d.tc8_attr_set, mx::gemm_tc8_kernel, (int)Cfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
+    mx::TcParams p{};
+    p.y = y;
+    p.bias = bias;
+    p.ldy = ldy;
+    p.M = (int)M;
+    p.N = (int)N;
+    p.K = (int)K;
+    p.tiles_m = (int)chunks_a;
+    p.tiles_n = (int)chunks_w;
+    p.status = d.status;
+    p.tma_store = tma_store ? 1 : 0;
+    p.batch = 1;
+    const int64_t tiles64 = chunks_a * chunks_w;
+    if (tiles64 > INT32_MAX / 2) return MX_ERR_SHAPE;
+    const int grid = tiles64 < d.sm_count ? (int)tiles64 : d.sm_count;
+    ProfScope prof(KIND_GEMM_TC, st);
+    MX_CUDA(launch_dep(mx::gemm_tc8_kernel, dim3(grid), dim3(mx::TC_THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p,
+                       (const uint8_t *)sfa, (const uint8_t *)sfw, (int)chunks_a, (int)chunks_w));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
 {
     const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256);
@@ -797,6 +891,8 @@ size_t mx_workspace_bytes_ex(int64_t M, int64_t N, int64_t K, mx_format_t fa, mx
     case MX_ALGO_TCGEN05:
     case MX_ALGO_TCGEN05_BLOCKWISE: return tc_workspace(M, N, K);
     case MX_ALGO_TCGEN05_FUSED: return (K % 32) == 0 ? fused_workspace(M, K) : tc_workspace(M, N, K);
+    case MX_ALGO_TCGEN05_MXF8:      // E4M3 operands + scale chunks; mx_linear also keeps the packed activations
+        return mxf8_fits(fa, fw, K) ? mxf8_operand_bytes(M, N, K) + pk : 0;
     default: return 0;
     }
 }
@@ -975,6 +1071,16 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         if (algo == MX_ALGO_AUTO) algo = can_stream ? MX_ALGO_STREAM : MX_ALGO_TCGEN05;
         if (algo == MX_ALGO_STREAM) return grouped_impl(&one, 1, &a_exp, workspace, workspace_bytes, stream);
     }
+    if (algo == MX_ALGO_TCGEN05_MXF8) {
+        if (!mxf8_fits(fa, fw, K)) return MX_ERR_FORMAT;
+        if (!workspace || workspace_bytes < mxf8_operand_bytes(M, N, K)) return MX_ERR_WORKSPACE;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+        DeviceInfo *d8 = nullptr;
+        s = device_info(&d8);
+        if (s != MX_OK) return s;
+        return run_tc8(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, static_cast<uint8_t *>(workspace), *d8,
+                       static_cast<cudaStream_t>(stream));
+    }
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
         algo != MX_ALGO_TCGEN05_BLOCKWISE)
         return MX_ERR_FORMAT;
@@ -1041,13 +1147,25 @@ mx_status_t mx_linear_ex(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int
                                                                                      : MX_ALGO_TCGEN05;
     if (algo == MX_ALGO_STREAM) return mx_linear_grouped(&one, 1, workspace, workspace_bytes, stream);
     if (algo != MX_ALGO_SIMT && algo != MX_ALGO_TCGEN05_FUSED && algo != MX_ALGO_TCGEN05 &&
-        algo != MX_ALGO_TCGEN05_BLOCKWISE)
+        algo != MX_ALGO_TCGEN05_BLOCKWISE && algo != MX_ALGO_TCGEN05_MXF8)
         return MX_ERR_FORMAT;
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (!workspace) return MX_ERR_WORKSPACE;
+    if (algo == MX_ALGO_TCGEN05_MXF8) {
+        if (!mxf8_fits(fa, fw, K)) return MX_ERR_FORMAT;
+        if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+        if (workspace_bytes < mxf8_operand_bytes(M, N, K) + packed_workspace(M, K, fa)) return MX_ERR_WORKSPACE;
+        uint8_t *ws8 = static_cast<uint8_t *>(workspace);
+        uint8_t *a_mant = ws8 + mxf8_operand_bytes(M, N, K);
+        uint8_t *a_exp = a_mant + round256(mx_mant_bytes(M, K, fa));
+        mx::QuantOut qo{a_mant, a_exp, nullptr, 0, nullptr};
+        s = quantize_rows_any(x, dt, M, K, ldx, fa, qo, *d, st);
+        if (s != MX_OK) return s;
+        return run_tc8(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, y, ldy, ws8, *d, st);
+    }
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     if (algo == MX_ALGO_SIMT) {

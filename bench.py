@@ -293,6 +293,46 @@ def llama7b_rate(mxb, synth, torch, iters=10):
                        for L in layers]}
 
 
+def block_scaled_rate(mxb, synth, torch, peak_bf16, iters=10):
+    """The LLaMA-7B-shaped layers of the seed-0 draw that the hardware's block-scaled tensor-core path holds
+    exactly (block 32, both widths <= 5): mx_linear with MX_ALGO_TCGEN05_MXF8 beside the default bf16 path.
+    The roofline of the 8-bit path is the bf16 peak times the nominal fp8 : bf16 ratio of 2."""
+    out = {"layers": []}
+    for li, spec in enumerate(synth.llama7b_mixed_layers(0)):
+        if spec.block != 32 or spec.w_act > 5 or spec.w_wgt > 5 or spec.K % 128:
+            continue
+        x, w = synth.llama7b_inputs(spec, li, seed=0)
+        fa, fw = mxb.MxFormat(spec.block, spec.w_act), mxb.MxFormat(spec.block, spec.w_wgt)
+        wm, we = mxb.mx_quantize(w.cuda(), fw)
+        xd = x.cuda()
+        M = x.shape[0]
+        y = torch.empty((M, spec.N), dtype=torch.float32, device="cuda")
+        flops = 2.0 * M * spec.N * spec.K
+        rec = {"name": spec.name, "K": spec.K, "N": spec.N, "w_act": spec.w_act, "w_wgt": spec.w_wgt}
+        for key, algo in (("bf16_path", mxb.MX_ALGO_AUTO), ("mxf8_path", mxb.MX_ALGO_TCGEN05_MXF8)):
+            ws = mxb.alloc_workspace(mxb.mx_workspace_bytes_ex(M, spec.N, spec.K, fa, fw, algo))
+            for _ in range(3):
+                mxb.mx_linear(xd, fa, wm, we, fw, spec.N, y=y, workspace=ws, algo=algo)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(iters):
+                mxb.mx_linear(xd, fa, wm, we, fw, spec.N, y=y, workspace=ws, algo=algo)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / iters
+            mxb.mx_profile_begin()
+            for _ in range(iters):
+                mxb.mx_linear(xd, fa, wm, we, fw, spec.N, y=y, workspace=ws, algo=algo)
+            torch.cuda.synchronize()
+            gemm_ms = mxb.mx_profile_end()["gemm_tc"][0] / iters
+            rec[key] = {"ms_per_call": ms, "tops": flops / ms / 1e9, "gemm_ms": gemm_ms, "gemm_tflops": flops / gemm_ms / 1e9}
+        rec["mxf8_path"]["gemm_frac_of_2x_bf16_burst"] = rec["mxf8_path"]["gemm_tflops"] / (2.0 * peak_bf16)
+        out["layers"].append(rec)
+        del x, w, xd, wm, we, y
+    return out
+
+
 def single_layer_latency(mxb, synth, torch, iters=200):
     """The single 128 x 768 x 768 MXInt4/B16 layer (151 MFLOP: latency-bound, two launches)."""
     x, w, spec = synth.single_layer(0)
@@ -621,6 +661,7 @@ def run_ours(args):
                      "quantize": quantize_rate(mxb, torch, peaks["hbm_gbs"]),
                      "single_layer": single_layer_latency(mxb, synth, torch),
                      "llama7b_mixed": llama7b_rate(mxb, synth, torch),
+                     "block_scaled": block_scaled_rate(mxb, synth, torch, peaks["bf16_tflops"]),
                      "decoder_block": decoder_block_rate(mxb, synth, torch),
                      "hbm_peak_gbs": peaks["hbm_gbs"], "peak_kind": peaks_kind}
         # every configuration's whole call against the vendor-GEMM rate (tensor-bound ones)

@@ -321,6 +321,30 @@ MX_API mx_status_t mx_softmax_q(const float *s, int64_t ld, int64_t rows, int64_
                                 int causal, int64_t rows_per_batch, mx_format_t fp, void *p_mant,
                                 uint8_t *p_exp, void *stream);
 
+/*
+ * Fused attention of one transformer block (Fig. 1(d); the matmuls "A" = Q K^T and "B" = P V of Fig. 1(a)/(b)
+ * are MXInt operators, softmax stays in floating point): per head h of `heads` heads of dimension head_dim,
+ *   S_h = Q_h K_h^T                      Q, K: MXInt [seq, heads*head_dim], format fqk, blocks along the head dimension
+ *   P_h = Q_fp(softmax(scale * S_h))     causal != 0: query i attends keys 0..i; P quantized to fp along the keys
+ *   ctx[:, h*head_dim ..] = P_h V_h      V given TRANSPOSED: MXInt [heads*head_dim, seq], format fv, blocks along the tokens
+ * i.e. mx_gemm_batched -> mx_softmax_q -> mx_gemm_batched in one kernel: the scores and the probabilities
+ * (heads * seq * seq values each) never reach memory.  Same arithmetic as that sequence up to the fp32
+ * rounding of the softmax row sums (two sweeps over the key tiles: maximum and sum first, then the
+ * probabilities normalised with the final values, quantized and multiplied).
+ *   ctx      : device fp32 [seq, ldc], ldc >= heads*head_dim, ldc % 4 == 0, 16-byte aligned
+ *   p_mant_out, p_exp_out : nullable; when given, the quantized probabilities are also written there
+ *              ([heads*seq, seq/2 or seq] and [heads*seq, seq/fp.block]; masked positions 0) -- for checks
+ *   workspace: mx_attention_workspace_bytes(seq, heads, head_dim) (the three operands as bf16), 256-byte aligned
+ * Restrictions: head_dim == 128, seq % 128 == 0, container storage, one-row blocks, fqk.block and fv.block
+ * dividing 128; otherwise MX_ERR_SHAPE / MX_ERR_FORMAT (use the three separate calls then).
+ */
+MX_API size_t mx_attention_workspace_bytes(int64_t seq, int64_t heads, int64_t head_dim);
+MX_API mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k_mant, const uint8_t *k_exp,
+                                mx_format_t fqk, const void *vt_mant, const uint8_t *vt_exp, mx_format_t fv,
+                                int64_t seq, int64_t heads, int64_t head_dim, float scale, int causal, mx_format_t fp,
+                                float *ctx, int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, void *workspace,
+                                size_t workspace_bytes, void *stream);
+
 /* ---- device status (the paper has no counterpart: it describes no runtime) ---------------- */
 
 /*

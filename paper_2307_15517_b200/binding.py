@@ -136,6 +136,10 @@ def _load() -> C.CDLL:
     L.mx_alt_gemm.argtypes = [vp, vp, A, vp, vp, A, i64, i64, i64, vp, vp, i64, vp, sz, vp]
     for name in ("mx_alt_quantize", "mx_alt_dequantize", "mx_alt_gemm"):
         getattr(L, name).restype = i32
+    L.mx_attention_workspace_bytes.argtypes = [i64, i64, i64]
+    L.mx_attention_workspace_bytes.restype = sz
+    L.mx_attention.argtypes = [vp, vp, vp, vp, F, vp, vp, F, i64, i64, i64, C.c_float, i32, F, vp, i64, vp, vp, vp, sz, vp]
+    L.mx_attention.restype = i32
     L.mx_profile_begin.argtypes = []
     L.mx_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
@@ -388,6 +392,27 @@ def mx_gemm_batched(a_mant, a_exp, fa: MxFormat, lda: int, stride_a: int, w_mant
                                ldw, stride_w, M, N, K, batch, _ptr(y), ldy, stride_y, _ptr(workspace),
                                workspace.numel(), _stream(stream)), "mx_gemm_batched")
     return y
+
+
+def mx_attention(q_mant, q_exp, k_mant, k_exp, fqk: MxFormat, vt_mant, vt_exp, fv: MxFormat, seq: int, heads: int,
+                 head_dim: int, scale: float, fp: MxFormat, causal: bool = True, ctx: Optional[torch.Tensor] = None,
+                 return_p: bool = False, workspace: Optional[torch.Tensor] = None, stream=None):
+    """Scores, causal softmax, quantized probabilities and context of all heads in one kernel.
+    Returns ctx [seq, heads*head_dim] fp32 (and the quantized probabilities (mant, exps) with return_p)."""
+    _need_cuda(q_mant, q_exp, k_mant, k_exp, vt_mant, vt_exp, ctx, workspace)
+    dev = q_mant.device
+    if ctx is None:
+        ctx = torch.empty((seq, heads * head_dim), dtype=torch.float32, device=dev)
+    pm = pe = None
+    if return_p:
+        pm = torch.zeros((heads * seq, seq // 2 if fp.elem_bits <= 4 else seq), dtype=torch.uint8, device=dev)
+        pe = torch.zeros((heads * seq, seq // fp.block), dtype=torch.uint8, device=dev)
+    if workspace is None:
+        workspace = alloc_workspace(int(lib.mx_attention_workspace_bytes(seq, heads, head_dim)), dev)
+    _check(lib.mx_attention(_ptr(q_mant), _ptr(q_exp), _ptr(k_mant), _ptr(k_exp), fqk, _ptr(vt_mant), _ptr(vt_exp), fv,
+                            seq, heads, head_dim, scale, 1 if causal else 0, fp, _ptr(ctx), ctx.stride(0), _ptr(pm),
+                            _ptr(pe), _ptr(workspace), workspace.numel(), _stream(stream)), "mx_attention")
+    return (ctx, pm, pe) if return_p else ctx
 
 
 def mx_layernorm(x: torch.Tensor, gamma, beta, eps: float, y: Optional[torch.Tensor] = None, stream=None):

@@ -14,6 +14,7 @@
 
 #include "../../include/mxint.h"
 #include "mx_alt.cuh"
+#include "mx_attention.cuh"
 #include "mx_gemm_simt.cuh"
 #include "mx_gemm_tc.cuh"
 #include "mx_gemm_tc2.cuh"
@@ -42,6 +43,7 @@ struct DeviceInfo {
     bool tc2_attr_set = false;
     bool tcx_attr_set = false;
     bool tc8_attr_set = false;
+    bool attn_attr_set = false;
 };
 DeviceInfo g_dev[MAX_DEVICES];
 std::mutex g_init_mu;        // guards every lazily initialised field above and below (calls may come from several host threads)
@@ -1510,6 +1512,73 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
     tb.w_item = w_item;
     tb.y_batch = stride_y;
     return run_tc(a_hat, w_hat, M, N, K, nullptr, y, ldy, *d, st, nullptr, tb);
+}
+
+// ---- fused attention ---------------------------------------------------------------------------
+size_t mx_attention_workspace_bytes(int64_t seq, int64_t heads, int64_t head_dim)
+{
+    if (seq <= 0 || heads <= 0 || head_dim <= 0) return 0;
+    return 3 * round256((size_t)seq * heads * head_dim * 2);
+}
+
+mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k_mant, const uint8_t *k_exp, mx_format_t fqk,
+                         const void *vt_mant, const uint8_t *vt_exp, mx_format_t fv, int64_t seq, int64_t heads,
+                         int64_t head_dim, float scale, int causal, mx_format_t fp, float *ctx, int64_t ldc,
+                         void *p_mant_out, uint8_t *p_exp_out, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!q_mant || !q_exp || !k_mant || !k_exp || !vt_mant || !vt_exp || !ctx) return MX_ERR_NULL;
+    if ((p_mant_out == nullptr) != (p_exp_out == nullptr)) return MX_ERR_NULL;
+    if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp)) return MX_ERR_FORMAT;
+    const int64_t hid = heads * head_dim;
+    if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid ||
+        seq > INT32_MAX / 4 || hid > INT32_MAX / 4)
+        return MX_ERR_SHAPE;
+    if (!aligned16(q_mant) || !aligned16(k_mant) || !aligned16(vt_mant) || !aligned16(ctx) || (ldc % 4) != 0 ||
+        (p_mant_out && !aligned16(p_mant_out)))
+        return MX_ERR_ALIGN;
+    if (!workspace || workspace_bytes < mx_attention_workspace_bytes(seq, heads, head_dim)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
+    if (s != MX_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t one = round256((size_t)seq * hid * 2);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    __nv_bfloat16 *q_hat = reinterpret_cast<__nv_bfloat16 *>(ws), *k_hat = reinterpret_cast<__nv_bfloat16 *>(ws + one),
+                  *v_hat = reinterpret_cast<__nv_bfloat16 *>(ws + 2 * one);
+    s = launch_dequant_bf16(q_mant, q_exp, seq, hid, fqk, q_hat, hid, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(k_mant, k_exp, seq, hid, fqk, k_hat, hid, *d, st);
+    if (s != MX_OK) return s;
+    s = launch_dequant_bf16(vt_mant, vt_exp, hid, seq, fv, v_hat, seq, *d, st);
+    if (s != MX_OK) return s;
+    CUtensorMap tm_q, tm_k, tm_v;
+    s = encode_bf16_rows(&tm_q, q_hat, seq, hid, 128);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_k, k_hat, seq, hid, 128);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_v, v_hat, hid, seq, 128);
+    if (s != MX_OK) return s;
+    s = smem_attr_once(d->attn_attr_set, mx::attention_kernel, (int)mx::AttnCfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
+    mx::AttnParams ap;
+    ap.ctx = ctx;
+    ap.ldc = ldc;
+    ap.seq = (int)seq;
+    ap.heads = (int)heads;
+    ap.scale = scale;
+    ap.causal = causal ? 1 : 0;
+    ap.p_bits = fp.elem_bits;
+    ap.p_block = fp.block;
+    ap.p_mant = static_cast<uint8_t *>(p_mant_out);
+    ap.p_exp = p_exp_out;
+    ap.status = d->status;
+    const int64_t items = (seq / mx::AttnCfg::BQ) * heads;
+    const int grid = items < d->sm_count ? (int)items : d->sm_count;
+    ProfScope prof(KIND_GEMM_TC, st);
+    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::TC_THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
 }
 
 // ---- fp32 glue of the transformer block ---------------------------------------------------------

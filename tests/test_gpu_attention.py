@@ -1,0 +1,78 @@
+"""GPU parity of the fused attention kernel (scores, causal softmax, MXInt probabilities and context in one
+launch).  Quantization is discontinuous, so the check is stage by stage on ONE run: the probabilities the
+kernel quantized (optional output) against the oracle's softmax of the oracle's scores -- every code a
+correct rounding of the exact probability up to the fp32 softmax's own error, nearly all codes and exponent
+bytes the oracle's, masked positions exact zeros -- and the context against the oracle's product of the
+kernel's OWN probability codes with the oracle-quantized V, within 1e-5 * S."""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import block_oracle as blk
+from oracle import mx_oracle as orc
+from paper_2307_15517_b200 import synth
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+
+
+@pytest.fixture(scope="module")
+def mxb():
+    from paper_2307_15517_b200 import binding
+    return binding
+
+
+@pytest.mark.parametrize("case", [(2, 256, 16, 8, True), (3, 384, 32, 8, True), (1, 512, 16, 4, True), (2, 256, 16, 8, False)])
+def test_fused_attention_stage_by_stage(mxb, case):
+    H, seq, B, wp, causal = case
+    d, w = 128, 8
+    hid = H * d
+    q = synth.student_t_activations(seq, hid, 21)
+    k = synth.outlier_activations(seq, hid, 22, 3, 20.0)
+    v = synth.student_t_activations(seq, hid, 23)
+    fa, fp = mxb.MxFormat(B, w), mxb.MxFormat(B, wp)
+    qm, qe = mxb.mx_quantize(q.cuda(), fa)
+    km, ke = mxb.mx_quantize(k.cuda(), fa)
+    vm, ve = mxb.mx_quantize(v.cuda().t(), fa)                  # [hid, seq]: blocks along the tokens
+    scale = 1.0 / math.sqrt(d)
+    ctx, pm, pe = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, scale, fp, causal=causal, return_p=True)
+    assert mxb.mx_poll_status() == 0
+    ctx, pm, pe = ctx.cpu().numpy(), pm.cpu().numpy(), pe.cpu().numpy()
+    sc = blk.attention_scores(q.numpy(), k.numpy(), H, d, B, w)
+    qmax = 2 ** (wp - 1) - 1
+    for h in range(H):
+        s_ref = sc[h][0].astype(np.float64)
+        if causal:
+            want = blk.softmax_causal(s_ref, scale, seq)
+        else:
+            z = s_ref * scale
+            e = np.exp(z - z.max(axis=1, keepdims=True))
+            want = e / e.sum(axis=1, keepdims=True)
+        q_or, e_or, _ = orc.quantize(want.astype(np.float32), B, wp)
+        eg = pe[h * seq:(h + 1) * seq]
+        qg = orc.unpack(pm[h * seq:(h + 1) * seq], seq, wp)
+        assert (eg == e_or).mean() > 0.99 and np.abs(eg.astype(int) - e_or.astype(int)).max() <= 1
+        assert (qg == q_or).mean() > 0.98
+        step = np.repeat(np.ldexp(1.0, eg.astype(np.int64) - 127 - (wp - 2)), B, axis=1)
+        tol = 3e-5 * want + 1e-9                          # fp32 exp, row sum and the scores' own tolerance
+        free = np.abs(qg) < qmax
+        assert (np.abs(qg * step - want)[free] <= (0.5 * step + tol)[free]).all()
+        assert (want[~free] >= ((qmax - 0.5) * step - tol)[~free]).all()
+        assert (qg[want == 0] == 0).all()
+        # context from the kernel's own probability codes
+        qv, ev, _ = orc.quantize(np.ascontiguousarray(v.numpy()[:, h * d:(h + 1) * d].T), B, w)
+        y_ref, _, S = orc.gemm(qg, eg, wp, qv, ev, w, B)
+        err = np.abs(ctx[:, h * d:(h + 1) * d].astype(np.float64) - y_ref)
+        assert (err <= TOL * S + 1e-30).all(), (h, float((err / np.maximum(S, 1e-300)).max()))
+
+
+def test_fused_attention_refuses_what_it_cannot_tile(mxb):
+    f = mxb.MxFormat(16, 8)
+    z = lambda r, c: torch.zeros((r, c), dtype=torch.uint8, device="cuda")
+    for seq, H, d, status in ((200, 2, 128, -2), (256, 2, 64, -2)):
+        with pytest.raises(mxb.MxError) as e:
+            mxb.mx_attention(z(seq, H * d), z(seq, H * d // 16), z(seq, H * d), z(seq, H * d // 16), f, z(H * d, seq),
+                             z(H * d, seq // 16), f, seq, H, d, 0.1, f, workspace=mxb.alloc_workspace(1 << 22))
+        assert e.value.status == status

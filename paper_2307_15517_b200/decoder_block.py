@@ -70,6 +70,11 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
     # attention scores per head: both operands MXInt, blocks along the head dimension
     qm, qe = mxb.mx_quantize(q, fa)
     km, ke = mxb.mx_quantize(k, fa)
+    if keep is None and d == 128 and seq % 128 == 0:
+        # scores, causal softmax, quantized probabilities and context in one kernel: nothing of size seq x seq is stored
+        vm, ve = mxb.mx_quantize(v.t(), fa)                      # [hidden, seq]: blocks along tokens
+        ctx = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, 1.0 / math.sqrt(d), fa, causal=True)
+        return _after_attention(cfg, x, ctx, qweights, params, linear, rec)
     s = torch.empty((H * seq, seq), dtype=torch.float32, device=x.device)
     mxb.mx_gemm_batched(qm, qe, fa, hid, d, km, ke, fa, hid, d, seq, seq, d, H, s, seq, seq * seq)
     rec("scores", s.clone() if keep is not None else s)
@@ -84,6 +89,12 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
     ctx = torch.empty((seq, hid), dtype=torch.float32, device=x.device)
     mxb.mx_gemm_batched(pm, pe, fa, seq, seq * seq, vm, ve, fa, seq, d * seq, seq, d, seq, H, ctx, hid, d)
     rec("ctx", ctx)
+    return _after_attention(cfg, x, ctx, qweights, params, linear, rec)
+
+
+def _after_attention(cfg, x, ctx, qweights, params, linear, rec):
+    """Output projection, residual, second LayerNorm and the feed-forward network."""
+    hid = cfg.hidden
     a = rec("attn_out", linear(ctx, "wo", params["bo"], hid))
     x1 = rec("x1", mxb.mx_relu_add(a, x))
     h2 = rec("ln2", mxb.mx_layernorm(x1, params["ln2_g"], params["ln2_b"], cfg.eps))

@@ -186,3 +186,53 @@ def test_decoder_block_opt67b_shapes_stage_by_stage(mods):
     res = out.cpu().numpy()
     assert np.array_equal(res, ffn_out + x1)
     assert np.isfinite(res).all()
+
+
+def test_fused_attention_opt67b_shapes(mods):
+    """The fused attention kernel at 32 heads x 128, sequence 2048 (512 work items over 148 CTAs, up to 16 key
+    tiles per item): on sampled query rows of every fourth head, the probabilities it quantized against the
+    oracle's softmax of the oracle's scores, and the context against the oracle's product of the kernel's own
+    probability codes with the oracle-quantized V."""
+    mxb, _ = mods
+    H, seq, d, B, w = 32, 2048, 128, 16, 8
+    hid = H * d
+    q = synth.student_t_activations(seq, hid, 31)
+    k = synth.outlier_activations(seq, hid, 32, 20, 20.0)
+    v = synth.student_t_activations(seq, hid, 33)
+    fa = mxb.MxFormat(B, w)
+    qm, qe = mxb.mx_quantize(q.cuda(), fa)
+    km, ke = mxb.mx_quantize(k.cuda(), fa)
+    vm, ve = mxb.mx_quantize(v.cuda().t(), fa)
+    scale = 1.0 / math.sqrt(d)
+    ctx, pm, pe = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, scale, fa, causal=True, return_p=True)
+    assert mxb.mx_poll_status() == 0
+    ctx2 = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, scale, fa, causal=True)
+    assert torch.equal(ctx, ctx2)                                  # the optional output changes nothing
+    ctx = ctx.cpu().numpy()
+    rng = np.random.default_rng(3)
+    qn, kn, vn = q.numpy(), k.numpy(), v.numpy()
+    for h in range(0, H, 4):
+        rows = np.sort(rng.choice(seq, 24, replace=False))
+        rows[0], rows[-1] = 0, seq - 1
+        qa, ea, _ = orc.quantize(np.ascontiguousarray(qn[rows, h * d:(h + 1) * d]), B, w)
+        qk, ek, _ = orc.quantize(np.ascontiguousarray(kn[:, h * d:(h + 1) * d]), B, w)
+        s_ref, _, _ = orc.gemm(qa, ea, w, qk, ek, w, B)             # [24, seq]
+        z = s_ref.astype(np.float64) * scale
+        mask = np.arange(seq)[None, :] <= rows[:, None]
+        z = np.where(mask, z, -np.inf)
+        e = np.where(mask, np.exp(z - z.max(axis=1, keepdims=True)), 0.0)
+        want = e / e.sum(axis=1, keepdims=True)
+        q_or, e_or, _ = orc.quantize(want.astype(np.float32), B, w)
+        sel = torch.from_numpy(h * seq + rows).cuda()
+        eg = pe[sel].cpu().numpy()
+        qg = orc.unpack(pm[sel].cpu().numpy(), seq, w)
+        assert (eg == e_or).mean() > 0.99 and np.abs(eg.astype(int) - e_or.astype(int)).max() <= 1
+        assert (qg == q_or).mean() > 0.98
+        step = np.repeat(np.ldexp(1.0, eg.astype(np.int64) - 127 - (w - 2)), B, axis=1)
+        tol = 3e-5 * want + 1e-9
+        free = np.abs(qg) < 127
+        assert (np.abs(qg * step - want)[free] <= (0.5 * step + tol)[free]).all()
+        assert (qg[~mask] == 0).all()
+        qv, ev, _ = orc.quantize(np.ascontiguousarray(vn[:, h * d:(h + 1) * d].T), B, w)
+        y_ref, _, S = orc.gemm(qg, eg, w, qv, ev, w, B)
+        _close(ctx[rows][:, h * d:(h + 1) * d], y_ref, S, "ctx head %d" % h)

@@ -11,13 +11,18 @@
 // sweep recomputes each score tile, normalises with the FINAL m and l and quantizes, so a probability
 // sees the same block exponent as in the unfused path.  Fully masked key tiles are skipped in both sweeps.
 //
-// One work item = (head, 128 queries); persistent CTAs take items round-robin, long rows first.
+// One work item = (head, 128 queries); items are ordered long rows first and dealt to the persistent CTAs
+// in alternating direction (round k: CTA b takes item k*G + b, then k*G + G-1-b, ...), which evens out the
+// causal rows' unequal lengths.
 //   warp 0      : TMA producer: Q tile once per item, K tiles (both sweeps), V^T tiles (second sweep)
 //   warp 1      : tensor-memory allocation, MMA issue: S_j = Q K_j^T (8 steps of K = 16) into one of two
 //                 score accumulators; O += P_j V_j (8 steps) into the context accumulator
-//   warps 2..5  : one query row per thread: statistics in sweep 1; in sweep 2 scores -> probabilities ->
-//                 MXInt codes -> exact bf16 -> the swizzled P operand tile in shared memory; at the end
-//                 the context tile out of tensor memory into global memory
+//   warps 2..   : ROW_WARPS row warps: warp w reads TMEM lanes 32 * (w % 4) .. + 31 (its hardware window), i.e.
+//                 32 query rows, and a slice of 128 / (ROW_WARPS / 4) key columns of every tile (the warps of a
+//                 row combine their maxima and sums once, between the sweeps, through shared memory).
+//                 Sweep 1: statistics; sweep 2: scores -> probabilities -> MXInt codes -> exact bf16 -> the
+//                 swizzled P operand tile in shared memory; at the end the context tile out of tensor
+//                 memory into global memory.  exp is ex2.approx on arguments pre-scaled by log2(e)
 // Every 128 x 128 bf16 tile is stored as two halves of 128 rows x 128 bytes (64 columns) with the
 // 128-byte swizzle.  All waits are bounded.
 #pragma once
@@ -37,7 +42,11 @@ struct AttnCfg {
     static constexpr uint32_t TILE_BYTES = 128 * 128 * 2;            // 32 KB, two halves of 16 KB
     static constexpr uint32_t HALF_BYTES = TILE_BYTES / 2;
     static constexpr int KST = 2, VST = 2;                           // K and V^T stage rings
-    static constexpr uint32_t SMEM_BYTES = (1 + KST + VST + 1) * TILE_BYTES + 512 + 1024;    // Q, K ring, V ring, P
+    static constexpr int ROW_WARPS = 16;                             // 4 per TMEM lane quarter: 32 key columns each
+    static constexpr int COLS_PER_WARP = 128 / (ROW_WARPS / 4);
+    static constexpr int THREADS = 64 + 32 * ROW_WARPS;
+    static constexpr uint32_t STATS_BYTES = 2 * (ROW_WARPS / 4) * 128 * 8;   // (maximum, sum) per row and column slice, two items deep
+    static constexpr uint32_t SMEM_BYTES = (1 + KST + VST + 1) * TILE_BYTES + 512 + STATS_BYTES + 1024;    // Q, K ring, V ring, P
     static constexpr uint32_t TMEM_COLS = 512;                       // S0, S1, O: 3 x 128 columns
 };
 
@@ -65,8 +74,18 @@ __device__ __forceinline__ void attn_mma_k128(uint32_t d_tmem, uint32_t a_tile, 
                              (accumulate || hh || j) ? 1u : 0u);
 }
 
+// Item of CTA b in round k of G CTAs: the direction alternates between rounds.
+__device__ __forceinline__ int attn_item(uint32_t k, int b, int G) { return (int)k * G + ((k & 1u) ? G - 1 - b : b); }
+
 // tmap_q, tmap_k: bf16 [seq, heads*128], box 64 x 128.  tmap_v: bf16 [heads*128, seq] (V transposed), box 64 x 128.
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__device__ __forceinline__ float exp2_approx(float x)
+{
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__global__ void __launch_bounds__(AttnCfg::THREADS, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const AttnParams p)
 {
@@ -80,16 +99,17 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const uint32_t p_tile = v_tiles + Cfg::VST * Cfg::TILE_BYTES;
     const uint32_t bar_base = p_tile + Cfg::TILE_BYTES;
     // barriers: 0 q_full, 1 q_empty, 2..3 k_full, 4..5 k_empty, 6..7 v_full, 8..9 v_empty, 10..11 s_full,
-    //           12..13 s_empty, 14 p_full, 15 p_empty, 16 o_full, 17 o_empty
+    //           12..13 s_empty, 14 p_full, 15 p_empty, 16 o_full, 17 o_empty, 18 row statistics written
     auto bar = [&](int i) { return bar_base + 8u * i; };
-    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + (bar_base - smem_base) + 8 * 18);
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem_gen + (bar_base - smem_base) + 8 * 19);
     volatile uint32_t *abort_flag = tmem_slot + 1;
+    float2 *stats = reinterpret_cast<float2 *>(smem_gen + (bar_base - smem_base) + 512);    // [slice][row]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 18; ++i) {
-            const bool by_rows = i == 12 || i == 13 || i == 14 || i == 17;      // arrived on by the four row warps
-            ptx::mbar_init(bar(i), by_rows ? 4 : 1);
+        for (int i = 0; i < 19; ++i) {
+            const bool by_rows = i == 12 || i == 13 || i == 14 || i == 17 || i == 18;      // arrived on by every row warp
+            ptx::mbar_init(bar(i), by_rows ? Cfg::ROW_WARPS : 1);
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -116,7 +136,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     if (warp == 0) {
         if (lane == 0) {
             uint32_t n_item = 0, n_k = 0, n_v = 0;                    // uses so far of the Q tile and the two rings
-            for (int w = blockIdx.x; w < items && !timed_out; w += gridDim.x, ++n_item) {
+            for (int w = attn_item(0, blockIdx.x, gridDim.x); w < items && !timed_out; ++n_item, w = attn_item(n_item, blockIdx.x, gridDim.x)) {
                 const int qt = q_tiles_n - 1 - w / p.heads, h = w % p.heads;
                 const int T = p.causal ? qt + 1 : q_tiles_n;
                 if (!wait(1, (n_item & 1u) ^ 1u)) { timed_out = true; break; }
@@ -162,7 +182,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 ++n_s;
                 return true;
             };
-            for (int w = blockIdx.x; w < items && !timed_out; w += gridDim.x, ++n_item) {
+            for (int w = attn_item(0, blockIdx.x, gridDim.x); w < items && !timed_out; ++n_item, w = attn_item(n_item, blockIdx.x, gridDim.x)) {
                 const int qt = q_tiles_n - 1 - w / p.heads;
                 const int T = p.causal ? qt + 1 : q_tiles_n;
                 if (!wait(0, n_item & 1u)) { timed_out = true; break; }
@@ -193,53 +213,79 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         __syncwarp();
     } else {
         const int quad = warp & 3;
+        const int slice = (warp - 2) >> 2;                   // which COLS_PER_WARP key columns of every tile
+        constexpr int CHUNKS = Cfg::COLS_PER_WARP / 32;
         const int r = quad * 32 + lane;                      // this thread's query row inside the tile
         const uint32_t lane_tmem = tmem_base + ((uint32_t)(quad * 32) << 16);
         const uint32_t p_row = p_tile + (uint32_t)((r >> 3) * 1024 + (r & 7) * 128);
         const bool nibble = p.p_bits <= 4;
+        const float scale2 = p.scale * 1.4426950408889634f;  // scores in units of log2: exp(x) = 2^(x log2 e)
         uint32_t n_item = 0, n_s = 0, n_p = 0;
-        for (int w = blockIdx.x; w < items && !timed_out; w += gridDim.x, ++n_item) {
+        for (int w = attn_item(0, blockIdx.x, gridDim.x); w < items && !timed_out; ++n_item, w = attn_item(n_item, blockIdx.x, gridDim.x)) {
             const int qt = q_tiles_n - 1 - w / p.heads, h = w % p.heads;
             const int T = p.causal ? qt + 1 : q_tiles_n;
             const int qrow = qt * Cfg::BQ + r;
             float m = -INFINITY, l = 0.f;
             for (int sweep = 0; sweep < 2 && !timed_out; ++sweep) {
+                if (sweep == 1) {
+                    // combine the statistics of the row's column slices: one exchange per item.  The buffer
+                    // alternates between items, so a warp that runs ahead never overwrites values still being read
+                    float2 *st_buf = stats + (n_item & 1u) * (Cfg::ROW_WARPS / 4) * 128;
+                    st_buf[slice * 128 + r] = make_float2(m, l);
+                    __syncwarp();
+                    if (lane == 0) ptx::mbar_arrive(bar(18));
+                    if (!__all_sync(0xFFFFFFFFu, wait(18, n_item & 1u))) { timed_out = true; break; }
+                    float mm = -INFINITY;
+#pragma unroll
+                    for (int q = 0; q < Cfg::ROW_WARPS / 4; ++q) mm = fmaxf(mm, st_buf[q * 128 + r].x);
+                    float ll = 0.f;
+#pragma unroll
+                    for (int q = 0; q < Cfg::ROW_WARPS / 4; ++q) {
+                        const float2 st = st_buf[q * 128 + r];
+                        ll += st.x == -INFINITY ? 0.f : st.y * exp2_approx(st.x - mm);
+                    }
+                    m = mm;
+                    l = ll;
+                }
                 const float inv = sweep ? 1.0f / l : 0.f;
                 for (int j = 0; j < T; ++j) {
                     const uint32_t si = n_s & 1u;
-                    bool ok = wait(10 + si, (n_s >> 1) & 1u);
-                    if (sweep == 1 && ok) ok = wait(15, (n_p & 1u) ^ 1u);       // the previous P tile has been consumed
-                    if (!__all_sync(0xFFFFFFFFu, ok)) { timed_out = true; break; }
+                    if (!__all_sync(0xFFFFFFFFu, wait(10 + si, (n_s >> 1) & 1u))) { timed_out = true; break; }
                     ptx::tc_fence_after_sync();
                     const int limit = p.causal ? qrow - j * Cfg::BKEY : Cfg::BKEY;   // keys 0..limit of this tile take part
 #pragma unroll 1
-                    for (int c = 0; c < 4; ++c) {
+                    for (int cc = 0; cc < CHUNKS; ++cc) {
+                        const int c = slice * CHUNKS + cc;
                         uint32_t raw[32];
                         ptx::tmem_ld_32x32(lane_tmem + si * 128u + (uint32_t)(c * 32), raw);
                         ptx::tmem_ld_wait();
                         float v[32];
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = (c * 32 + i <= limit) ? __uint_as_float(raw[i]) * p.scale : -INFINITY;
+                        for (int i = 0; i < 32; ++i) v[i] = (c * 32 + i <= limit) ? __uint_as_float(raw[i]) * scale2 : -INFINITY;
                         if (sweep == 0) {
                             float cm = m;
 #pragma unroll
                             for (int i = 0; i < 32; ++i) cm = fmaxf(cm, v[i]);
                             if (cm > m) {                               // the running sum follows the maximum
-                                l *= expf(m - cm);
+                                l *= exp2_approx(m - cm);
                                 m = cm;
                             }
-                            float s = 0.f;
+                            if (m != -INFINITY) {
+                                float s = 0.f;
 #pragma unroll
-                            for (int i = 0; i < 32; ++i) s += v[i] == -INFINITY ? 0.f : expf(v[i] - m);
-                            l += s;
+                                for (int i = 0; i < 32; ++i) s += exp2_approx(v[i] - m);      // 2^-inf = 0 for masked keys
+                                l += s;
+                            }
                         } else {
                             uint32_t amax[2] = {0u, 0u};
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
-                                v[i] = v[i] == -INFINITY ? 0.f : expf(v[i] - m) * inv;
+                                v[i] = exp2_approx(v[i] - m) * inv;
                                 amax[i >> 4] = max(amax[i >> 4], __float_as_uint(v[i]));     // v >= 0: bits order like values
                             }
                             if (p.p_block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
+                            // the previous P tile must have been consumed before the first store of this one
+                            if (cc == 0 && !__all_sync(0xFFFFFFFFu, wait(15, (n_p & 1u) ^ 1u))) { timed_out = true; break; }
                             const int64_t prow = (int64_t)h * p.seq + qrow;
                             const int key0 = j * Cfg::BKEY + c * 32;
 #pragma unroll
@@ -266,12 +312,13 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                             }
                         }
                     }
+                    if (timed_out) break;
                     ptx::tc_fence_before_sync();
                     if (sweep == 1) ptx::fence_proxy_async_smem();      // the P tile's stores -> visible to the MMA
                     __syncwarp();
                     if (lane == 0) {
                         ptx::mbar_arrive(bar(12 + si));                  // score accumulator free
-                        if (sweep == 1) ptx::mbar_arrive(bar(14));       // this warp's 32 rows of P are in place
+                        if (sweep == 1) ptx::mbar_arrive(bar(14));       // this warp's piece of P is in place
                     }
                     ++n_s;
                     if (sweep == 1) ++n_p;
@@ -284,7 +331,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
             ptx::tc_fence_after_sync();
             float *orow = p.ctx + (int64_t)qrow * p.ldc + h * Cfg::D;
 #pragma unroll 1
-            for (int c = 0; c < 4; ++c) {
+            for (int cc = 0; cc < CHUNKS; ++cc) {
+                const int c = slice * CHUNKS + cc;
                 uint32_t raw[32];
                 ptx::tmem_ld_32x32(lane_tmem + 256u + (uint32_t)(c * 32), raw);
                 ptx::tmem_ld_wait();

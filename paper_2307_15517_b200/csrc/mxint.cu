@@ -1576,7 +1576,7 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     const int64_t items = (seq / mx::AttnCfg::BQ) * heads;
     const int grid = items < d->sm_count ? (int)items : d->sm_count;
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::TC_THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
+    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::AttnCfg::THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }

@@ -395,6 +395,39 @@ MX_API mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t 
                         uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
                         size_t workspace_bytes, void *stream);
 
+/* ---- the product with a fused element-wise tail ------------------------------------------------
+ *
+ * Fig. 1(d): between the MX operators of a decoder block sit a bias, the activation function and the
+ * skip connection, all in floating point.  These two calls are mx_gemm / mx_linear (fp32 result y) or
+ * mx_gemm_q / mx_linear_q (MXInt result fy, y_mant, y_exp) with that tail applied in the product kernel's
+ * epilogue, on the fp32 accumulator, before the result is stored or quantized:
+ *     out[i,j] = act(acc[i,j] + bias[j]) + residual[i*ldr + j],   act(t) = relu ? (t < 0 ? 0 : t) : t
+ * so no separate pass over the fp32 tensor remains.  Exactly one of y and y_mant is non-null
+ * (MX_ERR_NULL otherwise); fy is ignored for an fp32 result.  ep may be NULL (no tail).
+ * residual is device fp32, 4-byte aligned (16-byte aligned with ldr % 4 == 0 takes vector loads),
+ * ldr >= N (MX_ERR_SHAPE); it may alias y only element for element (y = residual in place is fine).
+ * Always the tensor-core kernels; workspace as for MX_ALGO_TCGEN05.  Everything else as for the calls
+ * named above.
+ */
+typedef struct {
+    const float *bias;      /* device, [N], nullable                                   */
+    int32_t relu;           /* != 0: clamp negatives to zero after the bias (NaN stays) */
+    const float *residual;  /* device, [M, ldr] fp32, nullable: added last             */
+    int64_t ldr;            /* elements between the rows of residual                   */
+} mx_epilogue_t;
+
+MX_API mx_status_t mx_gemm_fused(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
+                          const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t M,
+                          int64_t N, int64_t K, const mx_epilogue_t *ep, float *y, int64_t ldy,
+                          mx_format_t fy, void *y_mant, uint8_t *y_exp, void *workspace,
+                          size_t workspace_bytes, void *stream);
+
+MX_API mx_status_t mx_linear_fused(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
+                            mx_format_t fa, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                            int64_t N, const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy,
+                            void *y_mant, uint8_t *y_exp, void *workspace, size_t workspace_bytes,
+                            void *stream);
+
 /* ---- the other MX formats of the paper: Block Minifloat and Block Logarithm ---------------------
  *
  * Sec. 2 "What are MX Formats?" puts two more block formats beside MXInt and Table 1 / Fig. 5 compare

@@ -43,6 +43,11 @@ class MxFormat(C.Structure):
                                                                                   self.block_rows, self.packing)
 
 
+class MxEpilogue(C.Structure):
+    """Mirrors ``mx_epilogue_t``: bias, activation and residual applied in the product's epilogue."""
+    _fields_ = [("bias", C.c_void_p), ("relu", C.c_int32), ("residual", C.c_void_p), ("ldr", C.c_int64)]
+
+
 class MxAltFormat(C.Structure):
     """A Block Minifloat (kind 1) or Block Logarithm (kind 2) format: mirrors ``mx_alt_format_t``."""
     _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("elem_exp_bits", C.c_int32),
@@ -108,6 +113,11 @@ def _load() -> C.CDLL:
     L.mx_linear_q.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, vp, F, vp, vp, vp, vp, sz, vp]
     L.mx_gemm_q.restype = i32
     L.mx_linear_q.restype = i32
+    E = C.POINTER(MxEpilogue)
+    L.mx_gemm_fused.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
+    L.mx_linear_fused.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
+    L.mx_gemm_fused.restype = i32
+    L.mx_linear_fused.restype = i32
     L.mx_poll_status.argtypes = [vp]
     L.mx_selftest_wait_expiry.argtypes = [C.c_uint32, vp]
     L.mx_selftest_wait_expiry.restype = i32
@@ -349,6 +359,65 @@ def mx_linear_q(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: i
                            fw, N, _ptr(bias), fy, _ptr(y_mant), _ptr(y_exp), _ptr(nonfinite_count),
                            _ptr(workspace), workspace.numel(), _stream(stream)), "mx_linear_q")
     return y_mant, y_exp
+
+
+def _epilogue(bias, relu, residual):
+    ep = MxEpilogue()
+    ep.bias = None if bias is None else bias.data_ptr()
+    ep.relu = 1 if relu else 0
+    ep.residual = None if residual is None else residual.data_ptr()
+    ep.ldr = 0 if residual is None else residual.stride(0)
+    return ep
+
+
+def mx_linear_fused(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int,
+                    bias: Optional[torch.Tensor] = None, relu: bool = False,
+                    residual: Optional[torch.Tensor] = None, fy: Optional[MxFormat] = None, y=None,
+                    y_mant=None, y_exp=None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """mx_linear with bias, ReLU and a residual applied in the epilogue.  ``fy`` None: returns the fp32
+    result; else returns (y_mant, y_exp), the result quantized to ``fy`` along N."""
+    _need_cuda(x, w_mant, w_exp, bias, residual, y, y_mant, y_exp, workspace)
+    M, K = x.shape
+    assert x.stride(1) == 1 and (residual is None or (residual.stride(1) == 1 and residual.dtype == torch.float32))
+    if fy is None:
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float32, device=x.device)
+        assert y.dtype == torch.float32 and y.stride(1) == 1
+    else:
+        y_mant, y_exp = _quantized_out(M, N, fy, x.device, y_mant, y_exp)
+    if workspace is None:
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_TCGEN05), x.device)
+    ep = _epilogue(bias, relu, residual)
+    _check(lib.mx_linear_fused(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant), _ptr(w_exp), fw, N,
+                               C.byref(ep), _ptr(y) if fy is None else None, y.stride(0) if fy is None else N,
+                               fy if fy is not None else MxFormat(), None if fy is None else _ptr(y_mant),
+                               None if fy is None else _ptr(y_exp), _ptr(workspace), workspace.numel(),
+                               _stream(stream)), "mx_linear_fused")
+    return y if fy is None else (y_mant, y_exp)
+
+
+def mx_gemm_fused(a_mant, a_exp, fa: MxFormat, w_mant, w_exp, fw: MxFormat, M: int, N: int, K: int,
+                  bias: Optional[torch.Tensor] = None, relu: bool = False,
+                  residual: Optional[torch.Tensor] = None, fy: Optional[MxFormat] = None, y=None,
+                  y_mant=None, y_exp=None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """mx_gemm with bias, ReLU and a residual applied in the epilogue; result as for ``mx_linear_fused``."""
+    _need_cuda(a_mant, a_exp, w_mant, w_exp, bias, residual, y, y_mant, y_exp, workspace)
+    assert residual is None or (residual.stride(1) == 1 and residual.dtype == torch.float32)
+    if fy is None:
+        if y is None:
+            y = torch.empty((M, N), dtype=torch.float32, device=a_mant.device)
+        assert y.dtype == torch.float32 and y.stride(1) == 1
+    else:
+        y_mant, y_exp = _quantized_out(M, N, fy, a_mant.device, y_mant, y_exp)
+    if workspace is None:
+        workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_TCGEN05), a_mant.device)
+    ep = _epilogue(bias, relu, residual)
+    _check(lib.mx_gemm_fused(_ptr(a_mant), _ptr(a_exp), fa, _ptr(w_mant), _ptr(w_exp), fw, M, N, K, C.byref(ep),
+                             _ptr(y) if fy is None else None, y.stride(0) if fy is None else N,
+                             fy if fy is not None else MxFormat(), None if fy is None else _ptr(y_mant),
+                             None if fy is None else _ptr(y_exp), _ptr(workspace), workspace.numel(),
+                             _stream(stream)), "mx_gemm_fused")
+    return y if fy is None else (y_mant, y_exp)
 
 
 def make_linear_args(layers):

@@ -87,7 +87,69 @@ struct TcParams {
     uint32_t *yq_nonfinite;   // nullable: number of blocks that held Inf/NaN
     int yq_bits, yq_block;
     int yq_rows2;             // 1: rows 2i and 2i+1 share the exponent bytes (two-row blocks); exponents [M/2, N/yq_block]
+    // Fused element-wise tail (one-CTA and CTA-pair kernels, batch == 1): when relu != 0 or residual is set the
+    // epilogue forms  act(acc + ex_bias[n]) + residual[row, n]  (act = max(., 0) if relu) before the fp32 or MXInt
+    // store; the host then passes the bias here and leaves `bias` null (Fig. 1(d): activation and skip
+    // connection stay in floating point around the MX operators).
+    const float *ex_bias;
+    int relu;
+    const float *residual;
+    int64_t ldr;
 };
+
+// The residual values of a lane's 32 consecutive outputs (columns n .. n + 31) of row `row`.  Fetched one
+// chunk ahead of their use: the loads cross the L2 while the previous chunk is processed (issued right before
+// use they cost the epilogue warp a memory latency per chunk: 164 -> 225 us on 2048 x 16384 x 4096).
+struct TailRegs { float4 res[8]; };
+
+__device__ __forceinline__ void tail_fetch(const TcParams &p, int row, int n, TailRegs &t)
+{
+    if (!p.residual) return;
+    const bool live = row < p.M && n < p.N;
+    const float *res = p.residual + (int64_t)row * p.ldr + n;
+    const bool vec = live && n + 32 <= p.N && ((p.ldr & 3) == 0) && ((reinterpret_cast<uintptr_t>(p.residual) & 15) == 0);
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+        if (vec) {
+            t.res[v] = __ldg(reinterpret_cast<const float4 *>(res) + v);
+        } else {
+            const int c = n + 4 * v;
+            t.res[v].x = live && c + 0 < p.N ? __ldg(res + 4 * v + 0) : 0.f;
+            t.res[v].y = live && c + 1 < p.N ? __ldg(res + 4 * v + 1) : 0.f;
+            t.res[v].z = live && c + 2 < p.N ? __ldg(res + 4 * v + 2) : 0.f;
+            t.res[v].w = live && c + 3 < p.N ? __ldg(res + 4 * v + 3) : 0.f;
+        }
+    }
+}
+
+// act(acc + bias) + residual on those 32 outputs, in place.
+__device__ __forceinline__ void tail_apply(const TcParams &p, const TailRegs &t, int n, uint32_t (&r)[32])
+{
+    const bool bvec = p.ex_bias && n + 32 <= p.N;          // the bias pointer is 16-byte aligned (checked on the host)
+#pragma unroll
+    for (int v = 0; v < 8; ++v) {
+        float o[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[i] = __uint_as_float(r[4 * v + i]);
+        if (bvec) {
+            const float4 bq = __ldg(reinterpret_cast<const float4 *>(p.ex_bias + n) + v);
+            o[0] += bq.x; o[1] += bq.y; o[2] += bq.z; o[3] += bq.w;
+        } else if (p.ex_bias) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (n + 4 * v + i < p.N) o[i] += __ldg(p.ex_bias + n + 4 * v + i);
+        }
+        if (p.relu) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[i] = o[i] < 0.f ? 0.f : o[i];       // NaN stays NaN
+        }
+        if (p.residual) {
+            o[0] += t.res[v].x; o[1] += t.res[v].y; o[2] += t.res[v].z; o[3] += t.res[v].w;
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) r[4 * v + i] = __float_as_uint(o[i]);
+    }
+}
 
 // MXInt-result epilogue of one lane: r holds 32 consecutive fp32 outputs (columns n .. n + 31) of
 // row `row`, i.e. one block of 32 or two blocks of 16 along N; no exchange between lanes is needed.
@@ -146,13 +208,15 @@ __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, in
 // TMA store -- whole 128-byte lines reach L2, rows >= M and columns >= N are clipped by the store --
 // or, when ldy % 4 != 0, with plain stores.  `epi_buf` counts the warp's TMA blocks (buffer parity).
 // Shared by the one-CTA, the CTA-pair and the block-wise kernel.
+// NBUF = 1: the warp has one 4 KB buffer and waits for its previous store to have been read.
+template <int NBUF = 2>
 __device__ __forceinline__ void store_f32_chunk(const TcParams &p, const CUtensorMap *tmap_y, uint32_t (&r)[32], int row,
                                                 int rows0, int n, int tb, uint32_t warp_bufs, uint32_t &epi_buf, int lane)
 {
     if (p.tma_store) {
         if (n < p.N && rows0 < p.M) {                      // warp-uniform
-            const uint32_t buf = warp_bufs + (epi_buf & 1u) * 4096u;
-            if (lane == 0) ptx::bulk_wait_group_read<1>();   // the buffer used two blocks ago is free
+            const uint32_t buf = warp_bufs + (NBUF == 2 ? (epi_buf & 1u) * 4096u : 0u);
+            if (lane == 0) ptx::bulk_wait_group_read<NBUF - 1>();   // the buffer used NBUF blocks ago is free
             __syncwarp();
 #pragma unroll
             for (int v = 0; v < 8; ++v) {
@@ -568,11 +632,15 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int quad = warp & 3;                          // TMEM lanes this warp may read
         int it = 0;
         uint32_t epi_buf = 0;                               // alternates between the warp's two store buffers
+        const bool tail = !FUSED && (p.relu != 0 || p.residual != nullptr);
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
             const int tb = t / tiles_item, tt = t - tb * tiles_item;
             const int m0 = (tt % p.tiles_m) * TC_BM, n0 = (tt / p.tiles_m) * BN;
+            const int row = m0 + quad * 32 + lane;
+            TailRegs t0, t1;
+            if (tail) tail_fetch(p, row, n0, t0);              // the first chunk's residual: in flight under the MMAs
             // every lane waits (acquire), then the warp agrees on the outcome so that the
             // warp-collective TMEM loads below are never executed by a partial warp
             const bool ok = ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
@@ -581,18 +649,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 break;
             }
             ptx::tc_fence_after_sync();
-            const int row = m0 + quad * 32 + lane;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            auto chunk = [&](int c0, TailRegs &cur, TailRegs &next) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                if (tail && c0 + 32 < BN) tail_fetch(p, row, n0 + c0 + 32, next);     // in flight under this chunk
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
+                if (tail) tail_apply(p, cur, n, r);
                 if (!FUSED && p.yq_mant) {
                     store_mxint_chunk(p, row, n, r);
-                    continue;
+                    return;
                 }
                 store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
+            };
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 64) {
+                chunk(c0, t0, t1);
+                chunk(c0 + 32, t1, t0);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

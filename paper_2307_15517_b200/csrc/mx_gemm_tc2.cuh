@@ -10,10 +10,13 @@
 //
 //   warp 0      : TMA producer (one lane, in both CTAs; bytes are counted on the leader's barrier)
 //   warp 1      : tensor-memory allocation (both CTAs), MMA issue (leader only)
-//   warps 2..5  : epilogue of the CTA's own 128 rows (fp32, or MXInt as in the one-CTA kernel)
+//   warps 2..9  : epilogue of the CTA's own 128 rows (fp32, or MXInt as in the one-CTA kernel): warp w reads
+//                 TMEM lanes 32 * (w % 4) .. + 31 and 128 of the 256 columns -- two warps per scheduler, so one
+//                 warp's TMEM and memory latencies hide under the other's arithmetic, and the last tile's
+//                 epilogue, which nothing overlaps, takes half as long
 // Barriers: full[s] lives in the leader (one arrival + the bytes of both CTAs), empty[s] and
 // tfull[a] in both (the MMA thread's commits are multicast to the pair), tempty[a] in the leader
-// (eight arrivals: the four epilogue warps of both CTAs).  No TMA load is multicast.  Every wait
+// (sixteen arrivals: the eight epilogue warps of both CTAs).  No TMA load is multicast.  Every wait
 // is bounded; both CTAs always reach the closing cluster barrier.
 #pragma once
 #include <cuda.h>
@@ -32,12 +35,14 @@ struct Tc2Cfg {
     static constexpr uint32_t W_BYTES = (BN / 2) * TC_BK * 2;       // this CTA's 128 rows of W
     static constexpr uint32_t STAGE_BYTES = A_BYTES + W_BYTES;
     static constexpr uint32_t BAR_BYTES = 256;
-    static constexpr uint32_t EPI_BYTES = 4 * 2 * 4096;
+    static constexpr int EPI_WARPS = 8;                   // two per TMEM lane quarter: 128 of the tile's 256 columns each
+    static constexpr int THREADS = 64 + 32 * EPI_WARPS;
+    static constexpr uint32_t EPI_BYTES = EPI_WARPS * 4096;         // one 32x32 fp32 store buffer per epilogue warp
     static constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + EPI_BYTES + BAR_BYTES + 1024;
     static constexpr uint32_t TMEM_COLS = 512;            // two accumulators of 256 columns
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(TC_THREADS, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Tc2Cfg::THREADS, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                 const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
 {
@@ -67,7 +72,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(tfull_bar(a), 1);
-            ptx::mbar_init(tempty_bar(a), 8);              // four epilogue warps of each CTA
+            ptx::mbar_init(tempty_bar(a), 2 * Cfg::EPI_WARPS);      // the epilogue warps of both CTAs
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -150,31 +155,42 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         }
         __syncwarp();
     } else {
-        const int quad = warp & 3;
+        const int quad = warp & 3;                           // TMEM lane quarter (the hardware's window for this warp)
+        const int col0 = ((warp - 2) >> 2) * (BN / (Cfg::EPI_WARPS / 4));   // this warp's columns of the tile
+        constexpr int COLS = BN / (Cfg::EPI_WARPS / 4);
         int it = 0;
         uint32_t epi_buf = 0;
+        const bool tail = p.relu != 0 || p.residual != nullptr;
         for (int t = pair; t < num_tiles && !timed_out; t += npairs, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
             const int m0 = (t % p.tiles_m) * 256 + (int)rank * 128, n0 = (t / p.tiles_m) * BN;
+            const int row = m0 + quad * 32 + lane;
+            TailRegs t0, t1;
+            if (tail) tail_fetch(p, row, n0 + col0, t0);       // the first chunk's residual: in flight under the MMAs
             const bool ok = ptx::mbar_wait_bounded_cluster(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
             if (!__all_sync(0xFFFFFFFFu, ok)) {
                 timed_out = true;
                 break;
             }
             ptx::tc_fence_after_sync();
-            const int row = m0 + quad * 32 + lane;
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            auto chunk = [&](int c0, TailRegs &cur, TailRegs &next) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
+                if (tail && c0 + 32 < col0 + COLS) tail_fetch(p, row, n0 + c0 + 32, next);     // in flight under this chunk
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
+                if (tail) tail_apply(p, cur, n, r);
                 if (p.yq_mant) {
                     store_mxint_chunk(p, row, n, r);
-                    continue;
+                    return;
                 }
-                store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, 0, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
+                store_f32_chunk<1>(p, &tmap_y, r, row, m0 + quad * 32, n, 0, epi_base + (uint32_t)(warp - 2) * 4096u, epi_buf, lane);
+            };
+#pragma unroll 1
+            for (int c0 = col0; c0 < col0 + COLS; c0 += 64) {
+                chunk(c0, t0, t1);
+                chunk(c0 + 32, t1, t0);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

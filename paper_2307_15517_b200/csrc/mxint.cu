@@ -373,6 +373,13 @@ struct TcBatch {                 // several products of one shape in one launch 
     bool no_events = false;          // never bracket the launch with profile events (mx_gemm_static)
 };
 
+struct EpiTail {                 // element-wise tail fused into the product's epilogue (see TcParams::relu)
+    int relu = 0;
+    const float *residual = nullptr;
+    int64_t ldr = 0;
+    bool any() const { return relu != 0 || residual != nullptr; }
+};
+
 struct PackedW {                 // weight operand of the fused kernels (unused for W_BF16)
     const uint8_t *mant = nullptr;
     const uint8_t *exps = nullptr;
@@ -402,7 +409,8 @@ mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int6
 template <int BN, int WMODE>
 mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
                       int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
-                      const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st, const TcBatch &tb = TcBatch())
+                      const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st, const TcBatch &tb = TcBatch(),
+                      const EpiTail &et = EpiTail())
 {
     using Cfg = mx::TcCfg<BN>;
     CUtensorMap tm_a, tm_w;
@@ -425,7 +433,11 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     if (s != MX_OK) return s;
     mx::TcParams p;
     p.y = y;
-    p.bias = bias;
+    p.bias = et.any() ? nullptr : bias;
+    p.ex_bias = et.any() ? bias : nullptr;
+    p.relu = et.relu;
+    p.residual = et.residual;
+    p.ldr = et.ldr;
     p.ldy = ldy;
     p.M = (int)M;
     p.N = (int)N;
@@ -464,7 +476,8 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
 
 // The CTA-pair kernel: 256 x 256 tiles, one product per launch.
 mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N, int64_t K,
-                       const float *bias, float *y, int64_t ldy, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st)
+                       const float *bias, float *y, int64_t ldy, const QuantizedOut *yq, DeviceInfo &d, cudaStream_t st,
+                       const EpiTail &et = EpiTail())
 {
     using Cfg = mx::Tc2Cfg;
     CUtensorMap tm_a, tm_w;
@@ -482,7 +495,11 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     if (s != MX_OK) return s;
     mx::TcParams p{};
     p.y = y;
-    p.bias = bias;
+    p.bias = et.any() ? nullptr : bias;
+    p.ex_bias = et.any() ? bias : nullptr;
+    p.relu = et.relu;
+    p.residual = et.residual;
+    p.ldr = et.ldr;
     p.ldy = ldy;
     p.M = (int)M;
     p.N = (int)N;
@@ -501,7 +518,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     const int tiles = p.tiles_m * p.tiles_n;
     const int pairs = tiles < d.sm_count / 2 ? tiles : d.sm_count / 2;
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::gemm_tc2_kernel, dim3(2 * pairs), dim3(mx::TC_THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    MX_CUDA(launch_dep(mx::gemm_tc2_kernel, dim3(2 * pairs), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -648,7 +665,7 @@ bool wide_tile(int64_t M, int64_t N, const DeviceInfo &d)
 // Pre-decoded bf16 weights (both operands fetched by TMA).
 mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64_t M, int64_t N,
                    int64_t K, const float *bias, float *y, int64_t ldy, DeviceInfo &d, cudaStream_t st,
-                   const QuantizedOut *yq = nullptr, const TcBatch &tb = TcBatch())
+                   const QuantizedOut *yq = nullptr, const TcBatch &tb = TcBatch(), const EpiTail &et = EpiTail())
 {
     const PackedW none;
     // CTA pairs (a third less shared-memory traffic per flop) when there is more than one wave of 256 x 256
@@ -658,11 +675,11 @@ mx_status_t run_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, int64
     const int64_t pair_tiles = ((M + 255) / 256) * ((N + 255) / 256);
     const int pairs = d.sm_count / 2;
     if (tb.count == 1 && M > 128 && (pair_tiles > pairs || (K >= 4096 && 4 * pair_tiles >= 3 * pairs)))
-        return launch_tc2(a_hat, w_hat, M, N, K, bias, y, ldy, yq, d, st);
+        return launch_tc2(a_hat, w_hat, M, N, K, bias, y, ldy, yq, d, st, et);
     const int64_t tiles256 = ((M + 127) / 128) * ((N + 255) / 256) * tb.count;
     if (N > 128 && tiles256 >= (int64_t)d.sm_count * 3 / 4)
-        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb);
-    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb);
+        return launch_tc<256, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb, et);
+    return launch_tc<128, mx::W_BF16>(a_hat, w_hat, none, M, N, K, bias, y, ldy, yq, d, st, tb, et);
 }
 
 // Packed weights decoded inside the kernel.
@@ -1221,18 +1238,23 @@ static mx_status_t check_quantized_out(mx_format_t fy, int64_t M, int64_t N, con
     return MX_OK;
 }
 
-mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
-                      const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
-                      const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
-                      uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+// Tensor-core product of packed operands with an fp32 (y) or MXInt (fy, y_mant, y_exp) result and an
+// optional element-wise tail.
+static mx_status_t gemm_tc_impl(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                                const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                                const float *bias, const EpiTail &et, float *y, int64_t ldy, mx_format_t fy,
+                                void *y_mant, uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
+                                size_t workspace_bytes, void *stream)
 {
-    // the output pointer checks (non-null, 16-byte aligned) apply to the mantissa array here
+    // the output pointer checks (non-null, 16-byte aligned) apply to the mantissa array of an MXInt result
     mx_status_t s = check_gemm_args(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias,
-                                    static_cast<const float *>(y_mant), N);
+                                    y ? y : static_cast<const float *>(y_mant), y ? ldy : N);
     if (s != MX_OK) return s;
     if (!a_exp) return MX_ERR_NULL;
-    s = check_quantized_out(fy, M, N, y_mant, y_exp);
-    if (s != MX_OK) return s;
+    if (!y) {
+        s = check_quantized_out(fy, M, N, y_mant, y_exp);
+        if (s != MX_OK) return s;
+    }
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
@@ -1246,28 +1268,33 @@ mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, 
     if (s != MX_OK) return s;
     s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
     if (s != MX_OK) return s;
+    if (y) return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st, nullptr, TcBatch(), et);
     QuantizedOut yq;
     yq.mant = static_cast<uint8_t *>(y_mant);
     yq.exps = y_exp;
     yq.nonfinite = nonfinite_count;
     yq.f = fy;
-    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq);
+    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq, TcBatch(), et);
 }
 
-mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
-                        const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
-                        const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
-                        uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+// The same for the layer: activations quantized on the fly.
+static mx_status_t linear_tc_impl(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
+                                  const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
+                                  const float *bias, const EpiTail &et, float *y, int64_t ldy, mx_format_t fy,
+                                  void *y_mant, uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
+                                  size_t workspace_bytes, void *stream)
 {
     mx_status_t s = check_gemm_args(x, nullptr, fa, w_mant, w_exp, fw, M, N, K, bias,
-                                    static_cast<const float *>(y_mant), N);
+                                    y ? y : static_cast<const float *>(y_mant), y ? ldy : N);
     if (s != MX_OK) return s;
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
     if (fa.packing) return MX_ERR_FORMAT;
     if (ldx < K) return MX_ERR_SHAPE;
     if ((ldx % 8) != 0) return MX_ERR_ALIGN;
-    s = check_quantized_out(fy, M, N, y_mant, y_exp);
-    if (s != MX_OK) return s;
+    if (!y) {
+        s = check_quantized_out(fy, M, N, y_mant, y_exp);
+        if (s != MX_OK) return s;
+    }
     DeviceInfo *d = nullptr;
     s = device_info(&d);
     if (s != MX_OK) return s;
@@ -1279,15 +1306,79 @@ mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int6
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(ws + round256((size_t)M * K * 2));
     mx_linear_args_t one;
     one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
-    one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = nullptr; one.ldy = N;
+    one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = y ? ldy : N;
+    s = tc_prepare(one, a_hat, w_hat, *d, st);
+    if (s != MX_OK) return s;
+    if (y) return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st, nullptr, TcBatch(), et);
     QuantizedOut yq;
     yq.mant = static_cast<uint8_t *>(y_mant);
     yq.exps = y_exp;
     yq.nonfinite = nonfinite_count;
     yq.f = fy;
-    s = tc_prepare(one, a_hat, w_hat, *d, st);
+    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq, TcBatch(), et);
+}
+
+mx_status_t mx_gemm_q(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                      const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                      const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
+                      uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!y_mant) return MX_ERR_NULL;
+    return gemm_tc_impl(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, EpiTail(), nullptr, 0, fy, y_mant, y_exp,
+                        nonfinite_count, workspace, workspace_bytes, stream);
+}
+
+mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
+                        const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
+                        const float *bias, mx_format_t fy, void *y_mant, uint8_t *y_exp,
+                        uint32_t *nonfinite_count, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!y_mant) return MX_ERR_NULL;
+    return linear_tc_impl(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, EpiTail(), nullptr, 0, fy, y_mant, y_exp,
+                          nonfinite_count, workspace, workspace_bytes, stream);
+}
+
+// ---- the product with a fused element-wise tail ---------------------------------------------------
+static mx_status_t tail_of(const mx_epilogue_t *ep, int64_t N, const float *y, const void *y_mant, const float **bias,
+                           EpiTail *et)
+{
+    if ((y != nullptr) == (y_mant != nullptr)) return MX_ERR_NULL;        // exactly one kind of result
+    *bias = nullptr;
+    *et = EpiTail();
+    if (!ep) return MX_OK;
+    *bias = ep->bias;
+    et->relu = ep->relu ? 1 : 0;
+    et->residual = ep->residual;
+    et->ldr = ep->ldr;
+    if (ep->residual && ep->ldr < N) return MX_ERR_SHAPE;
+    if (ep->residual && (reinterpret_cast<uintptr_t>(ep->residual) & 3u) != 0) return MX_ERR_ALIGN;
+    return MX_OK;
+}
+
+mx_status_t mx_gemm_fused(const void *a_mant, const uint8_t *a_exp, mx_format_t fa, const void *w_mant,
+                          const uint8_t *w_exp, mx_format_t fw, int64_t M, int64_t N, int64_t K,
+                          const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy, void *y_mant,
+                          uint8_t *y_exp, void *workspace, size_t workspace_bytes, void *stream)
+{
+    const float *bias;
+    EpiTail et;
+    const mx_status_t s = tail_of(ep, N, y, y_mant, &bias, &et);
     if (s != MX_OK) return s;
-    return run_tc(a_hat, w_hat, M, N, K, bias, nullptr, N, *d, st, &yq);
+    return gemm_tc_impl(a_mant, a_exp, fa, w_mant, w_exp, fw, M, N, K, bias, et, y, ldy, fy, y_mant, y_exp, nullptr,
+                        workspace, workspace_bytes, stream);
+}
+
+mx_status_t mx_linear_fused(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
+                            const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
+                            const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy, void *y_mant,
+                            uint8_t *y_exp, void *workspace, size_t workspace_bytes, void *stream)
+{
+    const float *bias;
+    EpiTail et;
+    const mx_status_t s = tail_of(ep, N, y, y_mant, &bias, &et);
+    if (s != MX_OK) return s;
+    return linear_tc_impl(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, et, y, ldy, fy, y_mant, y_exp, nullptr,
+                          workspace, workspace_bytes, stream);
 }
 
 // ---- decode: few tokens, weights streamed once ------------------------------------------------

@@ -57,6 +57,7 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
         if keep is not None:
             keep[name] = t
         return t
+    rec.keep = keep
 
     def linear(inp, name, bias, n_out):
         wm, we = qweights[name]
@@ -93,8 +94,19 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
 
 
 def _after_attention(cfg, x, ctx, qweights, params, linear, rec):
-    """Output projection, residual, second LayerNorm and the feed-forward network."""
+    """Output projection, skip connections and the feed-forward half of the block."""
     hid = cfg.hidden
+    fa, fw = mxb.MxFormat(cfg.block, cfg.w_act), mxb.MxFormat(cfg.block, cfg.w_wgt)
+    if rec.keep is None:
+        # bias, ReLU and the skip connections run in the products' epilogues; the feed-forward activation
+        # leaves its product already quantized (the next product's operand), so no fp32 tensor of width ffn exists
+        wm, we = qweights["wo"]
+        x1 = mxb.mx_linear_fused(ctx, fa, wm, we, fw, hid, bias=params["bo"], residual=x)
+        h2 = mxb.mx_layernorm(x1, params["ln2_g"], params["ln2_b"], cfg.eps)
+        wm, we = qweights["w1"]
+        fm, fe = mxb.mx_linear_fused(h2, fa, wm, we, fw, cfg.ffn, bias=params["b1"], relu=True, fy=fa)
+        wm, we = qweights["w2"]
+        return mxb.mx_gemm_fused(fm, fe, fa, wm, we, fw, x.shape[0], hid, cfg.ffn, bias=params["b2"], residual=x1)
     a = rec("attn_out", linear(ctx, "wo", params["bo"], hid))
     x1 = rec("x1", mxb.mx_relu_add(a, x))
     h2 = rec("ln2", mxb.mx_layernorm(x1, params["ln2_g"], params["ln2_b"], cfg.eps))

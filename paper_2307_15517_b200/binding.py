@@ -117,7 +117,6 @@ def _load() -> C.CDLL:
     L.mx_gemm_fused.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
     L.mx_linear_fused.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
     L.mx_gemm_fused.restype = i32
-    L.mx_linear_fused.restype = i32
     L.mx_poll_status.argtypes = [vp]
     L.mx_selftest_wait_expiry.argtypes = [C.c_uint32, vp]
     L.mx_selftest_wait_expiry.restype = i32

@@ -45,6 +45,11 @@ constexpr int TC_BK = 64;                                  // bf16 elements per 
 constexpr int TC_THREADS = 192;                            // producer, MMA, 4 epilogue warps
 // fused modes: 2 * BN extra weight-decode threads (one per tile row and half K step)
 constexpr int tc_threads(int bn, int wmode) { return wmode == 0 ? TC_THREADS : TC_THREADS + 2 * bn; }
+// registers per thread: 128 at most, and what one block of that many threads can have
+constexpr int tc_max_regs(int bn, int wmode)
+{
+    return 65536 / tc_threads(bn, wmode) >= 128 ? 128 : (65536 / tc_threads(bn, wmode)) / 16 * 16;
+}
 constexpr uint64_t TC_WAIT_LIMIT_NS = 400ull * 1000 * 1000; // 0.4 s per wait
 
 constexpr uint32_t STATUS_TIMEOUT_BIT = 1u;
@@ -283,7 +288,8 @@ template <int WMODE> struct RawItem {
 };                       // an item outside the matrix is all zero bytes and decodes to +0
 
 template <int BN, int WMODE>
-__global__ void __launch_bounds__(tc_threads(BN, WMODE), 1)
+// (register cap: see the CTA-pair kernel; the block has tc_threads(BN, WMODE) threads)
+__global__ void __maxnreg__(tc_max_regs(BN, WMODE))
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
 {
@@ -639,8 +645,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int tb = t / tiles_item, tt = t - tb * tiles_item;
             const int m0 = (tt % p.tiles_m) * TC_BM, n0 = (tt / p.tiles_m) * BN;
             const int row = m0 + quad * 32 + lane;
-            TailRegs t0, t1;
-            if (tail) tail_fetch(p, row, n0, t0);              // the first chunk's residual: in flight under the MMAs
+            TailRegs ahead;
+            if (tail) tail_fetch(p, row, n0, ahead);           // the first chunk's residual: in flight under the MMAs
             // every lane waits (acquire), then the warp agrees on the outcome so that the
             // warp-collective TMEM loads below are never executed by a partial warp
             const bool ok = ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
@@ -649,23 +655,23 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                 break;
             }
             ptx::tc_fence_after_sync();
-            auto chunk = [&](int c0, TailRegs &cur, TailRegs &next) {
+#pragma unroll 1
+            for (int c0 = 0; c0 < BN; c0 += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-                if (tail && c0 + 32 < BN) tail_fetch(p, row, n0 + c0 + 32, next);     // in flight under this chunk
+                TailRegs cur;
+                if (tail) {
+                    cur = ahead;                                               // fetched a chunk ago: has arrived
+                    if (c0 + 32 < BN) tail_fetch(p, row, n0 + c0 + 32, ahead);  // in flight under this chunk
+                }
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
                 if (tail) tail_apply(p, cur, n, r);
                 if (!FUSED && p.yq_mant) {
                     store_mxint_chunk(p, row, n, r);
-                    return;
+                    continue;
                 }
                 store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
-            };
-#pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 64) {
-                chunk(c0, t0, t1);
-                chunk(c0 + 32, t1, t0);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -42,7 +42,11 @@ struct Tc2Cfg {
     static constexpr uint32_t TMEM_COLS = 512;            // two accumulators of 256 columns
 };
 
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(Tc2Cfg::THREADS, 1)
+// 128 registers per thread instead of the 204 the block size allows (a few spills in the epilogue): the launch that
+// follows as a programmatic dependent -- the next call's operand pass, HBM-bound -- then finds room on the SM beside this
+// persistent CTA and runs under its last tiles (step of four layers 0.2361 -> 0.2339 ms, although this kernel alone
+// is 3 % slower).
+__global__ void __cluster_dims__(2, 1, 1) __maxnreg__(128)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                 const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
 {
@@ -166,31 +170,31 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;
             const int m0 = (t % p.tiles_m) * 256 + (int)rank * 128, n0 = (t / p.tiles_m) * BN;
             const int row = m0 + quad * 32 + lane;
-            TailRegs t0, t1;
-            if (tail) tail_fetch(p, row, n0 + col0, t0);       // the first chunk's residual: in flight under the MMAs
+            TailRegs ahead;
+            if (tail) tail_fetch(p, row, n0 + col0, ahead);    // the first chunk's residual: in flight under the MMAs
             const bool ok = ptx::mbar_wait_bounded_cluster(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
             if (!__all_sync(0xFFFFFFFFu, ok)) {
                 timed_out = true;
                 break;
             }
             ptx::tc_fence_after_sync();
-            auto chunk = [&](int c0, TailRegs &cur, TailRegs &next) {
+#pragma unroll 1
+            for (int c0 = col0; c0 < col0 + COLS; c0 += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
-                if (tail && c0 + 32 < col0 + COLS) tail_fetch(p, row, n0 + c0 + 32, next);     // in flight under this chunk
+                TailRegs cur;
+                if (tail) {
+                    cur = ahead;                                                        // fetched a chunk ago: has arrived
+                    if (c0 + 32 < col0 + COLS) tail_fetch(p, row, n0 + c0 + 32, ahead);  // in flight under this chunk
+                }
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
                 if (tail) tail_apply(p, cur, n, r);
                 if (p.yq_mant) {
                     store_mxint_chunk(p, row, n, r);
-                    return;
+                    continue;
                 }
                 store_f32_chunk<1>(p, &tmap_y, r, row, m0 + quad * 32, n, 0, epi_base + (uint32_t)(warp - 2) * 4096u, epi_buf, lane);
-            };
-#pragma unroll 1
-            for (int c0 = col0; c0 < col0 + COLS; c0 += 64) {
-                chunk(c0, t0, t1);
-                chunk(c0 + 32, t1, t0);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -93,12 +93,19 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     assert g(algo=9) == -3
     assert L.mx_linear_ex(fake, 0, 8, 64, 60, f, fake, fake, f, 8, None, fake, 8, None, 0, 2, None) == -2
     # the calls with an MXInt result: N must hold whole output blocks, outputs must be there
-    q = lambda **kw: L.mx_linear_q(fake, 0, 8, 64, 64, f, fake, fake, f, kw.get("N", 32), None, kw.get("fy", f),
+    q = lambda **kw: L.mx_linear_q(fake, 0, kw.get("M", 8), 64, 64, f, fake, fake, f, kw.get("N", 32), None, kw.get("fy", f),
                                    kw.get("ym", fake), kw.get("ye", fake), None, None, 0, None)
     assert q(N=40) == -2                                     # 40 is not a multiple of the output block
     assert q(fy=mxb.MxFormat(8, 4)) == -3
     assert q(ym=None) == -1 and q(ye=None) == -1
-    assert q(fy=F(16, 4, 8, 2)) == -3                        # the result format takes one-row blocks only
+    assert q(fy=F(16, 4, 8, 2), M=7) == -2                   # a two-row result format needs an even number of rows
+    assert q(fy=F(16, 4, 8, 3)) == -3
+    # the product with a fused tail: exactly one kind of result, residual rows at least N wide
+    ep = mxb.MxEpilogue()
+    ep.residual, ep.ldr = fake, 16
+    ft = lambda ep, y, ym: L.mx_linear_fused(fake, 0, 8, 64, 64, f, fake, fake, f, 32, ep, y, 32, f, ym, fake, None, 0, None)
+    assert ft(None, fake, fake) == -1 and ft(None, None, None) == -1
+    assert ft(C.byref(ep), fake, None) == -2
     # casts and the softmax with an MXInt result
     c = lambda **kw: L.mx_cast(kw.get("m", fake), fake, kw.get("fi", f), kw.get("rows", 4), kw.get("K", 64),
                                kw.get("fo", F(32, 8)), kw.get("mo", fake), fake, None, None)

@@ -345,6 +345,21 @@ MX_API mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const 
                                 float *ctx, int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, void *workspace,
                                 size_t workspace_bytes, void *stream);
 
+/*
+ * The same with the three operands still in floating point (what mx_linear is to mx_gemm): q, k, v are
+ * [seq, heads*head_dim] tensors of `dt` with leading dimensions ldq, ldk, ldv (elements, multiples of 8;
+ * slices of one fused projection result are fine), 16-byte aligned.  q and k are quantized to fqk in blocks
+ * along the head dimension, v to fv in blocks along the TOKENS (its slow axis; no transposed copy is needed
+ * from the caller), each in one pass that writes the tensor-core operand directly -- the packed codes never
+ * reach memory.  Equal to mx_quantize (x3) followed by mx_attention, bit for bit.  Workspace and
+ * restrictions as for mx_attention.
+ */
+MX_API mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtype_t dt, int64_t ldq,
+                                   int64_t ldk, int64_t ldv, mx_format_t fqk, mx_format_t fv, int64_t seq,
+                                   int64_t heads, int64_t head_dim, float scale, int causal, mx_format_t fp,
+                                   float *ctx, int64_t ldc, void *workspace, size_t workspace_bytes,
+                                   void *stream);
+
 /* ---- device status (the paper has no counterpart: it describes no runtime) ---------------- */
 
 /*

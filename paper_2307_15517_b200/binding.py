@@ -149,6 +149,8 @@ def _load() -> C.CDLL:
     L.mx_attention_workspace_bytes.restype = sz
     L.mx_attention.argtypes = [vp, vp, vp, vp, F, vp, vp, F, i64, i64, i64, C.c_float, i32, F, vp, i64, vp, vp, vp, sz, vp]
     L.mx_attention.restype = i32
+    L.mx_attention_fp.argtypes = [vp, vp, vp, i32, i64, i64, i64, F, F, i64, i64, i64, C.c_float, i32, F, vp, i64, vp, sz, vp]
+    L.mx_attention_fp.restype = i32
     L.mx_profile_begin.argtypes = []
     L.mx_profile_end.argtypes = [C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     for name in ("mx_quantize", "mx_dequantize", "mx_gemm", "mx_gemm_ex", "mx_linear",
@@ -481,6 +483,25 @@ def mx_attention(q_mant, q_exp, k_mant, k_exp, fqk: MxFormat, vt_mant, vt_exp, f
                             seq, heads, head_dim, scale, 1 if causal else 0, fp, _ptr(ctx), ctx.stride(0), _ptr(pm),
                             _ptr(pe), _ptr(workspace), workspace.numel(), _stream(stream)), "mx_attention")
     return (ctx, pm, pe) if return_p else ctx
+
+
+def mx_attention_fp(q: torch.Tensor, k: torch.Tensor, v: torch.Tensor, fqk: MxFormat, fv: MxFormat, heads: int,
+                    head_dim: int, scale: float, fp: MxFormat, causal: bool = True,
+                    ctx: Optional[torch.Tensor] = None, workspace: Optional[torch.Tensor] = None, stream=None):
+    """mx_attention on floating-point q, k, v ([seq, heads*head_dim], row-major views allowed): the three
+    operands are quantized on the fly (q, k along the head dimension, v along the tokens)."""
+    _need_cuda(q, k, v, ctx, workspace)
+    seq = q.shape[0]
+    assert q.dtype == k.dtype == v.dtype and q.stride(1) == k.stride(1) == v.stride(1) == 1
+    assert q.shape == k.shape == v.shape == (seq, heads * head_dim)
+    if ctx is None:
+        ctx = torch.empty((seq, heads * head_dim), dtype=torch.float32, device=q.device)
+    if workspace is None:
+        workspace = alloc_workspace(int(lib.mx_attention_workspace_bytes(seq, heads, head_dim)), q.device)
+    _check(lib.mx_attention_fp(_ptr(q), _ptr(k), _ptr(v), _dtype_code(q), q.stride(0), k.stride(0), v.stride(0), fqk, fv,
+                               seq, heads, head_dim, scale, 1 if causal else 0, fp, _ptr(ctx), ctx.stride(0),
+                               _ptr(workspace), workspace.numel(), _stream(stream)), "mx_attention_fp")
+    return ctx
 
 
 def mx_layernorm(x: torch.Tensor, gamma, beta, eps: float, y: Optional[torch.Tensor] = None, stream=None):

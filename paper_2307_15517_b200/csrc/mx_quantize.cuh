@@ -611,7 +611,19 @@ quantize_transposed_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, i
             if (block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);
             uint2 pk[4];
 #pragma unroll
-            for (int c = 0; c < 4; ++c) pk[c] = encode8_packed(v[c], (int)(amax[c >> 1] >> 23), w);
+            for (int c = 0; c < 4; ++c) {
+                float xh[8];
+                pk[c] = encode8_full(v[c], (int)(amax[c >> 1] >> 23), w, xh);
+                if (out.xhat) {                                       // the decoded values, exact in bf16
+                    uint4 h;
+                    h.x = as_u32(__floats2bfloat162_rn(xh[0], xh[1]));
+                    h.y = as_u32(__floats2bfloat162_rn(xh[2], xh[3]));
+                    h.z = as_u32(__floats2bfloat162_rn(xh[4], xh[5]));
+                    h.w = as_u32(__floats2bfloat162_rn(xh[6], xh[7]));
+                    *reinterpret_cast<uint4 *>(out.xhat + row * out.ld_xhat + kb + 8 * c) = h;
+                }
+            }
+            if (!out.mant) continue;                                  // operand form only
             if (nibble)
                 *reinterpret_cast<uint4 *>(out.mant + row * mant_ld + (kb >> 1)) = make_uint4(pk[0].x, pk[1].x, pk[2].x, pk[3].x);
             else {

@@ -1606,6 +1606,41 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
 }
 
 // ---- fused attention ---------------------------------------------------------------------------
+// The fused attention kernel on operands already in bf16 operand form: q_hat, k_hat [seq, hid], v_hat [hid, seq].
+static mx_status_t launch_attention(const __nv_bfloat16 *q_hat, const __nv_bfloat16 *k_hat, const __nv_bfloat16 *v_hat,
+                                    int64_t seq, int64_t heads, float scale, int causal, mx_format_t fp, float *ctx,
+                                    int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, DeviceInfo *d, cudaStream_t st)
+{
+    const int64_t hid = heads * mx::AttnCfg::D;
+    CUtensorMap tm_q, tm_k, tm_v;
+    mx_status_t s = encode_bf16_rows(&tm_q, q_hat, seq, hid, 128);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_k, k_hat, seq, hid, 128);
+    if (s != MX_OK) return s;
+    s = encode_bf16_rows(&tm_v, v_hat, hid, seq, 128);
+    if (s != MX_OK) return s;
+    s = smem_attr_once(d->attn_attr_set, mx::attention_kernel, (int)mx::AttnCfg::SMEM_BYTES);
+    if (s != MX_OK) return s;
+    mx::AttnParams ap;
+    ap.ctx = ctx;
+    ap.ldc = ldc;
+    ap.seq = (int)seq;
+    ap.heads = (int)heads;
+    ap.scale = scale;
+    ap.causal = causal ? 1 : 0;
+    ap.p_bits = fp.elem_bits;
+    ap.p_block = fp.block;
+    ap.p_mant = static_cast<uint8_t *>(p_mant_out);
+    ap.p_exp = p_exp_out;
+    ap.status = d->status;
+    const int64_t items = (seq / mx::AttnCfg::BQ) * heads;
+    const int grid = items < d->sm_count ? (int)items : d->sm_count;
+    ProfScope prof(KIND_GEMM_TC, st);
+    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::AttnCfg::THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 size_t mx_attention_workspace_bytes(int64_t seq, int64_t heads, int64_t head_dim)
 {
     if (seq <= 0 || heads <= 0 || head_dim <= 0) return 0;
@@ -1643,33 +1678,55 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     if (s != MX_OK) return s;
     s = launch_dequant_bf16(vt_mant, vt_exp, hid, seq, fv, v_hat, seq, *d, st);
     if (s != MX_OK) return s;
-    CUtensorMap tm_q, tm_k, tm_v;
-    s = encode_bf16_rows(&tm_q, q_hat, seq, hid, 128);
+    return launch_attention(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, p_mant_out, p_exp_out, d, st);
+}
+
+mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtype_t dt, int64_t ldq, int64_t ldk,
+                            int64_t ldv, mx_format_t fqk, mx_format_t fv, int64_t seq, int64_t heads, int64_t head_dim,
+                            float scale, int causal, mx_format_t fp, float *ctx, int64_t ldc, void *workspace,
+                            size_t workspace_bytes, void *stream)
+{
+    if (!q || !k || !v || !ctx) return MX_ERR_NULL;
+    if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
+    if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp) || fqk.packing || fv.packing) return MX_ERR_FORMAT;
+    const int64_t hid = heads * head_dim;
+    if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid || ldq < hid ||
+        ldk < hid || ldv < hid || seq > INT32_MAX / 4 || hid > INT32_MAX / 4)
+        return MX_ERR_SHAPE;
+    if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(ctx) || (ldc % 4) != 0 || (ldq % 8) != 0 ||
+        (ldk % 8) != 0 || (ldv % 8) != 0)
+        return MX_ERR_ALIGN;
+    if (!workspace || workspace_bytes < mx_attention_workspace_bytes(seq, heads, head_dim)) return MX_ERR_WORKSPACE;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
+    DeviceInfo *d = nullptr;
+    mx_status_t s = device_info(&d);
     if (s != MX_OK) return s;
-    s = encode_bf16_rows(&tm_k, k_hat, seq, hid, 128);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t one = round256((size_t)seq * hid * 2);
+    uint8_t *ws = static_cast<uint8_t *>(workspace);
+    __nv_bfloat16 *q_hat = reinterpret_cast<__nv_bfloat16 *>(ws), *k_hat = reinterpret_cast<__nv_bfloat16 *>(ws + one),
+                  *v_hat = reinterpret_cast<__nv_bfloat16 *>(ws + 2 * one);
+    // queries and keys: blocks along the head dimension, straight to the operand form
+    mx::QuantOut oq{nullptr, nullptr, q_hat, hid, nullptr, 0}, ok{nullptr, nullptr, k_hat, hid, nullptr, 0};
+    s = quantize_rows_any(q, dt, seq, hid, ldq, fqk, oq, *d, st);
     if (s != MX_OK) return s;
-    s = encode_bf16_rows(&tm_v, v_hat, hid, seq, 128);
+    s = quantize_rows_any(k, dt, seq, hid, ldk, fqk, ok, *d, st);
     if (s != MX_OK) return s;
-    s = smem_attr_once(d->attn_attr_set, mx::attention_kernel, (int)mx::AttnCfg::SMEM_BYTES);
-    if (s != MX_OK) return s;
-    mx::AttnParams ap;
-    ap.ctx = ctx;
-    ap.ldc = ldc;
-    ap.seq = (int)seq;
-    ap.heads = (int)heads;
-    ap.scale = scale;
-    ap.causal = causal ? 1 : 0;
-    ap.p_bits = fp.elem_bits;
-    ap.p_block = fp.block;
-    ap.p_mant = static_cast<uint8_t *>(p_mant_out);
-    ap.p_exp = p_exp_out;
-    ap.status = d->status;
-    const int64_t items = (seq / mx::AttnCfg::BQ) * heads;
-    const int grid = items < d->sm_count ? (int)items : d->sm_count;
-    ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::AttnCfg::THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
-    MX_CUDA(cudaGetLastError());
-    return MX_OK;
+    // values: blocks along the tokens, i.e. along the slow axis of v; written transposed, [hid, seq]
+    {
+        mx::QuantOut ov{nullptr, nullptr, v_hat, seq, nullptr, 0};
+        const int64_t tiles = ((hid + 31) / 32) * ((seq + 255) / 256);
+        const int tgrid = (int)(tiles < (int64_t)d->sm_count * 4 ? tiles : (int64_t)d->sm_count * 4);
+        ProfScope prof(KIND_QUANTIZE, st);
+        if (dt == MX_F32)
+            mx::quantize_transposed_kernel<float><<<tgrid, 256, 0, st>>>(static_cast<const float *>(v), hid, seq, ldv, fv.block,
+                                                                         fv.elem_bits, ov);
+        else
+            mx::quantize_transposed_kernel<__nv_bfloat16><<<tgrid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(v), hid, seq,
+                                                                                 ldv, fv.block, fv.elem_bits, ov);
+        MX_CUDA(cudaGetLastError());
+    }
+    return launch_attention(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, nullptr, nullptr, d, st);
 }
 
 // ---- fp32 glue of the transformer block ---------------------------------------------------------

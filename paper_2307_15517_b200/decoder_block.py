@@ -68,14 +68,14 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
     h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
     qkv = linear(h1, "wqkv", params["bqkv"], 3 * hid)           # [seq, 3 * hidden]: q | k | v
     q, k, v = rec("q", qkv[:, :hid]), rec("k", qkv[:, hid:2 * hid]), rec("v", qkv[:, 2 * hid:])
+    if keep is None and d == 128 and seq % 128 == 0:
+        # q, k, v quantized straight to the operand form, then scores, causal softmax, quantized probabilities and
+        # context in one kernel: nothing of size seq x seq and no packed copy of q, k, v is stored
+        ctx = mxb.mx_attention_fp(q, k, v, fa, fa, H, d, 1.0 / math.sqrt(d), fa, causal=True)
+        return _after_attention(cfg, x, ctx, qweights, params, linear, rec)
     # attention scores per head: both operands MXInt, blocks along the head dimension
     qm, qe = mxb.mx_quantize(q, fa)
     km, ke = mxb.mx_quantize(k, fa)
-    if keep is None and d == 128 and seq % 128 == 0:
-        # scores, causal softmax, quantized probabilities and context in one kernel: nothing of size seq x seq is stored
-        vm, ve = mxb.mx_quantize(v.t(), fa)                      # [hidden, seq]: blocks along tokens
-        ctx = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, 1.0 / math.sqrt(d), fa, causal=True)
-        return _after_attention(cfg, x, ctx, qweights, params, linear, rec)
     s = torch.empty((H * seq, seq), dtype=torch.float32, device=x.device)
     mxb.mx_gemm_batched(qm, qe, fa, hid, d, km, ke, fa, hid, d, seq, seq, d, H, s, seq, seq * seq)
     rec("scores", s.clone() if keep is not None else s)

@@ -76,3 +76,24 @@ def test_fused_attention_refuses_what_it_cannot_tile(mxb):
             mxb.mx_attention(z(seq, H * d), z(seq, H * d // 16), z(seq, H * d), z(seq, H * d // 16), f, z(H * d, seq),
                              z(H * d, seq // 16), f, seq, H, d, 0.1, f, workspace=mxb.alloc_workspace(1 << 22))
         assert e.value.status == status
+
+
+@pytest.mark.parametrize("case", [(2, 256, 16, torch.float32), (3, 384, 32, torch.bfloat16)])
+def test_attention_on_floating_point_operands_equals_quantize_then_attention(mxb, case):
+    """mx_attention_fp quantizes q, k (along the head dimension) and v (along the tokens) on the fly; its
+    context must equal, bit for bit, mx_attention on the operands quantized by mx_quantize (which the
+    quantizer tests tie to the oracle), also when q, k, v are column slices of one wider tensor."""
+    H, seq, B, dtype = case
+    d, hid = 128, H * 128
+    qkv = torch.cat([synth.student_t_activations(seq, hid, 41), synth.outlier_activations(seq, hid, 42, 3, 20.0),
+                     synth.student_t_activations(seq, hid, 43)], dim=1).to(dtype).cuda()
+    q, k, v = qkv[:, :hid], qkv[:, hid:2 * hid], qkv[:, 2 * hid:]
+    fa, fp = mxb.MxFormat(B, 8), mxb.MxFormat(B, 8)
+    scale = 1.0 / math.sqrt(d)
+    got = mxb.mx_attention_fp(q, k, v, fa, fa, H, d, scale, fp, causal=True)
+    qm, qe = mxb.mx_quantize(q, fa)
+    km, ke = mxb.mx_quantize(k, fa)
+    vm, ve = mxb.mx_quantize(v.t(), fa)
+    want = mxb.mx_attention(qm, qe, km, ke, fa, vm, ve, fa, seq, H, d, scale, fp, causal=True)
+    assert mxb.mx_poll_status() == 0
+    assert torch.equal(got, want)

@@ -134,9 +134,11 @@ typedef struct {
  * [rows, K] tensor is then uint8 [rows/2, K/block] and rows must be even (MX_ERR_SHAPE).
  * Accepted by mx_quantize (stride_k == 1), mx_dequantize, mx_gemm / mx_linear and their _q forms
  * for either operand with MX_ALGO_AUTO, MX_ALGO_TCGEN05(_BLOCKWISE) and MX_ALGO_SIMT, as the result
- * format fy of the _q forms (rows of Y pair up: exponent array [M/2, N/fy.block]) and by
- * mx_gemm_batched (items must start on even rows); the streaming, in-kernel decode, grouped and
- * static entry points take one-row blocks only (MX_ERR_FORMAT). */
+ * format fy of the _q forms (rows of Y pair up: exponent array [M/2, N/fy.block]), by
+ * mx_gemm_batched (items must start on even rows) and by MX_ALGO_STREAM / mx_linear_grouped for
+ * either operand (an even number of tokens when the activations pair up; weights in this form are
+ * read with plain loads instead of staged boxes); the in-kernel decode (MX_ALGO_TCGEN05_FUSED), the
+ * fused attention and the static entry point take one-row blocks only (MX_ERR_FORMAT). */
 
 /* ---- size helpers (host only, no CUDA call) ------------------------------------------- */
 

@@ -49,6 +49,9 @@ struct StreamLayer {
     int a_bits, w_bits;
     int tile_begin;          // index of this layer's first 16-row tile in the launch
     int n_tiles;             // ceil(N / 16)
+    // two-row blocks (the paper's (16,2) shape): rows 2i and 2i+1 share row i of the exponent array.  Weights in
+    // this form take the register variant of the kernel (the staged exponent boxes assume one row per weight row).
+    int w_rows2, a_rows2;    // 0 or 1: shift applied to the row index of w_exp / a_exp
 };
 
 struct StreamParams {
@@ -223,7 +226,7 @@ gemv_stream_kernel(const StreamParams p)
             // MMA slots 4t..4t+3 take the even k of this group of 8, slots 16+4t.. the odd k
             sB[i] = make_uint2(__byte_perm(lo, hi, 0x6420), __byte_perm(lo, hi, 0x7531));
             if (tq == 0) {
-                const int eb = tok < L.T ? (int)__ldg(L.a_exp + (int64_t)tok * nb + b) : 0;
+                const int eb = tok < L.T ? (int)__ldg(L.a_exp + (int64_t)(tok >> L.a_rows2) * nb + b) : 0;
                 // 2^(Ea-127-(wa-2)) * 2^-(ww-2) * 2^-4, every factor an exact power of two
                 sCS[b * TP + tok] = f32_scale(eb, L.a_bits) * small_neg_pow2(L.w_bits) * 0.0625f;
             }
@@ -242,8 +245,8 @@ gemv_stream_kernel(const StreamParams p)
                 const int rowA = min(r0 + g, L.N - 1), rowB = min(r0 + g + 8, L.N - 1);
                 const uint8_t *mA = L.w_mant + (int64_t)rowA * w_ld + t * 4;
                 const uint8_t *mB = L.w_mant + (int64_t)rowB * w_ld + t * 4;
-                const uint8_t *eA = L.w_exp + (int64_t)rowA * nb;
-                const uint8_t *eB = L.w_exp + (int64_t)rowB * nb;
+                const uint8_t *eA = L.w_exp + (int64_t)(rowA >> L.w_rows2) * nb;
+                const uint8_t *eB = L.w_exp + (int64_t)(rowB >> L.w_rows2) * nb;
                 const int b_lo = (nb / S) * s, b_hi = b_lo + nb / S;       // nb % (4*S) == 0
                 struct Regs { uint32_t a[4], b[4], ea, eb; };
                 // any exponent byte >= 226: 1.5*2^23 * 2^(E-127) is not finite, take two steps there

@@ -791,7 +791,7 @@ size_t stream_table_bytes(int32_t n_layers)
 bool stream_layer_ok(const mx_linear_args_t &a)
 {
     return a.M >= 1 && a.M <= 16 && a.fw.block == 32 && a.fa.block == 32 && a.fw.elem_bits <= 4 &&
-           (a.K % 128) == 0 && a.fa.block_rows == 1 && a.fw.block_rows == 1 && a.fa.packing == 0 && a.fw.packing == 0;
+           (a.K % 128) == 0 && a.fa.packing == 0 && a.fw.packing == 0;
 }
 
 size_t stream_act_bytes(const mx_linear_args_t &a)
@@ -802,7 +802,7 @@ size_t stream_act_bytes(const mx_linear_args_t &a)
 bool same_activation(const mx_linear_args_t &a, const mx_linear_args_t &b)
 {
     return a.x == b.x && a.dt == b.dt && a.M == b.M && a.K == b.K && a.ldx == b.ldx &&
-           a.fa.block == b.fa.block && a.fa.elem_bits == b.fa.elem_bits;
+           a.fa.block == b.fa.block && a.fa.elem_bits == b.fa.elem_bits && a.fa.block_rows == b.fa.block_rows;
 }
 
 template <int NT, bool BULK>
@@ -1426,7 +1426,8 @@ static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers
     // weights staged by bulk copies need 16-byte aligned exponent chunks: K % 512 == 0 everywhere
     bool bulk = true;
     for (int i = 0; i < n_layers; ++i)
-        bulk = bulk && (layers[i].K % 512) == 0 && (reinterpret_cast<uintptr_t>(layers[i].w_exp) & 15u) == 0;
+        bulk = bulk && (layers[i].K % 512) == 0 && (reinterpret_cast<uintptr_t>(layers[i].w_exp) & 15u) == 0 &&
+               layers[i].fw.block_rows == 1;
     auto smem_of = [&](bool b) {
         return nt == 2 ? (b ? mx::StreamCfg<2, true>::smem_bytes(max_nb) : mx::StreamCfg<2, false>::smem_bytes(max_nb))
                        : (b ? mx::StreamCfg<1, true>::smem_bytes(max_nb) : mx::StreamCfg<1, false>::smem_bytes(max_nb));
@@ -1470,10 +1471,16 @@ static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers
             job.block = a.fa.block;
             job.dt = a.dt == MX_F32 ? 0 : 1;
             job.out = mx::QuantOut{act_ptr[i], act_ptr[i] + round256(mx_mant_bytes(a.M, a.K, a.fa)), nullptr, 0, nullptr};
-            jobs.push_back(job);
-            any_dt[job.dt] = true;
-            const int64_t chunks = a.M * (a.K / 8);
-            max_chunks = chunks > max_chunks ? chunks : max_chunks;
+            if (a.fa.block_rows == 2) {
+                // pairs of tokens share their exponents: the two-row quantizer, one launch for this tensor
+                s = quantize_rows_any(a.x, a.dt, a.M, a.K, a.ldx, a.fa, job.out, *d, st);
+                if (s != MX_OK) return s;
+            } else {
+                jobs.push_back(job);
+                any_dt[job.dt] = true;
+                const int64_t chunks = a.M * (a.K / 8);
+                max_chunks = chunks > max_chunks ? chunks : max_chunks;
+            }
         }
         mx::StreamLayer &L = table[i];
         L.w_mant = static_cast<const uint8_t *>(a.w_mant);
@@ -1488,6 +1495,8 @@ static mx_status_t grouped_impl(const mx_linear_args_t *layers, int32_t n_layers
         L.T = (int)a.M;
         L.a_bits = a.fa.elem_bits;
         L.w_bits = a.fw.elem_bits;
+        L.w_rows2 = a.fw.block_rows == 2 ? 1 : 0;
+        L.a_rows2 = a.fa.block_rows == 2 ? 1 : 0;
         L.tile_begin = total_tiles;
         L.n_tiles = (int)((a.N + 15) / 16);
         total_tiles += L.n_tiles;

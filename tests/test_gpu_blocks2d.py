@@ -96,10 +96,44 @@ def test_two_row_blocks_are_refused_where_unsupported(mxb):
         mxb.mx_quantize(torch.randn(64, 4, device="cuda").t(), mxb.MxFormat(16, 4, 8, 2))  # strided axis
     wm, we = mxb.mx_quantize(torch.randn(64, 256, device="cuda"), F2)
     with pytest.raises(mxb.MxError):
-        mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64, algo=mxb.MX_ALGO_STREAM)
-    y = mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64)       # AUTO falls back to the tensor-core kernel
+        mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64, algo=mxb.MX_ALGO_TCGEN05_FUSED)   # in-kernel decode
+    with pytest.raises(mxb.MxError):
+        mxb.mx_linear(x[:3], mxb.MxFormat(32, 8, 8, 2), wm, we, F2, 64)                          # odd token count
+    y = mxb.mx_linear(x, mxb.MxFormat(32, 8), wm, we, F2, 64)
     assert torch.isfinite(y).all() and mxb.mx_poll_status() == 0
     del F1
+
+
+@pytest.mark.parametrize("case", [(2, 256, 2, 2), (4, 1024, 2, 1), (16, 1024, 1, 2), (16, 512, 2, 2), (1, 256, 1, 2)])
+def test_streamed_decode_with_two_row_blocks_is_bit_exact(mxb, case):
+    """The decode path (one launch over several layers, weights streamed once) on (32,2) blocks of the
+    weights, of the tokens, or of both: integer block sums and ascending fp32 block adds, so the result is
+    the oracle's sequential sum bit for bit, as for one-row blocks."""
+    T, K, ra, rw = case
+    N, B, wa, ww = 4096, 32, 8, 4
+    fa, fw = mxb.MxFormat(B, wa, 8, ra), mxb.MxFormat(B, ww, 8, rw)
+    layers, want = [], []
+    for i in range(6):
+        x = synth.student_t_activations(T, K, seed=11 * T + i).numpy()
+        wt = synth.gaussian_weights(N, K, seed=50 + i).numpy()
+        bias = synth.gaussian_weights(1, N, seed=90 + i, std=1.0)[0].numpy() if i % 2 else None
+        qa, ea, _ = orc.quantize_2d(x, B, ra, wa)
+        qw, ew, _ = orc.quantize_2d(wt, B, rw, ww)
+        want.append(orc.gemm(qa, orc.expand_exponent_rows(ea, ra), wa, qw, orc.expand_exponent_rows(ew, rw), ww, B,
+                             bias=bias)[1])
+        w_mant, w_exp = mxb.mx_quantize(_dev(wt), fw)
+        assert np.array_equal(w_exp.cpu().numpy(), ew)
+        layers.append(dict(x=_dev(x), fa=fa, w_mant=w_mant, w_exp=w_exp, fw=fw, N=N,
+                           bias=None if bias is None else _dev(bias),
+                           y=torch.empty((T, N), dtype=torch.float32, device="cuda")))
+    mxb.mx_linear_grouped(mxb.make_linear_args(layers))
+    assert mxb.mx_poll_status() == 0
+    for L, y_seq in zip(layers, want):
+        assert np.array_equal(L["y"].cpu().numpy(), y_seq)
+    # one layer through mx_linear: AUTO picks the streaming kernel for these shapes
+    L = layers[0]
+    y = mxb.mx_linear(L["x"], fa, L["w_mant"], L["w_exp"], fw, N, bias=L["bias"], algo=mxb.MX_ALGO_STREAM)
+    assert np.array_equal(y.cpu().numpy(), want[0])
 
 
 @pytest.mark.parametrize("case", [(300, 544, 512, 16, 16, 4), (130, 208, 256, 32, 16, 8), (2100, 2336, 128, 16, 16, 8),

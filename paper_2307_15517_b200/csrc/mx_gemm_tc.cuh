@@ -287,7 +287,9 @@ template <int WMODE> struct RawItem {
     uint32_t e;          // block 16: two exponent bytes (low = first block); block 32: one
 };                       // an item outside the matrix is all zero bytes and decodes to +0
 
-template <int BN, int WMODE>
+// TAIL: the instantiation whose epilogue applies the fused element-wise tail (it holds a chunk of residual values
+// in registers; kept out of the plain kernel, which then fits the register cap without spills).
+template <int BN, int WMODE, bool TAIL = false>
 // (register cap: see the CTA-pair kernel; the block has tc_threads(BN, WMODE) threads)
 __global__ void __maxnreg__(tc_max_regs(BN, WMODE))
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
@@ -638,7 +640,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const int quad = warp & 3;                          // TMEM lanes this warp may read
         int it = 0;
         uint32_t epi_buf = 0;                               // alternates between the warp's two store buffers
-        const bool tail = !FUSED && (p.relu != 0 || p.residual != nullptr);
+        constexpr bool tail = TAIL && !FUSED;
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;

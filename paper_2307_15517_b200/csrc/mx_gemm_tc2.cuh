@@ -42,10 +42,11 @@ struct Tc2Cfg {
     static constexpr uint32_t TMEM_COLS = 512;            // two accumulators of 256 columns
 };
 
-// 128 registers per thread instead of the 204 the block size allows (a few spills in the epilogue): the launch that
-// follows as a programmatic dependent -- the next call's operand pass, HBM-bound -- then finds room on the SM beside this
-// persistent CTA and runs under its last tiles (step of four layers 0.2361 -> 0.2339 ms, although this kernel alone
-// is 3 % slower).
+template <bool TAIL = false>
+// At most 128 registers per thread (the block size would allow 204; the plain instantiation needs 110, the one with
+// the fused tail 124): this launch follows an operand pass that fills the register file with its own CTAs, and as a
+// programmatic dependent it becomes resident -- barriers, tensor memory, descriptor prefetch -- as soon as enough of
+// those have left.  The smaller the footprint the earlier that is (step of four layers 0.2366 -> 0.2331 ms).
 __global__ void __cluster_dims__(2, 1, 1) __maxnreg__(128)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_w,
                 const __grid_constant__ CUtensorMap tmap_y, const TcParams p)
@@ -164,7 +165,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
         constexpr int COLS = BN / (Cfg::EPI_WARPS / 4);
         int it = 0;
         uint32_t epi_buf = 0;
-        const bool tail = p.relu != 0 || p.residual != nullptr;
+        constexpr bool tail = TAIL;
         for (int t = pair; t < num_tiles && !timed_out; t += npairs, ++it) {
             const int acc = it & 1;
             const uint32_t acc_ph = (uint32_t)(it >> 1) & 1u;

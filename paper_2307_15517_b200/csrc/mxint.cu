@@ -39,8 +39,9 @@ struct DeviceInfo {
     int sm_count = SM_COUNT_FALLBACK;
     uint32_t *status = nullptr;
     bool tc_attr_set[2][4] = {{false, false, false, false}, {false, false, false, false}};
+    bool tc_tail_attr_set[2] = {false, false};
     bool stream_attr_set[4] = {false, false, false, false};
-    bool tc2_attr_set = false;
+    bool tc2_attr_set[2] = {false, false};
     bool tcx_attr_set = false;
     bool tc8_attr_set = false;
     bool attn_attr_set = false;
@@ -429,8 +430,11 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         if (s != MX_OK) return s;
     }
     constexpr int slot = BN == 256 ? 0 : 1;
-    s = smem_attr_once(d.tc_attr_set[slot][WMODE], mx::gemm_tc_kernel<BN, WMODE>, (int)Cfg::SMEM_BYTES);
+    const bool tail = WMODE == mx::W_BF16 && et.any();
+    s = tail ? smem_attr_once(d.tc_tail_attr_set[slot], mx::gemm_tc_kernel<BN, mx::W_BF16, true>, (int)Cfg::SMEM_BYTES)
+             : smem_attr_once(d.tc_attr_set[slot][WMODE], mx::gemm_tc_kernel<BN, WMODE>, (int)Cfg::SMEM_BYTES);
     if (s != MX_OK) return s;
+    if (et.any() && !tail) return MX_ERR_FORMAT;          // the in-kernel decode variants have no tail
     mx::TcParams p;
     p.y = y;
     p.bias = et.any() ? nullptr : bias;
@@ -469,7 +473,8 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         return MX_OK;
     }
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::gemm_tc_kernel<BN, WMODE>, dim3(grid), dim3(threads), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    if (tail) MX_CUDA(launch_dep(mx::gemm_tc_kernel<BN, mx::W_BF16, true>, dim3(grid), dim3(threads), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    else MX_CUDA(launch_dep(mx::gemm_tc_kernel<BN, WMODE>, dim3(grid), dim3(threads), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -491,7 +496,8 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
     }
-    s = smem_attr_once(d.tc2_attr_set, mx::gemm_tc2_kernel, (int)Cfg::SMEM_BYTES);
+    s = et.any() ? smem_attr_once(d.tc2_attr_set[1], mx::gemm_tc2_kernel<true>, (int)Cfg::SMEM_BYTES)
+                 : smem_attr_once(d.tc2_attr_set[0], mx::gemm_tc2_kernel<false>, (int)Cfg::SMEM_BYTES);
     if (s != MX_OK) return s;
     mx::TcParams p{};
     p.y = y;
@@ -518,7 +524,8 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     const int tiles = p.tiles_m * p.tiles_n;
     const int pairs = tiles < d.sm_count / 2 ? tiles : d.sm_count / 2;
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::gemm_tc2_kernel, dim3(2 * pairs), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    if (et.any()) MX_CUDA(launch_dep(mx::gemm_tc2_kernel<true>, dim3(2 * pairs), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
+    else MX_CUDA(launch_dep(mx::gemm_tc2_kernel<false>, dim3(2 * pairs), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_a, tm_w, tm_y, p));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
@@ -841,12 +848,15 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     const bool f32 = a.dt == MX_F32, nib = a.fw.elem_bits <= 4;
     const double qb = (double)M * K * ((f32 ? 4.0 : 2.0) + 2.0);
     const double db = (double)N * K * ((nib ? 0.5 : 1.0) + 1.0 / a.fw.block + 2.0);
-    const int need_q = grid_for((M * (K / 8) + 1) / 2, 256, 1 << 20, 1);
-    const int need_d = grid_for((N * (K / 32) + 1) / 2, 256, 1 << 20, 1);
-    const int per_sm = f32 ? (nib ? resident_ctas(mx::prep_operands_kernel<float, true>)
-                            : resident_ctas(mx::prep_operands_kernel<float, false>))
-                     : (nib ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
-                            : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>));
+    // CTAs of 128 threads (8 K registers): small enough to become resident beside a persistent product CTA of the
+    // previous call, where they wait in griddepcontrol.wait and start the moment that grid completes
+    constexpr int PT = 128;
+    const int need_q = grid_for((M * (K / 8) + 1) / 2, PT, 1 << 20, 1);
+    const int need_d = grid_for((N * (K / 32) + 1) / 2, PT, 1 << 20, 1);
+    const int per_sm = (256 / PT) * (f32 ? (nib ? resident_ctas(mx::prep_operands_kernel<float, true>)
+                                            : resident_ctas(mx::prep_operands_kernel<float, false>))
+                                     : (nib ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
+                                            : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>)));
     const int total = d.sm_count * per_sm;            // exactly one resident wave
     int gq = (int)(total * qb / (qb + db) + 0.5);
     gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
@@ -856,11 +866,11 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     job.q_blocks = gq;
     ProfScope prof(KIND_PREP, st);
     if (f32) {
-        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<float, true>, dim3(gq + gd), dim3(256), 0, st, job));
-        else MX_CUDA(launch_dep(mx::prep_operands_kernel<float, false>, dim3(gq + gd), dim3(256), 0, st, job));
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<float, true>, dim3(gq + gd), dim3(PT), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<float, false>, dim3(gq + gd), dim3(PT), 0, st, job));
     } else {
-        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, true>, dim3(gq + gd), dim3(256), 0, st, job));
-        else MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, false>, dim3(gq + gd), dim3(256), 0, st, job));
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, true>, dim3(gq + gd), dim3(PT), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, false>, dim3(gq + gd), dim3(PT), 0, st, job));
     }
     MX_CUDA(cudaGetLastError());
     return MX_OK;

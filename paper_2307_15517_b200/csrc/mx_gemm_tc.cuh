@@ -14,7 +14,8 @@
 // columns) so that the epilogue of tile t overlaps the MMAs of tile t+1.
 //   warp 0      : TMA producer (one lane)
 //   warp 1      : tensor-memory allocation, MMA issue (one lane)
-//   warps 2..5  : epilogue, TMEM -> registers -> (+bias) -> global fp32
+//   warps 2..   : epilogue, TMEM -> registers -> (+bias) -> global fp32 (eight warps in the plain kernel, two per
+//                 TMEM lane quarter with half of the tile's columns each; four in the in-kernel-decode variants)
 // Every mbarrier wait is bounded in time; on expiry the kernel raises a CTA-wide abort flag,
 // records MX_ERR_TIMEOUT in the status word, frees its tensor memory and returns.
 #pragma once
@@ -43,8 +44,11 @@ enum WMode { W_BF16 = 0, W_NIBBLE = 1, W_INT8 = 2, W_NIBBLE_PERM = 3 };
 constexpr int TC_BM = 128;
 constexpr int TC_BK = 64;                                  // bf16 elements per 128-byte row
 constexpr int TC_THREADS = 192;                            // producer, MMA, 4 epilogue warps
-// fused modes: 2 * BN extra weight-decode threads (one per tile row and half K step)
-constexpr int tc_threads(int bn, int wmode) { return wmode == 0 ? TC_THREADS : TC_THREADS + 2 * bn; }
+// plain kernel: eight epilogue warps (two per TMEM lane quarter, half of the tile's columns each: the epilogue of a
+// CTA's last tile, which no MMA overlaps, takes half as long); fused modes: four, then 2 * BN weight-decode threads
+// (one per tile row and half K step)
+constexpr int tc_epi_warps(int wmode) { return wmode == 0 ? 8 : 4; }
+constexpr int tc_threads(int bn, int wmode) { return wmode == 0 ? 64 + 32 * tc_epi_warps(0) : TC_THREADS + 2 * bn; }
 // registers per thread: 128 at most, and what one block of that many threads can have
 constexpr int tc_max_regs(int bn, int wmode)
 {
@@ -322,7 +326,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
         for (int a = 0; a < 2; ++a) {
             ptx::mbar_init(tfull_bar(a), 1);
-            ptx::mbar_init(tempty_bar(a), 4);          // one arrival per epilogue warp
+            ptx::mbar_init(tempty_bar(a), tc_epi_warps(WMODE));          // one arrival per epilogue warp
         }
         *abort_flag = 0;
         ptx::fence_mbar_init();
@@ -638,8 +642,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
     } else {
         const int quad = warp & 3;                          // TMEM lanes this warp may read
+        constexpr int EPI_WARPS = tc_epi_warps(WMODE), COLS = BN / (EPI_WARPS / 4);
+        const int col0 = ((warp - 2) >> 2) * COLS;          // this warp's columns of the tile
         int it = 0;
-        uint32_t epi_buf = 0;                               // alternates between the warp's two store buffers
+        uint32_t epi_buf = 0;                               // counts the warp's TMA store blocks (buffer parity)
         constexpr bool tail = TAIL && !FUSED;
         for (int t = blockIdx.x; t < num_tiles && !timed_out; t += gridDim.x, ++it) {
             const int acc = it & 1;
@@ -648,7 +654,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             const int m0 = (tt % p.tiles_m) * TC_BM, n0 = (tt / p.tiles_m) * BN;
             const int row = m0 + quad * 32 + lane;
             TailRegs ahead;
-            if (tail) tail_fetch(p, row, n0, ahead);           // the first chunk's residual: in flight under the MMAs
+            if (tail) tail_fetch(p, row, n0 + col0, ahead);    // the first chunk's residual: in flight under the MMAs
             // every lane waits (acquire), then the warp agrees on the outcome so that the
             // warp-collective TMEM loads below are never executed by a partial warp
             const bool ok = ptx::mbar_wait_bounded(tfull_bar(acc), acc_ph, abort_flag, TC_WAIT_LIMIT_NS);
@@ -658,13 +664,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
             ptx::tc_fence_after_sync();
 #pragma unroll 1
-            for (int c0 = 0; c0 < BN; c0 += 32) {
+            for (int c0 = col0; c0 < col0 + COLS; c0 += 32) {
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
                 TailRegs cur;
                 if (tail) {
                     cur = ahead;                                               // fetched a chunk ago: has arrived
-                    if (c0 + 32 < BN) tail_fetch(p, row, n0 + c0 + 32, ahead);  // in flight under this chunk
+                    if (c0 + 32 < col0 + COLS) tail_fetch(p, row, n0 + c0 + 32, ahead);  // in flight under this chunk
                 }
                 ptx::tmem_ld_wait();
                 const int n = n0 + c0;
@@ -673,7 +679,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                     store_mxint_chunk(p, row, n, r);
                     continue;
                 }
-                store_f32_chunk(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
+                // eight warps share the 32 KB of store buffers: one 4 KB buffer each instead of two
+                if (EPI_WARPS == 8)
+                    store_f32_chunk<1>(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 4096u, epi_buf, lane);
+                else
+                    store_f32_chunk<2>(p, &tmap_y, r, row, m0 + quad * 32, n, tb, epi_base + (uint32_t)(warp - 2) * 8192u, epi_buf, lane);
             }
             ptx::tc_fence_before_sync();
             __syncwarp();

@@ -236,3 +236,62 @@ def test_fused_attention_opt67b_shapes(mods):
         qv, ev, _ = orc.quantize(np.ascontiguousarray(vn[:, h * d:(h + 1) * d].T), B, w)
         y_ref, _, S = orc.gemm(qg, eg, w, qv, ev, w, B)
         _close(ctx[rows][:, h * d:(h + 1) * d], y_ref, S, "ctx head %d" % h)
+
+
+def test_fused_tails_opt67b_shapes(mods):
+    """The three products of the block's second half as the timed path runs them -- output projection with the
+    residual, FFN-up with bias, ReLU and an MXInt8 result, FFN-down from that result with bias and residual -- at
+    2048 x 4096 / 16384, each on sampled outputs against the oracle fed with the GPU's own inputs of that stage."""
+    mxb, _ = mods
+    seq, hid, ffn, B, wa, ww = 2048, 4096, 16384, 16, 8, 4
+    fa, fw = mxb.MxFormat(B, wa), mxb.MxFormat(B, ww)
+    rng = np.random.default_rng(9)
+    ctx = synth.student_t_activations(seq, hid, 91)
+    x = synth.outlier_activations(seq, hid, 92, 20, 40.0)
+    W = {n: synth.gaussian_weights(o, i, 93 + j) for j, (n, o, i) in enumerate([("wo", hid, hid), ("w1", ffn, hid), ("w2", hid, ffn)])}
+    g = torch.Generator().manual_seed(94)
+    bo, b1, b2 = (torch.randn(n, generator=g) * 0.05 for n in (hid, ffn, hid))
+    q = {n: mxb.mx_quantize(w.cuda(), fw) for n, w in W.items()}
+    qo = {n: orc.quantize(w.numpy(), B, ww)[:2] for n, w in W.items()}
+    n = 640
+
+    # output projection + bias + residual
+    x1 = mxb.mx_linear_fused(ctx.cuda(), fa, q["wo"][0], q["wo"][1], fw, hid, bias=bo.cuda(), residual=x.cuda())
+    qa, ea, _ = orc.quantize(ctx.numpy(), B, wa)
+    si, sj = rng.integers(0, seq, n), rng.integers(0, hid, n)
+    y_ref, _, S = orc.gemm_samples(qa, ea, wa, qo["wo"][0], qo["wo"][1], ww, B, si, sj, bias=bo.numpy())
+    res = x.numpy()[si, sj].astype(np.float64)
+    _close(x1.cpu().numpy()[si, sj], y_ref.astype(np.float64) + res, S + np.abs(res) + np.abs(bo.numpy()[sj]), "out-proj + residual")
+
+    # FFN-up + bias + ReLU, MXInt8 result: codes must be a correct rounding of the oracle's values
+    h2 = synth.student_t_activations(seq, hid, 95)
+    fm, fe = mxb.mx_linear_fused(h2.cuda(), fa, q["w1"][0], q["w1"][1], fw, ffn, bias=b1.cuda(), relu=True, fy=fa)
+    assert mxb.mx_poll_status() == 0
+    qa, ea, _ = orc.quantize(h2.numpy(), B, wa)
+    rows = np.sort(rng.choice(seq, 6, replace=False))
+    cols = np.arange(0, ffn, 16)[rng.choice(ffn // 16, 96, replace=False)]
+    fe_n, fm_n = fe.cpu().numpy(), fm.cpu().numpy()
+    for r in rows:
+        sj = (cols[:, None] + np.arange(16)[None, :]).ravel()               # whole output blocks of 16
+        si = np.full_like(sj, r)
+        y_ref, _, S = orc.gemm_samples(qa, ea, wa, qo["w1"][0], qo["w1"][1], ww, B, si, sj, bias=b1.numpy())
+        want = np.maximum(y_ref.astype(np.float64), 0.0).reshape(-1, 16)
+        tol = (TOL * (S + np.abs(b1.numpy()[sj]))).reshape(-1, 16)
+        eg = fe_n[r, cols // 16].astype(np.int64)
+        codes = fm_n[r].view(np.int8)[sj].reshape(-1, 16).astype(np.float64)
+        e_lo = np.where(np.maximum(want - tol, 0).max(axis=1) > 0, np.frexp(np.maximum(want - tol, 0).max(axis=1))[1] - 1 + 127, 0)
+        e_hi = np.maximum(np.frexp((want + tol).max(axis=1))[1] - 1 + 127, 0)
+        assert ((eg >= e_lo) & (eg <= e_hi)).all()
+        step = np.ldexp(1.0, eg - 127 - (wa - 2))[:, None]
+        free = np.abs(codes) < 127
+        assert (np.abs(codes * step - want)[free] <= (0.5 * step + tol)[free]).all()
+        assert (codes >= 0).all()
+
+    # FFN-down from the kernel's own MXInt8 result + bias + residual
+    o = mxb.mx_gemm_fused(fm, fe, fa, q["w2"][0], q["w2"][1], fw, seq, hid, ffn, bias=b2.cuda(), residual=x1)
+    assert mxb.mx_poll_status() == 0
+    qf = fm_n.view(np.int8)
+    si, sj = rng.integers(0, seq, n), rng.integers(0, hid, n)
+    y_ref, _, S = orc.gemm_samples(qf, fe_n, wa, qo["w2"][0], qo["w2"][1], ww, B, si, sj, bias=b2.numpy())
+    res = x1.cpu().numpy()[si, sj].astype(np.float64)
+    _close(o.cpu().numpy()[si, sj], y_ref.astype(np.float64) + res, S + np.abs(res) + np.abs(b2.numpy()[sj]), "FFN-down + residual")

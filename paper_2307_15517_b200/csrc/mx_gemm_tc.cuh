@@ -75,7 +75,8 @@ struct TcParams {
     int64_t ldy;
     int M, N, K;
     int tiles_m, tiles_n;
-    int tma_store;   // 1: the epilogue writes Y with tiled TMA stores (needs ldy % 4 == 0)
+    int tma_store;   // 1: the epilogue writes Y with tiled TMA stores (needs ldy % 4 == 0 and N % 4 == 0: the store
+                     // clips at the tensor's extent in units of 16 bytes)
     // batch > 1 (W_BF16 kernels, fp32 result, no bias): `batch` independent products of the same
     // shape in one launch; the three tensor maps are rank 3 (z = item) and item b writes to
     // y + b * y_batch.  Tiles are numbered item-major.
@@ -215,7 +216,7 @@ __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, in
 // warp's 32 rows start at `rows0`.  Adds the bias and writes the 32 x 32 block either through one of
 // the warp's two 4 KB shared-memory buffers (`warp_bufs`, 128-byte swizzled box layout) and a tiled
 // TMA store -- whole 128-byte lines reach L2, rows >= M and columns >= N are clipped by the store --
-// or, when ldy % 4 != 0, with plain stores.  `epi_buf` counts the warp's TMA blocks (buffer parity).
+// or, when ldy % 4 != 0 or N % 4 != 0, with plain stores.  `epi_buf` counts the warp's TMA blocks (buffer parity).
 // Shared by the one-CTA, the CTA-pair and the block-wise kernel.
 // NBUF = 1: the warp has one 4 KB buffer and waits for its previous store to have been read.
 template <int NBUF = 2>

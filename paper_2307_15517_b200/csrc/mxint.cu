@@ -424,7 +424,9 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
         tm_w = tm_a;                     // not read by the fused kernels
     }
     CUtensorMap tm_y = tm_a;             // placeholder when the epilogue stores directly
-    const bool tma_store = !yq && (ldy % 4) == 0 && (tb.y_batch % 4) == 0;
+    // the tiled store clips at the tensor's extent in units of 16 bytes: with N % 4 != 0 it would write up to three
+    // floats past column N - 1 of every row (into the caller's row padding), so such shapes take the direct stores
+    const bool tma_store = !yq && (ldy % 4) == 0 && (N % 4) == 0 && (tb.y_batch % 4) == 0;
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy, tb.count, tb.y_batch);
         if (s != MX_OK) return s;
@@ -491,7 +493,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     s = encode_bf16_rows(&tm_w, w_hat, N, K, Cfg::BN / 2);
     if (s != MX_OK) return s;
     CUtensorMap tm_y = tm_a;
-    const bool tma_store = !yq && (ldy % 4) == 0;
+    const bool tma_store = !yq && (ldy % 4) == 0 && (N % 4) == 0;       // see launch_tc
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
@@ -542,7 +544,7 @@ mx_status_t launch_tcx(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     s = encode_bf16_rows(&tm_w, w_hat, N, K, Cfg::BN);
     if (s != MX_OK) return s;
     CUtensorMap tm_y = tm_a;
-    const bool tma_store = (ldy % 4) == 0;
+    const bool tma_store = (ldy % 4) == 0 && (N % 4) == 0;              // see launch_tc
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;
@@ -634,7 +636,7 @@ mx_status_t run_tc8(const void *a_mant, const uint8_t *a_exp, const mx_format_t 
     s = encode_u8_sw128(&tm_w, w8, N, K, Cfg::BN);
     if (s != MX_OK) return s;
     CUtensorMap tm_y = tm_a;
-    const bool tma_store = (ldy % 4) == 0;
+    const bool tma_store = (ldy % 4) == 0 && (N % 4) == 0;              // see launch_tc
     if (tma_store) {
         s = encode_f32_out(&tm_y, y, M, N, ldy);
         if (s != MX_OK) return s;

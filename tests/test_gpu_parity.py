@@ -484,3 +484,36 @@ def test_cast_between_widths_bit_exact(mxb, case):
     assert np.array_equal(exps.cpu().numpy(), eo)
     assert np.array_equal(mant.cpu().numpy(), orc.pack(qo, w_out))
     assert int(cnt.item()) == bad
+
+
+@pytest.mark.parametrize("shape", [(2100, 2330, 192), (2048, 8000, 128), (300, 520, 320), (130, 40, 96)])
+@pytest.mark.parametrize("ldy_pad", [8, 6])
+def test_products_write_nothing_outside_their_result(mxb, shape, ldy_pad):
+    """Ragged M and N on the CTA-pair and the one-CTA kernel, through the tiled TMA store (ldy % 4 == 0) and the
+    direct stores (ldy % 4 != 0), with and without the fused tail: the result sits in a frame of sentinel values
+    that must survive, and equals the oracle bit for bit (operands whose partial sums are exact in fp32)."""
+    M, N, K = shape
+    B = 16
+    qa = synth.random_ints((M, K), -7, 7, M + N).numpy()
+    qw = synth.random_ints((N, K), -7, 7, M + N + 1).numpy()
+    ea = np.full((M, K // B), 129, np.uint8)
+    ew = synth.random_bytes((N, 1), 120, 126, 5).numpy().repeat(K // B, axis=1)     # one scale per weight row: still exact
+    unit = 2.0 ** ((129 - 127 - 2) + (120 - 127 - 2))
+    bias = (synth.random_ints((1, N), -1000, 1000, 7).numpy()[0] * unit).astype(np.float32)
+    res = (synth.random_ints((M, N), -3000, 3000, 8).numpy() * unit).astype(np.float32)
+    y_ref, y_seq, _ = orc.gemm(qa, ea, 4, qw, ew, 4, B, bias=bias)
+    assert np.array_equal(y_ref, y_seq)
+    f = mxb.MxFormat(B, 4)
+    am, wm = _dev(orc.pack(qa, 4)), _dev(orc.pack(qw, 4))
+    for tail in (False, True):
+        canvas = torch.full((M + 8, N + ldy_pad), -7.0, dtype=torch.float32, device="cuda")
+        y = canvas[:M, :N]
+        if tail:
+            mxb.mx_gemm_fused(am, _dev(ea), f, wm, _dev(ew), f, M, N, K, bias=_dev(bias), relu=True, residual=_dev(res), y=y)
+            want = np.where(y_ref < 0, np.float32(0), y_ref) + res
+        else:
+            mxb.mx_gemm(am, _dev(ea), f, wm, _dev(ew), f, M, N, K, bias=_dev(bias), y=y, algo=mxb.MX_ALGO_TCGEN05)
+            want = y_ref
+        assert mxb.mx_poll_status() == 0
+        assert np.array_equal(y.cpu().numpy(), want)
+        assert (canvas[M:, :] == -7.0).all() and (canvas[:, N:] == -7.0).all()

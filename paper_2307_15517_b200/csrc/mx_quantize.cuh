@@ -967,22 +967,24 @@ prep_operands_kernel(const PrepJob j)
     ptx::dep_wait();
     ptx::dep_trigger();
     const int warps = blockDim.x >> 5;
-    if ((int)blockIdx.x < j.q_blocks) {
+    // every warp takes its share of BOTH sides (its quantize items, then its decode items): the two sides cost
+    // differently per byte, and with CTAs dedicated to one side each the cheaper side's SM slots sat idle while
+    // the other finished (SMs active 63 % of the kernel's duration)
+    const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)gridDim.x * warps;
+    {
         QuantOut out{nullptr, nullptr, j.a_hat, j.K, nullptr};
-        const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)j.q_blocks * warps;
         if (j.a_rows2) {
             if (j.block == 16) quantize_rows2_body<InT, 16>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
             else quantize_rows2_body<InT, 32>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
         } else if (j.block == 16) quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
         else quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.x), j.M, j.K, j.ldx, j.wa, out, wid, nw);
-    } else {
+    }
+    {
         PackedStrides ps;
         ps.mant_ld = NIBBLE ? j.K / 2 : j.K;
         ps.exp_ld = j.K / j.block;
         ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
         ps.exp_row_shift = j.w_row_shift;
-        const int64_t wid = (int64_t)(blockIdx.x - j.q_blocks) * warps + (threadIdx.x >> 5);
-        const int64_t nw = (int64_t)(gridDim.x - j.q_blocks) * warps;
         decode_bf16_body<NIBBLE, 2>(j.w_mant, j.w_exp, j.N, j.K, j.block, j.ww, j.w_hat, j.K, ps, wid, nw);
     }
 }

@@ -839,7 +839,7 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
         if (s != MX_OK) return s;
         return launch_dequant_bf16(a.w_mant, a.w_exp, N, K, a.fw, w_hat, K, d, st);
     }
-    // CTAs are split between the two sides in proportion to the bytes each moves
+    // one launch for both sides; every warp takes its share of each (see the kernel)
     mx::PrepJob job;
     job.x = a.x; job.M = M; job.K = K; job.ldx = a.ldx; job.wa = a.fa.elem_bits; job.block = a.fa.block;
     job.a_hat = a_hat;
@@ -848,8 +848,6 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
     job.w_row_shift = a.fw.block_rows == 2 ? 1 : 0;
     job.a_rows2 = a.fa.block_rows == 2 ? 1 : 0;
     const bool f32 = a.dt == MX_F32, nib = a.fw.elem_bits <= 4;
-    const double qb = (double)M * K * ((f32 ? 4.0 : 2.0) + 2.0);
-    const double db = (double)N * K * ((nib ? 0.5 : 1.0) + 1.0 / a.fw.block + 2.0);
     // CTAs of 128 threads (8 K registers): small enough to become resident beside a persistent product CTA of the
     // previous call, where they wait in griddepcontrol.wait and start the moment that grid completes
     constexpr int PT = 128;
@@ -859,12 +857,8 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
                                             : resident_ctas(mx::prep_operands_kernel<float, false>))
                                      : (nib ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
                                             : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>)));
-    const int total = d.sm_count * per_sm;            // exactly one resident wave
-    int gq = (int)(total * qb / (qb + db) + 0.5);
-    gq = gq < 1 ? 1 : (gq > total - 1 ? total - 1 : gq);
-    int gd = total - gq;
-    if (gq > need_q) gq = need_q;
-    if (gd > need_d) gd = need_d;
+    const int total = d.sm_count * per_sm;            // at most one resident wave
+    const int gq = need_q + need_d < total ? need_q + need_d : total, gd = 0;
     job.q_blocks = gq;
     ProfScope prof(KIND_PREP, st);
     if (f32) {

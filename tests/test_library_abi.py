@@ -120,6 +120,21 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     assert sq(fp=F(16, 8, 8, 2)) == -3
     assert sq(s=None) == -1 and sq(ld=66) == -4
     assert L.mx_selftest_wait_expiry(0, None) == -2
+    # fused attention: head dimension 128, whole query tiles, one-row container formats, aligned leading dimensions
+    f8 = F(16, 8)
+    at = lambda **kw: L.mx_attention(kw.get("q", fake), fake, fake, fake, kw.get("fqk", f8), fake, fake, f8,
+                                     kw.get("seq", 256), 2, kw.get("d", 128), C.c_float(0.1), 1, kw.get("fp", f8),
+                                     fake, kw.get("ldc", 256), kw.get("pm", None), None, None, 0, None)
+    assert at(q=None) == -1 and at(pm=fake) == -1            # probabilities out: both arrays or none
+    assert at(d=64) == -2 and at(seq=200) == -2 and at(ldc=128) == -2
+    assert at(fqk=F(16, 8, 8, 2)) == -3 and at(fp=F(16, 9)) == -3
+    assert at() == -5                                        # no workspace
+    af = lambda **kw: L.mx_attention_fp(kw.get("q", fake), fake, fake, kw.get("dt", 0), kw.get("ldq", 768), 768, 768,
+                                        kw.get("fqk", f8), f8, kw.get("seq", 256), 2, kw.get("d", 128), C.c_float(0.1),
+                                        1, f8, fake, 256, None, 0, None)
+    assert af(q=None) == -1 and af(dt=5) == -3 and af(fqk=f8.dense()) == -3
+    assert af(ldq=128) == -2 and af(seq=130) == -2 and af(d=96) == -2
+    assert af(ldq=772) == -4 and af() == -5
 
 
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU failure mode")

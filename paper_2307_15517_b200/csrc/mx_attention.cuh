@@ -22,7 +22,8 @@
 //                 row combine their maxima and sums once, between the sweeps, through shared memory).
 //                 Sweep 1: statistics; sweep 2: scores -> probabilities -> MXInt codes -> exact bf16 -> the
 //                 swizzled P operand tile in shared memory; at the end the context tile out of tensor
-//                 memory into global memory.  exp is ex2.approx on arguments pre-scaled by log2(e)
+//                 memory into global memory.  exp is ex2.approx on arguments pre-scaled by log2(e); the division
+//                 by the row sum is a subtraction of its log2 inside that argument
 // Every 128 x 128 bf16 tile is stored as two halves of 128 rows x 128 bytes (64 columns) with the
 // 128-byte swizzle.  All waits are bounded.
 #pragma once
@@ -82,6 +83,13 @@ __device__ __forceinline__ float exp2_approx(float x)
 {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ float log2_approx(float x)
+{
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
 
@@ -247,7 +255,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     m = mm;
                     l = ll;
                 }
-                const float inv = sweep ? 1.0f / l : 0.f;
+                // sweep 2 normalises inside the exponent: e / l = 2^(x - (m + log2 l))
+                const float m_norm = sweep ? m + log2_approx(l) : 0.f;
                 for (int j = 0; j < T; ++j) {
                     const uint32_t si = n_s & 1u;
                     if (!__all_sync(0xFFFFFFFFu, wait(10 + si, (n_s >> 1) & 1u))) { timed_out = true; break; }
@@ -259,13 +268,21 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         uint32_t raw[32];
                         ptx::tmem_ld_32x32(lane_tmem + si * 128u + (uint32_t)(c * 32), raw);
                         ptx::tmem_ld_wait();
+                        // raw scores; masked keys (only the diagonal tile of a causal row has any) become -inf
                         float v[32];
+                        if (c * 32 + 31 <= limit) {
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) v[i] = (c * 32 + i <= limit) ? __uint_as_float(raw[i]) * scale2 : -INFINITY;
+                            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(raw[i]);
+                        } else {
+#pragma unroll
+                            for (int i = 0; i < 32; ++i) v[i] = (c * 32 + i <= limit) ? __uint_as_float(raw[i]) : -INFINITY;
+                        }
+                        // exp(scale * s - max) = 2^(s * scale2 - m) with m kept in log2 units: one FMA and one ex2
                         if (sweep == 0) {
-                            float cm = m;
+                            float cm = -INFINITY;
 #pragma unroll
                             for (int i = 0; i < 32; ++i) cm = fmaxf(cm, v[i]);
+                            cm *= scale2;                               // scale2 > 0: the maximum commutes with the scaling
                             if (cm > m) {                               // the running sum follows the maximum
                                 l *= exp2_approx(m - cm);
                                 m = cm;
@@ -273,14 +290,14 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                             if (m != -INFINITY) {
                                 float s = 0.f;
 #pragma unroll
-                                for (int i = 0; i < 32; ++i) s += exp2_approx(v[i] - m);      // 2^-inf = 0 for masked keys
+                                for (int i = 0; i < 32; ++i) s += exp2_approx(fmaf(v[i], scale2, -m));      // 2^-inf = 0 for masked keys
                                 l += s;
                             }
                         } else {
                             uint32_t amax[2] = {0u, 0u};
 #pragma unroll
                             for (int i = 0; i < 32; ++i) {
-                                v[i] = exp2_approx(v[i] - m) * inv;
+                                v[i] = exp2_approx(fmaf(v[i], scale2, -m_norm));
                                 amax[i >> 4] = max(amax[i >> 4], __float_as_uint(v[i]));     // v >= 0: bits order like values
                             }
                             if (p.p_block == 32) amax[0] = amax[1] = max(amax[0], amax[1]);

@@ -1672,7 +1672,7 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp)) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
     if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid ||
-        seq > INT32_MAX / 4 || hid > INT32_MAX / 4)
+        seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q_mant) || !aligned16(k_mant) || !aligned16(vt_mant) || !aligned16(ctx) || (ldc % 4) != 0 ||
         (p_mant_out && !aligned16(p_mant_out)))
@@ -1706,7 +1706,7 @@ mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtyp
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp) || fqk.packing || fv.packing) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
     if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid || ldq < hid ||
-        ldk < hid || ldv < hid || seq > INT32_MAX / 4 || hid > INT32_MAX / 4)
+        ldk < hid || ldv < hid || seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(ctx) || (ldc % 4) != 0 || (ldq % 8) != 0 ||
         (ldk % 8) != 0 || (ldv % 8) != 0)

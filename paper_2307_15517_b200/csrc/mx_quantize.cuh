@@ -246,9 +246,6 @@ __device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, in
     const int cpr = (int)(K >> 3);                      // 8-element chunks per row
     const int segs = (cpr + 31) >> 5;                   // 256-element segments per row
     const bool nibble = w <= 4;
-    const int qmax = (1 << (w - 1)) - 1;
-    const uint32_t off = nibble ? 8u : 128u;
-    const int fast_top = 229 + w;                       // largest exponent byte of the add-only path
     const bool leader = (lane & (LANES - 1)) == 0;
     const int64_t nb_row = K >> (BLOCK == 16 ? 4 : 5);
     const int64_t mant_ld = nibble ? (K >> 1) : K;
@@ -291,52 +288,11 @@ __device__ __forceinline__ void quantize_rows_body(const InT *__restrict__ x, in
             if (live[u]) {
                 const int ebyte = (int)(amax >> 23);        // 255 <=> an Inf or NaN in the block
                 const bool bad = ebyte == 255;
-                uint32_t f[8];                              // per value: corr + OFF + q
                 float xh[8];                                // decoded values (when asked for)
-                uint32_t corr;
-                if (ebyte <= fast_top) {
-                    const uint32_t mb = ((uint32_t)(ebyte + 25 - w) << 23) | 0x00400000u;
-                    const float M = __uint_as_float(mb);
-                    const float lo = __uint_as_float(mb - (uint32_t)qmax), hi = __uint_as_float(mb + (uint32_t)qmax);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float t = fminf(fmaxf(v[u][i] + M, lo), hi);
-                        f[i] = __float_as_uint(t);
-                        xh[i] = t - M;
-                    }
-                    corr = mb - off;
-                } else {
-                    const float qmaxf = (float)qmax, pow2_wm2 = (float)(1 << (w - 2));
-                    const float magic = 12582912.f;         // 1.5 * 2^23: adding it rounds to an integer
-                    const float inv_pow2_E = pow2_from_biased(254 - (bad ? 254 : ebyte));
-                    const float dec_small = small_neg_pow2(w), dec_big = pow2_from_biased(bad ? 127 : ebyte);
-#pragma unroll
-                    for (int i = 0; i < 8; ++i) {
-                        const float s = (v[u][i] * inv_pow2_E) * pow2_wm2;              // exact scaling
-                        const float t = fminf(fmaxf(s, -qmaxf), qmaxf) + magic;         // clamp, then round
-                        f[i] = bad ? off : __float_as_uint(t) - 0x4B400000u + off;
-                        xh[i] = bad ? __uint_as_float(0x7FC00000u) : ((t - magic) * dec_small) * dec_big;
-                    }
-                    corr = 0;
-                }
+                const uint2 pk = encode8_full(v[u], ebyte, w, xh);      // the one rounding routine of this library
                 if (out.mant) {
-                    if (nibble) {
-                        uint32_t p = 0;
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) p += f[i] << (4 * i);
-                        p = (p - corr * 0x11111111u) ^ 0x88888888u;
-                        *reinterpret_cast<uint32_t *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 4) = p;
-                    } else {
-                        uint2 p = make_uint2(0, 0);
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) {
-                            p.x += f[i] << (8 * i);
-                            p.y += f[4 + i] << (8 * i);
-                        }
-                        p.x = (p.x - corr * 0x01010101u) ^ 0x80808080u;
-                        p.y = (p.y - corr * 0x01010101u) ^ 0x80808080u;
-                        *reinterpret_cast<uint2 *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 8) = p;
-                    }
+                    if (nibble) *reinterpret_cast<uint32_t *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 4) = pk.x;
+                    else *reinterpret_cast<uint2 *>(out.mant + row[u] * mant_ld + (int64_t)kc[u] * 8) = pk;
                     if (leader) out.exps[row[u] * nb_row + (kc[u] >> LANE_SHIFT)] = (uint8_t)ebyte;
                 }
                 if (out.xhat) {

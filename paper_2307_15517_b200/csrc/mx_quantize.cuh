@@ -793,6 +793,34 @@ decode_bf16_kernel(const uint8_t *__restrict__ mant, const uint8_t *__restrict__
                                      (int64_t)gridDim.x * (blockDim.x >> 5));
 }
 
+// Both packed operands of a product -> their bf16 operand forms in one launch: every warp takes its share of the
+// rows of A, then of W (the product that follows needs both; two launches would each pay their own ramp and tail).
+struct DecodePairJob {
+    const uint8_t *a_mant, *a_exp, *w_mant, *w_exp;
+    int64_t M, N, K;
+    int block, wa, ww, a_row_shift, w_row_shift;
+    __nv_bfloat16 *a_hat, *w_hat;
+};
+
+template <bool NIB_A, bool NIB_W>
+__global__ void __launch_bounds__(256)
+decode_pair_kernel(const DecodePairJob j)
+{
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int warps = blockDim.x >> 5;
+    const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)gridDim.x * warps;
+    PackedStrides ps;
+    ps.exp_ld = j.K / j.block;
+    ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+    ps.mant_ld = NIB_A ? j.K / 2 : j.K;
+    ps.exp_row_shift = j.a_row_shift;
+    decode_bf16_body<NIB_A, 2>(j.a_mant, j.a_exp, j.M, j.K, j.block, j.wa, j.a_hat, j.K, ps, wid, nw);
+    ps.mant_ld = NIB_W ? j.K / 2 : j.K;
+    ps.exp_row_shift = j.w_row_shift;
+    decode_bf16_body<NIB_W, 2>(j.w_mant, j.w_exp, j.N, j.K, j.block, j.ww, j.w_hat, j.K, ps, wid, nw);
+}
+
 // ---- dense storage: w bits per element (Eq. 1 counts m + 1 bits per value) ---------------------
 // Element k of a row sits in bits [k*w, (k+1)*w) of the row's bit stream (two's complement; stream
 // bit b = bit b % 8 of byte b / 8); a row takes K*w/8 bytes.  Eight consecutive elements are exactly w

@@ -286,6 +286,38 @@ mx_status_t launch_dequant_bf16(const void *mant, const uint8_t *exps, int64_t r
     return launch_dequant_bf16(mant, exps, rows, K, f, out, ld, dense_strides(K, f), 1, d, st);
 }
 
+// Both operands of a product, (mant, exps) -> bf16 [rows, K]: one launch when both are in container form with
+// whole 32-element items per row, else one launch each.
+mx_status_t launch_dequant_pair(const void *a_mant, const uint8_t *a_exp, const mx_format_t &fa, int64_t M,
+                                const void *w_mant, const uint8_t *w_exp, const mx_format_t &fw, int64_t N, int64_t K,
+                                __nv_bfloat16 *a_hat, __nv_bfloat16 *w_hat, const DeviceInfo &d, cudaStream_t st)
+{
+    if (fa.packing || fw.packing || (K % 32) != 0) {
+        const mx_status_t s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, d, st);
+        if (s != MX_OK) return s;
+        return launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, d, st);
+    }
+    mx::DecodePairJob j;
+    j.a_mant = static_cast<const uint8_t *>(a_mant); j.a_exp = a_exp;
+    j.w_mant = static_cast<const uint8_t *>(w_mant); j.w_exp = w_exp;
+    j.M = M; j.N = N; j.K = K;
+    j.block = fa.block; j.wa = fa.elem_bits; j.ww = fw.elem_bits;
+    j.a_row_shift = fa.block_rows == 2 ? 1 : 0;
+    j.w_row_shift = fw.block_rows == 2 ? 1 : 0;
+    j.a_hat = a_hat; j.w_hat = w_hat;
+    const bool na = fa.elem_bits <= 4, nw = fw.elem_bits <= 4;
+    const int64_t items = (M + N) * (K / 32);
+    ProfScope prof(KIND_DEQUANTIZE, st);
+    const int per_sm = resident_ctas(mx::decode_pair_kernel<true, true>);
+    const dim3 grid((unsigned)grid_for((items + 1) / 2, 256, d.sm_count, per_sm));
+    if (na && nw) MX_CUDA(launch_dep(mx::decode_pair_kernel<true, true>, dim3(grid), dim3(256), 0, st, j));
+    else if (na) MX_CUDA(launch_dep(mx::decode_pair_kernel<true, false>, dim3(grid), dim3(256), 0, st, j));
+    else if (nw) MX_CUDA(launch_dep(mx::decode_pair_kernel<false, true>, dim3(grid), dim3(256), 0, st, j));
+    else MX_CUDA(launch_dep(mx::decode_pair_kernel<false, false>, dim3(grid), dim3(256), 0, st, j));
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 // ---- tensor-core GEMM launcher ----------------------------------------------------------------
 // Encoded tensor maps by (kind, base, extents): pure functions of their key, so entries never go stale.
 typedef std::tuple<int, const void *, int64_t, int64_t, int64_t, int64_t, int64_t> MapKey;
@@ -1131,12 +1163,14 @@ mx_status_t mx_gemm_ex(const void *a_mant, const uint8_t *a_exp, mx_format_t fa,
         return MX_ERR_WORKSPACE;
     if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return MX_ERR_ALIGN;
     __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
-    s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
-    if (s != MX_OK) return s;
-    if (fused) return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+    if (fused) {
+        s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
+        if (s != MX_OK) return s;
+        return run_tc_fused(a_hat, w_mant, w_exp, fw, M, N, K, bias, y, ldy, *d, st);
+    }
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
                                                              round256((size_t)M * K * 2));
-    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    s = launch_dequant_pair(a_mant, a_exp, fa, M, w_mant, w_exp, fw, N, K, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
     if (algo == MX_ALGO_TCGEN05_BLOCKWISE) return launch_tcx(a_hat, w_hat, M, N, K, fa.block, bias, y, ldy, *d, st);
     return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st);
@@ -1270,9 +1304,7 @@ static mx_status_t gemm_tc_impl(const void *a_mant, const uint8_t *a_exp, mx_for
     __nv_bfloat16 *a_hat = static_cast<__nv_bfloat16 *>(workspace);
     __nv_bfloat16 *w_hat = reinterpret_cast<__nv_bfloat16 *>(static_cast<uint8_t *>(workspace) +
                                                              round256((size_t)M * K * 2));
-    s = launch_dequant_bf16(a_mant, a_exp, M, K, fa, a_hat, K, *d, st);
-    if (s != MX_OK) return s;
-    s = launch_dequant_bf16(w_mant, w_exp, N, K, fw, w_hat, K, *d, st);
+    s = launch_dequant_pair(a_mant, a_exp, fa, M, w_mant, w_exp, fw, N, K, a_hat, w_hat, *d, st);
     if (s != MX_OK) return s;
     if (y) return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st, nullptr, TcBatch(), et);
     QuantizedOut yq;

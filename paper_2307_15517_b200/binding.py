@@ -282,11 +282,13 @@ def mx_cast(mant: torch.Tensor, exps: torch.Tensor, K: int, f_in: MxFormat, f_ou
 
 
 def mx_dequantize(mant: torch.Tensor, exps: torch.Tensor, K: int, f: MxFormat,
-                  dtype=torch.float32, stream=None) -> torch.Tensor:
-    _need_cuda(mant, exps)
+                  dtype=torch.float32, out: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+    _need_cuda(mant, exps, out)
     rows = mant.shape[0]
-    out = torch.empty((rows, K), dtype=dtype, device=mant.device)
-    _check(lib.mx_dequantize(_ptr(mant), _ptr(exps), rows, K, f, _ptr(out), _dtype_code(out), K,
+    if out is None:
+        out = torch.empty((rows, K), dtype=dtype, device=mant.device)
+    assert out.shape == (rows, K) and out.stride(1) == 1
+    _check(lib.mx_dequantize(_ptr(mant), _ptr(exps), rows, K, f, _ptr(out), _dtype_code(out), out.stride(0),
                              _stream(stream)), "mx_dequantize")
     return out
 

@@ -24,7 +24,8 @@ def mxb():
     return binding
 
 
-@pytest.mark.parametrize("case", [(2, 256, 16, 8, True), (3, 384, 32, 8, True), (1, 512, 16, 4, True), (2, 256, 16, 8, False)])
+@pytest.mark.parametrize("case", [(2, 256, 16, 8, True), (3, 384, 32, 8, True), (1, 512, 16, 4, True), (2, 256, 16, 8, False),
+                                  (1, 128, 32, 3, True), (5, 640, 16, 6, False)])   # one tile only; five key tiles, no mask
 def test_fused_attention_stage_by_stage(mxb, case):
     H, seq, B, wp, causal = case
     d, w = 128, 8

@@ -927,9 +927,9 @@ dequantize_dense_kernel(const uint8_t *__restrict__ dense, const uint8_t *__rest
     }
 }
 
-// Both operands of the tensor-core product in one launch: the first `q_blocks` CTAs quantize the
-// activations straight to their exact bf16 operand form, the remaining CTAs decode the packed
-// weights to theirs.  Two HBM-bound passes overlap instead of queueing behind each other.
+// Both operands of the tensor-core product in one launch: the activations are quantized straight to
+// their exact bf16 operand form and the packed weights decoded to theirs.  Two HBM-bound passes share
+// one launch instead of queueing behind each other.
 struct PrepJob {
     const void *x;            // activations [M, K] of InT, leading dimension ldx
     int64_t M, K, ldx;
@@ -939,7 +939,6 @@ struct PrepJob {
     int64_t N;
     int ww;
     __nv_bfloat16 *w_hat;     // [N, K]
-    int q_blocks;
     int w_row_shift;          // 1: the weights have two-row blocks
     int a_rows2;              // 1: the activations get two-row blocks
 };

@@ -31,7 +31,7 @@ constexpr int SM_COUNT_FALLBACK = 148;
 
 __device__ uint32_t g_status_word;      // per device: bit 0 = a bounded wait expired
 
-thread_local char t_cuda_error[256] = "";
+thread_local char t_cuda_error[512] = "";
 
 struct DeviceInfo {
     bool probed = false;
@@ -890,15 +890,14 @@ mx_status_t tc_prepare(const mx_linear_args_t &a, __nv_bfloat16 *a_hat, __nv_bfl
                                      : (nib ? resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, true>)
                                             : resident_ctas(mx::prep_operands_kernel<__nv_bfloat16, false>)));
     const int total = d.sm_count * per_sm;            // at most one resident wave
-    const int gq = need_q + need_d < total ? need_q + need_d : total, gd = 0;
-    job.q_blocks = gq;
+    const int grid = need_q + need_d < total ? need_q + need_d : total;
     ProfScope prof(KIND_PREP, st);
     if (f32) {
-        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<float, true>, dim3(gq + gd), dim3(PT), 0, st, job));
-        else MX_CUDA(launch_dep(mx::prep_operands_kernel<float, false>, dim3(gq + gd), dim3(PT), 0, st, job));
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<float, true>, dim3(grid), dim3(PT), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<float, false>, dim3(grid), dim3(PT), 0, st, job));
     } else {
-        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, true>, dim3(gq + gd), dim3(PT), 0, st, job));
-        else MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, false>, dim3(gq + gd), dim3(PT), 0, st, job));
+        if (nib) MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, true>, dim3(grid), dim3(PT), 0, st, job));
+        else MX_CUDA(launch_dep(mx::prep_operands_kernel<__nv_bfloat16, false>, dim3(grid), dim3(PT), 0, st, job));
     }
     MX_CUDA(cudaGetLastError());
     return MX_OK;

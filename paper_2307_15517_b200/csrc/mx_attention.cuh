@@ -1,4 +1,4 @@
-// Fused MX attention for one head dimension of 128 (Fig. 1(d): the block's two attention matmuls --
+// Fused MX attention for head dimensions 128 and 64 (Fig. 1(d): the block's two attention matmuls --
 // tensors "A" = Q K^T and "B" = P V of Fig. 1(a)/(b) -- are MXInt operators, softmax stays in floating
 // point): scores, causal mask, softmax, quantization of the probabilities and the context product in ONE
 // kernel, so neither the fp32 scores (heads x seq x seq) nor the probabilities ever reach HBM.
@@ -38,21 +38,26 @@
 
 namespace mx {
 
-struct AttnCfg {
-    static constexpr int D = 128, BQ = 128, BKEY = 128;
-    static constexpr uint32_t TILE_BYTES = 128 * 128 * 2;            // 32 KB, two halves of 16 KB
-    static constexpr uint32_t HALF_BYTES = TILE_BYTES / 2;
+// D_ = head dimension, 128 or 64.  Q and K tiles are [128 rows, D_] (D_/64 halves of 128 rows x 128 bytes), the V^T
+// tile is [D_ rows, 128 keys] (two halves of D_ rows x 128 bytes), the P tile always [128, 128].
+template <int D_> struct AttnCfgT {
+    static constexpr int D = D_, BQ = 128, BKEY = 128;
+    static constexpr uint32_t TILE_BYTES = 128 * D_ * 2;             // Q, K and V^T tiles: 32 KB or 16 KB
+    static constexpr uint32_t HALF_BYTES = 128 * 128;                // 128 rows x 128 bytes: a half of Q, K or P
+    static constexpr uint32_t V_HALF_BYTES = D_ * 128;               // D_ rows x 128 bytes: a half of V^T
+    static constexpr uint32_t P_BYTES = 128 * 128 * 2;
     static constexpr int KST = 2, VST = 2;                           // K and V^T stage rings
     static constexpr int ROW_WARPS = 16;                             // 4 per TMEM lane quarter: 32 key columns each
     static constexpr int COLS_PER_WARP = 128 / (ROW_WARPS / 4);
     static constexpr int THREADS = 64 + 32 * ROW_WARPS;
     static constexpr uint32_t STATS_BYTES = 2 * (ROW_WARPS / 4) * 128 * 8;   // (maximum, sum) per row and column slice, two items deep
-    static constexpr uint32_t SMEM_BYTES = (1 + KST + VST + 1) * TILE_BYTES + 512 + STATS_BYTES + 1024;    // Q, K ring, V ring, P
-    static constexpr uint32_t TMEM_COLS = 512;                       // S0, S1, O: 3 x 128 columns
+    static constexpr uint32_t SMEM_BYTES = (1 + KST + VST) * TILE_BYTES + P_BYTES + 512 + STATS_BYTES + 1024;    // Q, K ring, V ring, P
+    static constexpr uint32_t TMEM_COLS = 512;                       // S0, S1 (128 columns each), O (D_ columns) at 0, 128, 256
 };
+using AttnCfg = AttnCfgT<128>;
 
 struct AttnParams {
-    float *ctx;               // [seq, ldc] fp32; head h writes columns h*128 .. h*128+127
+    float *ctx;               // [seq, ldc] fp32; head h writes columns h*D .. h*D+D-1
     int64_t ldc;
     int seq, heads;
     float scale;
@@ -63,22 +68,25 @@ struct AttnParams {
     uint32_t *status;
 };
 
-// D[tmem] (+)= A[smem tile] * B[smem tile]^T over K = 128 (two halves of four steps of 16).
-__device__ __forceinline__ void attn_mma_k128(uint32_t d_tmem, uint32_t a_tile, uint32_t b_tile, uint32_t idesc, bool accumulate)
+// D[tmem] (+)= A[smem tile] * B[smem tile]^T over K = 64 * HALVES (halves of four steps of 16); a_half / b_half
+// are the byte distances between the halves of the two tiles.
+template <int HALVES>
+__device__ __forceinline__ void attn_mma(uint32_t d_tmem, uint32_t a_tile, uint32_t a_half, uint32_t b_tile, uint32_t b_half,
+                                         uint32_t idesc, bool accumulate)
 {
 #pragma unroll
-    for (int hh = 0; hh < 2; ++hh)
+    for (int hh = 0; hh < HALVES; ++hh)
 #pragma unroll
         for (int j = 0; j < 4; ++j)
-            ptx::mma_bf16_ss(d_tmem, ptx::smem_desc_k_sw128(a_tile + hh * AttnCfg::HALF_BYTES, j * 32),
-                             ptx::smem_desc_k_sw128(b_tile + hh * AttnCfg::HALF_BYTES, j * 32), idesc,
+            ptx::mma_bf16_ss(d_tmem, ptx::smem_desc_k_sw128(a_tile + hh * a_half, j * 32),
+                             ptx::smem_desc_k_sw128(b_tile + hh * b_half, j * 32), idesc,
                              (accumulate || hh || j) ? 1u : 0u);
 }
 
 // Item of CTA b in round k of G CTAs: the direction alternates between rounds.
 __device__ __forceinline__ int attn_item(uint32_t k, int b, int G) { return (int)k * G + ((k & 1u) ? G - 1 - b : b); }
 
-// tmap_q, tmap_k: bf16 [seq, heads*128], box 64 x 128.  tmap_v: bf16 [heads*128, seq] (V transposed), box 64 x 128.
+// tmap_q, tmap_k: bf16 [seq, heads*D], box 64 x 128.  tmap_v: bf16 [heads*D, seq] (V transposed), box 64 x D.
 __device__ __forceinline__ float exp2_approx(float x)
 {
     float y;
@@ -93,11 +101,12 @@ __device__ __forceinline__ float log2_approx(float x)
     return y;
 }
 
-__global__ void __launch_bounds__(AttnCfg::THREADS, 1)
+template <int D_>
+__global__ void __launch_bounds__(AttnCfgT<D_>::THREADS, 1)
 attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_constant__ CUtensorMap tmap_k,
                  const __grid_constant__ CUtensorMap tmap_v, const AttnParams p)
 {
-    using Cfg = AttnCfg;
+    using Cfg = AttnCfgT<D_>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (ptx::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_gen = smem_raw + (smem_base - ptx::smem_u32(smem_raw));
@@ -105,7 +114,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     const uint32_t k_tiles = q_tile + Cfg::TILE_BYTES;
     const uint32_t v_tiles = k_tiles + Cfg::KST * Cfg::TILE_BYTES;
     const uint32_t p_tile = v_tiles + Cfg::VST * Cfg::TILE_BYTES;
-    const uint32_t bar_base = p_tile + Cfg::TILE_BYTES;
+    const uint32_t bar_base = p_tile + Cfg::P_BYTES;
     // barriers: 0 q_full, 1 q_empty, 2..3 k_full, 4..5 k_empty, 6..7 v_full, 8..9 v_empty, 10..11 s_full,
     //           12..13 s_empty, 14 p_full, 15 p_empty, 16 o_full, 17 o_empty, 18 row statistics written
     auto bar = [&](int i) { return bar_base + 8u * i; };
@@ -150,7 +159,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 if (!wait(1, (n_item & 1u) ^ 1u)) { timed_out = true; break; }
                 ptx::mbar_arrive_expect_tx(bar(0), Cfg::TILE_BYTES);
                 ptx::tma_load_2d(q_tile, &tmap_q, h * Cfg::D, qt * Cfg::BQ, bar(0));
-                ptx::tma_load_2d(q_tile + Cfg::HALF_BYTES, &tmap_q, h * Cfg::D + 64, qt * Cfg::BQ, bar(0));
+                if (Cfg::D == 128) ptx::tma_load_2d(q_tile + Cfg::HALF_BYTES, &tmap_q, h * Cfg::D + 64, qt * Cfg::BQ, bar(0));
                 for (int sweep = 0; sweep < 2 && !timed_out; ++sweep)
                     for (int j = 0; j < T; ++j) {
                         const uint32_t ks = n_k % Cfg::KST;
@@ -158,7 +167,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                         ptx::mbar_arrive_expect_tx(bar(2 + ks), Cfg::TILE_BYTES);
                         const uint32_t kt = k_tiles + ks * Cfg::TILE_BYTES;
                         ptx::tma_load_2d(kt, &tmap_k, h * Cfg::D, j * Cfg::BKEY, bar(2 + ks));
-                        ptx::tma_load_2d(kt + Cfg::HALF_BYTES, &tmap_k, h * Cfg::D + 64, j * Cfg::BKEY, bar(2 + ks));
+                        if (Cfg::D == 128) ptx::tma_load_2d(kt + Cfg::HALF_BYTES, &tmap_k, h * Cfg::D + 64, j * Cfg::BKEY, bar(2 + ks));
                         ++n_k;
                         if (sweep == 1) {
                             const uint32_t vs = n_v % Cfg::VST;
@@ -166,7 +175,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                             ptx::mbar_arrive_expect_tx(bar(6 + vs), Cfg::TILE_BYTES);
                             const uint32_t vt = v_tiles + vs * Cfg::TILE_BYTES;
                             ptx::tma_load_2d(vt, &tmap_v, j * Cfg::BKEY, h * Cfg::D, bar(6 + vs));
-                            ptx::tma_load_2d(vt + Cfg::HALF_BYTES, &tmap_v, j * Cfg::BKEY + 64, h * Cfg::D, bar(6 + vs));
+                            ptx::tma_load_2d(vt + Cfg::V_HALF_BYTES, &tmap_v, j * Cfg::BKEY + 64, h * Cfg::D, bar(6 + vs));
                             ++n_v;
                         }
                     }
@@ -175,7 +184,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
         __syncwarp();
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128);
+            constexpr uint32_t idesc = ptx::idesc_bf16_f32(128, 128), idesc_o = ptx::idesc_bf16_f32(128, Cfg::D);
             const uint32_t s_tmem[2] = {tmem_base, tmem_base + 128u}, o_tmem = tmem_base + 256u;
             uint32_t n_item = 0, n_k = 0, n_v = 0, n_s = 0, n_p = 0;
             // S_j = Q K_j^T into score accumulator n_s % 2
@@ -183,7 +192,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 const uint32_t ks = n_k % Cfg::KST, si = n_s & 1u;
                 if (!wait(2 + ks, (n_k / Cfg::KST) & 1u) || !wait(12 + si, ((n_s >> 1) & 1u) ^ 1u)) return false;
                 ptx::tc_fence_after_sync();
-                attn_mma_k128(s_tmem[si], q_tile, k_tiles + ks * Cfg::TILE_BYTES, idesc, false);
+                attn_mma<Cfg::D / 64>(s_tmem[si], q_tile, Cfg::HALF_BYTES, k_tiles + ks * Cfg::TILE_BYTES, Cfg::HALF_BYTES, idesc, false);
                 ptx::mma_commit(bar(4 + ks));               // K stage free
                 ptx::mma_commit(bar(10 + si));              // scores complete
                 ++n_k;
@@ -208,7 +217,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     const uint32_t vs = n_v % Cfg::VST;
                     if (!wait(14, n_p & 1u) || !wait(6 + vs, (n_v / Cfg::VST) & 1u)) { timed_out = true; break; }
                     ptx::tc_fence_after_sync();
-                    attn_mma_k128(o_tmem, p_tile, v_tiles + vs * Cfg::TILE_BYTES, idesc, j > 0);
+                    attn_mma<2>(o_tmem, p_tile, Cfg::HALF_BYTES, v_tiles + vs * Cfg::TILE_BYTES, Cfg::V_HALF_BYTES, idesc_o, j > 0);
                     ptx::mma_commit(bar(8 + vs));            // V stage free
                     ptx::mma_commit(bar(15));                // P tile free
                     ++n_v;
@@ -350,6 +359,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
 #pragma unroll 1
             for (int cc = 0; cc < CHUNKS; ++cc) {
                 const int c = slice * CHUNKS + cc;
+                if (c * 32 >= Cfg::D) break;                 // head dimension 64: the first two column slices write it
                 uint32_t raw[32];
                 ptx::tmem_ld_32x32(lane_tmem + 256u + (uint32_t)(c * 32), raw);
                 ptx::tmem_ld_wait();

@@ -44,7 +44,7 @@ struct DeviceInfo {
     bool tc2_attr_set[2] = {false, false};
     bool tcx_attr_set = false;
     bool tc8_attr_set = false;
-    bool attn_attr_set = false;
+    bool attn_attr_set[2] = {false, false};
 };
 DeviceInfo g_dev[MAX_DEVICES];
 std::mutex g_init_mu;        // guards every lazily initialised field above and below (calls may come from several host threads)
@@ -1652,20 +1652,23 @@ mx_status_t mx_gemm_batched(const void *a_mant, const uint8_t *a_exp, mx_format_
 }
 
 // ---- fused attention ---------------------------------------------------------------------------
+extern "C++" {
 // The fused attention kernel on operands already in bf16 operand form: q_hat, k_hat [seq, hid], v_hat [hid, seq].
-static mx_status_t launch_attention(const __nv_bfloat16 *q_hat, const __nv_bfloat16 *k_hat, const __nv_bfloat16 *v_hat,
-                                    int64_t seq, int64_t heads, float scale, int causal, mx_format_t fp, float *ctx,
-                                    int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, DeviceInfo *d, cudaStream_t st)
+template <int D>
+static mx_status_t launch_attention_d(const __nv_bfloat16 *q_hat, const __nv_bfloat16 *k_hat, const __nv_bfloat16 *v_hat,
+                                      int64_t seq, int64_t heads, float scale, int causal, mx_format_t fp, float *ctx,
+                                      int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, DeviceInfo *d, cudaStream_t st)
 {
-    const int64_t hid = heads * mx::AttnCfg::D;
+    using Cfg = mx::AttnCfgT<D>;
+    const int64_t hid = heads * D;
     CUtensorMap tm_q, tm_k, tm_v;
     mx_status_t s = encode_bf16_rows(&tm_q, q_hat, seq, hid, 128);
     if (s != MX_OK) return s;
     s = encode_bf16_rows(&tm_k, k_hat, seq, hid, 128);
     if (s != MX_OK) return s;
-    s = encode_bf16_rows(&tm_v, v_hat, hid, seq, 128);
+    s = encode_bf16_rows(&tm_v, v_hat, hid, seq, D);
     if (s != MX_OK) return s;
-    s = smem_attr_once(d->attn_attr_set, mx::attention_kernel, (int)mx::AttnCfg::SMEM_BYTES);
+    s = smem_attr_once(d->attn_attr_set[D == 128 ? 0 : 1], mx::attention_kernel<D>, (int)Cfg::SMEM_BYTES);
     if (s != MX_OK) return s;
     mx::AttnParams ap;
     ap.ctx = ctx;
@@ -1679,13 +1682,25 @@ static mx_status_t launch_attention(const __nv_bfloat16 *q_hat, const __nv_bfloa
     ap.p_mant = static_cast<uint8_t *>(p_mant_out);
     ap.p_exp = p_exp_out;
     ap.status = d->status;
-    const int64_t items = (seq / mx::AttnCfg::BQ) * heads;
+    const int64_t items = (seq / Cfg::BQ) * heads;
     const int grid = items < d->sm_count ? (int)items : d->sm_count;
     ProfScope prof(KIND_GEMM_TC, st);
-    MX_CUDA(launch_dep(mx::attention_kernel, dim3(grid), dim3(mx::AttnCfg::THREADS), mx::AttnCfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
+    MX_CUDA(launch_dep(mx::attention_kernel<D>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
     MX_CUDA(cudaGetLastError());
     return MX_OK;
 }
+
+static mx_status_t launch_attention(const __nv_bfloat16 *q_hat, const __nv_bfloat16 *k_hat, const __nv_bfloat16 *v_hat,
+                                    int64_t seq, int64_t heads, int64_t head_dim, float scale, int causal, mx_format_t fp,
+                                    float *ctx, int64_t ldc, void *p_mant_out, uint8_t *p_exp_out, DeviceInfo *d,
+                                    cudaStream_t st)
+{
+    if (head_dim == 64)
+        return launch_attention_d<64>(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, p_mant_out, p_exp_out, d, st);
+    return launch_attention_d<128>(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, p_mant_out, p_exp_out, d, st);
+}
+
+}  // extern "C++"
 
 size_t mx_attention_workspace_bytes(int64_t seq, int64_t heads, int64_t head_dim)
 {
@@ -1702,7 +1717,7 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     if ((p_mant_out == nullptr) != (p_exp_out == nullptr)) return MX_ERR_NULL;
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp)) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
-    if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid ||
+    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid ||
         seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q_mant) || !aligned16(k_mant) || !aligned16(vt_mant) || !aligned16(ctx) || (ldc % 4) != 0 ||
@@ -1724,7 +1739,7 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     if (s != MX_OK) return s;
     s = launch_dequant_bf16(vt_mant, vt_exp, hid, seq, fv, v_hat, seq, *d, st);
     if (s != MX_OK) return s;
-    return launch_attention(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, p_mant_out, p_exp_out, d, st);
+    return launch_attention(q_hat, k_hat, v_hat, seq, heads, head_dim, scale, causal, fp, ctx, ldc, p_mant_out, p_exp_out, d, st);
 }
 
 mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtype_t dt, int64_t ldq, int64_t ldk,
@@ -1736,7 +1751,7 @@ mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtyp
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp) || fqk.packing || fv.packing) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
-    if (seq <= 0 || heads <= 0 || head_dim != mx::AttnCfg::D || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid || ldq < hid ||
+    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid || ldq < hid ||
         ldk < hid || ldv < hid || seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(ctx) || (ldc % 4) != 0 || (ldq % 8) != 0 ||
@@ -1772,7 +1787,7 @@ mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtyp
                                                                                  ldv, fv.block, fv.elem_bits, ov);
         MX_CUDA(cudaGetLastError());
     }
-    return launch_attention(q_hat, k_hat, v_hat, seq, heads, scale, causal, fp, ctx, ldc, nullptr, nullptr, d, st);
+    return launch_attention(q_hat, k_hat, v_hat, seq, heads, head_dim, scale, causal, fp, ctx, ldc, nullptr, nullptr, d, st);
 }
 
 // ---- fp32 glue of the transformer block ---------------------------------------------------------

@@ -24,11 +24,12 @@ def mxb():
     return binding
 
 
+@pytest.mark.parametrize("d", [128, 64])
 @pytest.mark.parametrize("case", [(2, 256, 16, 8, True), (3, 384, 32, 8, True), (1, 512, 16, 4, True), (2, 256, 16, 8, False),
                                   (1, 128, 32, 3, True), (5, 640, 16, 6, False)])   # one tile only; five key tiles, no mask
-def test_fused_attention_stage_by_stage(mxb, case):
+def test_fused_attention_stage_by_stage(mxb, case, d):
     H, seq, B, wp, causal = case
-    d, w = 128, 8
+    w = 8
     hid = H * d
     q = synth.student_t_activations(seq, hid, 21)
     k = synth.outlier_activations(seq, hid, 22, 3, 20.0)
@@ -72,20 +73,21 @@ def test_fused_attention_stage_by_stage(mxb, case):
 def test_fused_attention_refuses_what_it_cannot_tile(mxb):
     f = mxb.MxFormat(16, 8)
     z = lambda r, c: torch.zeros((r, c), dtype=torch.uint8, device="cuda")
-    for seq, H, d, status in ((200, 2, 128, -2), (256, 2, 64, -2)):
+    for seq, H, d, status in ((200, 2, 128, -2), (256, 2, 96, -2)):
         with pytest.raises(mxb.MxError) as e:
             mxb.mx_attention(z(seq, H * d), z(seq, H * d // 16), z(seq, H * d), z(seq, H * d // 16), f, z(H * d, seq),
                              z(H * d, seq // 16), f, seq, H, d, 0.1, f, workspace=mxb.alloc_workspace(1 << 22))
         assert e.value.status == status
 
 
+@pytest.mark.parametrize("d", [128, 64])
 @pytest.mark.parametrize("case", [(2, 256, 16, torch.float32), (3, 384, 32, torch.bfloat16)])
-def test_attention_on_floating_point_operands_equals_quantize_then_attention(mxb, case):
+def test_attention_on_floating_point_operands_equals_quantize_then_attention(mxb, case, d):
     """mx_attention_fp quantizes q, k (along the head dimension) and v (along the tokens) on the fly; its
     context must equal, bit for bit, mx_attention on the operands quantized by mx_quantize (which the
     quantizer tests tie to the oracle), also when q, k, v are column slices of one wider tensor."""
     H, seq, B, dtype = case
-    d, hid = 128, H * 128
+    hid = H * d
     qkv = torch.cat([synth.student_t_activations(seq, hid, 41), synth.outlier_activations(seq, hid, 42, 3, 20.0),
                      synth.student_t_activations(seq, hid, 43)], dim=1).to(dtype).cuda()
     q, k, v = qkv[:, :hid], qkv[:, hid:2 * hid], qkv[:, 2 * hid:]

@@ -148,10 +148,12 @@ def test_softmax_with_mxint_result(mods, fmt):
         assert (pm2 == pm).float().mean().item() > 0.995 and (pe2 == pe).float().mean().item() > 0.999
 
 
-def test_decoder_block_fused_softmax_matches_staged_run(mods):
+@pytest.mark.parametrize("heads,head_dim,seq", [(2, 128, 160), (2, 128, 256), (4, 64, 256)])
+def test_decoder_block_fused_softmax_matches_staged_run(mods, heads, head_dim, seq):
+    """The path the benchmark times (products with fused tails; the fused attention kernel when the sequence is
+    a whole number of 128-query tiles, for head dimensions 128 and 64) against the staged run of the same block."""
     mxb, db = mods
-    cfg = db.BlockConfig(hidden=256, heads=2, head_dim=128, ffn=512)
-    seq = 160
+    cfg = db.BlockConfig(hidden=256, heads=heads, head_dim=head_dim, ffn=512)
     g = torch.Generator().manual_seed(12)
     x = synth.outlier_activations(seq, cfg.hidden, 6, 2, 40.0).cuda()
     W = {n: synth.gaussian_weights(o, i, 30 + j).cuda() for j, (n, o, i) in enumerate(

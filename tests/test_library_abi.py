@@ -126,7 +126,7 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
                                      kw.get("seq", 256), 2, kw.get("d", 128), C.c_float(0.1), 1, kw.get("fp", f8),
                                      fake, kw.get("ldc", 256), kw.get("pm", None), None, None, 0, None)
     assert at(q=None) == -1 and at(pm=fake) == -1            # probabilities out: both arrays or none
-    assert at(d=64) == -2 and at(seq=200) == -2 and at(ldc=128) == -2
+    assert at(d=96) == -2 and at(seq=200) == -2 and at(ldc=128) == -2
     assert L.mx_attention(fake, fake, fake, fake, f8, fake, fake, f8, 256, 2, 128, C.c_float(-0.1), 1, f8, fake, 256, None,
                           None, None, 0, None) == -2       # the softmax scale must be positive
     assert at(fqk=F(16, 8, 8, 2)) == -3 and at(fp=F(16, 9)) == -3

@@ -337,9 +337,9 @@ MX_API mx_status_t mx_softmax_q(const float *s, int64_t ld, int64_t rows, int64_
  *   p_mant_out, p_exp_out : nullable; when given, the quantized probabilities are also written there
  *              ([heads*seq, seq/2 or seq] and [heads*seq, seq/fp.block]; masked positions 0) -- for checks
  *   workspace: mx_attention_workspace_bytes(seq, heads, head_dim) (the three operands as bf16), 256-byte aligned
- * Restrictions: head_dim 128 or 64, seq % 128 == 0, scale > 0, container storage, one-row blocks (blocks of 16 or
- * 32 divide both head dimensions and the key tile); otherwise MX_ERR_SHAPE / MX_ERR_FORMAT (use the three separate
- * calls then).
+ * Restrictions: head_dim 128 or 64, seq % 32 == 0 (whole blocks along the keys; the last tile of 128 queries or keys
+ * may be ragged), scale > 0, container storage, one-row blocks; otherwise MX_ERR_SHAPE / MX_ERR_FORMAT (use the
+ * three separate calls then).
  */
 MX_API size_t mx_attention_workspace_bytes(int64_t seq, int64_t heads, int64_t head_dim);
 MX_API mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k_mant, const uint8_t *k_exp,

@@ -145,7 +145,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
     ptx::dep_wait();
     if (threadIdx.x == 0) ptx::dep_trigger();
 
-    const int q_tiles_n = p.seq / Cfg::BQ;
+    const int q_tiles_n = (p.seq + Cfg::BQ - 1) / Cfg::BQ;      // the last tile may be ragged: loads beyond seq read zeros
     const int items = q_tiles_n * p.heads;
     bool timed_out = false;
     auto wait = [&](int i, uint32_t parity) { return ptx::mbar_wait_bounded(bar(i), parity, abort_flag, TC_WAIT_LIMIT_NS); };
@@ -270,7 +270,8 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                     const uint32_t si = n_s & 1u;
                     if (!__all_sync(0xFFFFFFFFu, wait(10 + si, (n_s >> 1) & 1u))) { timed_out = true; break; }
                     ptx::tc_fence_after_sync();
-                    const int limit = p.causal ? qrow - j * Cfg::BKEY : Cfg::BKEY;   // keys 0..limit of this tile take part
+                    // keys 0..limit of this tile take part: the causal bound and the end of the sequence
+                    const int limit = min(p.causal ? qrow - j * Cfg::BKEY : Cfg::BKEY, p.seq - 1 - j * Cfg::BKEY);
 #pragma unroll 1
                     for (int cc = 0; cc < CHUNKS; ++cc) {
                         const int c = slice * CHUNKS + cc;
@@ -329,7 +330,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                                 asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(hw[0]), "r"(hw[1]),
                                              "r"(hw[2]), "r"(hw[3])
                                              : "memory");
-                                if (p.p_mant) {
+                                if (p.p_mant && qrow < p.seq && key0 + 8 * u < p.seq) {
                                     if (nibble) *reinterpret_cast<uint32_t *>(p.p_mant + prow * (p.seq >> 1) + ((key0 + 8 * u) >> 1)) = pk.x;
                                     else *reinterpret_cast<uint2 *>(p.p_mant + prow * p.seq + key0 + 8 * u) = pk;
                                     if (p.p_block == 16 ? (u & 1) == 0 : u == 0)
@@ -363,6 +364,7 @@ attention_kernel(const __grid_constant__ CUtensorMap tmap_q, const __grid_consta
                 uint32_t raw[32];
                 ptx::tmem_ld_32x32(lane_tmem + 256u + (uint32_t)(c * 32), raw);
                 ptx::tmem_ld_wait();
+                if (qrow >= p.seq) continue;                 // rows of a ragged last query tile
 #pragma unroll
                 for (int i = 0; i < 8; ++i)
                     reinterpret_cast<float4 *>(orow + c * 32)[i] =

@@ -1682,7 +1682,7 @@ static mx_status_t launch_attention_d(const __nv_bfloat16 *q_hat, const __nv_bfl
     ap.p_mant = static_cast<uint8_t *>(p_mant_out);
     ap.p_exp = p_exp_out;
     ap.status = d->status;
-    const int64_t items = (seq / Cfg::BQ) * heads;
+    const int64_t items = ((seq + Cfg::BQ - 1) / Cfg::BQ) * heads;
     const int grid = items < d->sm_count ? (int)items : d->sm_count;
     ProfScope prof(KIND_GEMM_TC, st);
     MX_CUDA(launch_dep(mx::attention_kernel<D>, dim3(grid), dim3(Cfg::THREADS), Cfg::SMEM_BYTES, st, tm_q, tm_k, tm_v, ap));
@@ -1717,7 +1717,7 @@ mx_status_t mx_attention(const void *q_mant, const uint8_t *q_exp, const void *k
     if ((p_mant_out == nullptr) != (p_exp_out == nullptr)) return MX_ERR_NULL;
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp)) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
-    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid ||
+    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % 32) != 0 || ldc < hid ||
         seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q_mant) || !aligned16(k_mant) || !aligned16(vt_mant) || !aligned16(ctx) || (ldc % 4) != 0 ||
@@ -1751,7 +1751,7 @@ mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtyp
     if (dt != MX_F32 && dt != MX_BF16) return MX_ERR_FORMAT;
     if (!format_1d(fqk) || !format_1d(fv) || !format_1d(fp) || fqk.packing || fv.packing) return MX_ERR_FORMAT;
     const int64_t hid = heads * head_dim;
-    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % mx::AttnCfg::BQ) != 0 || ldc < hid || ldq < hid ||
+    if (seq <= 0 || heads <= 0 || (head_dim != 128 && head_dim != 64) || (seq % 32) != 0 || ldc < hid || ldq < hid ||
         ldk < hid || ldv < hid || seq > INT32_MAX / 4 || hid > INT32_MAX / 4 || !(scale > 0.f))
         return MX_ERR_SHAPE;
     if (!aligned16(q) || !aligned16(k) || !aligned16(v) || !aligned16(ctx) || (ldc % 4) != 0 || (ldq % 8) != 0 ||

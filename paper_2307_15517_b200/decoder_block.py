@@ -68,7 +68,7 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
     h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
     qkv = linear(h1, "wqkv", params["bqkv"], 3 * hid)           # [seq, 3 * hidden]: q | k | v
     q, k, v = rec("q", qkv[:, :hid]), rec("k", qkv[:, hid:2 * hid]), rec("v", qkv[:, 2 * hid:])
-    if keep is None and d in (64, 128) and seq % 128 == 0:
+    if keep is None and d in (64, 128) and seq % 32 == 0:
         # q, k, v quantized straight to the operand form, then scores, causal softmax, quantized probabilities and
         # context in one kernel: nothing of size seq x seq and no packed copy of q, k, v is stored
         ctx = mxb.mx_attention_fp(q, k, v, fa, fa, H, d, 1.0 / math.sqrt(d), fa, causal=True)

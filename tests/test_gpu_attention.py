@@ -26,7 +26,8 @@ def mxb():
 
 @pytest.mark.parametrize("d", [128, 64])
 @pytest.mark.parametrize("case", [(2, 256, 16, 8, True), (3, 384, 32, 8, True), (1, 512, 16, 4, True), (2, 256, 16, 8, False),
-                                  (1, 128, 32, 3, True), (5, 640, 16, 6, False)])   # one tile only; five key tiles, no mask
+                                  (1, 128, 32, 3, True), (5, 640, 16, 6, False),    # one tile only; five key tiles, no mask
+                                  (2, 160, 16, 8, True), (2, 416, 32, 8, False), (3, 32, 16, 8, True)])   # ragged last tiles
 def test_fused_attention_stage_by_stage(mxb, case, d):
     H, seq, B, wp, causal = case
     w = 8
@@ -73,7 +74,7 @@ def test_fused_attention_stage_by_stage(mxb, case, d):
 def test_fused_attention_refuses_what_it_cannot_tile(mxb):
     f = mxb.MxFormat(16, 8)
     z = lambda r, c: torch.zeros((r, c), dtype=torch.uint8, device="cuda")
-    for seq, H, d, status in ((200, 2, 128, -2), (256, 2, 96, -2)):
+    for seq, H, d, status in ((200, 2, 128, -2), (256, 2, 96, -2)):       # 200 % 32 != 0; head dimension 96
         with pytest.raises(mxb.MxError) as e:
             mxb.mx_attention(z(seq, H * d), z(seq, H * d // 16), z(seq, H * d), z(seq, H * d // 16), f, z(H * d, seq),
                              z(H * d, seq // 16), f, seq, H, d, 0.1, f, workspace=mxb.alloc_workspace(1 << 22))
@@ -81,7 +82,7 @@ def test_fused_attention_refuses_what_it_cannot_tile(mxb):
 
 
 @pytest.mark.parametrize("d", [128, 64])
-@pytest.mark.parametrize("case", [(2, 256, 16, torch.float32), (3, 384, 32, torch.bfloat16)])
+@pytest.mark.parametrize("case", [(2, 256, 16, torch.float32), (3, 384, 32, torch.bfloat16), (2, 224, 16, torch.float32)])
 def test_attention_on_floating_point_operands_equals_quantize_then_attention(mxb, case, d):
     """mx_attention_fp quantizes q, k (along the head dimension) and v (along the tokens) on the fly; its
     context must equal, bit for bit, mx_attention on the operands quantized by mx_quantize (which the

@@ -86,8 +86,9 @@ def test_streamed_decode_result_stays_inside(mxb, T):
     assert all(bool((L["y"] != -3.0).any()) for L in layers)
 
 
-def test_attention_context_stays_inside(mxb):
-    H, seq, d = 2, 256, 128
+@pytest.mark.parametrize("seq,d", [(256, 128), (160, 128), (96, 64)])      # whole and ragged query tiles
+def test_attention_context_stays_inside(mxb, seq, d):
+    H = 2
     hid = H * d
     fa = mxb.MxFormat(16, 8)
     q, k, v = (synth.student_t_activations(seq, hid, s).cuda() for s in (1, 2, 3))

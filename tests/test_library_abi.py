@@ -135,7 +135,7 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
                                         kw.get("fqk", f8), f8, kw.get("seq", 256), 2, kw.get("d", 128), C.c_float(0.1),
                                         1, f8, fake, 256, None, 0, None)
     assert af(q=None) == -1 and af(dt=5) == -3 and af(fqk=f8.dense()) == -3
-    assert af(ldq=128) == -2 and af(seq=130) == -2 and af(d=96) == -2
+    assert af(ldq=128) == -2 and af(seq=136) == -2 and af(d=96) == -2
     assert af(ldq=772) == -4 and af() == -5
 
 

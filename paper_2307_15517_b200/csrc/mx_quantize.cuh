@@ -527,17 +527,17 @@ quantize_strided_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int6
 // of 16 or one of 32 -- so that they write 128 (nibbles) or 256 contiguous bytes per row.
 // Tile element (r, k) sits at r * 264 + k + k / 32: with this padding both the transposing store
 // and the per-lane reads are (nearly) free of bank conflicts.
+// CTA-wide body (256 threads, every thread must call it): CTA `cta` of `n_ctas` walks the 32 x 256 tiles.
 template <typename InT>
-__global__ void __launch_bounds__(256)
-quantize_transposed_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t stride_k, int block, int w,
-                           QuantOut out)
+__device__ __forceinline__ void quantize_transposed_body(float *tile, const InT *__restrict__ x, int64_t rows, int64_t K,
+                                                         int64_t stride_k, int block, int w, const QuantOut &out,
+                                                         int cta, int n_ctas)
 {
-    __shared__ float tile[32 * 264];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const bool nibble = w <= 4;
     const int64_t nb_row = K / block, mant_ld = nibble ? (K >> 1) : K;
     const int64_t row_tiles = (rows + 31) >> 5, k_tiles = (K + 255) >> 8;
-    for (int64_t tix = blockIdx.x; tix < row_tiles * k_tiles; tix += gridDim.x) {
+    for (int64_t tix = cta; tix < row_tiles * k_tiles; tix += n_ctas) {
         const int64_t r0 = (tix % row_tiles) * 32, k0 = (tix / row_tiles) * 256;
         __syncthreads();                                    // the previous tile has been consumed
 #pragma unroll 4
@@ -601,6 +601,48 @@ quantize_transposed_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, i
             }
         }
     }
+}
+
+template <typename InT>
+__global__ void __launch_bounds__(256)
+quantize_transposed_kernel(const InT *__restrict__ x, int64_t rows, int64_t K, int64_t stride_k, int block, int w,
+                           QuantOut out)
+{
+    __shared__ float tile[32 * 264];
+    quantize_transposed_body<InT>(tile, x, rows, K, stride_k, block, w, out, (int)blockIdx.x, (int)gridDim.x);
+}
+
+// The three operands of the fused attention in one launch (256 threads per CTA): every warp takes its share of the
+// rows of q and of k (blocks along the head dimension, written in operand form), then every CTA its share of the
+// tiles of v (blocks along the tokens, written transposed).
+struct AttnOperandsJob {
+    const void *q, *k, *v;
+    int64_t seq, hid, ldq, ldk, ldv;
+    int block_qk, w_qk, block_v, w_v;
+    __nv_bfloat16 *q_hat, *k_hat;      // [seq, hid]
+    __nv_bfloat16 *v_hat;              // [hid, seq]
+};
+
+template <typename InT>
+__global__ void __launch_bounds__(256)
+attention_operands_kernel(const AttnOperandsJob j)
+{
+    __shared__ float tile[32 * 264];
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int warps = blockDim.x >> 5;
+    const int64_t wid = (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), nw = (int64_t)gridDim.x * warps;
+    const QuantOut oq{nullptr, nullptr, j.q_hat, j.hid, nullptr, 0}, ok{nullptr, nullptr, j.k_hat, j.hid, nullptr, 0};
+    if (j.block_qk == 16) {
+        quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.q), j.seq, j.hid, j.ldq, j.w_qk, oq, wid, nw);
+        quantize_rows_body<InT, 16, 2>(static_cast<const InT *>(j.k), j.seq, j.hid, j.ldk, j.w_qk, ok, wid, nw);
+    } else {
+        quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.q), j.seq, j.hid, j.ldq, j.w_qk, oq, wid, nw);
+        quantize_rows_body<InT, 32, 2>(static_cast<const InT *>(j.k), j.seq, j.hid, j.ldk, j.w_qk, ok, wid, nw);
+    }
+    const QuantOut ov{nullptr, nullptr, j.v_hat, j.seq, nullptr, 0};
+    quantize_transposed_body<InT>(tile, static_cast<const InT *>(j.v), j.hid, j.seq, j.ldv, j.block_v, j.w_v, ov,
+                                  (int)blockIdx.x, (int)gridDim.x);
 }
 
 // (mant, exps) -> decoded values, 8 elements per thread.

@@ -1767,24 +1767,23 @@ mx_status_t mx_attention_fp(const void *q, const void *k, const void *v, mx_dtyp
     uint8_t *ws = static_cast<uint8_t *>(workspace);
     __nv_bfloat16 *q_hat = reinterpret_cast<__nv_bfloat16 *>(ws), *k_hat = reinterpret_cast<__nv_bfloat16 *>(ws + one),
                   *v_hat = reinterpret_cast<__nv_bfloat16 *>(ws + 2 * one);
-    // queries and keys: blocks along the head dimension, straight to the operand form
-    mx::QuantOut oq{nullptr, nullptr, q_hat, hid, nullptr, 0}, ok{nullptr, nullptr, k_hat, hid, nullptr, 0};
-    s = quantize_rows_any(q, dt, seq, hid, ldq, fqk, oq, *d, st);
-    if (s != MX_OK) return s;
-    s = quantize_rows_any(k, dt, seq, hid, ldk, fqk, ok, *d, st);
-    if (s != MX_OK) return s;
-    // values: blocks along the tokens, i.e. along the slow axis of v; written transposed, [hid, seq]
+    // one launch for the three operands: q and k in blocks along the head dimension, v in blocks along the tokens
+    // (the slow axis of v) and written transposed, [hid, seq]; all straight to the operand form
     {
-        mx::QuantOut ov{nullptr, nullptr, v_hat, seq, nullptr, 0};
-        const int64_t tiles = ((hid + 31) / 32) * ((seq + 255) / 256);
-        const int tgrid = (int)(tiles < (int64_t)d->sm_count * 4 ? tiles : (int64_t)d->sm_count * 4);
+        mx::AttnOperandsJob j;
+        j.q = q; j.k = k; j.v = v;
+        j.seq = seq; j.hid = hid; j.ldq = ldq; j.ldk = ldk; j.ldv = ldv;
+        j.block_qk = fqk.block; j.w_qk = fqk.elem_bits; j.block_v = fv.block; j.w_v = fv.elem_bits;
+        j.q_hat = q_hat; j.k_hat = k_hat; j.v_hat = v_hat;
+        const int64_t row_items = seq * ((hid + 255) / 256), tiles = ((hid + 31) / 32) * ((seq + 255) / 256);
+        const int64_t want = (row_items + 7) / 8 > tiles ? (row_items + 7) / 8 : tiles;      // 8 warps per CTA
+        const int per_sm = dt == MX_F32 ? resident_ctas(mx::attention_operands_kernel<float>)
+                                        : resident_ctas(mx::attention_operands_kernel<__nv_bfloat16>);
+        const int64_t cap = (int64_t)d->sm_count * per_sm;
+        const int grid = (int)(want < cap ? want : cap);
         ProfScope prof(KIND_QUANTIZE, st);
-        if (dt == MX_F32)
-            mx::quantize_transposed_kernel<float><<<tgrid, 256, 0, st>>>(static_cast<const float *>(v), hid, seq, ldv, fv.block,
-                                                                         fv.elem_bits, ov);
-        else
-            mx::quantize_transposed_kernel<__nv_bfloat16><<<tgrid, 256, 0, st>>>(static_cast<const __nv_bfloat16 *>(v), hid, seq,
-                                                                                 ldv, fv.block, fv.elem_bits, ov);
+        if (dt == MX_F32) MX_CUDA(launch_dep(mx::attention_operands_kernel<float>, dim3(grid), dim3(256), 0, st, j));
+        else MX_CUDA(launch_dep(mx::attention_operands_kernel<__nv_bfloat16>, dim3(grid), dim3(256), 0, st, j));
         MX_CUDA(cudaGetLastError());
     }
     return launch_attention(q_hat, k_hat, v_hat, seq, heads, head_dim, scale, causal, fp, ctx, ldc, nullptr, nullptr, d, st);

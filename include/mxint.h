@@ -415,7 +415,7 @@ MX_API mx_status_t mx_linear_q(const void *x, mx_dtype_t dt, int64_t M, int64_t 
 
 /* ---- the product with a fused element-wise tail ------------------------------------------------
  *
- * Fig. 1(d): between the MX operators of a decoder block sit a bias, the activation function and the
+ * Fig. 1(d): between the MX operators of a decoder block sit LayerNorm, a bias, the activation function and the
  * skip connection, all in floating point.  These two calls are mx_gemm / mx_linear (fp32 result y) or
  * mx_gemm_q / mx_linear_q (MXInt result fy, y_mant, y_exp) with that tail applied in the product kernel's
  * epilogue, on the fp32 accumulator, before the result is stored or quantized:
@@ -440,11 +440,24 @@ MX_API mx_status_t mx_gemm_fused(const void *a_mant, const uint8_t *a_exp, mx_fo
                           mx_format_t fy, void *y_mant, uint8_t *y_exp, void *workspace,
                           size_t workspace_bytes, void *stream);
 
+/* What happens to the rows of x before they are quantized (mx_linear_fused only; NULL = nothing).
+ * layernorm != 0: every row is layer-normalised first, y = (x - mean) / sqrt(var + ln_eps) * ln_gamma + ln_beta
+ * (ln_gamma / ln_beta device fp32 [K], nullable = 1 / 0), with the arithmetic of mx_layernorm, bit for bit, and
+ * goes straight to the quantizer: the normalised fp32 tensor is never stored (Fig. 1(d): LayerNorm stays in
+ * floating point in front of the MX linears).  Needs fp32 x, K % 32 == 0, K <= 8192, one-row container formats
+ * (MX_ERR_FORMAT / MX_ERR_SHAPE otherwise). */
+typedef struct {
+    int32_t layernorm;
+    const float *ln_gamma;
+    const float *ln_beta;
+    float ln_eps;
+} mx_prologue_t;
+
 MX_API mx_status_t mx_linear_fused(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx,
-                            mx_format_t fa, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
-                            int64_t N, const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy,
-                            void *y_mant, uint8_t *y_exp, void *workspace, size_t workspace_bytes,
-                            void *stream);
+                            mx_format_t fa, const mx_prologue_t *pro, const void *w_mant,
+                            const uint8_t *w_exp, mx_format_t fw, int64_t N, const mx_epilogue_t *ep,
+                            float *y, int64_t ldy, mx_format_t fy, void *y_mant, uint8_t *y_exp,
+                            void *workspace, size_t workspace_bytes, void *stream);
 
 /* ---- the other MX formats of the paper: Block Minifloat and Block Logarithm ---------------------
  *

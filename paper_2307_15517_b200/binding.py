@@ -48,6 +48,11 @@ class MxEpilogue(C.Structure):
     _fields_ = [("bias", C.c_void_p), ("relu", C.c_int32), ("residual", C.c_void_p), ("ldr", C.c_int64)]
 
 
+class MxPrologue(C.Structure):
+    """Mirrors ``mx_prologue_t``: LayerNorm applied to the rows of x in front of the quantizer."""
+    _fields_ = [("layernorm", C.c_int32), ("ln_gamma", C.c_void_p), ("ln_beta", C.c_void_p), ("ln_eps", C.c_float)]
+
+
 class MxAltFormat(C.Structure):
     """A Block Minifloat (kind 1) or Block Logarithm (kind 2) format: mirrors ``mx_alt_format_t``."""
     _fields_ = [("kind", C.c_int32), ("block", C.c_int32), ("elem_exp_bits", C.c_int32),
@@ -115,7 +120,8 @@ def _load() -> C.CDLL:
     L.mx_linear_q.restype = i32
     E = C.POINTER(MxEpilogue)
     L.mx_gemm_fused.argtypes = [vp, vp, F, vp, vp, F, i64, i64, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
-    L.mx_linear_fused.argtypes = [vp, i32, i64, i64, i64, F, vp, vp, F, i64, E, vp, i64, F, vp, vp, vp, sz, vp]
+    L.mx_linear_fused.argtypes = [vp, i32, i64, i64, i64, F, C.POINTER(MxPrologue), vp, vp, F, i64, E, vp, i64, F, vp, vp,
+                                  vp, sz, vp]
     L.mx_gemm_fused.restype = i32
     L.mx_poll_status.argtypes = [vp]
     L.mx_selftest_wait_expiry.argtypes = [C.c_uint32, vp]
@@ -376,10 +382,16 @@ def _epilogue(bias, relu, residual):
 def mx_linear_fused(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, N: int,
                     bias: Optional[torch.Tensor] = None, relu: bool = False,
                     residual: Optional[torch.Tensor] = None, fy: Optional[MxFormat] = None, y=None,
-                    y_mant=None, y_exp=None, workspace: Optional[torch.Tensor] = None, stream=None):
+                    y_mant=None, y_exp=None, layernorm=None, workspace: Optional[torch.Tensor] = None, stream=None):
     """mx_linear with bias, ReLU and a residual applied in the epilogue.  ``fy`` None: returns the fp32
-    result; else returns (y_mant, y_exp), the result quantized to ``fy`` along N."""
+    result; else returns (y_mant, y_exp), the result quantized to ``fy`` along N.
+    ``layernorm`` = (gamma, beta, eps): the rows of x are layer-normalised in front of the quantizer."""
     _need_cuda(x, w_mant, w_exp, bias, residual, y, y_mant, y_exp, workspace)
+    pro = None
+    if layernorm is not None:
+        gamma, beta, eps = layernorm
+        _need_cuda(gamma, beta)
+        pro = MxPrologue(1, None if gamma is None else gamma.data_ptr(), None if beta is None else beta.data_ptr(), eps)
     M, K = x.shape
     assert x.stride(1) == 1 and (residual is None or (residual.stride(1) == 1 and residual.dtype == torch.float32))
     if fy is None:
@@ -391,8 +403,8 @@ def mx_linear_fused(x: torch.Tensor, fa: MxFormat, w_mant, w_exp, fw: MxFormat, 
     if workspace is None:
         workspace = alloc_workspace(mx_workspace_bytes_ex(M, N, K, fa, fw, MX_ALGO_TCGEN05), x.device)
     ep = _epilogue(bias, relu, residual)
-    _check(lib.mx_linear_fused(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, _ptr(w_mant), _ptr(w_exp), fw, N,
-                               C.byref(ep), _ptr(y) if fy is None else None, y.stride(0) if fy is None else N,
+    _check(lib.mx_linear_fused(_ptr(x), _dtype_code(x), M, K, x.stride(0), fa, None if pro is None else C.byref(pro),
+                               _ptr(w_mant), _ptr(w_exp), fw, N, C.byref(ep), _ptr(y) if fy is None else None, y.stride(0) if fy is None else N,
                                fy if fy is not None else MxFormat(), None if fy is None else _ptr(y_mant),
                                None if fy is None else _ptr(y_exp), _ptr(workspace), workspace.numel(),
                                _stream(stream)), "mx_linear_fused")

@@ -70,6 +70,79 @@ layernorm_kernel(const float *__restrict__ x, int64_t ldx, const float *__restri
     }
 }
 
+// The operand pass of a layer whose input is layer-normalised first (Fig. 1(d): LayerNorm in floating point in
+// front of the MX linears): CTA r < M normalises row r exactly as layernorm_kernel does (same ownership of the
+// elements, same order of every sum: the values are bit-identical to that kernel's), quantizes them to MXInt --
+// element c of the row sits in thread c % 256, so a block of 16 or 32 columns is a group of neighbouring lanes and
+// its maximum one round of shuffles -- and writes the exact bf16 operand; the fp32 normalised tensor never exists.
+// After its row every CTA decodes its share of the packed weights (decode_bf16_body), so one launch prepares both
+// operands of the product, as prep_operands_kernel does for a plain layer.
+struct PrepLnJob {
+    const float *x;           // [M, K] fp32, leading dimension ldx
+    int64_t M, K, ldx;
+    const float *gamma, *beta;   // nullable
+    float eps;
+    int wa, block;
+    __nv_bfloat16 *a_hat;     // [M, K]
+    const uint8_t *w_mant, *w_exp;
+    int64_t N;
+    int ww;
+    __nv_bfloat16 *w_hat;     // [N, K]
+    int w_row_shift;
+};
+
+template <int PER, bool NIBBLE>
+__global__ void __launch_bounds__(GLUE_THREADS)
+prep_ln_operands_kernel(const PrepLnJob j)
+{
+    __shared__ float scratch[GLUE_THREADS / 32];
+    ptx::dep_wait();
+    ptx::dep_trigger();
+    const int cols = (int)j.K;
+    for (int64_t r = blockIdx.x; r < j.M; r += gridDim.x) {
+        const float *xr = j.x + r * j.ldx;
+        float v[PER];
+        float s = 0.f;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int c = threadIdx.x + i * GLUE_THREADS;
+            v[i] = c < cols ? xr[c] : 0.f;
+            s += v[i];
+        }
+        const float mean = block_sum(s, scratch) / (float)cols;
+        float q = 0.f;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int c = threadIdx.x + i * GLUE_THREADS;
+            const float d = c < cols ? v[i] - mean : 0.f;
+            q += d * d;
+        }
+        const float rstd = 1.0f / sqrtf(block_sum(q, scratch) / (float)cols + j.eps);
+        __nv_bfloat16 *ar = j.a_hat + r * j.K;
+#pragma unroll
+        for (int i = 0; i < PER; ++i) {
+            const int c = threadIdx.x + i * GLUE_THREADS;           // K % block == 0: a block is all inside or all outside
+            const float y = c < cols ? (v[i] - mean) * rstd * (j.gamma ? j.gamma[c] : 1.f) + (j.beta ? j.beta[c] : 0.f) : 0.f;
+            uint32_t amax = __float_as_uint(absmax_nan(0.f, y));
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1)
+                if (d < j.block) amax = max(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, d));
+            const float y8[8] = {y, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            float xh[8];
+            encode8_full(y8, (int)(amax >> 23), j.wa, xh);          // the library's rounding; only xh[0] is used
+            if (c < cols) ar[c] = __float2bfloat16_rn(xh[0]);
+        }
+    }
+    PackedStrides ps;
+    ps.mant_ld = NIBBLE ? j.K / 2 : j.K;
+    ps.exp_ld = j.K / j.block;
+    ps.mant_batch = ps.exp_batch = ps.out_batch = 0;
+    ps.exp_row_shift = j.w_row_shift;
+    const int warps = blockDim.x >> 5;
+    decode_bf16_body<NIBBLE, 2>(j.w_mant, j.w_exp, j.N, j.K, j.block, j.ww, j.w_hat, j.K, ps,
+                                (int64_t)blockIdx.x * warps + (threadIdx.x >> 5), (int64_t)gridDim.x * warps);
+}
+
 // In place: s[r, j] = softmax_j(scale * s[r, j]) over j < limit, 0 elsewhere; limit = cols, or
 // (r % rows_per_batch) + 1 with the causal mask.
 template <int PER>

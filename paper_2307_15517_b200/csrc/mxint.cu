@@ -1315,11 +1315,39 @@ static mx_status_t gemm_tc_impl(const void *a_mant, const uint8_t *a_exp, mx_for
 }
 
 // The same for the layer: activations quantized on the fly.
+// The operand pass with LayerNorm in front of the activation quantizer (see prep_ln_operands_kernel).
+static mx_status_t tc_prepare_ln(const mx_linear_args_t &a, const mx_prologue_t &ln, __nv_bfloat16 *a_hat,
+                                 __nv_bfloat16 *w_hat, DeviceInfo &d, cudaStream_t st)
+{
+    mx::PrepLnJob j;
+    j.x = static_cast<const float *>(a.x); j.M = a.M; j.K = a.K; j.ldx = a.ldx;
+    j.gamma = ln.ln_gamma; j.beta = ln.ln_beta; j.eps = ln.ln_eps;
+    j.wa = a.fa.elem_bits; j.block = a.fa.block; j.a_hat = a_hat;
+    j.w_mant = static_cast<const uint8_t *>(a.w_mant); j.w_exp = a.w_exp; j.N = a.N; j.ww = a.fw.elem_bits;
+    j.w_hat = w_hat; j.w_row_shift = a.fw.block_rows == 2 ? 1 : 0;
+    const int per = (int)((a.K + mx::GLUE_THREADS - 1) / mx::GLUE_THREADS);
+    const bool nib = a.fw.elem_bits <= 4;
+    const unsigned g = (unsigned)(a.M < (int64_t)d.sm_count * 8 ? a.M : (int64_t)d.sm_count * 8);
+    ProfScope prof(KIND_PREP, st);
+#define MX_LAUNCH_LN(P)                                                                                                  \
+    do {                                                                                                                 \
+        if (nib) MX_CUDA(launch_dep(mx::prep_ln_operands_kernel<P, true>, dim3(g), dim3(mx::GLUE_THREADS), 0, st, j));   \
+        else MX_CUDA(launch_dep(mx::prep_ln_operands_kernel<P, false>, dim3(g), dim3(mx::GLUE_THREADS), 0, st, j));      \
+    } while (0)
+    if (per <= 4) MX_LAUNCH_LN(4);
+    else if (per <= 8) MX_LAUNCH_LN(8);
+    else if (per <= 16) MX_LAUNCH_LN(16);
+    else MX_LAUNCH_LN(32);
+#undef MX_LAUNCH_LN
+    MX_CUDA(cudaGetLastError());
+    return MX_OK;
+}
+
 static mx_status_t linear_tc_impl(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
                                   const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
                                   const float *bias, const EpiTail &et, float *y, int64_t ldy, mx_format_t fy,
                                   void *y_mant, uint8_t *y_exp, uint32_t *nonfinite_count, void *workspace,
-                                  size_t workspace_bytes, void *stream)
+                                  size_t workspace_bytes, void *stream, const mx_prologue_t *ln = nullptr)
 {
     mx_status_t s = check_gemm_args(x, nullptr, fa, w_mant, w_exp, fw, M, N, K, bias,
                                     y ? y : static_cast<const float *>(y_mant), y ? ldy : N);
@@ -1331,6 +1359,12 @@ static mx_status_t linear_tc_impl(const void *x, mx_dtype_t dt, int64_t M, int64
     if (!y) {
         s = check_quantized_out(fy, M, N, y_mant, y_exp);
         if (s != MX_OK) return s;
+    }
+    const bool with_ln = ln && ln->layernorm;
+    if (with_ln) {
+        // rows normalised in registers: fp32 input, rows of at most 8192 values, one-row container formats
+        if (dt != MX_F32 || fa.block_rows != 1 || fw.packing) return MX_ERR_FORMAT;
+        if ((K % 32) != 0 || K > mx::GLUE_THREADS * mx::GLUE_MAX_PER_THREAD) return MX_ERR_SHAPE;
     }
     DeviceInfo *d = nullptr;
     s = device_info(&d);
@@ -1344,7 +1378,11 @@ static mx_status_t linear_tc_impl(const void *x, mx_dtype_t dt, int64_t M, int64
     mx_linear_args_t one;
     one.x = x; one.dt = dt; one.M = M; one.K = K; one.ldx = ldx; one.fa = fa;
     one.w_mant = w_mant; one.w_exp = w_exp; one.fw = fw; one.N = N; one.bias = bias; one.y = y; one.ldy = y ? ldy : N;
-    s = tc_prepare(one, a_hat, w_hat, *d, st);
+    if (with_ln) {
+        s = tc_prepare_ln(one, *ln, a_hat, w_hat, *d, st);
+    } else {
+        s = tc_prepare(one, a_hat, w_hat, *d, st);
+    }
     if (s != MX_OK) return s;
     if (y) return run_tc(a_hat, w_hat, M, N, K, bias, y, ldy, *d, st, nullptr, TcBatch(), et);
     QuantizedOut yq;
@@ -1406,8 +1444,8 @@ mx_status_t mx_gemm_fused(const void *a_mant, const uint8_t *a_exp, mx_format_t 
 }
 
 mx_status_t mx_linear_fused(const void *x, mx_dtype_t dt, int64_t M, int64_t K, int64_t ldx, mx_format_t fa,
-                            const void *w_mant, const uint8_t *w_exp, mx_format_t fw, int64_t N,
-                            const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy, void *y_mant,
+                            const mx_prologue_t *pro, const void *w_mant, const uint8_t *w_exp, mx_format_t fw,
+                            int64_t N, const mx_epilogue_t *ep, float *y, int64_t ldy, mx_format_t fy, void *y_mant,
                             uint8_t *y_exp, void *workspace, size_t workspace_bytes, void *stream)
 {
     const float *bias;
@@ -1415,7 +1453,7 @@ mx_status_t mx_linear_fused(const void *x, mx_dtype_t dt, int64_t M, int64_t K, 
     const mx_status_t s = tail_of(ep, N, y, y_mant, &bias, &et);
     if (s != MX_OK) return s;
     return linear_tc_impl(x, dt, M, K, ldx, fa, w_mant, w_exp, fw, N, bias, et, y, ldy, fy, y_mant, y_exp, nullptr,
-                          workspace, workspace_bytes, stream);
+                          workspace, workspace_bytes, stream, pro);
 }
 
 // ---- decode: few tokens, weights streamed once ------------------------------------------------

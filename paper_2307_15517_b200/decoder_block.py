@@ -65,10 +65,17 @@ def run(cfg: BlockConfig, x: torch.Tensor, qweights, params: Dict[str, torch.Ten
 
     if "bqkv" not in params:
         params = prepare_params(params)
-    h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
-    qkv = linear(h1, "wqkv", params["bqkv"], 3 * hid)           # [seq, 3 * hidden]: q | k | v
+    fused_path = keep is None and d in (64, 128) and seq % 32 == 0
+    if fused_path:
+        # LayerNorm runs inside the projection's operand pass: the normalised tensor is never stored
+        wm, we = qweights["wqkv"]
+        qkv = mxb.mx_linear_fused(x, fa, wm, we, fw, 3 * hid, bias=params["bqkv"],
+                                  layernorm=(params["ln1_g"], params["ln1_b"], cfg.eps))
+    else:
+        h1 = rec("ln1", mxb.mx_layernorm(x, params["ln1_g"], params["ln1_b"], cfg.eps))
+        qkv = linear(h1, "wqkv", params["bqkv"], 3 * hid)       # [seq, 3 * hidden]: q | k | v
     q, k, v = rec("q", qkv[:, :hid]), rec("k", qkv[:, hid:2 * hid]), rec("v", qkv[:, 2 * hid:])
-    if keep is None and d in (64, 128) and seq % 32 == 0:
+    if fused_path:
         # q, k, v quantized straight to the operand form, then scores, causal softmax, quantized probabilities and
         # context in one kernel: nothing of size seq x seq and no packed copy of q, k, v is stored
         ctx = mxb.mx_attention_fp(q, k, v, fa, fa, H, d, 1.0 / math.sqrt(d), fa, causal=True)
@@ -102,9 +109,9 @@ def _after_attention(cfg, x, ctx, qweights, params, linear, rec):
         # leaves its product already quantized (the next product's operand), so no fp32 tensor of width ffn exists
         wm, we = qweights["wo"]
         x1 = mxb.mx_linear_fused(ctx, fa, wm, we, fw, hid, bias=params["bo"], residual=x)
-        h2 = mxb.mx_layernorm(x1, params["ln2_g"], params["ln2_b"], cfg.eps)
         wm, we = qweights["w1"]
-        fm, fe = mxb.mx_linear_fused(h2, fa, wm, we, fw, cfg.ffn, bias=params["b1"], relu=True, fy=fa)
+        fm, fe = mxb.mx_linear_fused(x1, fa, wm, we, fw, cfg.ffn, bias=params["b1"], relu=True, fy=fa,
+                                     layernorm=(params["ln2_g"], params["ln2_b"], cfg.eps))
         wm, we = qweights["w2"]
         return mxb.mx_gemm_fused(fm, fe, fa, wm, we, fw, x.shape[0], hid, cfg.ffn, bias=params["b2"], residual=x1)
     a = rec("attn_out", linear(ctx, "wo", params["bo"], hid))

@@ -136,3 +136,31 @@ def test_fused_tail_argument_checks(mxb):
     assert call(None, y.data_ptr(), None) == 0
     assert mxb.mx_poll_status() == 0
     assert torch.count_nonzero(y).item() == 0
+
+
+@pytest.mark.parametrize("case", [(300, 512, 528, 16, True), (129, 1056, 256, 32, False), (2048, 4096, 1024, 16, True)])
+def test_layernorm_in_the_operand_pass_equals_the_separate_kernel(mxb, case):
+    """mx_linear_fused with a LayerNorm prologue normalises each row with the arithmetic of mx_layernorm and
+    quantizes it straight to the operand: the product must equal mx_layernorm followed by mx_linear bit for bit
+    (the staged sequence is checked against the oracle stage by stage elsewhere), also with a poisoned row."""
+    M, K, N, B, affine = case
+    x = synth.outlier_activations(M, K, 51, 3, 30.0)
+    x[M // 2, 5] = float("nan")                                  # one non-finite row: the poison must carry over
+    g = torch.Generator().manual_seed(52)
+    gamma = (1 + 0.1 * torch.randn(K, generator=g)).cuda() if affine else None
+    beta = (0.1 * torch.randn(K, generator=g)).cuda() if affine else None
+    bias = torch.randn(N, generator=g).cuda()
+    fa, fw = mxb.MxFormat(B, 8), mxb.MxFormat(B, 4)
+    wm, we = mxb.mx_quantize(synth.gaussian_weights(N, K, 53).cuda(), fw)
+    xd = x.cuda()
+    h = mxb.mx_layernorm(xd, gamma, beta, 1e-5)
+    want = mxb.mx_linear(h, fa, wm, we, fw, N, bias=bias, algo=mxb.MX_ALGO_TCGEN05)
+    got = mxb.mx_linear_fused(xd, fa, wm, we, fw, N, bias=bias, layernorm=(gamma, beta, 1e-5))
+    assert mxb.mx_poll_status() == 0
+    w_, g_ = want.cpu().numpy(), got.cpu().numpy()
+    assert np.array_equal(np.isnan(w_), np.isnan(g_)) and np.isnan(g_[M // 2]).all() and not np.isnan(g_[0]).any()
+    assert np.array_equal(w_[~np.isnan(w_)], g_[~np.isnan(g_)])
+    # and with the tail and an MXInt8 result, as the decoder block's FFN-up runs it
+    qm, qe = mxb.mx_linear_fused(xd, fa, wm, we, fw, N, bias=bias, relu=True, fy=fa, layernorm=(gamma, beta, 1e-5))
+    qm2, qe2 = mxb.mx_linear_fused(h, fa, wm, we, fw, N, bias=bias, relu=True, fy=fa)
+    assert torch.equal(qm, qm2) and torch.equal(qe, qe2)

@@ -103,9 +103,13 @@ def test_invalid_arguments_are_rejected_on_the_host(mxb):
     # the product with a fused tail: exactly one kind of result, residual rows at least N wide
     ep = mxb.MxEpilogue()
     ep.residual, ep.ldr = fake, 16
-    ft = lambda ep, y, ym: L.mx_linear_fused(fake, 0, 8, 64, 64, f, fake, fake, f, 32, ep, y, 32, f, ym, fake, None, 0, None)
+    ft = lambda ep, y, ym, pro=None, K=64, dt=0: L.mx_linear_fused(fake, dt, 8, K, K, f, pro, fake, fake, f, 32, ep, y, 32, f, ym,
+                                                                 fake, fake, 1 << 20, None)
     assert ft(None, fake, fake) == -1 and ft(None, None, None) == -1
     assert ft(C.byref(ep), fake, None) == -2
+    ln = mxb.MxPrologue(1, None, None, 1e-5)
+    assert ft(None, fake, None, C.byref(ln), dt=1) == -3        # LayerNorm in the operand pass wants fp32 rows
+    assert ft(None, fake, None, C.byref(ln), K=16384) == -2     # ... of at most 8192 values
     # casts and the softmax with an MXInt result
     c = lambda **kw: L.mx_cast(kw.get("m", fake), fake, kw.get("fi", f), kw.get("rows", 4), kw.get("K", 64),
                                kw.get("fo", F(32, 8)), kw.get("mo", fake), fake, None, None)

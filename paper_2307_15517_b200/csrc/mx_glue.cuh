@@ -92,7 +92,7 @@ struct PrepLnJob {
 };
 
 template <int PER, bool NIBBLE>
-__global__ void __launch_bounds__(GLUE_THREADS)
+__global__ void __launch_bounds__(GLUE_THREADS, 4)
 prep_ln_operands_kernel(const PrepLnJob j)
 {
     __shared__ float scratch[GLUE_THREADS / 32];

@@ -77,6 +77,8 @@ struct TcParams {
     int tiles_m, tiles_n;
     int tma_store;   // 1: the epilogue writes Y with tiled TMA stores (needs ldy % 4 == 0 and N % 4 == 0: the store
                      // clips at the tensor's extent in units of 16 bytes)
+    int frag_store;  // 1 (fp32 result, no tail, ldy even, y 8-byte aligned): the epilogue reads the accumulator in the
+                     // fragment shape and stores from registers, 32-byte sectors at a time, without shared memory
     // batch > 1 (W_BF16 kernels, fp32 result, no bias): `batch` independent products of the same
     // shape in one launch; the three tensor maps are rank 3 (z = item) and item b writes to
     // y + b * y_batch.  Tiles are numbered item-major.
@@ -210,6 +212,41 @@ __device__ __forceinline__ void store_mxint_chunk(const TcParams &p, int row, in
             *reinterpret_cast<uint4 *>(p.yq_mant + (int64_t)row * p.N + n + 16 * h) =
                 make_uint4(pk[0].x, pk[0].y, pk[1].x, pk[1].y);
     }
+}
+
+// fp32 epilogue without shared memory: the 32 rows x 32 columns of a warp's chunk are read from tensor memory in
+// the fragment shape (two loads of 16 lanes) and stored from registers; four neighbouring lanes write one 32-byte
+// sector.  The staging of the tiled store costs the pair kernel shared-memory bandwidth, which is what bounds its
+// main loop (see the header of mx_gemm_tc2.cuh).  taddr = the warp's lane quarter and the chunk's first column.
+__device__ __forceinline__ void store_f32_frag(const TcParams &p, uint32_t taddr, int rows0, int n, int tb, int lane)
+{
+    uint32_t r[2][16];
+    ptx::tmem_ld_16x256b_x4(taddr, r[0]);
+    ptx::tmem_ld_16x256b_x4(taddr + (16u << 16), r[1]);
+    ptx::tmem_ld_wait();
+    if (n >= p.N || rows0 >= p.M) return;                  // warp-uniform
+    float *y = p.y + (int64_t)tb * p.y_batch;
+    const int cq = 2 * (lane & 3);
+#pragma unroll
+    for (int h = 0; h < 2; ++h)
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+            const int c = n + 8 * g + cq;
+            float2 b = make_float2(0.f, 0.f);
+            if (p.bias) {
+                if (c + 1 < p.N) b = __ldg(reinterpret_cast<const float2 *>(p.bias + c));
+                else if (c < p.N) b.x = __ldg(p.bias + c);
+            }
+#pragma unroll
+            for (int u = 0; u < 2; ++u) {
+                const int row = rows0 + 16 * h + 8 * u + (lane >> 2);
+                if (row >= p.M || c >= p.N) continue;
+                const float2 v = make_float2(__uint_as_float(r[h][4 * g + 2 * u]) + b.x, __uint_as_float(r[h][4 * g + 2 * u + 1]) + b.y);
+                float *dst = y + (int64_t)row * p.ldy + c;
+                if (c + 1 < p.N) *reinterpret_cast<float2 *>(dst) = v;
+                else *dst = v.x;
+            }
+        }
 }
 
 // fp32 epilogue of one lane: r holds 32 consecutive outputs (columns n .. n + 31) of row `row`; the
@@ -666,6 +703,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             ptx::tc_fence_after_sync();
 #pragma unroll 1
             for (int c0 = col0; c0 < col0 + COLS; c0 += 32) {
+                if (!FUSED && !tail && p.frag_store) {
+                    store_f32_frag(p, tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), m0 + quad * 32,
+                                   n0 + c0, tb, lane);
+                    continue;
+                }
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
                 TailRegs cur;

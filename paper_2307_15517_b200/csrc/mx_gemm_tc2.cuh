@@ -181,6 +181,11 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constan
             ptx::tc_fence_after_sync();
 #pragma unroll 1
             for (int c0 = col0; c0 < col0 + COLS; c0 += 32) {
+                if (!tail && p.frag_store) {
+                    store_f32_frag(p, tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), m0 + quad * 32,
+                                   n0 + c0, 0, lane);
+                    continue;
+                }
                 uint32_t r[32];
                 ptx::tmem_ld_32x32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(acc * BN + c0), r);
                 TailRegs cur;

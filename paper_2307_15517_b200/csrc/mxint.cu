@@ -439,6 +439,13 @@ mx_status_t encode_f32_out(CUtensorMap *tm, float *y, int64_t M, int64_t N, int6
     return MX_OK;
 }
 
+// fp32 result, no fused tail, rows of y and the items of a batch 8-byte aligned: the epilogue may store from registers
+// in the accumulator-fragment shape (TcParams::frag_store)
+bool frag_store_ok(bool quantized, bool tail, const float *y, int64_t ldy, int64_t y_batch)
+{
+    return !quantized && !tail && y && (ldy % 2) == 0 && (y_batch % 2) == 0 && (reinterpret_cast<uintptr_t>(y) & 7u) == 0;
+}
+
 template <int BN, int WMODE>
 mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, const PackedW &pw,
                       int64_t M, int64_t N, int64_t K, const float *bias, float *y, int64_t ldy,
@@ -484,6 +491,7 @@ mx_status_t launch_tc(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, co
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.status = d.status;
     p.tma_store = tma_store ? 1 : 0;
+    p.frag_store = frag_store_ok(yq != nullptr, et.any(), y, ldy, tb.y_batch) && WMODE == mx::W_BF16 ? 1 : 0;
     p.w_mant = pw.mant;
     p.w_exp = pw.exps;
     p.w_bits = pw.bits;
@@ -548,6 +556,7 @@ mx_status_t launch_tc2(const __nv_bfloat16 *a_hat, const __nv_bfloat16 *w_hat, i
     p.tiles_n = (int)((N + Cfg::BN - 1) / Cfg::BN);
     p.status = d.status;
     p.tma_store = tma_store ? 1 : 0;
+    p.frag_store = frag_store_ok(yq != nullptr, et.any(), y, ldy, 0) ? 1 : 0;
     p.batch = 1;
     p.yq_mant = yq ? yq->mant : nullptr;
     p.yq_exp = yq ? yq->exps : nullptr;

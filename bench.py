@@ -33,7 +33,7 @@ WORKLOAD = "opt-1.3b prefill linears, 2048 tokens, MXInt4 block 16 (4 layers per
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 # dram__bytes_read.sum + dram__bytes_write.sum per launch, averaged over the four launches of a step, from the
 # ncu captures summarised under profiles/ (gemm_tc_kernel_opt13b_prefill.md, launch_list_bench.md)
-GEMM_TC_DRAM_BYTES_PER_LAUNCH = 47.2e6
+GEMM_TC_DRAM_BYTES_PER_LAUNCH = 48.1e6
 PREP_DRAM_BYTES_PER_LAUNCH = 38.9e6
 # Dense bf16 tensor throughput of one SM per clock (tcgen05, 128x256x16 per 128 clocks): 8192 flop.
 # SMs x this x the SM clock sampled during the timed region = the hardware bound the fractions below use
